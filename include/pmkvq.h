@@ -1,0 +1,121 @@
+/*
+ * pmkvq.h - C ABI of the B200-native PM-KVQ decode hot path.
+ *
+ * PM-KVQ (Progressive Mixed-precision KV cache Quantization) stores a transformer block's
+ * KV cache as integer codes with a per-token fp32 scale and zero-point, starts at 16 bit and
+ * halves the width of the existing cache (16 -> 8 -> 4 -> 2) each time the block's memory
+ * budget fills, down to the block's final width "Fbit" (Sec. 3.1).  Keys are channel-equalized
+ * before quantization and the scale is migrated into the Query (Eq. 9, Sec. 3.3).
+ *
+ * Conventions
+ *  - Pointers named d_* are DEVICE pointers owned by the caller; h_* are HOST pointers.
+ *    The library never frees caller memory and never allocates device memory: the whole
+ *    cache (codes, scales, zero-points, split-K partials) lives in one caller-supplied arena.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Kernel launches are
+ *    asynchronous on that stream; an asynchronous CUDA error surfaces as PMKVQ_ERR_CUDA from a
+ *    later call.
+ *  - Every call returns a status; nothing throws, aborts or traps.  Argument errors are
+ *    detected on the host before any launch and leave the cache state unchanged.
+ *  - All sequences of the batch share one length.  head_dim is 128 (one quantization group =
+ *    one token x one KV head x 128 channels, group size 128, Sec. 4.1.3).
+ *  - A cache handle is not thread-safe.
+ */
+#ifndef PMKVQ_H_
+#define PMKVQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pmkvq_cache pmkvq_cache; /* opaque; host heap; created / destroyed by the library */
+
+typedef enum {
+  PMKVQ_OK = 0,
+  PMKVQ_ERR_INVALID_ARG = 1,     /* bad pointer, size, layer index, bit width ... */
+  PMKVQ_ERR_ARENA_TOO_SMALL = 2, /* arena_bytes < pmkvq_arena_bytes_required()   */
+  PMKVQ_ERR_BUDGET_FULL = 3,     /* append would exceed the block budget and cur_bits > Fbit:
+                                    call pmkvq_progressive_reduce and retry (or set auto_reduce) */
+  PMKVQ_ERR_AT_FBIT = 4,         /* progressive_reduce on a block already at its Fbit */
+  PMKVQ_ERR_CAPACITY = 5,        /* over budget at Fbit, or past max_tokens */
+  PMKVQ_ERR_CUDA = 6,            /* a CUDA runtime call or launch failed */
+  PMKVQ_ERR_STATE = 7            /* internal invariant violated */
+} pmkvq_status;
+
+typedef struct {
+  int32_t layers;       /* number of transformer blocks */
+  int32_t q_heads;      /* query heads; q_heads / kv_heads (the GQA group) must be 1..8 */
+  int32_t kv_heads;
+  int32_t head_dim;     /* must be 128 */
+  int32_t batch;
+  int32_t max_tokens;   /* maximum context length the budget is derived from (Sec. 3.1) */
+  const uint8_t *fbit;           /* HOST [layers], each in {2,4,8,16}: per-block bit schedule (Sec. 3.2) */
+  const uint64_t *budget_bytes;  /* HOST [layers], bytes per block for the whole batch (K+V, codes +
+                                    fp32 scale + fp32 zero); NULL => size of max_tokens tokens with the
+                                    body at Fbit (Sec. 3.1) */
+  const float *lambda;           /* HOST [layers][kv_heads][128], > 0 and finite: Eq. 9's Lambda;
+                                    NULL => all ones */
+  int32_t n_sink;         /* leading tokens kept INT16 (Sec. 2.2: the first token); default 1 */
+  int32_t window;         /* most recent tokens kept INT16 (Sec. 4.1.2: 128) */
+  int32_t evict_chunk;    /* tokens leave the window in groups of this many (>= 1) */
+  int32_t count_metadata; /* 1: budget accounting counts scale + zero bytes; 0: code bytes only */
+  int32_t auto_reduce;    /* 1: pmkvq_append reduces by itself when the budget is full */
+  float sm_scale;         /* softmax scale; 0 => 1/sqrt(head_dim) */
+  void *d_arena;          /* DEVICE, 256-byte aligned, caller-owned, must outlive the cache */
+  size_t arena_bytes;
+} pmkvq_config;
+
+/* Bytes of device arena a cache with this configuration needs (d_arena / arena_bytes are
+ * ignored).  Returns 0 for an invalid configuration. */
+size_t pmkvq_arena_bytes_required(const pmkvq_config *cfg);
+
+/* Problem statement of Sec. 3.1 / 3.4: create the (empty) cache of `layers` blocks, each with its
+ * Fbit and budget.  Copies lambda / fbit / budgets; zero-initialises its bookkeeping in the arena
+ * (synchronous).  *out is set only on PMKVQ_OK. */
+pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out);
+void pmkvq_cache_destroy(pmkvq_cache *cache);
+
+/* Quantize-on-append (Eq. 1-2 at 16 bit; Keys multiplied by Lambda^-1 first, Eq. 9) of n_new
+ * tokens, then window eviction: tokens leaving the INT16 window are shifted (Eq. 3, repeatedly)
+ * to the block's current width.
+ *   d_K_bf16, d_V_bf16: DEVICE bf16 [n_new][batch][kv_heads][128], read only.
+ * Returns BUDGET_FULL (state unchanged) if the block must be reduced first and auto_reduce is 0. */
+pmkvq_status pmkvq_append(pmkvq_cache *cache, int32_t layer, const void *d_K_bf16, const void *d_V_bf16,
+                          int32_t n_new, void *stream);
+
+/* One step of the progressive strategy (Sec. 3.1): shift every body token of the block from
+ * 2b to b bits with Eq. 3, S_b = (2^b+1) S_2b, Z unchanged; sink and window tokens stay INT16. */
+pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *cache, int32_t layer, void *stream);
+
+/* Decode-step attention of one block over all cached tokens (the one just appended included):
+ * out = softmax(sm_scale * (Q Lambda) dequant(K Lambda^-1)^T) dequant(V)  (Eq. 9 with GQA).
+ *   d_Q_bf16: DEVICE bf16 [batch][q_heads][128]; d_out: DEVICE fp32 [batch][q_heads][128]. */
+pmkvq_status pmkvq_decode_attention(pmkvq_cache *cache, int32_t layer, const void *d_Q_bf16, float *d_out,
+                                    void *stream);
+
+/* Host-side state of a block; any out pointer may be NULL. */
+pmkvq_status pmkvq_layer_state(const pmkvq_cache *cache, int32_t layer, int32_t *n_tokens, int32_t *cur_bits,
+                               uint64_t *bytes_used, uint64_t *budget_bytes);
+
+/* Algorithmic bytes one pmkvq_decode_attention call on this block moves in its current state:
+ * codes + fp32 scale + fp32 zero of every cached token of K and V, Q in, out, lambda. */
+uint64_t pmkvq_attention_bytes(const pmkvq_cache *cache, int32_t layer);
+
+/* Copy one (batch, kv_head) slice of K (is_value = 0) or V (1) to the host in token order, for
+ * bit-exact comparison.  Synchronises the device.  Any of the outputs may be NULL.
+ *   h_codes  [n_tokens][128] uint16, each < 2^bits of its token
+ *   h_scale, h_zero [n_tokens] fp32;  h_bits [n_tokens]
+ *   h_packed canonical packed bytes, token after token: token t takes 16*bits_t bytes, element i in
+ *            byte floor(i*bits/8) at bit (i*bits) mod 8 (16-bit codes little-endian). */
+pmkvq_status pmkvq_export_slice(pmkvq_cache *cache, int32_t layer, int32_t batch_idx, int32_t kv_head,
+                                int32_t is_value, uint16_t *h_codes, float *h_scale, float *h_zero,
+                                uint8_t *h_bits, uint8_t *h_packed);
+
+const char *pmkvq_status_string(pmkvq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PMKVQ_H_ */
