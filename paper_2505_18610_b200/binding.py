@@ -1,0 +1,199 @@
+"""Thin ctypes binding of the C ABI in ``include/pmkvq.h`` (same call names, argument
+marshalling only).  PyTorch supplies device memory (the arena, inputs, outputs) and the stream;
+every step of the path runs inside ``libpmkvq.so``.  There is no fallback: if the library is
+missing it is built with nvcc, and if that fails the import raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libpmkvq.so")
+
+STATUS_NAMES = ["OK", "INVALID_ARG", "ARENA_TOO_SMALL", "BUDGET_FULL", "AT_FBIT", "CAPACITY", "CUDA", "STATE"]
+OK, INVALID_ARG, ARENA_TOO_SMALL, BUDGET_FULL, AT_FBIT, CAPACITY, CUDA_ERROR, STATE = range(8)
+
+
+class PmkvqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: {STATUS_NAMES[status] if 0 <= status < 8 else status}")
+        self.status = status
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [
+        ("layers", ctypes.c_int32), ("q_heads", ctypes.c_int32), ("kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("batch", ctypes.c_int32), ("max_tokens", ctypes.c_int32),
+        ("fbit", ctypes.POINTER(ctypes.c_uint8)), ("budget_bytes", ctypes.POINTER(ctypes.c_uint64)),
+        ("lam", ctypes.POINTER(ctypes.c_float)),
+        ("n_sink", ctypes.c_int32), ("window", ctypes.c_int32), ("evict_chunk", ctypes.c_int32),
+        ("count_metadata", ctypes.c_int32), ("auto_reduce", ctypes.c_int32), ("sm_scale", ctypes.c_float),
+        ("d_arena", ctypes.c_void_p), ("arena_bytes", ctypes.c_size_t),
+    ]
+
+
+def load_library() -> ctypes.CDLL:
+    if _build.needs_build():
+        _build.build()
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, u64p, i32p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_int32)
+    lib.pmkvq_arena_bytes_required.restype = ctypes.c_size_t
+    lib.pmkvq_arena_bytes_required.argtypes = [ctypes.POINTER(_Config)]
+    lib.pmkvq_cache_create.restype = i32
+    lib.pmkvq_cache_create.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(vp)]
+    lib.pmkvq_cache_destroy.restype = None
+    lib.pmkvq_cache_destroy.argtypes = [vp]
+    lib.pmkvq_append.restype = i32
+    lib.pmkvq_append.argtypes = [vp, i32, vp, vp, i32, vp]
+    lib.pmkvq_progressive_reduce.restype = i32
+    lib.pmkvq_progressive_reduce.argtypes = [vp, i32, vp]
+    lib.pmkvq_decode_attention.restype = i32
+    lib.pmkvq_decode_attention.argtypes = [vp, i32, vp, vp, vp]
+    lib.pmkvq_set_attention_splits.restype = i32
+    lib.pmkvq_set_attention_splits.argtypes = [vp, i32]
+    lib.pmkvq_layer_state.restype = i32
+    lib.pmkvq_layer_state.argtypes = [vp, i32, i32p, i32p, u64p, u64p]
+    lib.pmkvq_attention_bytes.restype = ctypes.c_uint64
+    lib.pmkvq_attention_bytes.argtypes = [vp, i32]
+    lib.pmkvq_export_slice.restype = i32
+    lib.pmkvq_export_slice.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.pmkvq_status_string.restype = ctypes.c_char_p
+    lib.pmkvq_status_string.argtypes = [i32]
+    return lib
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = load_library()
+    return _lib
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+class Cache:
+    """A PM-KVQ cache of ``layers`` transformer blocks living in one torch-owned device arena."""
+
+    def __init__(self, layers: int, q_heads: int, kv_heads: int, batch: int, max_tokens: int,
+                 fbit: Sequence[int], budget_bytes: Optional[Sequence[int]] = None,
+                 lam: Optional[np.ndarray] = None, n_sink: int = 1, window: int = 128, evict_chunk: int = 1,
+                 count_metadata: bool = True, auto_reduce: bool = True, sm_scale: float = 0.0,
+                 device: str = "cuda:0"):
+        self._h = None
+        self.layers, self.q_heads, self.kv_heads, self.batch = layers, q_heads, kv_heads, batch
+        self._fbit = (ctypes.c_uint8 * layers)(*[int(b) for b in fbit])
+        self._budget = None if budget_bytes is None else (ctypes.c_uint64 * layers)(*[int(b) for b in budget_bytes])
+        self._lam = None
+        if lam is not None:
+            self._lam = np.ascontiguousarray(lam, dtype=np.float32).reshape(layers, kv_heads, 128)
+        cfg = _Config()
+        cfg.layers, cfg.q_heads, cfg.kv_heads, cfg.head_dim = layers, q_heads, kv_heads, 128
+        cfg.batch, cfg.max_tokens = batch, max_tokens
+        cfg.fbit = ctypes.cast(self._fbit, ctypes.POINTER(ctypes.c_uint8))
+        cfg.budget_bytes = None if self._budget is None else ctypes.cast(self._budget, ctypes.POINTER(ctypes.c_uint64))
+        cfg.lam = None if self._lam is None else self._lam.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+        cfg.n_sink, cfg.window, cfg.evict_chunk = n_sink, window, evict_chunk
+        cfg.count_metadata, cfg.auto_reduce, cfg.sm_scale = int(count_metadata), int(auto_reduce), float(sm_scale)
+        need = lib().pmkvq_arena_bytes_required(ctypes.byref(cfg))
+        if need == 0:
+            raise PmkvqError(INVALID_ARG, "pmkvq_arena_bytes_required")
+        self.arena_bytes = need
+        self.device = torch.device(device)
+        with torch.cuda.device(self.device):
+            self.arena = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+            base = self.arena.data_ptr()
+            cfg.d_arena = (base + 255) // 256 * 256
+            cfg.arena_bytes = need
+            h = ctypes.c_void_p()
+            st = lib().pmkvq_cache_create(ctypes.byref(cfg), ctypes.byref(h))
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_cache_create")
+        self._h = h
+
+    def close(self):
+        if self._h is not None:
+            lib().pmkvq_cache_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @staticmethod
+    def _check(t: torch.Tensor, dtype, what):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+            raise ValueError(f"{what} must be a contiguous CUDA tensor of {dtype}")
+
+    def append(self, layer: int, k: torch.Tensor, v: torch.Tensor, stream=None, check: bool = True) -> int:
+        """k, v: bf16 [n_new, batch, kv_heads, 128] (or [batch, kv_heads, 128] for one token)."""
+        self._check(k, torch.bfloat16, "k"); self._check(v, torch.bfloat16, "v")
+        n_new = 1 if k.dim() == 3 else k.shape[0]
+        if k.numel() != n_new * self.batch * self.kv_heads * 128 or v.numel() != k.numel():
+            raise ValueError("bad K/V shape")
+        st = lib().pmkvq_append(self._h, layer, k.data_ptr(), v.data_ptr(), n_new, _stream_ptr(stream))
+        if check and st != OK:
+            raise PmkvqError(st, "pmkvq_append")
+        return st
+
+    def progressive_reduce(self, layer: int, stream=None, check: bool = True) -> int:
+        st = lib().pmkvq_progressive_reduce(self._h, layer, _stream_ptr(stream))
+        if check and st != OK:
+            raise PmkvqError(st, "pmkvq_progressive_reduce")
+        return st
+
+    def decode_attention(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None):
+        """q: bf16 [batch, q_heads, 128] -> fp32 [batch, q_heads, 128]."""
+        self._check(q, torch.bfloat16, "q")
+        if q.numel() != self.batch * self.q_heads * 128:
+            raise ValueError("bad Q shape")
+        if out is None:
+            out = torch.empty(self.batch, self.q_heads, 128, dtype=torch.float32, device=q.device)
+        self._check(out, torch.float32, "out")
+        st = lib().pmkvq_decode_attention(self._h, layer, q.data_ptr(), out.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_decode_attention")
+        return out
+
+    def set_attention_splits(self, splits: int):
+        st = lib().pmkvq_set_attention_splits(self._h, splits)
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_set_attention_splits")
+
+    def layer_state(self, layer: int):
+        n, b = ctypes.c_int32(), ctypes.c_int32()
+        used, budget = ctypes.c_uint64(), ctypes.c_uint64()
+        st = lib().pmkvq_layer_state(self._h, layer, ctypes.byref(n), ctypes.byref(b), ctypes.byref(used), ctypes.byref(budget))
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_layer_state")
+        return {"n_tokens": n.value, "cur_bits": b.value, "bytes_used": used.value, "budget_bytes": budget.value}
+
+    def attention_bytes(self, layer: int) -> int:
+        return int(lib().pmkvq_attention_bytes(self._h, layer))
+
+    def export_slice(self, layer: int, batch_idx: int, kv_head: int, is_value: bool, packed: bool = False):
+        n = self.layer_state(layer)["n_tokens"]
+        codes = np.zeros((n, 128), np.uint16)
+        scale, zero, bits = np.zeros(n, np.float32), np.zeros(n, np.float32), np.zeros(n, np.uint8)
+        pk = np.zeros(n * 256, np.uint8) if packed else None
+        st = lib().pmkvq_export_slice(self._h, layer, batch_idx, kv_head, int(is_value), codes.ctypes.data,
+                                      scale.ctypes.data, zero.ctypes.data, bits.ctypes.data,
+                                      None if pk is None else pk.ctypes.data)
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_export_slice")
+        if packed:
+            return codes, scale, zero, bits, pk[: int(bits.astype(np.int64).sum()) * 16]
+        return codes, scale, zero, bits

@@ -1,0 +1,279 @@
+// Cache-maintenance kernels: quantize-on-append (Eq. 1-2 at 16 bit, Keys equalized per Eq. 9),
+// window eviction and the progressive reduce (Eq. 3).  All integer / IEEE-fp32 work is written
+// with explicit round-to-nearest intrinsics so that codes, scales and zero-points have exactly
+// one bit pattern.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "layout.cuh"
+
+namespace pmkvq {
+
+// Where one block's slices live inside the arena.
+struct LayerGeom {
+  uint8_t *base;        // first slice of this block
+  size_t slice_stride;  // bytes between (batch, kv_head) slices
+  size_t ring_off;      // byte offset of the INT16 window ring inside a slice
+  size_t body_off;      // byte offset of the body inside a slice
+  int n_sink;           // leading INT16 tokens (stored in tiles at offset 0)
+  int ring_tokens;      // ring capacity in tokens (multiple of 16)
+};
+
+struct TokenDest {
+  uint8_t *tile;
+  int row;
+  int bits;
+};
+
+// Tile, row and width of absolute token t, given the first window token `win_start`
+// (= n_sink + n_body) and the body width.
+__device__ __forceinline__ TokenDest token_dest(const LayerGeom &g, uint8_t *slice, int t, int win_start,
+                                                int cur_bits) {
+  TokenDest d;
+  if (t < g.n_sink) {
+    d.tile = slice + (size_t)(t >> 4) * tile_bytes(16);
+    d.row = t & 15;
+    d.bits = 16;
+  } else if (t < win_start) {
+    const int j = t - g.n_sink;
+    d.tile = slice + g.body_off + (size_t)(j >> 4) * tile_bytes(cur_bits);
+    d.row = j & 15;
+    d.bits = cur_bits;
+  } else {
+    const int rp = (t - g.n_sink) % g.ring_tokens;
+    d.tile = slice + g.ring_off + (size_t)(rp >> 4) * tile_bytes(16);
+    d.row = rp & 15;
+    d.bits = 16;
+  }
+  return d;
+}
+
+// Scale after the chain 16 -> ... -> bits: S_b = (2^b + 1) S_2b, one fp32 rounding per step (Sec. 3.1).
+__device__ __forceinline__ float chain_scale(float s16, int bits) {
+  float s = s16;
+  for (int w = 8; w >= bits; w >>= 1) s = __fmul_rn(s, (float)((1 << w) + 1));
+  return s;
+}
+
+// Write one token's 128 codes (given as INT16 codes in shared memory) into a tile at `bits`,
+// applying the Eq. 3 chain; one warp, every half-word of the token is written by one lane.
+__device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, const uint16_t *codes16, int is_value,
+                                            int lane) {
+  const int n = 16 / bits;
+  const int r = row >> 3;
+  for (int hw = lane; hw < 8 * bits; hw += 32) {
+    const int w = hw >> 3, sub = hw & 7;
+    int owner, h, chan0, chan_step = 8;
+    if (is_value) {  // sub = g ; channels 8*J + g
+      h = row & 1;
+      owner = sub * 4 + ((row & 7) >> 1);
+      chan0 = sub;
+    } else {  // sub = tig + 4*h ; channels 8*W + 2*tig + h
+      const int tig = sub & 3;
+      h = sub >> 2;
+      owner = (row & 7) * 4 + tig;
+      chan0 = 2 * tig + h;
+    }
+    uint32_t val = 0;
+    for (int j = 0; j < n; ++j) {
+      const int ch = chan_step * (w * n + j) + chan0;
+      val |= shift_chain(codes16[ch], bits) << (j * bits);
+    }
+    int byte_off, bit_off;
+    lane_slot(bits, owner, r, w * n, h, byte_off, bit_off);
+    *reinterpret_cast<uint16_t *>(part + byte_off) = (uint16_t)val;
+  }
+}
+
+// Read one token's INT16 codes from a 16-bit tile into shared memory; one warp.
+__device__ __forceinline__ void load_token16(const uint8_t *part, int row, uint16_t *codes16, int is_value, int lane) {
+  for (int ch = lane; ch < kHeadDim; ch += 32) {
+    int byte_off, bit_off;
+    if (is_value) v_slot(16, row, ch, byte_off, bit_off);
+    else k_slot(16, row, ch, byte_off, bit_off);
+    codes16[ch] = *reinterpret_cast<const uint16_t *>(part + byte_off);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Quantize-on-append.  One warp per (new token, slice, K|V).  Eq. 1-2 with b = 16 on the 128
+// channels of the token; Keys are first multiplied by Lambda^-1 (Eq. 9).  The token goes to the
+// sink, straight to the body (bulk appends; Eq. 3 chain to the body width) or to the window ring.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
+                                                     const float *__restrict__ inv_lambda, unsigned *vmax_bits,
+                                                     LayerGeom geom, int n_new, int n_slices, int kv_heads,
+                                                     int n_old, int win_start, int cur_bits) {
+  __shared__ uint16_t s_codes[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wid = (long long)blockIdx.x * 4 + warp;
+  const long long total = (long long)n_new * n_slices * 2;
+  if (wid >= total) return;
+  const int is_value = (int)(wid & 1);
+  const long long ts = wid >> 1;
+  const int slice = (int)(ts % n_slices);
+  const int i = (int)(ts / n_slices);
+  const uint16_t *src = (is_value ? V : K) + ((size_t)i * n_slices + slice) * kHeadDim + lane * 4;
+  const uint2 raw = *reinterpret_cast<const uint2 *>(src);
+  float x[4];
+  x[0] = __uint_as_float(raw.x << 16);
+  x[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+  x[2] = __uint_as_float(raw.y << 16);
+  x[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+  if (!is_value) {
+    const float4 il = *reinterpret_cast<const float4 *>(inv_lambda + (size_t)(slice % kv_heads) * kHeadDim + lane * 4);
+    x[0] = __fmul_rn(x[0], il.x);
+    x[1] = __fmul_rn(x[1], il.y);
+    x[2] = __fmul_rn(x[2], il.z);
+    x[3] = __fmul_rn(x[3], il.w);
+  }
+  float mn = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
+  float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  const float scale = __fdiv_rn(__fsub_rn(mx, mn), 65535.0f);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    int c = 0;
+    if (scale != 0.0f) {
+      c = __float2int_rn(__fdiv_rn(__fsub_rn(x[e], mn), scale));
+      c = min(max(c, 0), 65535);
+    }
+    s_codes[warp][lane * 4 + e] = (uint16_t)c;
+  }
+  __syncwarp();
+  uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
+  const TokenDest d = token_dest(geom, slice_base, n_old + i, win_start, cur_bits);
+  store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, s_codes[warp], is_value, lane);
+  if (lane == 0) {
+    float *meta = reinterpret_cast<float *>(d.tile + meta_offset(d.bits));
+    meta[meta_slot(is_value ? 2 : 0, d.row) >> 2] = chain_scale(scale, d.bits);
+    meta[meta_slot(is_value ? 3 : 1, d.row) >> 2] = mn;
+    if (is_value) atomicMax(vmax_bits + slice, __float_as_uint(scale));  // scale >= 0: uint order = float order
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Window eviction.  One warp per (evicted token, slice, K|V): the INT16 token leaves the ring and
+// enters the body at the body width through the Eq. 3 chain (16 -> 8 -> ... -> cur_bits).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) evict_kernel(LayerGeom geom, int n_slices, int first_token, int n_evict,
+                                                    int cur_bits) {
+  __shared__ uint16_t s_codes[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wid = (long long)blockIdx.x * 4 + warp;
+  const long long total = (long long)n_evict * n_slices * 2;
+  if (wid >= total) return;
+  const int is_value = (int)(wid & 1);
+  const long long ts = wid >> 1;
+  const int slice = (int)(ts % n_slices);
+  const int t = first_token + (int)(ts / n_slices);
+  uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
+  const int rp = (t - geom.n_sink) % geom.ring_tokens;
+  const uint8_t *src_tile = slice_base + geom.ring_off + (size_t)(rp >> 4) * tile_bytes(16);
+  const int src_row = rp & 15;
+  load_token16(src_tile + (is_value ? v_part_offset(16) : 0), src_row, s_codes[warp], is_value, lane);
+  const float *smeta = reinterpret_cast<const float *>(src_tile + meta_offset(16));
+  const float s16 = smeta[meta_slot(is_value ? 2 : 0, src_row) >> 2];
+  const float z = smeta[meta_slot(is_value ? 3 : 1, src_row) >> 2];
+  __syncwarp();
+  const int j = t - geom.n_sink;
+  uint8_t *dst_tile = slice_base + geom.body_off + (size_t)(j >> 4) * tile_bytes(cur_bits);
+  store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, s_codes[warp], is_value, lane);
+  if (lane == 0) {
+    float *meta = reinterpret_cast<float *>(dst_tile + meta_offset(cur_bits));
+    meta[meta_slot(is_value ? 2 : 0, j & 15) >> 2] = chain_scale(s16, cur_bits);
+    meta[meta_slot(is_value ? 3 : 1, j & 15) >> 2] = z;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Progressive reduce 2B -> B (Eq. 3) of one tile, by one warp.  Lane-local: two adjacent words of
+// a lane at 2B bits become one word at B bits.  Everything is read and transformed before the
+// first store, so the output may overlap this tile's own input.
+// ---------------------------------------------------------------------------------------------
+template <int B>
+__device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1) {
+  constexpr int NIN = 8 / B;  // codes per half-word at 2B bits
+  constexpr uint32_t MASK = (1u << (2 * B)) - 1u;
+  uint32_t out = 0;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int j = 0; j < NIN; ++j) {
+      const uint32_t c0 = (in0 >> (16 * h + j * 2 * B)) & MASK;
+      const uint32_t c1 = (in1 >> (16 * h + j * 2 * B)) & MASK;
+      out |= shift_step(c0, B) << (16 * h + j * B);
+      out |= shift_step(c1, B) << (16 * h + (NIN + j) * B);
+    }
+  }
+  return out;
+}
+
+template <int B>
+__device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int lane) {
+  constexpr int IN_CHUNKS = B;                          // 16-byte chunks per lane per part at 2B bits
+  constexpr int OUT_WORDS = 2 * B;                      // words per lane per part at B bits
+  constexpr int OUT_CHUNKS = (OUT_WORDS + 3) / 4;
+  uint32_t o[2][OUT_CHUNKS * 4];
+#pragma unroll
+  for (int part = 0; part < 2; ++part) {
+    const uint8_t *src = in + part * code_part_bytes(2 * B);
+    uint32_t w[IN_CHUNKS * 4];
+#pragma unroll
+    for (int q = 0; q < IN_CHUNKS; ++q) {
+      const uint4 v = *reinterpret_cast<const uint4 *>(src + (q * 32 + lane) * 16);
+      w[4 * q + 0] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+    }
+    // out lane-word r*B + w'  <-  in lane-words r*2B + 2w', r*2B + 2w' + 1
+#pragma unroll
+    for (int lw = 0; lw < OUT_WORDS; ++lw) {
+      const int r = lw / B, wp = lw % B;
+      o[part][lw] = merge_words<B>(w[r * 2 * B + 2 * wp], w[r * 2 * B + 2 * wp + 1]);
+    }
+  }
+  float2 m = *reinterpret_cast<const float2 *>(in + meta_offset(2 * B) + lane * 8);
+  const int kind = ((2 * lane) & 15) >> 2;  // 0 S_K, 1 Z_K, 2 S_V, 3 Z_V
+  if ((kind & 1) == 0) {
+    m.x = __fmul_rn(m.x, (float)((1 << B) + 1));
+    m.y = __fmul_rn(m.y, (float)((1 << B) + 1));
+  }
+  __syncwarp();  // every lane holds its transformed data: the tile's input is dead from here on
+#pragma unroll
+  for (int part = 0; part < 2; ++part) {
+    uint8_t *dst = out + part * code_part_bytes(B);
+#pragma unroll
+    for (int q = 0; q < OUT_CHUNKS; ++q) {
+      *reinterpret_cast<uint4 *>(dst + (q * 32 + lane) * 16) =
+          make_uint4(o[part][4 * q], o[part][4 * q + 1], o[part][4 * q + 2], o[part][4 * q + 3]);
+    }
+  }
+  *reinterpret_cast<float2 *>(out + meta_offset(B) + lane * 8) = m;
+}
+
+// First tiles of every slice, one warp per slice, in order (tile i's output overlaps inputs <= i only).
+template <int B>
+__global__ void __launch_bounds__(32) reduce_head_kernel(LayerGeom geom, int n_tiles) {
+  uint8_t *body = geom.base + (size_t)blockIdx.x * geom.slice_stride + geom.body_off;
+  const int lane = threadIdx.x;
+  for (int i = 0; i < n_tiles; ++i) {
+    reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), lane);
+    __syncwarp();
+  }
+}
+
+// One wave: tiles [lo, hi) of every slice, one warp per tile.  The host picks the waves so that
+// hi * tile_bytes(B) <= lo * tile_bytes(2B): no output of the wave lands on an input of the wave.
+template <int B>
+__global__ void __launch_bounds__(128) reduce_wave_kernel(LayerGeom geom, int lo, int hi) {
+  const int i = lo + blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (i >= hi) return;
+  uint8_t *body = geom.base + (size_t)blockIdx.y * geom.slice_stride + geom.body_off;
+  reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), threadIdx.x & 31);
+}
+
+}  // namespace pmkvq

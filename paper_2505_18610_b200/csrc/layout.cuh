@@ -1,0 +1,90 @@
+// Tile layout of the packed KV cache in HBM.
+//
+// A tile holds 16 consecutive tokens of one (batch, kv_head) slice, K and V together:
+//
+//   [ K codes : 256*b bytes ][ V codes : 256*b bytes ][ metadata : 256 bytes ]      b = bit width
+//
+// so tile_bytes(b) = 512*b + 256 = 16 tokens * 2 * (16*b code bytes + 4 scale + 4 zero): the bytes
+// the budget accounting of the progressive policy (Sec. 3.1) charges, nothing more.
+//
+// Codes are stored "lane-owned": the 32 lanes of a warp own 16-byte chunks, chunk q of lane l at
+// byte (q*32 + l)*16, so a warp reads a tile with fully coalesced 128-bit loads and every lane gets
+// exactly the codes its tensor-core fragments need, with no shuffle.  With lane = 4*g + tig:
+//
+//   K part: lane (g,tig) owns tokens {g, g+8} and channels {8*W + 2*tig + h : W=0..15, h=0,1}.
+//           The two 16-bit halves of a 32-bit word are two channels (h) of ONE token: exactly the
+//           k-pair of an m16n8k16 B fragment for S = Q K^T (k = channel, n = token).
+//   V part: lane (g,tig) owns tokens {2*tig + 8*r + h : r=0,1, h=0,1} and channels {8*J + g : J=0..15}.
+//           The two halves of a word are two consecutive tokens (h) of ONE channel: the k-pair of an
+//           m16n8k16 A fragment for O^T = V^T P^T (m = channel, k = token).
+//
+// In both parts a 16-bit half-word holds n = 16/b codes of one token: index W (or J) = w*n + j sits
+// in lane-word lw = r*b + w, at bits [j*b, j*b + b) of half h.  Going from 2b to b bits therefore
+// merges two adjacent words of a lane into one (Eq. 3 applied per field): the reduce is lane-local.
+//
+// Metadata: for tig = 0..3 a 64-byte record {S_K[4], Z_K[4], S_V[4], Z_V[4]} of the four tokens
+// {2tig, 2tig+1, 8+2tig, 9+2tig} a lane needs for its score / probability fragments.
+#pragma once
+#include <cstdint>
+
+#if defined(__CUDACC__)
+#define PMKVQ_HD __host__ __device__ __forceinline__
+#else
+#define PMKVQ_HD inline
+#endif
+
+namespace pmkvq {
+
+constexpr int kHeadDim = 128;
+constexpr int kTileTokens = 16;
+
+PMKVQ_HD constexpr int code_part_bytes(int bits) { return 256 * bits; }
+PMKVQ_HD constexpr int tile_bytes(int bits) { return 512 * bits + 256; }
+PMKVQ_HD constexpr int v_part_offset(int bits) { return 256 * bits; }
+PMKVQ_HD constexpr int meta_offset(int bits) { return 512 * bits; }
+
+// Byte offset (inside the K or V part) of the half-word that holds lane-element (lane, r, idx, h)
+// and the bit position of the code inside that half-word.  idx is W (K part) or J (V part).
+PMKVQ_HD void lane_slot(int bits, int lane, int r, int idx, int h, int &byte_off, int &bit_off) {
+  const int n = 16 / bits;
+  const int w = idx / n, j = idx % n;
+  const int lw = r * bits + w;
+  byte_off = ((lw >> 2) * 32 + lane) * 16 + (lw & 3) * 4 + h * 2;
+  bit_off = j * bits;
+}
+
+// K code of (token row 0..15, channel 0..127)
+PMKVQ_HD void k_slot(int bits, int row, int ch, int &byte_off, int &bit_off) {
+  const int g = row & 7, r = row >> 3;
+  const int W = ch >> 3, tig = (ch & 7) >> 1, h = ch & 1;
+  lane_slot(bits, g * 4 + tig, r, W, h, byte_off, bit_off);
+}
+
+// V code of (token row 0..15, channel 0..127)
+PMKVQ_HD void v_slot(int bits, int row, int ch, int &byte_off, int &bit_off) {
+  const int h = row & 1, tig = (row & 7) >> 1, r = row >> 3;
+  const int g = ch & 7, J = ch >> 3;
+  lane_slot(bits, g * 4 + tig, r, J, h, byte_off, bit_off);
+}
+
+// Byte offset inside the metadata block of kind (0 S_K, 1 Z_K, 2 S_V, 3 Z_V) of token row.
+PMKVQ_HD int meta_slot(int kind, int row) {
+  const int tig = (row & 7) >> 1;
+  const int i = (row >> 3) * 2 + (row & 1);
+  return tig * 64 + kind * 16 + i * 4;
+}
+
+// Eq. 3, one step 2b -> b on one code.  The product needs the full 32 unsigned bits at b = 8.
+PMKVQ_HD uint32_t shift_step(uint32_t c, int b) {
+  const uint32_t mult = (1u << (2 * b)) - (1u << b) + 1u;
+  return (mult * (c + (1u << (b - 1)))) >> (3 * b);
+}
+
+// 16-bit code -> `bits`-bit code through the chain 16 -> 8 -> 4 -> 2.
+PMKVQ_HD uint32_t shift_chain(uint32_t c16, int bits) {
+  uint32_t c = c16;
+  for (int w = 8; w >= bits; w >>= 1) c = shift_step(c, w);
+  return c;
+}
+
+}  // namespace pmkvq

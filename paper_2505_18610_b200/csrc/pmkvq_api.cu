@@ -1,0 +1,414 @@
+// C ABI of the PM-KVQ decode hot path: host-side cache state machine (progressive policy of
+// Sec. 3.1), arena layout, kernel launches, and the slice export used for bit-exact comparison.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/pmkvq.h"
+#include "kernels_attn.cuh"
+#include "kernels_cache.cuh"
+#include "layout.cuh"
+
+using namespace pmkvq;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kHeadTiles = 8;     // tiles the reduce handles in order before the parallel waves start
+constexpr int kTargetCtas = 1184;  // 148 SMs x 4 resident CTAs of 128 threads x 2 waves
+constexpr int kMaxSplits = 64;      // upper bound on body CTAs per slice (sizes the partials workspace)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool valid_bits(int b) { return b == 2 || b == 4 || b == 8 || b == 16; }
+
+struct Layer {
+  int fbit = 16;
+  int cur_bits = 16;
+  int n_tokens = 0;
+  uint64_t budget = 0;
+  size_t offset = 0;        // of the first slice inside the arena
+  size_t slice_stride = 0;
+  size_t body_cap = 0;      // bytes of body per slice
+};
+
+}  // namespace
+
+struct pmkvq_cache {
+  int layers, q_heads, kv_heads, batch, max_tokens, group, n_slices;
+  int n_sink, window, evict_chunk, count_metadata, auto_reduce;
+  float sm_scale;
+  uint8_t *arena;
+  size_t arena_bytes;
+  // arena sections
+  size_t off_lambda, off_inv_lambda, off_vmax, off_partials, partial_bytes;
+  int sink_tiles, ring_tiles, max_splits, auto_splits, user_splits;
+  std::vector<Layer> L;
+
+  // ---- policy arithmetic (Sec. 3.1) ----
+  int tokbytes(int bits) const { return 16 * bits + (count_metadata ? 8 : 0); }
+  int sink_at(int n) const { return std::min(n, n_sink); }
+  int body_at(int n) const {
+    const int excess = n - n_sink - window;
+    return excess <= 0 ? 0 : excess / evict_chunk * evict_chunk;
+  }
+  uint64_t bytes_at(int n, int bits) const {
+    const uint64_t nb = body_at(n), n16 = n - nb;
+    return 2ull * n_slices * (n16 * tokbytes(16) + nb * tokbytes(bits));
+  }
+  uint64_t default_budget(int fbit) const {
+    uint64_t best = 0;
+    for (int n = std::max(0, max_tokens - evict_chunk + 1); n <= max_tokens; ++n) best = std::max(best, bytes_at(n, fbit));
+    return best;
+  }
+  LayerGeom geom(const Layer &l) const {
+    LayerGeom g;
+    g.base = arena + l.offset;
+    g.slice_stride = l.slice_stride;
+    g.ring_off = (size_t)sink_tiles * tile_bytes(16);
+    g.body_off = g.ring_off + (size_t)ring_tiles * tile_bytes(16);
+    g.n_sink = n_sink;
+    g.ring_tokens = ring_tiles * 16;
+    return g;
+  }
+};
+
+namespace {
+
+bool check_config(const pmkvq_config *c) {
+  if (!c) return false;
+  if (c->layers <= 0 || c->q_heads <= 0 || c->kv_heads <= 0 || c->batch <= 0 || c->max_tokens <= 0) return false;
+  if (c->head_dim != kHeadDim) return false;
+  if (c->q_heads % c->kv_heads) return false;
+  const int g = c->q_heads / c->kv_heads;
+  if (g < 1 || g > kMaxGroup) return false;
+  if (!c->fbit) return false;
+  for (int i = 0; i < c->layers; ++i)
+    if (!valid_bits(c->fbit[i])) return false;
+  if (c->n_sink < 0 || c->window < 0 || c->evict_chunk < 1) return false;
+  if ((int64_t)c->n_sink + c->window + c->evict_chunk > (1 << 24)) return false;
+  if ((int64_t)c->batch * c->kv_heads > 65535) return false;
+  if (c->lambda) {
+    const size_t n = (size_t)c->layers * c->kv_heads * kHeadDim;
+    for (size_t i = 0; i < n; ++i)
+      if (!(c->lambda[i] > 0.0f) || !std::isfinite(c->lambda[i])) return false;
+  }
+  if (!(c->sm_scale >= 0.0f) || !std::isfinite(c->sm_scale)) return false;
+  return true;
+}
+
+// Fills everything of the handle that depends only on the configuration; returns the arena size.
+size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
+  k.layers = c->layers; k.q_heads = c->q_heads; k.kv_heads = c->kv_heads; k.batch = c->batch;
+  k.max_tokens = c->max_tokens; k.group = c->q_heads / c->kv_heads; k.n_slices = c->batch * c->kv_heads;
+  k.n_sink = c->n_sink; k.window = c->window; k.evict_chunk = c->evict_chunk;
+  k.count_metadata = c->count_metadata ? 1 : 0; k.auto_reduce = c->auto_reduce ? 1 : 0;
+  k.sm_scale = c->sm_scale > 0.0f ? c->sm_scale : 1.0f / std::sqrt((float)kHeadDim);
+  k.sink_tiles = (k.n_sink + 15) / 16;
+  k.ring_tiles = std::max(1, (k.window + k.evict_chunk - 1 + 15) / 16 + 1);
+  k.max_splits = kMaxSplits;
+  k.auto_splits = std::min(kMaxSplits, std::max(1, (kTargetCtas + k.n_slices - 1) / k.n_slices));
+  k.user_splits = 0;
+
+  size_t off = 0;
+  const size_t lam_bytes = (size_t)k.layers * k.kv_heads * kHeadDim * sizeof(float);
+  k.off_lambda = off; off = align_up(off + lam_bytes, kAlign);
+  k.off_inv_lambda = off; off = align_up(off + lam_bytes, kAlign);
+  k.off_vmax = off; off = align_up(off + (size_t)k.layers * k.n_slices * sizeof(unsigned), kAlign);
+  k.partial_bytes = (size_t)k.n_slices * (1 + k.max_splits) * kMaxGroup * kPartialStride * sizeof(float);
+  k.off_partials = off; off = align_up(off + k.partial_bytes, kAlign);
+
+  k.L.assign(k.layers, Layer());
+  for (int i = 0; i < k.layers; ++i) {
+    Layer &l = k.L[i];
+    l.fbit = c->fbit[i];
+    l.budget = c->budget_bytes ? c->budget_bytes[i] : k.default_budget(l.fbit);
+    // body capacity: the most tiles the policy can ever ask for at any width of the chain
+    size_t cap = 0;
+    for (int b = 16; b >= l.fbit; b >>= 1) {
+      int lo = 0, hi = k.max_tokens;  // largest n with bytes_at(n, b) <= budget (bytes_at is monotone enough
+      while (lo < hi) {               // for a bisection on the chunk-aligned body count below)
+        const int mid = (lo + hi + 1) / 2;
+        // the worst window phase for a given body count is right before the next chunk leaves
+        if (k.bytes_at(mid, b) <= l.budget) lo = mid; else hi = mid - 1;
+      }
+      int nb = 0;
+      for (int n = std::max(0, lo - 2 * k.evict_chunk); n <= std::min(k.max_tokens, lo + 2 * k.evict_chunk); ++n)
+        if (k.bytes_at(n, b) <= l.budget) nb = std::max(nb, k.body_at(n));
+      cap = std::max(cap, (size_t)((nb + 15) / 16) * tile_bytes(b));
+    }
+    l.body_cap = cap;
+    l.slice_stride = align_up((size_t)(k.sink_tiles + k.ring_tiles) * tile_bytes(16) + cap, kAlign);
+    l.offset = off;
+    off = align_up(off + l.slice_stride * k.n_slices, kAlign);
+  }
+  return off;
+}
+
+template <int B>
+cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStream_t st) {
+  const int head = std::min(n_tiles, kHeadTiles);
+  if (head > 0) reduce_head_kernel<B><<<n_slices, 32, 0, st>>>(g, head);
+  int lo = head;
+  while (lo < n_tiles) {
+    // outputs of tiles [lo, hi) end at hi * tile_bytes(B); inputs start at lo * tile_bytes(2B)
+    long long hi = (long long)lo * tile_bytes(2 * B) / tile_bytes(B);
+    hi = std::min<long long>(hi, n_tiles);
+    if (hi <= lo) return cudaErrorUnknown;
+    dim3 grid((unsigned)((hi - lo + 3) / 4), (unsigned)n_slices);
+    reduce_wave_kernel<B><<<grid, 128, 0, st>>>(g, lo, (int)hi);
+    lo = (int)hi;
+  }
+  return cudaGetLastError();
+}
+
+pmkvq_status do_reduce(pmkvq_cache *k, int layer, cudaStream_t st) {
+  Layer &l = k->L[layer];
+  const int b = l.cur_bits / 2;
+  const int n_body = k->body_at(l.n_tokens);
+  const int n_tiles = (n_body + 15) / 16;
+  const LayerGeom g = k->geom(l);
+  cudaError_t e = cudaSuccess;
+  if (n_tiles > 0) {
+    if (b == 8) e = launch_reduce<8>(g, k->n_slices, n_tiles, st);
+    else if (b == 4) e = launch_reduce<4>(g, k->n_slices, n_tiles, st);
+    else e = launch_reduce<2>(g, k->n_slices, n_tiles, st);
+  }
+  if (e != cudaSuccess) return PMKVQ_ERR_CUDA;
+  l.cur_bits = b;
+  return PMKVQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t pmkvq_arena_bytes_required(const pmkvq_config *cfg) {
+  if (!check_config(cfg)) return 0;
+  pmkvq_cache tmp{};
+  return plan(tmp, cfg);
+}
+
+pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
+  if (!out || !check_config(cfg) || !cfg->d_arena) return PMKVQ_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(cfg->d_arena) % kAlign) return PMKVQ_ERR_INVALID_ARG;
+  pmkvq_cache *k = new (std::nothrow) pmkvq_cache{};
+  if (!k) return PMKVQ_ERR_STATE;
+  const size_t need = plan(*k, cfg);
+  if (cfg->arena_bytes < need) {
+    delete k;
+    return PMKVQ_ERR_ARENA_TOO_SMALL;
+  }
+  k->arena = static_cast<uint8_t *>(cfg->d_arena);
+  k->arena_bytes = cfg->arena_bytes;
+  const size_t n_lam = (size_t)k->layers * k->kv_heads * kHeadDim;
+  std::vector<float> lam(n_lam, 1.0f), inv(n_lam, 1.0f);
+  if (cfg->lambda) {
+    for (size_t i = 0; i < n_lam; ++i) {
+      lam[i] = cfg->lambda[i];
+      inv[i] = 1.0f / cfg->lambda[i];  // one IEEE fp32 division; Keys are multiplied by this (Eq. 9)
+    }
+  }
+  cudaError_t e = cudaMemcpy(k->arena + k->off_lambda, lam.data(), n_lam * sizeof(float), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(k->arena + k->off_inv_lambda, inv.data(), n_lam * sizeof(float), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_vmax, 0, (size_t)k->layers * k->n_slices * sizeof(unsigned));
+  if (e != cudaSuccess) {
+    delete k;
+    return PMKVQ_ERR_CUDA;
+  }
+  *out = k;
+  return PMKVQ_OK;
+}
+
+void pmkvq_cache_destroy(pmkvq_cache *cache) { delete cache; }
+
+pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *k, int32_t layer, void *stream) {
+  if (!k || layer < 0 || layer >= k->layers) return PMKVQ_ERR_INVALID_ARG;
+  if (k->L[layer].cur_bits <= k->L[layer].fbit) return PMKVQ_ERR_AT_FBIT;
+  return do_reduce(k, layer, static_cast<cudaStream_t>(stream));
+}
+
+pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const void *d_V, int32_t n_new,
+                          void *stream) {
+  if (!k || layer < 0 || layer >= k->layers || !d_K || !d_V || n_new <= 0) return PMKVQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_K) | reinterpret_cast<uintptr_t>(d_V)) & 7) return PMKVQ_ERR_INVALID_ARG;
+  Layer &l = k->L[layer];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t n_after64 = (int64_t)l.n_tokens + n_new;
+  if (n_after64 > k->max_tokens) return PMKVQ_ERR_CAPACITY;
+  const int n_after = (int)n_after64;
+  // budget test before anything is mutated (Sec. 3.1: shrink when the budget is fully used)
+  int bits = l.cur_bits, n_reduce = 0;
+  while (k->bytes_at(n_after, bits) > l.budget) {
+    if (bits <= l.fbit) return PMKVQ_ERR_CAPACITY;
+    bits >>= 1;
+    ++n_reduce;
+  }
+  if (n_reduce && !k->auto_reduce) return PMKVQ_ERR_BUDGET_FULL;
+  const int new_body = k->body_at(n_after);
+  if ((size_t)((new_body + 15) / 16) * tile_bytes(bits) > l.body_cap) return PMKVQ_ERR_STATE;
+  for (int i = 0; i < n_reduce; ++i) {
+    const pmkvq_status s = do_reduce(k, layer, st);
+    if (s != PMKVQ_OK) return s;
+  }
+  const LayerGeom g = k->geom(l);
+  const int n_old = l.n_tokens;
+  const int old_win_start = k->sink_at(n_old) + k->body_at(n_old);
+  const int new_win_start = k->sink_at(n_after) + new_body;
+  // tokens already in the ring that now leave the window
+  const int ev_first = std::max(old_win_start, k->n_sink);
+  const int ev_last = std::min(new_win_start, n_old);
+  if (ev_last > ev_first) {
+    const long long warps = 2ll * (ev_last - ev_first) * k->n_slices;
+    evict_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(g, k->n_slices, ev_first, ev_last - ev_first, l.cur_bits);
+  }
+  {
+    const long long warps = 2ll * n_new * k->n_slices;
+    const float *inv_lam = reinterpret_cast<const float *>(k->arena + k->off_inv_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
+    unsigned *vmax = reinterpret_cast<unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
+    append_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(static_cast<const uint16_t *>(d_K),
+                                                              static_cast<const uint16_t *>(d_V), inv_lam, vmax, g, n_new,
+                                                              k->n_slices, k->kv_heads, n_old, new_win_start, l.cur_bits);
+  }
+  if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  l.n_tokens = n_after;
+  return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, void *stream) {
+  if (!k || layer < 0 || layer >= k->layers || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
+  const Layer &l = k->L[layer];
+  if (l.n_tokens <= 0) return PMKVQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  AttnParams p;
+  p.geom = k->geom(l);
+  p.Q = static_cast<const uint16_t *>(d_Q);
+  p.lambda = reinterpret_cast<const float *>(k->arena + k->off_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
+  p.vmax_bits = reinterpret_cast<const unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
+  p.partials = reinterpret_cast<float *>(k->arena + k->off_partials);
+  p.out = d_out;
+  p.kv_heads = k->kv_heads; p.group = k->group; p.q_heads = k->q_heads;
+  p.n_tokens = l.n_tokens;
+  p.n_sink_eff = k->sink_at(l.n_tokens);
+  p.n_body = k->body_at(l.n_tokens);
+  p.win_start = p.n_sink_eff + p.n_body;
+  p.cur_bits = l.cur_bits;
+  p.body_tiles = (p.n_body + 15) / 16;
+  // split the body: every CTA gets at least 8 tiles (2 per warp), at most max_splits CTAs per slice
+  int splits = std::min(k->user_splits > 0 ? k->user_splits : k->auto_splits, (p.body_tiles + 7) / 8);
+  splits = std::max(splits, p.body_tiles > 0 ? 1 : 0);
+  p.tiles_per_split = splits ? (p.body_tiles + splits - 1) / splits : 0;
+  if (splits) splits = (p.body_tiles + p.tiles_per_split - 1) / p.tiles_per_split;
+  p.body_splits = splits;
+  p.qk_scale = k->sm_scale * 1.4426950408889634f;
+  dim3 grid(1 + splits, k->n_slices);
+  switch (l.cur_bits) {
+    case 16: decode_attn_splitk_kernel<16><<<grid, 128, 0, st>>>(p); break;
+    case 8: decode_attn_splitk_kernel<8><<<grid, 128, 0, st>>>(p); break;
+    case 4: decode_attn_splitk_kernel<4><<<grid, 128, 0, st>>>(p); break;
+    default: decode_attn_splitk_kernel<2><<<grid, 128, 0, st>>>(p); break;
+  }
+  decode_combine_kernel<<<k->n_slices, 128, 0, st>>>(p);
+  if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_layer_state(const pmkvq_cache *k, int32_t layer, int32_t *n_tokens, int32_t *cur_bits,
+                               uint64_t *bytes_used, uint64_t *budget_bytes) {
+  if (!k || layer < 0 || layer >= k->layers) return PMKVQ_ERR_INVALID_ARG;
+  const Layer &l = k->L[layer];
+  if (n_tokens) *n_tokens = l.n_tokens;
+  if (cur_bits) *cur_bits = l.cur_bits;
+  if (bytes_used) *bytes_used = k->bytes_at(l.n_tokens, l.cur_bits);
+  if (budget_bytes) *budget_bytes = l.budget;
+  return PMKVQ_OK;
+}
+
+uint64_t pmkvq_attention_bytes(const pmkvq_cache *k, int32_t layer) {
+  if (!k || layer < 0 || layer >= k->layers) return 0;
+  const Layer &l = k->L[layer];
+  const uint64_t nb = k->body_at(l.n_tokens), n16 = l.n_tokens - nb;
+  const uint64_t kv = 2ull * k->n_slices * (n16 * (16 * 16 + 8) + nb * (16 * l.cur_bits + 8));
+  const uint64_t qo = (uint64_t)k->batch * k->q_heads * kHeadDim * (2 + 4);
+  return kv + qo + (uint64_t)k->kv_heads * kHeadDim * 4;
+}
+
+pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx, int32_t kv_head, int32_t is_value,
+                                uint16_t *h_codes, float *h_scale, float *h_zero, uint8_t *h_bits, uint8_t *h_packed) {
+  if (!k || layer < 0 || layer >= k->layers || batch_idx < 0 || batch_idx >= k->batch || kv_head < 0 ||
+      kv_head >= k->kv_heads)
+    return PMKVQ_ERR_INVALID_ARG;
+  const Layer &l = k->L[layer];
+  if (cudaDeviceSynchronize() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  const LayerGeom g = k->geom(l);
+  const int n = l.n_tokens, n_sink_eff = k->sink_at(n), n_body = k->body_at(n), win_start = n_sink_eff + n_body;
+  const size_t fixed = g.body_off;
+  const size_t body_bytes = (size_t)((n_body + 15) / 16) * tile_bytes(l.cur_bits);
+  std::vector<uint8_t> host(fixed + body_bytes);
+  const uint8_t *src = g.base + (size_t)(batch_idx * k->kv_heads + kv_head) * g.slice_stride;
+  if (cudaMemcpy(host.data(), src, host.size(), cudaMemcpyDeviceToHost) != cudaSuccess) return PMKVQ_ERR_CUDA;
+  size_t packed_off = 0;
+  for (int t = 0; t < n; ++t) {
+    const uint8_t *tile;
+    int row, bits;
+    if (t < k->n_sink) {
+      tile = host.data() + (size_t)(t >> 4) * tile_bytes(16); row = t & 15; bits = 16;
+    } else if (t < win_start) {
+      const int j = t - k->n_sink;
+      tile = host.data() + g.body_off + (size_t)(j >> 4) * tile_bytes(l.cur_bits); row = j & 15; bits = l.cur_bits;
+    } else {
+      const int rp = (t - k->n_sink) % g.ring_tokens;
+      tile = host.data() + g.ring_off + (size_t)(rp >> 4) * tile_bytes(16); row = rp & 15; bits = 16;
+    }
+    const uint8_t *part = tile + (is_value ? v_part_offset(bits) : 0);
+    const uint32_t cmask = (1u << bits) - 1u;
+    uint8_t packed[256];
+    std::memset(packed, 0, sizeof(packed));
+    for (int ch = 0; ch < kHeadDim; ++ch) {
+      int bo, sh;
+      if (is_value) v_slot(bits, row, ch, bo, sh); else k_slot(bits, row, ch, bo, sh);
+      uint16_t hw;
+      std::memcpy(&hw, part + bo, 2);
+      const uint32_t c = (hw >> sh) & cmask;
+      if (h_codes) h_codes[(size_t)t * kHeadDim + ch] = (uint16_t)c;
+      if (bits == 16) { packed[2 * ch] = c & 0xFF; packed[2 * ch + 1] = c >> 8; }
+      else packed[(ch * bits) >> 3] |= (uint8_t)(c << ((ch * bits) & 7));
+    }
+    float sc, ze;
+    std::memcpy(&sc, tile + meta_offset(bits) + meta_slot(is_value ? 2 : 0, row), 4);
+    std::memcpy(&ze, tile + meta_offset(bits) + meta_slot(is_value ? 3 : 1, row), 4);
+    if (h_scale) h_scale[t] = sc;
+    if (h_zero) h_zero[t] = ze;
+    if (h_bits) h_bits[t] = (uint8_t)bits;
+    if (h_packed) std::memcpy(h_packed + packed_off, packed, 16 * bits);
+    packed_off += 16 * bits;
+  }
+  return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_set_attention_splits(pmkvq_cache *k, int32_t splits) {
+  if (!k || splits < 0 || splits > kMaxSplits) return PMKVQ_ERR_INVALID_ARG;
+  k->user_splits = splits;
+  return PMKVQ_OK;
+}
+
+const char *pmkvq_status_string(pmkvq_status s) {
+  switch (s) {
+    case PMKVQ_OK: return "ok";
+    case PMKVQ_ERR_INVALID_ARG: return "invalid argument";
+    case PMKVQ_ERR_ARENA_TOO_SMALL: return "arena too small";
+    case PMKVQ_ERR_BUDGET_FULL: return "budget full: reduce the block first";
+    case PMKVQ_ERR_AT_FBIT: return "block is already at its final bit width";
+    case PMKVQ_ERR_CAPACITY: return "capacity exceeded";
+    case PMKVQ_ERR_CUDA: return "CUDA error";
+    case PMKVQ_ERR_STATE: return "internal state error";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

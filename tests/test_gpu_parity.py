@@ -1,0 +1,165 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+Codes, scales and zero-points bit-exact; attention outputs within max-abs 2e-3 and rel-L2 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_18610_b200 import synth
+from tests.helpers import Mirror, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _lam(layers, kv_heads, k_sample):
+    return np.stack([synth.make_lambda(k_sample).numpy() for _ in range(layers)])
+
+
+@pytest.mark.parametrize("fbit", [16, 8, 4, 2])
+@pytest.mark.parametrize("n", [1, 2, 3, 17])
+def test_tiny_token_counts(fbit, n):
+    """1-17 tokens, no window: sink + body at every width, brute-force sized."""
+    k, v = make_inputs(1, 0, n, 1, 1)
+    m = Mirror(1, 4, 1, 1, 64, [fbit], n_sink=1, window=0,
+               budget_bytes=[2 * (264 + (n - 1) * (16 * fbit + 8))])     # exactly n tokens with the body at Fbit
+    m.append(0, k, v, bulk=False)
+    assert m.cache.layer_state(0)["cur_bits"] == (fbit if n > 1 else 16)
+    m.check_state(0)
+    m.check_attention(0, synth.make_q(1, 0, 0, 1, 4, n))
+
+
+def test_config1_progressive_16_8_4():
+    """BASELINE config 1: 1 block, batch 1, 4 Q / 1 KV head, 4096 tokens fed one by one, 4 outlier channels
+    x20, default budget for Fbit = 4: the block goes 16 -> 8 -> 4.  Full parity after every reduce."""
+    n = 4096
+    k, v = make_inputs(0, 0, n, 1, 1, n_outlier=4, factor=20.0)
+    lam = _lam(1, 1, k[:512])
+    m = Mirror(1, 4, 1, 1, n, [4], lam=lam)
+    kd, vd = k.cuda(), v.cuda()
+    seen = [16]
+    for t in range(n):
+        m.cache.append(0, kd[t:t + 1], vd[t:t + 1])
+        bits = m.cache.layer_state(0)["cur_bits"]
+        if bits != seen[-1] or t in (0, 128, 129, 130, 500, n - 1):
+            # catch the oracle up token by token (literal process), then compare everything
+            o = m.oracles[0]
+            t0 = o.p.n_tokens
+            o.append(k[t0:t + 1].float().numpy().reshape(-1, 1, 128), v[t0:t + 1].float().numpy().reshape(-1, 1, 128))
+            if bits != seen[-1]:
+                seen.append(bits)
+            m.check_state(0)
+            m.check_attention(0, synth.make_q(0, 0, t, 1, 4, t + 1))
+    assert seen == [16, 8, 4]
+
+
+@pytest.mark.parametrize("group", [1, 4, 5, 7, 8])
+def test_gqa_groups(group):
+    kvh, batch, n = 2, 2, 333
+    k, v = make_inputs(2, 0, n, batch, kvh)
+    m = Mirror(1, group * kvh, kvh, batch, 400, [2], lam=_lam(1, kvh, k[:64]), window=32)
+    m.append(0, k, v)
+    m.check_state(0)
+    m.check_attention(0, synth.make_q(2, 0, 0, batch, group * kvh, n))
+
+
+@pytest.mark.parametrize("fbit,chunk,n_sink,window", [(2, 1, 1, 128), (4, 16, 1, 128), (2, 16, 0, 32), (8, 3, 4, 20),
+                                                     (2, 1, 0, 0), (4, 1, 17, 5)])
+def test_multi_layer_bulk_and_stepwise(fbit, chunk, n_sink, window):
+    """Several blocks / slices, ragged bulk appends followed by single-token decode steps."""
+    layers, kvh, batch, group, n_max = 2, 2, 3, 7, 1500
+    m = None
+    ks, vs = [], []
+    for l in range(layers):
+        k, v = make_inputs(3, l, n_max, batch, kvh)
+        ks.append(k); vs.append(v)
+    lam = np.stack([synth.make_lambda(ks[l][:256]).numpy() for l in range(layers)])
+    m = Mirror(layers, group * kvh, kvh, batch, n_max, [fbit, 16 if fbit == 16 else max(fbit, 4)], lam=lam,
+               n_sink=n_sink, window=window, evict_chunk=chunk)
+    cuts = [0, 1, 130, 131, 700, 1237, 1400]
+    for l in range(layers):
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            m.append(l, ks[l][a:b], vs[l][a:b])
+        m.check_state(l, slices=[0, 3, 5])
+        m.check_attention(l, synth.make_q(3, l, 0, batch, group * kvh, cuts[-1]))
+    for t in range(cuts[-1], cuts[-1] + 40):
+        for l in range(layers):
+            m.append(l, ks[l][t:t + 1], vs[l][t:t + 1])
+            if t % 13 == 0:
+                m.check_attention(l, synth.make_q(3, l, t, batch, group * kvh, t + 1))
+    for l in range(layers):
+        m.check_state(l, slices=[1, 4])
+
+
+def test_policy_thresholds_on_gpu():
+    """Code-bit accounting, no sink / window, Fbit = 2, 512 max tokens: reduces at 64, 128, 256 tokens."""
+    n = 512
+    k, v = make_inputs(4, 0, n, 1, 2)
+    m = Mirror(1, 8, 2, 1, n, [2], n_sink=0, window=0, count_metadata=False)
+    kd, vd = k.cuda(), v.cuda()
+    fired, bits = [], 16
+    for t in range(n):
+        m.cache.append(0, kd[t:t + 1], vd[t:t + 1])
+        b = m.cache.layer_state(0)["cur_bits"]
+        if b != bits:
+            fired.append(t); bits = b
+    assert fired == [64, 128, 256]
+    m.oracles[0].append(k.float().numpy().reshape(n, 2, 128), v.float().numpy().reshape(n, 2, 128))
+    m.check_state(0)
+    m.check_attention(0, synth.make_q(4, 0, 0, 1, 8, n))
+
+
+def test_manual_reduce_and_error_codes():
+    from paper_2505_18610_b200 import binding as B
+    k, v = make_inputs(5, 0, 80, 1, 1)
+    m = Mirror(1, 4, 1, 1, 64, [8], n_sink=0, window=0, count_metadata=False, auto_reduce=False)
+    kd, vd = k.cuda(), v.cuda()
+    for t in range(32):
+        assert m.cache.append(0, kd[t:t + 1], vd[t:t + 1], check=False) == B.OK
+    assert m.cache.append(0, kd[32:33], vd[32:33], check=False) == B.BUDGET_FULL
+    assert m.cache.layer_state(0) == {"n_tokens": 32, "cur_bits": 16, "bytes_used": 32 * 512, "budget_bytes": 64 * 256}
+    assert m.cache.progressive_reduce(0, check=False) == B.OK
+    assert m.cache.progressive_reduce(0, check=False) == B.AT_FBIT
+    for t in range(32, 64):
+        assert m.cache.append(0, kd[t:t + 1], vd[t:t + 1], check=False) == B.OK
+    assert m.cache.append(0, kd[64:65], vd[64:65], check=False) == B.CAPACITY
+    assert m.cache.append(5, kd[:1], vd[:1], check=False) == B.INVALID_ARG
+    o = m.oracles[0]
+    o.append(k[:32].float().numpy().reshape(32, 1, 128), v[:32].float().numpy().reshape(32, 1, 128), auto_reduce=False)
+    o.reduce()
+    o.append(k[32:64].float().numpy().reshape(32, 1, 128), v[32:64].float().numpy().reshape(32, 1, 128), auto_reduce=False)
+    m.check_state(0)
+    m.check_attention(0, synth.make_q(5, 0, 0, 1, 4, 64))
+    with pytest.raises(B.PmkvqError):
+        B.Cache(1, 4, 1, 1, 64, [3])
+    with pytest.raises(B.PmkvqError):
+        B.Cache(1, 18, 2, 1, 64, [4])          # GQA group of 9 is outside 1..8
+
+
+def test_split_invariance():
+    kvh, batch, n, group = 2, 2, 5000, 8
+    k, v = make_inputs(6, 0, n, batch, kvh)
+    m = Mirror(1, group * kvh, kvh, batch, n, [2], lam=_lam(1, kvh, k[:256]))
+    m.append(0, k, v)
+    q = synth.make_q(6, 0, 0, batch, group * kvh, n)
+    outs = []
+    for s in (1, 2, 3, 7, 64, 0):
+        m.cache.set_attention_splits(s)
+        m.check_attention(0, q)
+        outs.append(m.cache.decode_attention(0, q.cuda()).cpu().numpy())
+    for o in outs[1:]:
+        assert np.abs(o - outs[0]).max() < 2e-4
+
+
+def test_degenerate_values():
+    """Constant V groups (S = 0), zero K, zero Q, and a huge-range token."""
+    n, kvh = 200, 1
+    k, v = make_inputs(7, 0, n, 1, kvh)
+    v[5] = 1.5; v[150] = -2.0          # constant groups: scale 0
+    k[7] = 0.0
+    v[9] = v[9] * 1000.0               # one token with a huge value range
+    m = Mirror(1, 4, kvh, 1, n, [2], window=16)
+    m.append(0, k, v)
+    m.check_state(0)
+    q = synth.make_q(7, 0, 0, 1, 4, n)
+    m.check_attention(0, q, max_abs=2e-3 * 50)    # outputs reach O(1000) with the scaled token
+    q0 = torch.zeros_like(q)
+    m.check_attention(0, q0, max_abs=2e-3 * 50)
