@@ -104,6 +104,9 @@ pmkvq_status pmkvq_set_attention_splits(pmkvq_cache *cache, int32_t splits);
 pmkvq_status pmkvq_layer_state(const pmkvq_cache *cache, int32_t layer, int32_t *n_tokens, int32_t *cur_bits,
                                uint64_t *bytes_used, uint64_t *budget_bytes);
 
+/* Number of CUDA kernels this cache has launched since it was created (all calls). */
+uint64_t pmkvq_launch_count(const pmkvq_cache *cache);
+
 /* Algorithmic bytes one pmkvq_decode_attention call on this block moves in its current state:
  * codes + fp32 scale + fp32 zero of every cached token of K and V, Q in, out, lambda. */
 uint64_t pmkvq_attention_bytes(const pmkvq_cache *cache, int32_t layer);

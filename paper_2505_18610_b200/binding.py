@@ -59,6 +59,8 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_set_attention_splits.argtypes = [vp, i32]
     lib.pmkvq_layer_state.restype = i32
     lib.pmkvq_layer_state.argtypes = [vp, i32, i32p, i32p, u64p, u64p]
+    lib.pmkvq_launch_count.restype = ctypes.c_uint64
+    lib.pmkvq_launch_count.argtypes = [vp]
     lib.pmkvq_attention_bytes.restype = ctypes.c_uint64
     lib.pmkvq_attention_bytes.argtypes = [vp, i32]
     lib.pmkvq_export_slice.restype = i32
@@ -180,6 +182,9 @@ class Cache:
         if st != OK:
             raise PmkvqError(st, "pmkvq_layer_state")
         return {"n_tokens": n.value, "cur_bits": b.value, "bytes_used": used.value, "budget_bytes": budget.value}
+
+    def launch_count(self) -> int:
+        return int(lib().pmkvq_launch_count(self._h))
 
     def attention_bytes(self, layer: int) -> int:
         return int(lib().pmkvq_attention_bytes(self._h, layer))

@@ -47,6 +47,7 @@ struct pmkvq_cache {
   // arena sections
   size_t off_lambda, off_inv_lambda, off_vmax, off_partials, partial_bytes;
   int sink_tiles, ring_tiles, max_splits, auto_splits, user_splits;
+  uint64_t launches = 0;  // kernels launched so far
   std::vector<Layer> L;
 
   // ---- policy arithmetic (Sec. 3.1) ----
@@ -150,9 +151,9 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
 }
 
 template <int B>
-cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStream_t st) {
+cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStream_t st, uint64_t &launches) {
   const int head = std::min(n_tiles, kHeadTiles);
-  if (head > 0) reduce_head_kernel<B><<<n_slices, 32, 0, st>>>(g, head);
+  if (head > 0) { reduce_head_kernel<B><<<n_slices, 32, 0, st>>>(g, head); ++launches; }
   int lo = head;
   while (lo < n_tiles) {
     // outputs of tiles [lo, hi) end at hi * tile_bytes(B); inputs start at lo * tile_bytes(2B)
@@ -161,6 +162,7 @@ cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStr
     if (hi <= lo) return cudaErrorUnknown;
     dim3 grid((unsigned)((hi - lo + 3) / 4), (unsigned)n_slices);
     reduce_wave_kernel<B><<<grid, 128, 0, st>>>(g, lo, (int)hi);
+    ++launches;
     lo = (int)hi;
   }
   return cudaGetLastError();
@@ -174,9 +176,9 @@ pmkvq_status do_reduce(pmkvq_cache *k, int layer, cudaStream_t st) {
   const LayerGeom g = k->geom(l);
   cudaError_t e = cudaSuccess;
   if (n_tiles > 0) {
-    if (b == 8) e = launch_reduce<8>(g, k->n_slices, n_tiles, st);
-    else if (b == 4) e = launch_reduce<4>(g, k->n_slices, n_tiles, st);
-    else e = launch_reduce<2>(g, k->n_slices, n_tiles, st);
+    if (b == 8) e = launch_reduce<8>(g, k->n_slices, n_tiles, st, k->launches);
+    else if (b == 4) e = launch_reduce<4>(g, k->n_slices, n_tiles, st, k->launches);
+    else e = launch_reduce<2>(g, k->n_slices, n_tiles, st, k->launches);
   }
   if (e != cudaSuccess) return PMKVQ_ERR_CUDA;
   l.cur_bits = b;
@@ -266,6 +268,7 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
   if (ev_last > ev_first) {
     const long long warps = 2ll * (ev_last - ev_first) * k->n_slices;
     evict_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(g, k->n_slices, ev_first, ev_last - ev_first, l.cur_bits);
+    ++k->launches;
   }
   {
     const long long warps = 2ll * n_new * k->n_slices;
@@ -274,6 +277,7 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
     append_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(static_cast<const uint16_t *>(d_K),
                                                               static_cast<const uint16_t *>(d_V), inv_lam, vmax, g, n_new,
                                                               k->n_slices, k->kv_heads, n_old, new_win_start, l.cur_bits);
+    ++k->launches;
   }
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
   l.n_tokens = n_after;
@@ -314,6 +318,7 @@ pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d
     default: decode_attn_splitk_kernel<2><<<grid, 128, 0, st>>>(p); break;
   }
   decode_combine_kernel<<<k->n_slices, 128, 0, st>>>(p);
+  k->launches += 2;
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
   return PMKVQ_OK;
 }
@@ -328,6 +333,8 @@ pmkvq_status pmkvq_layer_state(const pmkvq_cache *k, int32_t layer, int32_t *n_t
   if (budget_bytes) *budget_bytes = l.budget;
   return PMKVQ_OK;
 }
+
+uint64_t pmkvq_launch_count(const pmkvq_cache *k) { return k ? k->launches : 0; }
 
 uint64_t pmkvq_attention_bytes(const pmkvq_cache *k, int32_t layer) {
   if (!k || layer < 0 || layer >= k->layers) return 0;
