@@ -3,7 +3,10 @@
 //
 // Per (batch, kv_head) slice the grid has one "aux" CTA for the INT16 tokens (sink + window ring)
 // and `body_splits` CTAs that share the body tiles.  A warp owns whole 16-token tiles and keeps its
-// own running (max, sum, accumulator); warps are merged in shared memory, CTAs by the combine kernel.
+// own running (max, sum, accumulator); warps are merged in shared memory.  Body tiles are staged
+// through a per-warp cp.async ring in shared memory (a tile is one contiguous run of bytes), so a
+// warp has several tiles in flight while it works on one.  The CTA that finishes last for a slice
+// (atomic ticket, no waiting) merges the slice's split partials and writes the output.
 //
 // The contraction runs on the tensor cores with mma.sync.m16n8k16 (f16 inputs, f32 accumulate) and
 // register operands: packed codes go from 128-bit global loads to MMA fragments with one AND (and
@@ -37,6 +40,7 @@ struct AttnParams {
   const unsigned *vmax_bits;  // [n_slices] running max of the INT16 V scales (fp32 bit patterns)
   float *partials;            // [n_slices][1 + body_splits][8][kPartialStride]
   float *out;                 // fp32 [batch][q_heads][128]
+  unsigned *tickets;          // [n_slices], zero between launches: CTAs of a slice that have finished
   int kv_heads, group, q_heads;
   int n_tokens, n_sink_eff, win_start, cur_bits;
   int n_body, body_tiles, body_splits, tiles_per_split;
@@ -55,6 +59,19 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1,
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -75,7 +92,7 @@ __device__ __forceinline__ uint32_t mul_half2(uint32_t a, float f) {
 // below 2^15 while products keep at least 20 significant bits inside the MMA's alignment window.
 template <int BITS> struct Fmt;
 template <> struct Fmt<2> {
-  static constexpr int N = 8, E = 14, SIGMA_LOG2 = 15;
+  static constexpr int N = 8, E = 14, SIGMA_LOG2 = 15, STAGES = 4;
   __device__ static constexpr int pos(int j) { return j < 3 ? 5 + 2 * j : (j < 5 ? 2 * j : 2 * j - 5); }
   __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[8]) {
     const uint32_t xl = x << 5, xr = x >> 5;
@@ -85,7 +102,7 @@ template <> struct Fmt<2> {
   }
 };
 template <> struct Fmt<4> {
-  static constexpr int N = 4, E = 14, SIGMA_LOG2 = 13;
+  static constexpr int N = 4, E = 14, SIGMA_LOG2 = 13, STAGES = 4;
   __device__ static constexpr int pos(int j) { return (j & 1) ? 7 : 3; }
   __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[4]) {
     const uint32_t xl = x << 3, xr = x >> 5;
@@ -94,7 +111,7 @@ template <> struct Fmt<4> {
   }
 };
 template <> struct Fmt<8> {
-  static constexpr int N = 2, E = 14, SIGMA_LOG2 = 9;
+  static constexpr int N = 2, E = 14, SIGMA_LOG2 = 9, STAGES = 3;
   __device__ static constexpr int pos(int) { return 0; }
   __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[2]) {
     e[0] = x & 0x00FF00FFu;
@@ -104,7 +121,7 @@ template <> struct Fmt<8> {
 // 16 bit: a code is split into its low byte (pos 0, weight 1) and its high byte moved to pos 3
 // (weight 256); the operand that multiplies the high bytes is the low one times 2^5.
 template <> struct Fmt<16> {
-  static constexpr int N = 1, E = 9, SIGMA_LOG2 = 0;
+  static constexpr int N = 1, E = 9, SIGMA_LOG2 = 0, STAGES = 0;  // 16-bit tiles are read straight from global memory
   __device__ static constexpr int pos(int) { return 0; }
 };
 
@@ -114,7 +131,7 @@ struct WarpState {
 };
 
 // One 16-token tile.  `mask` has bit r set when token row r of the tile is a live token.
-template <int BITS>
+template <int BITS, bool MASKED>
 __device__ __forceinline__ void process_tile(const uint8_t *tile, uint32_t mask, WarpState &st,
                                              const uint32_t (&qa)[8][4], float mu, float sumq, float sigma_u,
                                              float inv_sigma_e, int lane) {
@@ -174,11 +191,13 @@ __device__ __forceinline__ void process_tile(const uint8_t *tile, uint32_t mask,
     const int r = i >> 1, e = i & 1;
     const float dot = sacc[r][e] + sacc[r][2 + e];
     sc[i] = fmaf(sk[i] * mu, dot, zk[i] * sumq);
-    const bool live = (mask >> (8 * r + 2 * tig + e)) & 1u;
-    if (!live) {
-      sc[i] = -INFINITY;
-      sv[i] = 0.f;
-      zv[i] = 0.f;
+    if constexpr (MASKED) {
+      const bool live = (mask >> (8 * r + 2 * tig + e)) & 1u;
+      if (!live) {
+        sc[i] = -INFINITY;
+        sv[i] = 0.f;
+        zv[i] = 0.f;
+      }
     }
   }
   float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
@@ -201,7 +220,7 @@ __device__ __forceinline__ void process_tile(const uint8_t *tile, uint32_t mask,
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float s_e = (sv[i] == 0.f ? sigma_u : sv[i]) * inv_sigma_e;  // S_V / sigma_u * 2^E  (<= 2^E)
-    rs[i] = __frcp_rn(s_e);
+    rs[i] = rcp_approx(s_e);
     wv[i] = ex2(sc[i] - st.m) * s_e;
   }
   const uint32_t pb0 = pack_half2(wv[0], wv[1]);
@@ -237,11 +256,36 @@ __device__ __forceinline__ void process_tile(const uint8_t *tile, uint32_t mask,
   }
 }
 
+// Log-sum-exp merge of the split partials of one slice (all its CTAs have published theirs);
+// 128 threads = 128 channels.
+__device__ __forceinline__ void combine_slice(const AttnParams &p, int slice, float *s_w) {
+  const int tid = threadIdx.x;
+  const int b = slice / p.kv_heads, hkv = slice % p.kv_heads;
+  const int n_ctas = 1 + p.body_splits;
+  const float *part = p.partials + (size_t)slice * n_ctas * kMaxGroup * kPartialStride;
+  for (int h = 0; h < p.group; ++h) {
+    // weights 2^(m_c - M) of the CTAs, computed once by the first warps and shared
+    float M = kNegBig;
+    for (int c = 0; c < n_ctas; ++c) M = fmaxf(M, __ldcg(part + ((size_t)c * kMaxGroup + h) * kPartialStride));
+    __syncthreads();
+    for (int c = tid; c < n_ctas; c += 128) s_w[c] = ex2(__ldcg(part + ((size_t)c * kMaxGroup + h) * kPartialStride) - M);
+    __syncthreads();
+    float num = 0.f, den = 0.f;
+#pragma unroll 4
+    for (int c = 0; c < n_ctas; ++c) {
+      const float *pc = part + ((size_t)c * kMaxGroup + h) * kPartialStride;
+      den = fmaf(s_w[c], __ldcg(pc + 1), den);
+      num = fmaf(s_w[c], __ldcg(pc + 4 + tid), num);
+    }
+    p.out[((size_t)b * p.q_heads + hkv * p.group + h) * kHeadDim + tid] = num / den;
+  }
+}
+
 // Everything one CTA does at width BITS: build the query fragments, run its tiles, merge its warps
-// and write one partial (m, l, o[128]) per head.
+// and write one partial (m, l, o[128]) per head.  `ring` is the CTA's dynamic shared memory: the
+// per-warp cp.async stages while tiles stream, then the warps' outputs.
 template <int BITS>
-__device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadDim], float *s_stat,
-                                        float (*s_o)[kMaxGroup][kHeadDim]) {
+__device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadDim], float *s_stat, uint8_t *ring) {
   using F = Fmt<BITS>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
   const int slice = blockIdx.y;
@@ -341,7 +385,8 @@ __device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadD
             }
           }
         }
-        if (mask) process_tile<16>(tile, mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
+        if (mask == 0xFFFFu) process_tile<16, false>(tile, mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
+        else if (mask) process_tile<16, true>(tile, mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
       }
     }
   } else {
@@ -349,19 +394,60 @@ __device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadD
     const int t0 = split * p.tiles_per_split;
     const int t1 = min(p.body_tiles, t0 + p.tiles_per_split);
     const uint8_t *body = slice_base + p.geom.body_off;
-    for (int t = t0 + warp; t < t1; t += 4) {
-      uint32_t mask = 0xFFFFu;
-      if (t == p.body_tiles - 1 && (p.n_body & 15)) mask = (1u << (p.n_body & 15)) - 1u;
-      process_tile<BITS>(body + (size_t)t * tile_bytes(BITS), mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
+    const uint32_t tail_mask = (p.n_body & 15) ? (1u << (p.n_body & 15)) - 1u : 0xFFFFu;
+    if constexpr (F::STAGES == 0) {
+      for (int t = t0 + warp; t < t1; t += 4) {
+        const uint8_t *tile = body + (size_t)t * tile_bytes(BITS);
+        if (t == p.body_tiles - 1 && tail_mask != 0xFFFFu)
+          process_tile<BITS, true>(tile, tail_mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
+        else
+          process_tile<BITS, false>(tile, 0xFFFFu, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
+      }
+    } else {
+      // per-warp ring of STAGES tiles; tile i of this warp is body tile t0 + warp + 4 i
+      constexpr int TB = tile_bytes(BITS);
+      constexpr int S = F::STAGES;
+      uint8_t *my_ring = ring + (size_t)warp * S * TB;
+      const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
+      const int n_my = (t1 - t0 - warp + 3) >> 2;
+      const uint8_t *src0 = body + (size_t)(t0 + warp) * TB + lane * 16;
+      auto issue = [&](int i, int stage) {
+        const uint8_t *src = src0 + (size_t)i * 4 * TB;
+        const uint32_t dst = ring_addr + stage * TB + lane * 16;
+#pragma unroll
+        for (int c = 0; c < (TB / 16 + 31) / 32; ++c)
+          if (c * 32 + lane < TB / 16) cp_async16(dst + c * 512, src + c * 512);
+      };
+#pragma unroll
+      for (int i = 0; i < S - 1; ++i) {
+        if (i < n_my) issue(i, i);
+        cp_async_commit();
+      }
+      int stage = 0, fill = S - 1;
+      for (int i = 0; i < n_my; ++i) {
+        if (i + S - 1 < n_my) issue(i + S - 1, fill);
+        cp_async_commit();
+        cp_async_wait<S - 1>();
+        __syncwarp();
+        const uint8_t *tile = my_ring + stage * TB;
+        if (t0 + warp + 4 * i == p.body_tiles - 1 && tail_mask != 0xFFFFu)
+          process_tile<BITS, true>(tile, tail_mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
+        else
+          process_tile<BITS, false>(tile, 0xFFFFu, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
+        __syncwarp();
+        fill = stage;
+        stage = (stage + 1 == S) ? 0 : stage + 1;
+      }
     }
   }
 
-  // ---- warp epilogue: quad sums, real units, to shared memory ----
+  // ---- warp epilogue: quad sums, real units, to shared memory (the ring is free now) ----
   st.l += __shfl_xor_sync(0xffffffffu, st.l, 1);
   st.l += __shfl_xor_sync(0xffffffffu, st.l, 2);
   st.zs += __shfl_xor_sync(0xffffffffu, st.zs, 1);
   st.zs += __shfl_xor_sync(0xffffffffu, st.zs, 2);
-  __syncthreads();  // s_stat is reused below
+  __syncthreads();  // every warp is done with its stages; s_stat is reused below
+  float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(ring);
   if (tig == 0) {
     s_stat[16 + warp * 8 + g] = st.m;
     s_stat[48 + warp * 8 + g] = st.l;
@@ -381,49 +467,51 @@ __device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadD
   }
   __syncthreads();
 
-  // ---- merge the 4 warps, write the CTA's partial ----
+  // ---- merge the 4 warps, publish the CTA's partial ----
   float *part = p.partials + ((size_t)slice * (1 + p.body_splits) + blockIdx.x) * kMaxGroup * kPartialStride;
   for (int h = 0; h < p.group; ++h) {
     const float m0 = s_stat[16 + h], m1 = s_stat[24 + h], m2 = s_stat[32 + h], m3 = s_stat[40 + h];
     const float M = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     const float w0 = ex2(m0 - M), w1 = ex2(m1 - M), w2 = ex2(m2 - M), w3 = ex2(m3 - M);
     const float o = w0 * s_o[0][h][tid] + w1 * s_o[1][h][tid] + w2 * s_o[2][h][tid] + w3 * s_o[3][h][tid];
-    part[h * kPartialStride + 4 + tid] = o;
+    __stcg(part + h * kPartialStride + 4 + tid, o);
     if (tid == 0) {
-      part[h * kPartialStride] = M;
-      part[h * kPartialStride + 1] =
-          w0 * s_stat[48 + h] + w1 * s_stat[56 + h] + w2 * s_stat[64 + h] + w3 * s_stat[72 + h];
+      __stcg(part + h * kPartialStride, M);
+      __stcg(part + h * kPartialStride + 1,
+             w0 * s_stat[48 + h] + w1 * s_stat[56 + h] + w2 * s_stat[64 + h] + w3 * s_stat[72 + h]);
     }
   }
+
+  // ---- the last CTA of the slice to get here merges the slice (ticket, nobody waits) ----
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned t = atomicAdd(p.tickets + slice, 1u);
+    s_stat[79] = (t == (unsigned)p.body_splits) ? 1.f : 0.f;  // 1 + body_splits CTAs per slice
+  }
+  __syncthreads();
+  if (s_stat[79] != 0.f) {
+    __threadfence();
+    combine_slice(p, slice, s_stat + 80);
+    if (tid == 0) p.tickets[slice] = 0u;  // ready for the next launch (stream order)
+  }
+}
+
+constexpr int attn_ring_bytes(int bits) {
+  // per-warp stages while streaming; at least the 16 KB of warp outputs they are reused for
+  return bits == 16 ? 4 * kMaxGroup * kHeadDim * 4
+                    : (4 * (bits == 8 ? 3 : 4) * tile_bytes(bits) > 4 * kMaxGroup * kHeadDim * 4
+                           ? 4 * (bits == 8 ? 3 : 4) * tile_bytes(bits)
+                           : 4 * kMaxGroup * kHeadDim * 4);
 }
 
 template <int BODY_BITS>
-__global__ void __launch_bounds__(128) decode_attn_splitk_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(128, 4) decode_attn_splitk_kernel(const AttnParams p) {
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
-  __shared__ float s_stat[80];
-  __shared__ __align__(16) float s_o[4][kMaxGroup][kHeadDim];
-  if (blockIdx.x == 0) run_cta<16>(p, s_q, s_stat, s_o);
-  else run_cta<BODY_BITS>(p, s_q, s_stat, s_o);
-}
-
-// Log-sum-exp merge of the split partials of one slice; 128 threads = 128 channels.
-__global__ void __launch_bounds__(128) decode_combine_kernel(const AttnParams p) {
-  const int slice = blockIdx.x, tid = threadIdx.x;
-  const int b = slice / p.kv_heads, hkv = slice % p.kv_heads;
-  const int n_ctas = 1 + p.body_splits;
-  const float *part = p.partials + (size_t)slice * n_ctas * kMaxGroup * kPartialStride;
-  for (int h = 0; h < p.group; ++h) {
-    float M = kNegBig;
-    for (int c = 0; c < n_ctas; ++c) M = fmaxf(M, part[((size_t)c * kMaxGroup + h) * kPartialStride]);
-    float num = 0.f, den = 0.f;
-    for (int c = 0; c < n_ctas; ++c) {
-      const float *pc = part + ((size_t)c * kMaxGroup + h) * kPartialStride;
-      const float w = ex2(pc[0] - M);
-      den = fmaf(w, pc[1], den);
-      num = fmaf(w, pc[4 + tid], num);
-    }
-    p.out[((size_t)b * p.q_heads + hkv * p.group + h) * kHeadDim + tid] = num / den;
-  }
+  __shared__ float s_stat[80 + 72];  // head stats, warp stats, ticket flag, combine weights (<= 65 CTAs)
+  extern __shared__ __align__(128) uint8_t ring[];
+  if (blockIdx.x == 0) run_cta<16>(p, s_q, s_stat, ring);
+  else run_cta<BODY_BITS>(p, s_q, s_stat, ring);
 }
 
 }  // namespace pmkvq

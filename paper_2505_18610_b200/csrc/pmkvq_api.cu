@@ -45,7 +45,7 @@ struct pmkvq_cache {
   uint8_t *arena;
   size_t arena_bytes;
   // arena sections
-  size_t off_lambda, off_inv_lambda, off_vmax, off_partials, partial_bytes;
+  size_t off_lambda, off_inv_lambda, off_vmax, off_tickets, off_partials, partial_bytes;
   int sink_tiles, ring_tiles, max_splits, auto_splits, user_splits;
   uint64_t launches = 0;  // kernels launched so far
   std::vector<Layer> L;
@@ -120,6 +120,7 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.off_lambda = off; off = align_up(off + lam_bytes, kAlign);
   k.off_inv_lambda = off; off = align_up(off + lam_bytes, kAlign);
   k.off_vmax = off; off = align_up(off + (size_t)k.layers * k.n_slices * sizeof(unsigned), kAlign);
+  k.off_tickets = off; off = align_up(off + (size_t)k.n_slices * sizeof(unsigned), kAlign);
   k.partial_bytes = (size_t)k.n_slices * (1 + k.max_splits) * kMaxGroup * kPartialStride * sizeof(float);
   k.off_partials = off; off = align_up(off + k.partial_bytes, kAlign);
 
@@ -219,6 +220,10 @@ pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
   if (e == cudaSuccess)
     e = cudaMemcpy(k->arena + k->off_inv_lambda, inv.data(), n_lam * sizeof(float), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_vmax, 0, (size_t)k->layers * k->n_slices * sizeof(unsigned));
+  if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_tickets, 0, (size_t)k->n_slices * sizeof(unsigned));
+  if (e == cudaSuccess) {
+    e = cudaFuncSetAttribute(decode_attn_splitk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_ring_bytes(8));
+  }
   if (e != cudaSuccess) {
     delete k;
     return PMKVQ_ERR_CUDA;
@@ -296,6 +301,7 @@ pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d
   p.vmax_bits = reinterpret_cast<const unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
   p.partials = reinterpret_cast<float *>(k->arena + k->off_partials);
   p.out = d_out;
+  p.tickets = reinterpret_cast<unsigned *>(k->arena + k->off_tickets);
   p.kv_heads = k->kv_heads; p.group = k->group; p.q_heads = k->q_heads;
   p.n_tokens = l.n_tokens;
   p.n_sink_eff = k->sink_at(l.n_tokens);
@@ -312,13 +318,12 @@ pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d
   p.qk_scale = k->sm_scale * 1.4426950408889634f;
   dim3 grid(1 + splits, k->n_slices);
   switch (l.cur_bits) {
-    case 16: decode_attn_splitk_kernel<16><<<grid, 128, 0, st>>>(p); break;
-    case 8: decode_attn_splitk_kernel<8><<<grid, 128, 0, st>>>(p); break;
-    case 4: decode_attn_splitk_kernel<4><<<grid, 128, 0, st>>>(p); break;
-    default: decode_attn_splitk_kernel<2><<<grid, 128, 0, st>>>(p); break;
+    case 16: decode_attn_splitk_kernel<16><<<grid, 128, attn_ring_bytes(16), st>>>(p); break;
+    case 8: decode_attn_splitk_kernel<8><<<grid, 128, attn_ring_bytes(8), st>>>(p); break;
+    case 4: decode_attn_splitk_kernel<4><<<grid, 128, attn_ring_bytes(4), st>>>(p); break;
+    default: decode_attn_splitk_kernel<2><<<grid, 128, attn_ring_bytes(2), st>>>(p); break;
   }
-  decode_combine_kernel<<<k->n_slices, 128, 0, st>>>(p);
-  k->launches += 2;
+  k->launches += 1;
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
   return PMKVQ_OK;
 }
