@@ -256,7 +256,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="pmkvq", choices=["pmkvq", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS))
-    ap.add_argument("--splits", type=int, default=0, help="attention split-K override (0 = library default)")
+    ap.add_argument("--ctas", type=int, default=0, help="attention grid override (0 = library default: one wave)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
@@ -302,8 +302,8 @@ def main():
 
     # ---------------- device-resident leg ----------------
     cache = build_cache(wl, fbit, budgets, lam, n0, device)
-    if args.splits:
-        cache.set_attention_splits(args.splits)
+    if args.ctas:
+        cache.set_attention_ctas(args.ctas)
     run_steps(cache, wl, pool, warmup, 0)
     bits_before = [cache.layer_state(l)["cur_bits"] for l in range(wl["layers"])]
     barrier()
@@ -332,8 +332,8 @@ def main():
     e2e_ms, h2d, d2h = float("nan"), 0, 0
     if not args.no_e2e:
         cache = build_cache(wl, fbit, budgets, lam, n0, device)
-        if args.splits:
-            cache.set_attention_splits(args.splits)
+        if args.ctas:
+            cache.set_attention_ctas(args.ctas)
         K, V, Q = pool
         hk, hv, hq = K.cpu().pin_memory(), V.cpu().pin_memory(), Q.cpu().pin_memory()
         dk, dv, dq = torch.empty_like(K[0]), torch.empty_like(V[0]), torch.empty_like(Q[0])

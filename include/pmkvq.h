@@ -95,10 +95,10 @@ pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *cache, int32_t layer, void *s
 pmkvq_status pmkvq_decode_attention(pmkvq_cache *cache, int32_t layer, const void *d_Q_bf16, float *d_out,
                                     void *stream);
 
-/* Split-K tuning of pmkvq_decode_attention (flash-decoding partition over the sequence): the body
- * of every (batch, kv_head) slice is shared by at most `splits` CTAs (1..64); 0 restores the
- * default, which aims at two waves of resident CTAs on the GPU's 148 SMs. */
-pmkvq_status pmkvq_set_attention_splits(pmkvq_cache *cache, int32_t splits);
+/* Split-K tuning of pmkvq_decode_attention (flash-decoding partition over the sequence): the tiles
+ * of all (batch, kv_head) slices are cut into `n_ctas` equal contiguous pieces, one per CTA
+ * (1..2048); 0 restores the default, one wave of resident CTAs on the GPU's SMs. */
+pmkvq_status pmkvq_set_attention_ctas(pmkvq_cache *cache, int32_t n_ctas);
 
 /* Host-side state of a block; any out pointer may be NULL. */
 pmkvq_status pmkvq_layer_state(const pmkvq_cache *cache, int32_t layer, int32_t *n_tokens, int32_t *cur_bits,

@@ -55,8 +55,8 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_progressive_reduce.argtypes = [vp, i32, vp]
     lib.pmkvq_decode_attention.restype = i32
     lib.pmkvq_decode_attention.argtypes = [vp, i32, vp, vp, vp]
-    lib.pmkvq_set_attention_splits.restype = i32
-    lib.pmkvq_set_attention_splits.argtypes = [vp, i32]
+    lib.pmkvq_set_attention_ctas.restype = i32
+    lib.pmkvq_set_attention_ctas.argtypes = [vp, i32]
     lib.pmkvq_layer_state.restype = i32
     lib.pmkvq_layer_state.argtypes = [vp, i32, i32p, i32p, u64p, u64p]
     lib.pmkvq_launch_count.restype = ctypes.c_uint64
@@ -170,10 +170,10 @@ class Cache:
             raise PmkvqError(st, "pmkvq_decode_attention")
         return out
 
-    def set_attention_splits(self, splits: int):
-        st = lib().pmkvq_set_attention_splits(self._h, splits)
+    def set_attention_ctas(self, n_ctas: int):
+        st = lib().pmkvq_set_attention_ctas(self._h, n_ctas)
         if st != OK:
-            raise PmkvqError(st, "pmkvq_set_attention_splits")
+            raise PmkvqError(st, "pmkvq_set_attention_ctas")
 
     def layer_state(self, layer: int):
         n, b = ctypes.c_int32(), ctypes.c_int32()

@@ -1,24 +1,36 @@
 // Fused dequantize + GQA decode attention over the packed mixed-precision cache (Eq. 9 + softmax
-// attention), split over the sequence (flash-decoding) with a separate combine kernel.
+// attention), split over the sequence (flash-decoding) with a last-arriver combine.
 //
-// Per (batch, kv_head) slice the grid has one "aux" CTA for the INT16 tokens (sink + window ring)
-// and `body_splits` CTAs that share the body tiles.  A warp owns whole 16-token tiles and keeps its
-// own running (max, sum, accumulator); warps are merged in shared memory.  Body tiles are staged
-// through a per-warp cp.async ring in shared memory (a tile is one contiguous run of bytes), so a
-// warp has several tiles in flight while it works on one.  The CTA that finishes last for a slice
-// (atomic ticket, no waiting) merges the slice's split partials and writes the output.
+// Work decomposition.  Every (batch, kv_head) slice is two runs of 16-token tiles: the INT16 run
+// (sink tiles + window ring) and the body run at the block's current width.  A tile of the body
+// weighs one unit, an INT16 tile `w16` units (their byte ratio), and every slice starts with a few
+// empty units that stand for the fixed cost of a segment.  All units of all slices form one
+// line that is cut into equal contiguous pieces, one per CTA of a persistent grid (one CTA of 16
+// warps per SM), so every CTA streams the same number of bytes whatever the shape.  The part of a
+// CTA's piece that lies in one slice is a "segment": its 16 warps draw the segment's tiles from a
+// shared counter (INT16 tiles first, then body tiles, the accumulators changing units in between),
+// so they finish together however the SM shares its issue slots among them; each warp keeps its
+// own running (max, sum, accumulator), the warps are merged in shared memory and the segment
+// publishes one partial (m, l, o[128]) per head.  The CTA that publishes the
+// last partial of a slice (atomic ticket, nobody waits) merges the slice and writes the output.
+//
+// Body tiles are staged through a per-warp cp.async ring in shared memory (a tile is one
+// contiguous run of bytes); tiles are consumed two at a time at 2 and 4 bit so that the softmax
+// bookkeeping is paid once per 32 tokens.
 //
 // The contraction runs on the tensor cores with mma.sync.m16n8k16 (f16 inputs, f32 accumulate) and
-// register operands: packed codes go from 128-bit global loads to MMA fragments with one AND (and
-// a shared shift) per pair of codes - a code field left in place inside an fp16 bit pattern below
-// bit 11 is the exact value code * 2^(pos-24) (fp16 subnormals and the first binade are linear).
+// register operands: packed codes go from 128-bit loads to MMA fragments with one AND per pair of
+// codes - a code field left in place inside an fp16 bit pattern below bit 11 is the exact value
+// code * 2^(pos-24) (fp16 subnormals and the first binade are linear in the bit pattern).
 //   scores:  S[h, t]  = sum_i Q''[h, i] * c_K[t, i]      A = Q'' (rows 0-7: fp16 "hi" part of the 8 heads,
 //                                                        rows 8-15: the "lo" remainder), B = K codes
 //   output:  O^T[i,h] = sum_t c_V[t, i] * w[t, h]        A = V codes, B = w = p * S_V (one fp16)
 // The per-token scale and zero-point never touch the codes: q.k = S_K (q.c) + Z_K sum(q) and
-// sum_t p_t v_t = sum_t (p_t S_V,t) c_t + sum_t p_t Z_V,t.  The probability actually used for a token is
-// the fp16-rounded w divided by its scale, in numerator and denominator alike, so the fp16 rounding
-// of w is a consistent (softmax-invariant to first order) perturbation.
+// sum_t p_t v_t = sum_t (p_t S_V,t) c_t + sum_t p_t Z_V,t.
+//
+// Online softmax with a lazy reference: probabilities are taken relative to a per-head reference m
+// that is only moved (and the accumulators rescaled) when a score exceeds it by more than
+// kMaxAhead, so the common case has no cross-lane traffic at all.
 #pragma once
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -29,49 +41,71 @@
 
 namespace pmkvq {
 
-constexpr int kMaxGroup = 8;        // query heads per KV head handled by one MMA row block
-constexpr int kPartialStride = 132; // floats per (cta, head): m, l, 2 pad, o[128]
+constexpr int kMaxGroup = 8;         // query heads per KV head handled by one MMA row block
+constexpr int kPartialStride = 132;  // floats per (segment, head): m, l, 2 pad, o[128]
 constexpr float kNegBig = -1.0e30f;
+constexpr float kMaxAhead = 3.0f;    // a score may exceed the reference by this much (log2 units)
+constexpr int kAttnWarps = 16;      // one CTA per SM; its warps share the CTA's tiles dynamically
+constexpr int kAttnThreads = 32 * kAttnWarps;
 
 struct AttnParams {
   LayerGeom geom;
   const uint16_t *Q;          // bf16 [batch][q_heads][128]
   const float *lambda;        // [kv_heads][128] of this block
   const unsigned *vmax_bits;  // [n_slices] running max of the INT16 V scales (fp32 bit patterns)
-  float *partials;            // [n_slices][1 + body_splits][8][kPartialStride]
+  float *partials;            // [n_ctas + n_slices][8][kPartialStride]
   float *out;                 // fp32 [batch][q_heads][128]
-  unsigned *tickets;          // [n_slices], zero between launches: CTAs of a slice that have finished
-  int kv_heads, group, q_heads;
+  unsigned *tickets;          // [n_slices], zero between launches: partials of a slice published so far
+  int kv_heads, group, q_heads, n_slices;
   int n_tokens, n_sink_eff, win_start, cur_bits;
-  int n_body, body_tiles, body_splits, tiles_per_split;
-  float qk_scale;  // sm_scale * log2(e)
+  int n_body, body_tiles, aux_tiles, sink_tiles;
+  int w16;                    // units of one INT16 tile
+  int units_lead;             // empty units at the start of every slice: the fixed cost of one more segment
+  long long units_aux, units_slice, units_total, units_per_cta;  // units_aux includes units_lead
+  float qk_scale;             // sm_scale * log2(e)
 };
 
 __device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                         uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void *gptr) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gptr) : "memory");
 }
+// the same at byte offset OFF of both addresses (an immediate: no address arithmetic per copy)
+template <int OFF>
+__device__ __forceinline__ void cp_async16_at(uint32_t smem_addr, const void *gptr) {
+  asm volatile("cp.async.cg.shared.global [%0 + %2], [%1 + %2], 16;\n" ::"r"(smem_addr), "l"(gptr), "n"(OFF) : "memory");
+}
+template <int N, int I = 0>
+__device__ __forceinline__ void cp_async_run(uint32_t smem_addr, const void *gptr) {  // N copies, 512 bytes apart
+  if constexpr (I < N) {
+    cp_async16_at<I * 512>(smem_addr, gptr);
+    cp_async_run<N, I + 1>(smem_addr, gptr);
+  }
+}
+// lane 0 takes the next ticket of a shared-memory counter; every lane gets it
+__device__ __forceinline__ int claim_next(int *ctr, int lane) {
+  int j = 0;
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(ctr);
+  asm volatile(
+      "{\n .reg .pred p;\n setp.eq.s32 p, %2, 0;\n @p atom.shared.add.u32 %0, [%1], 1;\n}\n"
+      : "+r"(j)
+      : "r"(addr), "r"(lane)
+      : "memory");
+  return __shfl_sync(0xffffffffu, j, 0);
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ float rcp_approx(float x) {
-  float y;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -86,125 +120,160 @@ __device__ __forceinline__ uint32_t mul_half2(uint32_t a, float f) {
   const __half2 r = __hmul2(*reinterpret_cast<const __half2 *>(&a), __float2half2_rn(f));
   return *reinterpret_cast<const uint32_t *>(&r);
 }
+__device__ __forceinline__ uint32_t high_bytes(uint32_t x) { return __byte_perm(x, 0u, 0x4341); }  // {b1, 0, b3, 0}
 
-// Bit position of code j of a half-word after extraction, per width (see extract<>), and the fp16
-// exponent budget: A/B operands built from Q or w are scaled by 2^(E - pos) so that they stay
-// below 2^15 while products keep at least 20 significant bits inside the MMA's alignment window.
+// Per width: bit position of code j of a half-word after extraction, the fp16 exponent budgets
+// (Q fragments are scaled by 2^(EQ - pos - e_head) and stay below 2^EQ; w = p * S_V is scaled to at
+// most 2^(EP + kMaxAhead)), log2 of the bound on S_b / S_16, and the staging ring (NT tiles are
+// consumed per step, SLOTS steps are resident per warp; a warp holds SLOTS - 1 claimed steps, which
+// is also how far apart the warps of a CTA can finish, so the ring is kept shallow: 16 warps per SM
+// already keep about 70 KB in flight).
 template <int BITS> struct Fmt;
 template <> struct Fmt<2> {
-  static constexpr int N = 8, E = 14, SIGMA_LOG2 = 15, STAGES = 4;
-  __device__ static constexpr int pos(int j) { return j < 3 ? 5 + 2 * j : (j < 5 ? 2 * j : 2 * j - 5); }
+    static constexpr int N = 8, EQ = 14, EP = 12, SIGMA_LOG2 = 15, NT = 2, SLOTS = 2;
+  __host__ __device__ static constexpr int pos(int j) { return j < 5 ? 2 * j : 2 * j - 5; }
   __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[8]) {
-    const uint32_t xl = x << 5, xr = x >> 5;
-    e[0] = xl & 0x00600060u; e[1] = xl & 0x01800180u; e[2] = xl & 0x06000600u;
-    e[3] = x & 0x00C000C0u;  e[4] = x & 0x03000300u;
+    const uint32_t xr = x >> 5;
+    e[0] = x & 0x00030003u; e[1] = x & 0x000C000Cu; e[2] = x & 0x00300030u; e[3] = x & 0x00C000C0u;
+    e[4] = x & 0x03000300u;
     e[5] = xr & 0x00600060u; e[6] = xr & 0x01800180u; e[7] = xr & 0x06000600u;
   }
 };
 template <> struct Fmt<4> {
-  static constexpr int N = 4, E = 14, SIGMA_LOG2 = 13, STAGES = 4;
-  __device__ static constexpr int pos(int j) { return (j & 1) ? 7 : 3; }
+  static constexpr int N = 4, EQ = 14, EP = 12, SIGMA_LOG2 = 13, NT = 2, SLOTS = 2;
+  __host__ __device__ static constexpr int pos(int j) { return (j & 1) ? 4 : 0; }
   __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[4]) {
-    const uint32_t xl = x << 3, xr = x >> 5;
-    e[0] = xl & 0x00780078u; e[1] = xl & 0x07800780u;
-    e[2] = xr & 0x00780078u; e[3] = xr & 0x07800780u;
+    const uint32_t xr = x >> 8;
+    e[0] = x & 0x000F000Fu; e[1] = x & 0x00F000F0u;
+    e[2] = xr & 0x000F000Fu; e[3] = xr & 0x00F000F0u;
   }
 };
 template <> struct Fmt<8> {
-  static constexpr int N = 2, E = 14, SIGMA_LOG2 = 9, STAGES = 3;
-  __device__ static constexpr int pos(int) { return 0; }
+  static constexpr int N = 2, EQ = 14, EP = 12, SIGMA_LOG2 = 9, NT = 1, SLOTS = 2;
+  __host__ __device__ static constexpr int pos(int) { return 0; }
   __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[2]) {
     e[0] = x & 0x00FF00FFu;
-    e[1] = (x >> 8) & 0x00FF00FFu;
+    e[1] = high_bytes(x);
   }
 };
-// 16 bit: a code is split into its low byte (pos 0, weight 1) and its high byte moved to pos 3
-// (weight 256); the operand that multiplies the high bytes is the low one times 2^5.
+// 16 bit: a code is split into its two bytes.  Scores keep two accumulators (low bytes, high bytes)
+// against the same Q fragments; for the output the high bytes sit at bit 3 (weight 8) and are
+// multiplied by w * 32.  16-bit tiles are read straight from global memory.
 template <> struct Fmt<16> {
-  static constexpr int N = 1, E = 9, SIGMA_LOG2 = 0, STAGES = 0;  // 16-bit tiles are read straight from global memory
-  __device__ static constexpr int pos(int) { return 0; }
+  static constexpr int N = 1, EQ = 14, EP = 7, SIGMA_LOG2 = 0, NT = 1, SLOTS = 0;
+  __host__ __device__ static constexpr int pos(int) { return 0; }
 };
 
 struct WarpState {
-  float m, l, zs;      // running max (log2 units), sum of probabilities, sum of p * Z_V, for head g (this lane's quad)
-  float acc[8][4];     // O^T accumulators: [m-tile][channel row g / g+8 x head col 2tig / 2tig+1]
+  float m, l, zs;   // reference (log2 units), sum of probabilities, sum of p * Z_V, for head g (this lane's quad)
+  float acc[8][4];  // O^T accumulators: [m-tile][channel row g / g+8 x head col 2tig / 2tig+1]
 };
 
-// One 16-token tile.  `mask` has bit r set when token row r of the tile is a live token.
-template <int BITS, bool MASKED>
-__device__ __forceinline__ void process_tile(const uint8_t *tile, uint32_t mask, WarpState &st,
-                                             const uint32_t (&qa)[8][4], float mu, float sumq, float sigma_u,
-                                             float inv_sigma_e, int lane) {
+// NT consecutive 16-token tiles.  `mask` (NT == 1 only) has bit r set when token row r is live.
+template <int BITS, int NT, bool MASKED>
+__device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mask, WarpState &st,
+                                              const uint32_t (&qa)[8][4], float mu, float sumq, float inv_sigma_e,
+                                              int lane) {
   using F = Fmt<BITS>;
+  static_assert(!(MASKED && NT != 1), "masked tiles are processed one at a time");
+  constexpr int TB = tile_bytes(BITS);
   constexpr int CHUNKS = BITS / 2;
+  constexpr int NS = 4 * NT;  // scores per lane
   const int tig = lane & 3;
-  uint32_t kw[2 * BITS], vw[2 * BITS];
-  {
-    const uint8_t *kp = tile + lane * 16;
-    const uint8_t *vp = tile + v_part_offset(BITS) + lane * 16;
-#pragma unroll
-    for (int q = 0; q < CHUNKS; ++q) {
-      const uint4 a = *reinterpret_cast<const uint4 *>(kp + q * 512);
-      kw[4 * q] = a.x; kw[4 * q + 1] = a.y; kw[4 * q + 2] = a.z; kw[4 * q + 3] = a.w;
-    }
-#pragma unroll
-    for (int q = 0; q < CHUNKS; ++q) {
-      const uint4 a = *reinterpret_cast<const uint4 *>(vp + q * 512);
-      vw[4 * q] = a.x; vw[4 * q + 1] = a.y; vw[4 * q + 2] = a.z; vw[4 * q + 3] = a.w;
-    }
-  }
-  const float4 *mp = reinterpret_cast<const float4 *>(tile + meta_offset(BITS) + tig * 64);
-  const float4 sk4 = mp[0], zk4 = mp[1], sv4 = mp[2], zv4 = mp[3];
-  float sk[4] = {sk4.x, sk4.y, sk4.z, sk4.w}, zk[4] = {zk4.x, zk4.y, zk4.z, zk4.w};
-  float sv[4] = {sv4.x, sv4.y, sv4.z, sv4.w}, zv[4] = {zv4.x, zv4.y, zv4.z, zv4.w};
 
   // ---- scores: S = Q'' K^T, heads on M (hi rows 0-7, lo rows 8-15), tokens on N ----
-  float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+  float dot[NS];
   if constexpr (BITS == 16) {
+    const uint8_t *kp = tile0 + lane * 16;
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
+      uint32_t kw[16];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 a = *reinterpret_cast<const uint4 *>(kp + (4 * r + q) * 512);
+        kw[4 * q] = a.x; kw[4 * q + 1] = a.y; kw[4 * q + 2] = a.z; kw[4 * q + 3] = a.w;
+      }
+      float lo[4] = {0.f, 0.f, 0.f, 0.f}, hi[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int s = 0; s < 8; ++s) {
-        const uint32_t x0 = kw[r * 16 + 2 * s], x1 = kw[r * 16 + 2 * s + 1];
-        mma_f16(sacc[r], qa[s], x0 & 0x00FF00FFu, x1 & 0x00FF00FFu);
-        mma_f16(sacc[r], mul_half2(qa[s][0], 32.f), mul_half2(qa[s][1], 32.f), mul_half2(qa[s][2], 32.f),
-                mul_half2(qa[s][3], 32.f), (x0 >> 5) & 0x07F807F8u, (x1 >> 5) & 0x07F807F8u);
+        const uint32_t x0 = kw[2 * s], x1 = kw[2 * s + 1];
+        mma_f16(lo, qa[s], x0 & 0x00FF00FFu, x1 & 0x00FF00FFu);
+        mma_f16(hi, qa[s], high_bytes(x0), high_bytes(x1));
       }
+      dot[2 * r] = fmaf(256.f, hi[0] + hi[2], lo[0] + lo[2]);
+      dot[2 * r + 1] = fmaf(256.f, hi[1] + hi[3], lo[1] + lo[3]);
     }
   } else {
+    // the 2 NT (tile, token half) accumulators advance together: consecutive MMAs are independent
+    uint32_t kw[NT][2 * BITS];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
+    for (int nt = 0; nt < NT; ++nt) {
+      const uint8_t *kp = tile0 + nt * TB + lane * 16;
 #pragma unroll
-      for (int w = 0; w < BITS; ++w) {
-        uint32_t e[F::N];
-        F::extract(kw[r * BITS + w], e);
-#pragma unroll
-        for (int jj = 0; jj < F::N / 2; ++jj) mma_f16(sacc[r], qa[(w * F::N) / 2 + jj], e[2 * jj], e[2 * jj + 1]);
+      for (int q = 0; q < CHUNKS; ++q) {
+        const uint4 a = *reinterpret_cast<const uint4 *>(kp + q * 512);
+        kw[nt][4 * q] = a.x; kw[nt][4 * q + 1] = a.y; kw[nt][4 * q + 2] = a.z; kw[nt][4 * q + 3] = a.w;
       }
     }
+    float sacc[NT][2][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int r = 0; r < 2; ++r) sacc[nt][r][0] = sacc[nt][r][1] = sacc[nt][r][2] = sacc[nt][r][3] = 0.f;
+#pragma unroll
+    for (int w = 0; w < BITS; ++w) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          uint32_t e[F::N];
+          F::extract(kw[nt][r * BITS + w], e);
+#pragma unroll
+          for (int jj = 0; jj < F::N / 2; ++jj) mma_f16(sacc[nt][r], qa[(w * F::N) / 2 + jj], e[2 * jj], e[2 * jj + 1]);
+        }
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        dot[4 * nt + 2 * r] = sacc[nt][r][0] + sacc[nt][r][2];
+        dot[4 * nt + 2 * r + 1] = sacc[nt][r][1] + sacc[nt][r][3];
+      }
   }
 
-  // ---- online softmax for head g over this lane's 4 tokens {2tig, 2tig+1, 8+2tig, 9+2tig} ----
-  float sc[4];
+  // ---- per-token scale / zero-point of this lane's tokens {2tig, 2tig+1, 8+2tig, 9+2tig} of each tile ----
+  float sk[NS], zk[NS], sv[NS], zv[NS];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = i >> 1, e = i & 1;
-    const float dot = sacc[r][e] + sacc[r][2 + e];
-    sc[i] = fmaf(sk[i] * mu, dot, zk[i] * sumq);
+  for (int nt = 0; nt < NT; ++nt) {
+    const float4 *mp = reinterpret_cast<const float4 *>(tile0 + nt * TB + meta_offset(BITS) + tig * 64);
+    const float4 a = mp[0], b = mp[1], c = mp[2], d = mp[3];
+    sk[4 * nt] = a.x; sk[4 * nt + 1] = a.y; sk[4 * nt + 2] = a.z; sk[4 * nt + 3] = a.w;
+    zk[4 * nt] = b.x; zk[4 * nt + 1] = b.y; zk[4 * nt + 2] = b.z; zk[4 * nt + 3] = b.w;
+    sv[4 * nt] = c.x; sv[4 * nt + 1] = c.y; sv[4 * nt + 2] = c.z; sv[4 * nt + 3] = c.w;
+    zv[4 * nt] = d.x; zv[4 * nt + 1] = d.y; zv[4 * nt + 2] = d.z; zv[4 * nt + 3] = d.w;
+  }
+
+  // ---- true scores; the reference moves only when one of them runs ahead of it ----
+  float sc[NS];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < NS; ++i) {
+    sc[i] = fmaf(sk[i] * mu, dot[i], zk[i] * sumq);
     if constexpr (MASKED) {
-      const bool live = (mask >> (8 * r + 2 * tig + e)) & 1u;
+      const bool live = (mask >> (8 * ((i >> 1) & 1) + 2 * tig + (i & 1))) & 1u;
       if (!live) {
         sc[i] = -INFINITY;
         sv[i] = 0.f;
         zv[i] = 0.f;
       }
     }
+    mx = fmaxf(mx, sc[i]);
   }
-  float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
-  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-  const float m_new = fmaxf(st.m, mx);
-  if (__any_sync(0xffffffffu, m_new > st.m)) {
+  if (__any_sync(0xffffffffu, mx > st.m + kMaxAhead)) {
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float m_new = fmaxf(st.m, mx);
     const float f = ex2(st.m - m_new);
     st.l *= f;
     st.zs *= f;
@@ -216,97 +285,203 @@ __device__ __forceinline__ void process_tile(const uint8_t *tile, uint32_t mask,
     }
     st.m = m_new;
   }
-  float wv[4], rs[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float s_e = (sv[i] == 0.f ? sigma_u : sv[i]) * inv_sigma_e;  // S_V / sigma_u * 2^E  (<= 2^E)
-    rs[i] = rcp_approx(s_e);
-    wv[i] = ex2(sc[i] - st.m) * s_e;
-  }
-  const uint32_t pb0 = pack_half2(wv[0], wv[1]);
-  const uint32_t pb1 = pack_half2(wv[2], wv[3]);
+  uint32_t pb[2 * NT];
   {
-    const float2 w01 = __half22float2(*reinterpret_cast<const __half2 *>(&pb0));
-    const float2 w23 = __half22float2(*reinterpret_cast<const __half2 *>(&pb1));
-    const float p0 = w01.x * rs[0], p1 = w01.y * rs[1], p2 = w23.x * rs[2], p3 = w23.y * rs[3];
-    st.l += (p0 + p1) + (p2 + p3);
-    st.zs += fmaf(p0, zv[0], fmaf(p1, zv[1], fmaf(p2, zv[2], p3 * zv[3])));
+    float wv[NS];
+#pragma unroll
+    for (int i = 0; i < NS; ++i) {
+      const float p = ex2(sc[i] - st.m);
+      st.l += p;
+      st.zs = fmaf(p, zv[i], st.zs);
+      wv[i] = p * (sv[i] * inv_sigma_e);  // p * S_V / sigma_u * 2^EP
+    }
+#pragma unroll
+    for (int j = 0; j < 2 * NT; ++j) pb[j] = pack_half2(wv[2 * j], wv[2 * j + 1]);
   }
 
   // ---- output: O^T += V^T w, channels on M, tokens on K, heads on N ----
-  if constexpr (BITS == 16) {
-    const uint32_t ph0 = mul_half2(pb0, 32.f), ph1 = mul_half2(pb1, 32.f);
 #pragma unroll
-    for (int mt = 0; mt < 8; ++mt) {
-      const uint32_t a0 = vw[2 * mt], a1 = vw[2 * mt + 1], a2 = vw[16 + 2 * mt], a3 = vw[16 + 2 * mt + 1];
-      mma_f16(st.acc[mt], a0 & 0x00FF00FFu, a1 & 0x00FF00FFu, a2 & 0x00FF00FFu, a3 & 0x00FF00FFu, pb0, pb1);
-      mma_f16(st.acc[mt], (a0 >> 5) & 0x07F807F8u, (a1 >> 5) & 0x07F807F8u, (a2 >> 5) & 0x07F807F8u,
-              (a3 >> 5) & 0x07F807F8u, ph0, ph1);
+  for (int nt = 0; nt < NT; ++nt) {
+    const uint8_t *vp = tile0 + nt * TB + v_part_offset(BITS) + lane * 16;
+    uint32_t vw[2 * BITS];
+#pragma unroll
+    for (int q = 0; q < CHUNKS; ++q) {
+      const uint4 a = *reinterpret_cast<const uint4 *>(vp + q * 512);
+      vw[4 * q] = a.x; vw[4 * q + 1] = a.y; vw[4 * q + 2] = a.z; vw[4 * q + 3] = a.w;
     }
-  } else {
+    const uint32_t pb0 = pb[2 * nt], pb1 = pb[2 * nt + 1];
+    if constexpr (BITS == 16) {
+      const uint32_t ph0 = mul_half2(pb0, 32.f), ph1 = mul_half2(pb1, 32.f);
 #pragma unroll
-    for (int w = 0; w < BITS; ++w) {
-      uint32_t ea[F::N], eb[F::N];
-      F::extract(vw[w], ea);
-      F::extract(vw[BITS + w], eb);
+      for (int mt = 0; mt < 8; ++mt) {
+        const uint32_t a0 = vw[2 * mt], a1 = vw[2 * mt + 1], a2 = vw[16 + 2 * mt], a3 = vw[16 + 2 * mt + 1];
+        mma_f16(st.acc[mt], a0 & 0x00FF00FFu, a1 & 0x00FF00FFu, a2 & 0x00FF00FFu, a3 & 0x00FF00FFu, pb0, pb1);
+        mma_f16(st.acc[mt], (a0 >> 5) & 0x07F807F8u, (a1 >> 5) & 0x07F807F8u, (a2 >> 5) & 0x07F807F8u,
+                (a3 >> 5) & 0x07F807F8u, ph0, ph1);
+      }
+    } else {
 #pragma unroll
-      for (int jj = 0; jj < F::N / 2; ++jj)
-        mma_f16(st.acc[(w * F::N) / 2 + jj], ea[2 * jj], ea[2 * jj + 1], eb[2 * jj], eb[2 * jj + 1], pb0, pb1);
+      for (int w = 0; w < BITS; ++w) {
+        uint32_t ea[F::N], eb[F::N];
+        F::extract(vw[w], ea);
+        F::extract(vw[BITS + w], eb);
+#pragma unroll
+        for (int jj = 0; jj < F::N / 2; ++jj)
+          mma_f16(st.acc[(w * F::N) / 2 + jj], ea[2 * jj], ea[2 * jj + 1], eb[2 * jj], eb[2 * jj + 1], pb0, pb1);
+      }
     }
   }
 }
 
-// Log-sum-exp merge of the split partials of one slice (all its CTAs have published theirs);
-// 128 threads = 128 channels.
-__device__ __forceinline__ void combine_slice(const AttnParams &p, int slice, float *s_w) {
-  const int tid = threadIdx.x;
+// ---- where the partials of a slice live ------------------------------------------------------
+// Slice s covers units [s U, (s+1) U); the segment of CTA c in it publishes partial number c + s.
+__device__ __forceinline__ void slice_ctas(const AttnParams &p, int slice, int &c_first, int &c_last) {
+  const long long lo = (long long)slice * p.units_slice;
+  c_first = (int)((lo + p.units_lead) / p.units_per_cta);  // a CTA that only touches the lead units has no segment
+  c_last = (int)((lo + p.units_slice - 1) / p.units_per_cta);
+}
+
+// Log-sum-exp merge of the partials of one slice (all published).  Warp w merges head w;
+// a lane owns 4 channels, and the weights of up to 32 partials at a time (one per lane).
+__device__ __forceinline__ void combine_slice(const AttnParams &p, int slice) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = slice / p.kv_heads, hkv = slice % p.kv_heads;
-  const int n_ctas = 1 + p.body_splits;
-  const float *part = p.partials + (size_t)slice * n_ctas * kMaxGroup * kPartialStride;
-  for (int h = 0; h < p.group; ++h) {
-    // weights 2^(m_c - M) of the CTAs, computed once by the first warps and shared
+  int cf, cl;
+  slice_ctas(p, slice, cf, cl);
+  const int n_parts = cl - cf + 1;
+  const float *base = p.partials + (size_t)(cf + slice) * kMaxGroup * kPartialStride;
+  for (int h = warp; h < p.group; h += kAttnWarps) {
+    const float *ph = base + (size_t)h * kPartialStride;
     float M = kNegBig;
-    for (int c = 0; c < n_ctas; ++c) M = fmaxf(M, __ldcg(part + ((size_t)c * kMaxGroup + h) * kPartialStride));
-    __syncthreads();
-    for (int c = tid; c < n_ctas; c += 128) s_w[c] = ex2(__ldcg(part + ((size_t)c * kMaxGroup + h) * kPartialStride) - M);
-    __syncthreads();
-    float num = 0.f, den = 0.f;
-#pragma unroll 4
-    for (int c = 0; c < n_ctas; ++c) {
-      const float *pc = part + ((size_t)c * kMaxGroup + h) * kPartialStride;
-      den = fmaf(s_w[c], __ldcg(pc + 1), den);
-      num = fmaf(s_w[c], __ldcg(pc + 4 + tid), num);
+    for (int c = lane; c < n_parts; c += 32) M = fmaxf(M, __ldcg(ph + (size_t)c * kMaxGroup * kPartialStride));
+#pragma unroll
+    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+    for (int c0 = 0; c0 < n_parts; c0 += 32) {
+      float w = 0.f;
+      if (c0 + lane < n_parts) {
+        const float2 ml = __ldcg(reinterpret_cast<const float2 *>(ph + (size_t)(c0 + lane) * kMaxGroup * kPartialStride));
+        w = ex2(ml.x - M);
+        den = fmaf(w, ml.y, den);
+      }
+      const int nb = min(32, n_parts - c0);
+#pragma unroll 8
+      for (int j = 0; j < nb; ++j) {
+        const float wj = __shfl_sync(0xffffffffu, w, j);
+        const float4 o4 = __ldcg(reinterpret_cast<const float4 *>(ph + (size_t)(c0 + j) * kMaxGroup * kPartialStride + 4) + lane);
+        num.x = fmaf(wj, o4.x, num.x); num.y = fmaf(wj, o4.y, num.y);
+        num.z = fmaf(wj, o4.z, num.z); num.w = fmaf(wj, o4.w, num.w);
+      }
     }
-    p.out[((size_t)b * p.q_heads + hkv * p.group + h) * kHeadDim + tid] = num / den;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    const float inv = 1.0f / den;
+    float4 *dst = reinterpret_cast<float4 *>(p.out + ((size_t)b * p.q_heads + hkv * p.group + h) * kHeadDim) + lane;
+    *dst = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
   }
 }
 
-// Everything one CTA does at width BITS: build the query fragments, run its tiles, merge its warps
-// and write one partial (m, l, o[128]) per head.  `ring` is the CTA's dynamic shared memory: the
-// per-warp cp.async stages while tiles stream, then the warps' outputs.
+// Query fragments of head g at the code positions of width BITS, from Q'' in shared memory.
 template <int BITS>
-__device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadDim], float *s_stat, uint8_t *ring) {
+__device__ __forceinline__ void build_q_fragments(uint32_t (&qa)[8][4], const float (*s_q)[kHeadDim], int e_g, int g,
+                                                  int tig) {
   using F = Fmt<BITS>;
+#pragma unroll
+  for (int s = 0; s < 8; ++s) {
+#pragma unroll
+    for (int beta = 0; beta < 2; ++beta) {
+      const int W = 2 * s + beta;
+      const float scl = ldexpf(1.0f, F::EQ - F::pos(W % F::N) - e_g);
+      const int c0 = 16 * s + 8 * beta + 2 * tig;
+      const float x0 = s_q[g][c0] * scl, x1 = s_q[g][c0 + 1] * scl;
+      const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+      const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
+      const __half2 hi = __halves2half2(h0, h1), lo = __halves2half2(l0, l1);
+      qa[s][2 * beta] = *reinterpret_cast<const uint32_t *>(&hi);
+      qa[s][2 * beta + 1] = *reinterpret_cast<const uint32_t *>(&lo);
+    }
+  }
+}
+
+// One segment: the part [u_lo, u_hi) (units relative to the slice) of one slice that this CTA owns.
+// Builds the slice's query, runs the INT16 tiles and then the body tiles (width BITS) of the range,
+// merges the warps and publishes one partial per head; the CTA that publishes the slice's last
+// partial merges the slice.  The warps of the CTA draw work from two shared counters (INT16 tiles,
+// then body steps of NT tiles), so they all finish together whatever share of the issue slots
+// each of them gets.  `ring` is the CTA's dynamic shared memory: the per-warp cp.async stages while
+// tiles stream, then the warps' outputs.
+template <int BITS>
+__device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long long u_lo, long long u_hi,
+                                            float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint8_t *ring) {
+  using F = Fmt<BITS>;
+  using F16 = Fmt<16>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
-  const int slice = blockIdx.y;
   const int b = slice / p.kv_heads, hkv = slice % p.kv_heads;
-  const bool aux = (blockIdx.x == 0);
+
+  // (the previous segment ended with a CTA-wide barrier after its last use of s_q / s_stat / s_ctr / ring)
+  if (tid == 0) s_ctr[0] = s_ctr[1] = 0;
+  __syncthreads();
+
+  // ranges of this segment: INT16 tiles [a_lo, a_hi) (a tile belongs to the segment that holds its
+  // first unit) and body tiles [t_lo, t_hi)
+  int a_lo = 0, a_hi = 0, t_lo = 0, t_hi = 0;
+  if (u_lo < p.units_aux) {
+    a_lo = (int)((max(u_lo - p.units_lead, 0ll) + p.w16 - 1) / p.w16);
+    a_hi = (int)((min(u_hi, p.units_aux) - p.units_lead + p.w16 - 1) / p.w16);
+  }
+  if (u_hi > p.units_aux) {
+    t_lo = (int)(max(u_lo, p.units_aux) - p.units_aux);
+    t_hi = (int)(u_hi - p.units_aux);
+  }
+  const uint8_t *slice_base = p.geom.base + (size_t)slice * p.geom.slice_stride;
+
+  // ---- body stream set-up: claim the first steps and start their copies before anything else ----
+  constexpr int TB = tile_bytes(BITS);
+  constexpr int NT = F::NT, S = F::SLOTS > 0 ? F::SLOTS : 1, SB = NT * TB;
+  const int n_steps = (t_hi - t_lo + NT - 1) / NT;
+  const uint8_t *body = slice_base + p.geom.body_off;
+  uint8_t *my_ring = ring + (size_t)warp * S * SB;
+  const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
+  auto claim = [&](int which) { return claim_next(s_ctr + which, lane); };
+  auto issue = [&](int j, int slot) {
+    const int t = t_lo + NT * j;
+    const uint8_t *src = body + (size_t)t * TB + lane * 16;
+    const uint32_t dst = ring_addr + slot * SB + lane * 16;
+    const int n_tiles = t_hi - t;
+    if ((SB / 16) % 32 == 0 && n_tiles >= NT) {  // whole step, every lane copies the same number of chunks
+      cp_async_run<SB / 512>(dst, src);
+    } else {
+      const int n_chunks = min(NT, n_tiles) * (TB / 16);
+#pragma unroll
+      for (int c = 0; c < (SB / 16 + 31) / 32; ++c)
+        if (c * 32 + lane < n_chunks) cp_async16(dst + c * 512, src + c * 512);
+    }
+  };
+  int pending[S];  // steps claimed and in flight, oldest first (>= n_steps: none)
+  if constexpr (F::SLOTS > 0) {
+#pragma unroll
+    for (int i = 0; i < S - 1; ++i) {
+      pending[i] = n_steps > 0 ? claim(1) : 0;
+      if (pending[i] < n_steps) issue(pending[i], i);
+      cp_async_commit();
+    }
+  }
 
   // ---- Q'' = Q * lambda * sm_scale * log2(e)  (Eq. 9: the equalization scale migrates into Q) ----
-  {
-    const float lam = p.lambda[hkv * kHeadDim + tid];
-    for (int h = 0; h < kMaxGroup; ++h) {
-      float v = 0.f;
-      if (h < p.group) {
-        const uint16_t raw = p.Q[((size_t)b * p.q_heads + hkv * p.group + h) * kHeadDim + tid];
-        v = __fmul_rn(__fmul_rn(__uint_as_float((uint32_t)raw << 16), lam), p.qk_scale);
-      }
-      s_q[h][tid] = v;
+  for (int i = tid; i < kMaxGroup * kHeadDim; i += kAttnThreads) {
+    const int h = i >> 7, ch = i & 127;
+    float v = 0.f;
+    if (h < p.group) {
+      const uint16_t raw = p.Q[((size_t)b * p.q_heads + hkv * p.group + h) * kHeadDim + ch];
+      v = __fmul_rn(__fmul_rn(__uint_as_float((uint32_t)raw << 16), p.lambda[hkv * kHeadDim + ch]), p.qk_scale);
     }
+    s_q[h][ch] = v;
   }
   __syncthreads();
-  for (int h = warp; h < kMaxGroup; h += 4) {  // per-head max |q''| and sum q''
-    const float4 v = *reinterpret_cast<const float4 *>(&s_q[h][lane * 4]);
+
+  if (warp < kMaxGroup) {  // per-head max |q''| and sum q''
+    const float4 v = *reinterpret_cast<const float4 *>(&s_q[warp][lane * 4]);
     float mx = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
     float sm = (v.x + v.y) + (v.z + v.w);
 #pragma unroll
@@ -317,65 +492,50 @@ __device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadD
     if (lane == 0) {
       int e = 0;
       if (mx > 0.f) frexpf(mx, &e);  // mx = f * 2^e, f in [0.5, 1)
-      s_stat[h] = (float)e;
-      s_stat[8 + h] = sm;
+      s_stat[warp] = (float)e;
+      s_stat[8 + warp] = sm;
     }
   }
   __syncthreads();
   const int e_g = (int)s_stat[g];
   const float sumq = s_stat[8 + g];
-  const float mu = ldexpf(1.0f, 24 - F::E + e_g);
 
-  uint32_t qa[8][4];
-#pragma unroll
-  for (int s = 0; s < 8; ++s) {
-#pragma unroll
-    for (int beta = 0; beta < 2; ++beta) {
-      const int W = 2 * s + beta;
-      const float scl = ldexpf(1.0f, F::E - F::pos(W % F::N) - e_g);
-      const int c0 = 16 * s + 8 * beta + 2 * tig;
-      const float x0 = s_q[g][c0] * scl, x1 = s_q[g][c0 + 1] * scl;
-      const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
-      const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
-      const __half2 hi = __halves2half2(h0, h1), lo = __halves2half2(l0, l1);
-      qa[s][2 * beta] = *reinterpret_cast<const uint32_t *>(&hi);
-      qa[s][2 * beta + 1] = *reinterpret_cast<const uint32_t *>(&lo);
-    }
-  }
-
-  // ---- unit of the V accumulators: a power of two >= every V scale of this slice at this width ----
-  float sigma_u = 1.0f;
+  // ---- unit of the V accumulators: a power of two >= every INT16 V scale of this slice; at width b
+  //      the scales are at most 2^SIGMA_LOG2 times larger ----
+  float sigma16 = 1.0f;
   {
     const float s16 = __uint_as_float(p.vmax_bits[slice]);
     if (s16 > 0.f) {
       int e;
       frexpf(s16, &e);
-      sigma_u = ldexpf(1.0f, e + F::SIGMA_LOG2);
+      sigma16 = ldexpf(1.0f, e);
     }
   }
-  const float inv_sigma_e = ldexpf(1.0f, F::E) / sigma_u;
 
   WarpState st;
   st.m = kNegBig; st.l = 0.f; st.zs = 0.f;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
+  uint32_t qa[8][4];
 
-  const uint8_t *slice_base = p.geom.base + (size_t)slice * p.geom.slice_stride;
-  if (aux) {
-    if constexpr (BITS == 16) {
-      const int sink_tiles = (p.n_sink_eff + 15) >> 4;
-      const int ring_tiles = p.geom.ring_tokens >> 4;
+  // ---- INT16 tiles (sink + window ring) ----
+  if (a_hi > a_lo) {
+    int it = a_lo + claim(0);
+    if (it < a_hi) {
+      build_q_fragments<16>(qa, s_q, e_g, g, tig);
+      const float mu = ldexpf(1.0f, 24 - F16::EQ + e_g);
+      const float inv_sigma_e = ldexpf(1.0f, F16::EP) / sigma16;
       const int n_win = p.n_tokens - p.win_start;
-      const int first_slot = (p.win_start - p.geom.n_sink) % p.geom.ring_tokens;  // win_start >= n_sink when n_win > 0
-      for (int it = warp; it < sink_tiles + ring_tiles; it += 4) {
+      const int first_slot = n_win > 0 ? (p.win_start - p.geom.n_sink) % p.geom.ring_tokens : 0;
+      do {
         uint32_t mask = 0;
         const uint8_t *tile;
-        if (it < sink_tiles) {
-          const int live = min(16, p.n_sink_eff - 16 * it);
+        if (it < p.sink_tiles) {
+          const int live = max(0, min(16, p.n_sink_eff - 16 * it));
           mask = (1u << live) - 1u;
           tile = slice_base + (size_t)it * tile_bytes(16);
         } else {
-          const int rt = it - sink_tiles;
+          const int rt = it - p.sink_tiles;
           tile = slice_base + p.geom.ring_off + (size_t)rt * tile_bytes(16);
           if (n_win > 0) {
             for (int r = 0; r < 16; ++r) {
@@ -385,72 +545,83 @@ __device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadD
             }
           }
         }
-        if (mask == 0xFFFFu) process_tile<16, false>(tile, mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
-        else if (mask) process_tile<16, true>(tile, mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
-      }
-    }
-  } else {
-    const int split = blockIdx.x - 1;
-    const int t0 = split * p.tiles_per_split;
-    const int t1 = min(p.body_tiles, t0 + p.tiles_per_split);
-    const uint8_t *body = slice_base + p.geom.body_off;
-    const uint32_t tail_mask = (p.n_body & 15) ? (1u << (p.n_body & 15)) - 1u : 0xFFFFu;
-    if constexpr (F::STAGES == 0) {
-      for (int t = t0 + warp; t < t1; t += 4) {
-        const uint8_t *tile = body + (size_t)t * tile_bytes(BITS);
-        if (t == p.body_tiles - 1 && tail_mask != 0xFFFFu)
-          process_tile<BITS, true>(tile, tail_mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
-        else
-          process_tile<BITS, false>(tile, 0xFFFFu, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
-      }
-    } else {
-      // per-warp ring of STAGES tiles; tile i of this warp is body tile t0 + warp + 4 i
-      constexpr int TB = tile_bytes(BITS);
-      constexpr int S = F::STAGES;
-      uint8_t *my_ring = ring + (size_t)warp * S * TB;
-      const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
-      const int n_my = (t1 - t0 - warp + 3) >> 2;
-      const uint8_t *src0 = body + (size_t)(t0 + warp) * TB + lane * 16;
-      auto issue = [&](int i, int stage) {
-        const uint8_t *src = src0 + (size_t)i * 4 * TB;
-        const uint32_t dst = ring_addr + stage * TB + lane * 16;
+        if (mask == 0xFFFFu) process_tiles<16, 1, false>(tile, mask, st, qa, mu, sumq, inv_sigma_e, lane);
+        else if (mask) process_tiles<16, 1, true>(tile, mask, st, qa, mu, sumq, inv_sigma_e, lane);
+        it = a_lo + claim(0);
+      } while (it < a_hi);
+      if constexpr (BITS != 16) {
+        // accumulator units change with the width: INT16 units -> body units (exact powers of two)
 #pragma unroll
-        for (int c = 0; c < (TB / 16 + 31) / 32; ++c)
-          if (c * 32 + lane < TB / 16) cp_async16(dst + c * 512, src + c * 512);
-      };
+        for (int mt = 0; mt < 8; ++mt) {
 #pragma unroll
-      for (int i = 0; i < S - 1; ++i) {
-        if (i < n_my) issue(i, i);
-        cp_async_commit();
-      }
-      int stage = 0, fill = S - 1;
-      for (int i = 0; i < n_my; ++i) {
-        if (i + S - 1 < n_my) issue(i + S - 1, fill);
-        cp_async_commit();
-        cp_async_wait<S - 1>();
-        __syncwarp();
-        const uint8_t *tile = my_ring + stage * TB;
-        if (t0 + warp + 4 * i == p.body_tiles - 1 && tail_mask != 0xFFFFu)
-          process_tile<BITS, true>(tile, tail_mask, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
-        else
-          process_tile<BITS, false>(tile, 0xFFFFu, st, qa, mu, sumq, sigma_u, inv_sigma_e, lane);
-        __syncwarp();
-        fill = stage;
-        stage = (stage + 1 == S) ? 0 : stage + 1;
+          for (int rr = 0; rr < 2; ++rr) {
+            const float f = ldexpf(1.0f, F::EP - F16::EP + F::pos((2 * mt + rr) % F::N) - F::SIGMA_LOG2);
+            st.acc[mt][2 * rr] *= f;
+            st.acc[mt][2 * rr + 1] *= f;
+          }
+        }
       }
     }
   }
+
+  // ---- body tiles ----
+  const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
+  if (n_steps > 0) {
+    build_q_fragments<BITS>(qa, s_q, e_g, g, tig);
+    const float mu = ldexpf(1.0f, 24 - F::EQ + e_g);
+    const float inv_sigma_e = ldexpf(1.0f, F::EP) / sigma_u;
+    const uint32_t tail_mask = (p.n_body & 15) ? (1u << (p.n_body & 15)) - 1u : 0xFFFFu;
+    const int tail_tile = tail_mask != 0xFFFFu ? p.body_tiles - 1 : -1;  // the one tile with dead rows
+    if constexpr (F::SLOTS == 0) {
+      for (int t = t_lo + claim(1); t < t_hi; t = t_lo + claim(1)) {
+        const uint8_t *tile = body + (size_t)t * TB;
+        if (t == tail_tile) process_tiles<BITS, 1, true>(tile, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
+        else process_tiles<BITS, 1, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+      }
+    } else {
+      int slot = 0, fill = S - 1;
+      while (pending[0] < n_steps) {
+        const int nxt = claim(1);
+        if (nxt < n_steps) issue(nxt, fill);
+        cp_async_commit();
+        cp_async_wait<S - 1>();
+        __syncwarp();
+        const uint8_t *tile = my_ring + slot * SB;
+        const int t = t_lo + NT * pending[0];
+        if (NT == 2 && t + 1 < t_hi && t + 1 != tail_tile) {
+          process_tiles<BITS, NT, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+        } else {
+#pragma unroll
+          for (int k = 0; k < NT; ++k) {
+            if (t + k >= t_hi) break;
+            if (t + k == tail_tile)
+              process_tiles<BITS, 1, true>(tile + k * TB, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
+            else
+              process_tiles<BITS, 1, false>(tile + k * TB, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+          }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i + 2 < S; ++i) pending[i] = pending[i + 1];
+        pending[S - 2] = nxt;
+        fill = slot;
+        slot = (slot + 1 == S) ? 0 : slot + 1;
+      }
+    }
+  }
+  if constexpr (F::SLOTS > 0) cp_async_wait<0>();
 
   // ---- warp epilogue: quad sums, real units, to shared memory (the ring is free now) ----
   st.l += __shfl_xor_sync(0xffffffffu, st.l, 1);
   st.l += __shfl_xor_sync(0xffffffffu, st.l, 2);
   st.zs += __shfl_xor_sync(0xffffffffu, st.zs, 1);
   st.zs += __shfl_xor_sync(0xffffffffu, st.zs, 2);
-  __syncthreads();  // every warp is done with its stages; s_stat is reused below
+  __syncthreads();  // every warp is done with its stages
   float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(ring);
+  float *s_m = s_stat + 16, *s_l = s_stat + 16 + kAttnWarps * kMaxGroup;
   if (tig == 0) {
-    s_stat[16 + warp * 8 + g] = st.m;
-    s_stat[48 + warp * 8 + g] = st.l;
+    s_m[warp * 8 + g] = st.m;
+    s_l[warp * 8 + g] = st.l;
   }
   const float zs0 = __shfl_sync(0xffffffffu, st.zs, (2 * tig) * 4);
   const float zs1 = __shfl_sync(0xffffffffu, st.zs, (2 * tig + 1) * 4);
@@ -459,7 +630,7 @@ __device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadD
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
       const int J = 2 * mt + rr;
-      const float f = ldexpf(sigma_u, 24 - F::E - F::pos(J % F::N));
+      const float f = ldexpf(sigma_u, 24 - F::EP - F::pos(J % F::N));
       const int ch = 16 * mt + 8 * rr + g;
       s_o[warp][2 * tig][ch] = fmaf(st.acc[mt][2 * rr], f, zs0);
       s_o[warp][2 * tig + 1][ch] = fmaf(st.acc[mt][2 * rr + 1], f, zs1);
@@ -467,51 +638,68 @@ __device__ __forceinline__ void run_cta(const AttnParams &p, float (*s_q)[kHeadD
   }
   __syncthreads();
 
-  // ---- merge the 4 warps, publish the CTA's partial ----
-  float *part = p.partials + ((size_t)slice * (1 + p.body_splits) + blockIdx.x) * kMaxGroup * kPartialStride;
-  for (int h = 0; h < p.group; ++h) {
-    const float m0 = s_stat[16 + h], m1 = s_stat[24 + h], m2 = s_stat[32 + h], m3 = s_stat[40 + h];
-    const float M = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-    const float w0 = ex2(m0 - M), w1 = ex2(m1 - M), w2 = ex2(m2 - M), w3 = ex2(m3 - M);
-    const float o = w0 * s_o[0][h][tid] + w1 * s_o[1][h][tid] + w2 * s_o[2][h][tid] + w3 * s_o[3][h][tid];
-    __stcg(part + h * kPartialStride + 4 + tid, o);
-    if (tid == 0) {
+  // ---- merge the warps, publish the segment's partial ----
+  float *part = p.partials + (size_t)(blockIdx.x + slice) * kMaxGroup * kPartialStride;
+  for (int i = tid; i < p.group * kHeadDim; i += kAttnThreads) {
+    const int h = i >> 7, ch = i & 127;
+    float M = kNegBig;
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, s_m[w * 8 + h]);
+    float o = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) {
+      const float wt = ex2(s_m[w * 8 + h] - M);
+      o = fmaf(wt, s_o[w][h][ch], o);
+      l = fmaf(wt, s_l[w * 8 + h], l);
+    }
+    __stcg(part + h * kPartialStride + 4 + ch, o);
+    if (ch == 0) {
       __stcg(part + h * kPartialStride, M);
-      __stcg(part + h * kPartialStride + 1,
-             w0 * s_stat[48 + h] + w1 * s_stat[56 + h] + w2 * s_stat[64 + h] + w3 * s_stat[72 + h]);
+      __stcg(part + h * kPartialStride + 1, l);
     }
   }
 
-  // ---- the last CTA of the slice to get here merges the slice (ticket, nobody waits) ----
+  // ---- the segment that publishes the slice's last partial merges the slice (nobody waits) ----
   __threadfence();
   __syncthreads();
   if (tid == 0) {
+    int cf, cl;
+    slice_ctas(p, slice, cf, cl);
     const unsigned t = atomicAdd(p.tickets + slice, 1u);
-    s_stat[79] = (t == (unsigned)p.body_splits) ? 1.f : 0.f;  // 1 + body_splits CTAs per slice
+    s_ctr[2] = (t + 1u == (unsigned)(cl - cf + 1)) ? 1 : 0;
   }
   __syncthreads();
-  if (s_stat[79] != 0.f) {
+  if (s_ctr[2]) {
     __threadfence();
-    combine_slice(p, slice, s_stat + 80);
+    combine_slice(p, slice);
     if (tid == 0) p.tickets[slice] = 0u;  // ready for the next launch (stream order)
   }
+  __syncthreads();  // s_q, s_stat, s_ctr and the ring may be reused
 }
 
-constexpr int attn_ring_bytes(int bits) {
-  // per-warp stages while streaming; at least the 16 KB of warp outputs they are reused for
-  return bits == 16 ? 4 * kMaxGroup * kHeadDim * 4
-                    : (4 * (bits == 8 ? 3 : 4) * tile_bytes(bits) > 4 * kMaxGroup * kHeadDim * 4
-                           ? 4 * (bits == 8 ? 3 : 4) * tile_bytes(bits)
-                           : 4 * kMaxGroup * kHeadDim * 4);
+template <int BITS>
+constexpr int attn_ring_bytes() {
+  // per-warp stages while streaming; at least the warps' outputs they are reused for
+  constexpr int out_bytes = kAttnWarps * kMaxGroup * kHeadDim * 4;
+  constexpr int ring = kAttnWarps * Fmt<BITS>::SLOTS * Fmt<BITS>::NT * tile_bytes(BITS);
+  return ring > out_bytes ? ring : out_bytes;
 }
 
 template <int BODY_BITS>
-__global__ void __launch_bounds__(128, 4) decode_attn_splitk_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(const AttnParams p) {
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
-  __shared__ float s_stat[80 + 72];  // head stats, warp stats, ticket flag, combine weights (<= 65 CTAs)
+  __shared__ float s_stat[16 + 2 * kAttnWarps * kMaxGroup];  // head stats, per-warp (m, l)
+  __shared__ int s_ctr[4];                                    // work counters (INT16 tiles, body steps), combine flag
   extern __shared__ __align__(128) uint8_t ring[];
-  if (blockIdx.x == 0) run_cta<16>(p, s_q, s_stat, ring);
-  else run_cta<BODY_BITS>(p, s_q, s_stat, ring);
+  const long long u_begin = (long long)blockIdx.x * p.units_per_cta;
+  const long long u_end = min(u_begin + p.units_per_cta, p.units_total);
+  for (long long u = u_begin; u < u_end;) {
+    const int slice = (int)(u / p.units_slice);
+    const long long base = (long long)slice * p.units_slice;
+    const long long hi = min(u_end - base, p.units_slice);
+    if (hi > p.units_lead) run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, ring);
+    u = base + hi;
+  }
 }
 
 }  // namespace pmkvq

@@ -20,8 +20,9 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kHeadTiles = 8;     // tiles the reduce handles in order before the parallel waves start
-constexpr int kTargetCtas = 1184;  // 148 SMs x 4 resident CTAs of 128 threads x 2 waves
-constexpr int kMaxSplits = 64;      // upper bound on body CTAs per slice (sizes the partials workspace)
+constexpr int kMaxCtas = 2048;      // upper bound on the attention grid (sizes the partials workspace)
+constexpr int kSegmentCostBytes = 40 * 1024;  // set-up + merge + publish of one segment, in streamed bytes
+constexpr int kMinUnitsPerCta = 32;  // do not cut the work finer than two tiles per warp
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool valid_bits(int b) { return b == 2 || b == 4 || b == 8 || b == 16; }
@@ -46,7 +47,8 @@ struct pmkvq_cache {
   size_t arena_bytes;
   // arena sections
   size_t off_lambda, off_inv_lambda, off_vmax, off_tickets, off_partials, partial_bytes;
-  int sink_tiles, ring_tiles, max_splits, auto_splits, user_splits;
+  int sink_tiles, ring_tiles, user_ctas;
+  int resident_ctas[4];  // one wave of the attention kernel at body width 16, 8, 4, 2
   uint64_t launches = 0;  // kernels launched so far
   std::vector<Layer> L;
 
@@ -111,9 +113,7 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.sm_scale = c->sm_scale > 0.0f ? c->sm_scale : 1.0f / std::sqrt((float)kHeadDim);
   k.sink_tiles = (k.n_sink + 15) / 16;
   k.ring_tiles = std::max(1, (k.window + k.evict_chunk - 1 + 15) / 16 + 1);
-  k.max_splits = kMaxSplits;
-  k.auto_splits = std::min(kMaxSplits, std::max(1, (kTargetCtas + k.n_slices - 1) / k.n_slices));
-  k.user_splits = 0;
+  k.user_ctas = 0;
 
   size_t off = 0;
   const size_t lam_bytes = (size_t)k.layers * k.kv_heads * kHeadDim * sizeof(float);
@@ -121,7 +121,7 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.off_inv_lambda = off; off = align_up(off + lam_bytes, kAlign);
   k.off_vmax = off; off = align_up(off + (size_t)k.layers * k.n_slices * sizeof(unsigned), kAlign);
   k.off_tickets = off; off = align_up(off + (size_t)k.n_slices * sizeof(unsigned), kAlign);
-  k.partial_bytes = (size_t)k.n_slices * (1 + k.max_splits) * kMaxGroup * kPartialStride * sizeof(float);
+  k.partial_bytes = ((size_t)kMaxCtas + 2 * (size_t)k.n_slices) * kMaxGroup * kPartialStride * sizeof(float);
   k.off_partials = off; off = align_up(off + k.partial_bytes, kAlign);
 
   k.L.assign(k.layers, Layer());
@@ -167,6 +167,30 @@ cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStr
     lo = (int)hi;
   }
   return cudaGetLastError();
+}
+
+template <int BITS>
+cudaError_t attention_setup_one(int &resident, int sms) {
+  cudaError_t e = cudaFuncSetAttribute(decode_attn_splitk_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       attn_ring_bytes<BITS>());
+  int per_sm = 0;
+  if (e == cudaSuccess)
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_splitk_kernel<BITS>, kAttnThreads,
+                                                      attn_ring_bytes<BITS>());
+  resident = std::min(kMaxCtas, std::max(1, per_sm) * sms);
+  return e;
+}
+
+// Dynamic shared memory opt-in and the size of one wave of resident CTAs, per body width.
+cudaError_t attention_setup(pmkvq_cache *k) {
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = attention_setup_one<16>(k->resident_ctas[0], sms);
+  if (e == cudaSuccess) e = attention_setup_one<8>(k->resident_ctas[1], sms);
+  if (e == cudaSuccess) e = attention_setup_one<4>(k->resident_ctas[2], sms);
+  if (e == cudaSuccess) e = attention_setup_one<2>(k->resident_ctas[3], sms);
+  return e;
 }
 
 pmkvq_status do_reduce(pmkvq_cache *k, int layer, cudaStream_t st) {
@@ -221,9 +245,7 @@ pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
     e = cudaMemcpy(k->arena + k->off_inv_lambda, inv.data(), n_lam * sizeof(float), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_vmax, 0, (size_t)k->layers * k->n_slices * sizeof(unsigned));
   if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_tickets, 0, (size_t)k->n_slices * sizeof(unsigned));
-  if (e == cudaSuccess) {
-    e = cudaFuncSetAttribute(decode_attn_splitk_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_ring_bytes(8));
-  }
+  if (e == cudaSuccess) e = attention_setup(k);
   if (e != cudaSuccess) {
     delete k;
     return PMKVQ_ERR_CUDA;
@@ -309,19 +331,27 @@ pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d
   p.win_start = p.n_sink_eff + p.n_body;
   p.cur_bits = l.cur_bits;
   p.body_tiles = (p.n_body + 15) / 16;
-  // split the body: every CTA gets at least 8 tiles (2 per warp), at most max_splits CTAs per slice
-  int splits = std::min(k->user_splits > 0 ? k->user_splits : k->auto_splits, (p.body_tiles + 7) / 8);
-  splits = std::max(splits, p.body_tiles > 0 ? 1 : 0);
-  p.tiles_per_split = splits ? (p.body_tiles + splits - 1) / splits : 0;
-  if (splits) splits = (p.body_tiles + p.tiles_per_split - 1) / p.tiles_per_split;
-  p.body_splits = splits;
+  p.sink_tiles = k->sink_tiles;
+  p.aux_tiles = k->sink_tiles + k->ring_tiles;
+  p.n_slices = k->n_slices;
+  // one line of work units over all slices: a body tile is one unit, an INT16 tile their byte ratio
+  p.w16 = (tile_bytes(16) + tile_bytes(l.cur_bits) - 1) / tile_bytes(l.cur_bits);
+  // a segment costs about as much as streaming 40 KB: every slice starts with that many empty units
+  p.units_lead = kSegmentCostBytes / tile_bytes(l.cur_bits);
+  p.units_aux = p.units_lead + (long long)p.aux_tiles * p.w16;
+  p.units_slice = p.units_aux + p.body_tiles;
+  p.units_total = p.units_slice * k->n_slices;
+  const int width_idx = l.cur_bits == 16 ? 0 : l.cur_bits == 8 ? 1 : l.cur_bits == 4 ? 2 : 3;
+  const int want = k->user_ctas > 0 ? k->user_ctas : k->resident_ctas[width_idx];
+  long long per = std::max<long long>((p.units_total + want - 1) / want, k->user_ctas > 0 ? 1 : kMinUnitsPerCta);
+  p.units_per_cta = per;
+  const unsigned n_ctas = (unsigned)((p.units_total + per - 1) / per);
   p.qk_scale = k->sm_scale * 1.4426950408889634f;
-  dim3 grid(1 + splits, k->n_slices);
   switch (l.cur_bits) {
-    case 16: decode_attn_splitk_kernel<16><<<grid, 128, attn_ring_bytes(16), st>>>(p); break;
-    case 8: decode_attn_splitk_kernel<8><<<grid, 128, attn_ring_bytes(8), st>>>(p); break;
-    case 4: decode_attn_splitk_kernel<4><<<grid, 128, attn_ring_bytes(4), st>>>(p); break;
-    default: decode_attn_splitk_kernel<2><<<grid, 128, attn_ring_bytes(2), st>>>(p); break;
+    case 16: decode_attn_splitk_kernel<16><<<n_ctas, kAttnThreads, attn_ring_bytes<16>(), st>>>(p); break;
+    case 8: decode_attn_splitk_kernel<8><<<n_ctas, kAttnThreads, attn_ring_bytes<8>(), st>>>(p); break;
+    case 4: decode_attn_splitk_kernel<4><<<n_ctas, kAttnThreads, attn_ring_bytes<4>(), st>>>(p); break;
+    default: decode_attn_splitk_kernel<2><<<n_ctas, kAttnThreads, attn_ring_bytes<2>(), st>>>(p); break;
   }
   k->launches += 1;
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
@@ -403,9 +433,9 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
   return PMKVQ_OK;
 }
 
-pmkvq_status pmkvq_set_attention_splits(pmkvq_cache *k, int32_t splits) {
-  if (!k || splits < 0 || splits > kMaxSplits) return PMKVQ_ERR_INVALID_ARG;
-  k->user_splits = splits;
+pmkvq_status pmkvq_set_attention_ctas(pmkvq_cache *k, int32_t n_ctas) {
+  if (!k || n_ctas < 0 || n_ctas > kMaxCtas) return PMKVQ_ERR_INVALID_ARG;
+  k->user_ctas = n_ctas;
   return PMKVQ_OK;
 }
 

@@ -141,12 +141,14 @@ def test_split_invariance():
     m.append(0, k, v)
     q = synth.make_q(6, 0, 0, batch, group * kvh, n)
     outs = []
-    for s in (1, 2, 3, 7, 64, 0):
-        m.cache.set_attention_splits(s)
+    for s in (1, 2, 3, 7, 64, 333, 2048, 0):
+        m.cache.set_attention_ctas(s)
         m.check_attention(0, q)
         outs.append(m.cache.decode_attention(0, q.cuda()).cpu().numpy())
+    # partitions differ only by fp32 summation order and by where the fp16 rounding of p * S_V falls
+    # (relative 2^-12 per token, not averaged out when one token dominates the softmax)
     for o in outs[1:]:
-        assert np.abs(o - outs[0]).max() < 2e-4
+        assert np.abs(o - outs[0]).max() < 6e-4 * max(1.0, float(np.abs(outs[0]).max()))
 
 
 def test_degenerate_values():
