@@ -95,6 +95,17 @@ pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *cache, int32_t layer, void *s
 pmkvq_status pmkvq_decode_attention(pmkvq_cache *cache, int32_t layer, const void *d_Q_bf16, float *d_out,
                                     void *stream);
 
+/* One decode step of the whole model's attention path (Sec. 3.4, inference stage): for every block in
+ * order, pmkvq_append of one new token followed by pmkvq_decode_attention; everything is enqueued on
+ * `stream` without a host synchronisation.
+ *   d_K_bf16, d_V_bf16: DEVICE bf16 [layers][batch][kv_heads][128]
+ *   d_Q_bf16:           DEVICE bf16 [layers][batch][q_heads][128]
+ *   d_out:              DEVICE fp32 [layers][batch][q_heads][128]
+ * Stops at the first block whose call fails and returns its status; earlier blocks keep their new
+ * token.  With auto_reduce = 0 a block whose budget is full returns PMKVQ_ERR_BUDGET_FULL here. */
+pmkvq_status pmkvq_decode_step(pmkvq_cache *cache, const void *d_K_bf16, const void *d_V_bf16, const void *d_Q_bf16,
+                               float *d_out, void *stream);
+
 /* Split-K tuning of pmkvq_decode_attention (flash-decoding partition over the sequence): the tiles
  * of all (batch, kv_head) slices are cut into `n_ctas` equal contiguous pieces, one per CTA
  * (1..2048); 0 restores the default, one wave of resident CTAs on the GPU's SMs. */

@@ -55,6 +55,8 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_progressive_reduce.argtypes = [vp, i32, vp]
     lib.pmkvq_decode_attention.restype = i32
     lib.pmkvq_decode_attention.argtypes = [vp, i32, vp, vp, vp]
+    lib.pmkvq_decode_step.restype = i32
+    lib.pmkvq_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.pmkvq_set_attention_ctas.restype = i32
     lib.pmkvq_set_attention_ctas.argtypes = [vp, i32]
     lib.pmkvq_layer_state.restype = i32
@@ -168,6 +170,24 @@ class Cache:
         st = lib().pmkvq_decode_attention(self._h, layer, q.data_ptr(), out.data_ptr(), _stream_ptr(stream))
         if st != OK:
             raise PmkvqError(st, "pmkvq_decode_attention")
+        return out
+
+    def decode_step(self, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                    stream=None):
+        """One decode step over all blocks.  k, v: bf16 [layers, batch, kv_heads, 128]; q: bf16
+        [layers, batch, q_heads, 128] -> fp32 [layers, batch, q_heads, 128]."""
+        self._check(k, torch.bfloat16, "k"); self._check(v, torch.bfloat16, "v"); self._check(q, torch.bfloat16, "q")
+        if (k.numel() != self.layers * self.batch * self.kv_heads * 128 or v.numel() != k.numel()
+                or q.numel() != self.layers * self.batch * self.q_heads * 128):
+            raise ValueError("bad K/V/Q shape")
+        if out is None:
+            out = torch.empty(self.layers, self.batch, self.q_heads, 128, dtype=torch.float32, device=q.device)
+        self._check(out, torch.float32, "out")
+        if out.numel() != q.numel():
+            raise ValueError("bad out shape")
+        st = lib().pmkvq_decode_step(self._h, k.data_ptr(), v.data_ptr(), q.data_ptr(), out.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_decode_step")
         return out
 
     def set_attention_ctas(self, n_ctas: int):

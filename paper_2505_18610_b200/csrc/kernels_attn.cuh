@@ -107,6 +107,11 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -285,18 +290,28 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
     }
     st.m = m_new;
   }
+  // w = p * S_V goes to the tensor cores as one fp16; the probability that enters the denominator and
+  // the zero-point sum is that rounded w divided by the scale again, so numerator and denominator
+  // see the same (slightly perturbed) probabilities and the rounding cancels where it matters most,
+  // when a few tokens carry the whole softmax.
   uint32_t pb[2 * NT];
   {
-    float wv[NS];
+    float wv[NS], rs[NS];
 #pragma unroll
     for (int i = 0; i < NS; ++i) {
-      const float p = ex2(sc[i] - st.m);
-      st.l += p;
-      st.zs = fmaf(p, zv[i], st.zs);
-      wv[i] = p * (sv[i] * inv_sigma_e);  // p * S_V / sigma_u * 2^EP
+      // a constant V group has S_V = 0 and all codes 0: any finite unit will do for it
+      const float s_e = fmaf(sv[i], inv_sigma_e, sv[i] == 0.f ? 1.f : 0.f);  // S_V / sigma_u * 2^EP
+      rs[i] = rcp_approx(s_e);
+      wv[i] = ex2(sc[i] - st.m) * s_e;
     }
 #pragma unroll
-    for (int j = 0; j < 2 * NT; ++j) pb[j] = pack_half2(wv[2 * j], wv[2 * j + 1]);
+    for (int j = 0; j < 2 * NT; ++j) {
+      pb[j] = pack_half2(wv[2 * j], wv[2 * j + 1]);
+      const float2 wf = __half22float2(*reinterpret_cast<const __half2 *>(&pb[j]));
+      const float p0 = wf.x * rs[2 * j], p1 = wf.y * rs[2 * j + 1];
+      st.l += p0 + p1;
+      st.zs = fmaf(p0, zv[2 * j], fmaf(p1, zv[2 * j + 1], st.zs));
+    }
   }
 
   // ---- output: O^T += V^T w, channels on M, tokens on K, heads on N ----

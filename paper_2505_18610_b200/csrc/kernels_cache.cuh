@@ -101,15 +101,10 @@ __device__ __forceinline__ void load_token16(const uint8_t *part, int row, uint1
 // channels of the token; Keys are first multiplied by Lambda^-1 (Eq. 9).  The token goes to the
 // sink, straight to the body (bulk appends; Eq. 3 chain to the body width) or to the window ring.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
-                                                     const float *__restrict__ inv_lambda, unsigned *vmax_bits,
-                                                     LayerGeom geom, int n_new, int n_slices, int kv_heads,
-                                                     int n_old, int win_start, int cur_bits) {
-  __shared__ uint16_t s_codes[4][kHeadDim];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long wid = (long long)blockIdx.x * 4 + warp;
-  const long long total = (long long)n_new * n_slices * 2;
-  if (wid >= total) return;
+__device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int lane, const uint16_t *__restrict__ K,
+                                           const uint16_t *__restrict__ V, const float *__restrict__ inv_lambda,
+                                           unsigned *vmax_bits, const LayerGeom &geom, int n_slices, int kv_heads,
+                                           int n_old, int win_start, int cur_bits) {
   const int is_value = (int)(wid & 1);
   const long long ts = wid >> 1;
   const int slice = (int)(ts % n_slices);
@@ -143,12 +138,12 @@ __global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict_
       c = __float2int_rn(__fdiv_rn(__fsub_rn(x[e], mn), scale));
       c = min(max(c, 0), 65535);
     }
-    s_codes[warp][lane * 4 + e] = (uint16_t)c;
+    codes[lane * 4 + e] = (uint16_t)c;
   }
   __syncwarp();
   uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
   const TokenDest d = token_dest(geom, slice_base, n_old + i, win_start, cur_bits);
-  store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, s_codes[warp], is_value, lane);
+  store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, codes, is_value, lane);
   if (lane == 0) {
     float *meta = reinterpret_cast<float *>(d.tile + meta_offset(d.bits));
     meta[meta_slot(is_value ? 2 : 0, d.row) >> 2] = chain_scale(scale, d.bits);
@@ -157,17 +152,23 @@ __global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict_
   }
 }
 
+__global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
+                                                     const float *__restrict__ inv_lambda, unsigned *vmax_bits,
+                                                     LayerGeom geom, int n_new, int n_slices, int kv_heads,
+                                                     int n_old, int win_start, int cur_bits) {
+  __shared__ uint16_t s_codes[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wid = (long long)blockIdx.x * 4 + warp;
+  if (wid >= (long long)n_new * n_slices * 2) return;
+  append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Window eviction.  One warp per (evicted token, slice, K|V): the INT16 token leaves the ring and
 // enters the body at the body width through the Eq. 3 chain (16 -> 8 -> ... -> cur_bits).
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) evict_kernel(LayerGeom geom, int n_slices, int first_token, int n_evict,
-                                                    int cur_bits) {
-  __shared__ uint16_t s_codes[4][kHeadDim];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long wid = (long long)blockIdx.x * 4 + warp;
-  const long long total = (long long)n_evict * n_slices * 2;
-  if (wid >= total) return;
+__device__ __forceinline__ void evict_one(long long wid, uint16_t *codes, int lane, const LayerGeom &geom, int n_slices,
+                                          int first_token, int cur_bits) {
   const int is_value = (int)(wid & 1);
   const long long ts = wid >> 1;
   const int slice = (int)(ts % n_slices);
@@ -176,18 +177,48 @@ __global__ void __launch_bounds__(128) evict_kernel(LayerGeom geom, int n_slices
   const int rp = (t - geom.n_sink) % geom.ring_tokens;
   const uint8_t *src_tile = slice_base + geom.ring_off + (size_t)(rp >> 4) * tile_bytes(16);
   const int src_row = rp & 15;
-  load_token16(src_tile + (is_value ? v_part_offset(16) : 0), src_row, s_codes[warp], is_value, lane);
+  load_token16(src_tile + (is_value ? v_part_offset(16) : 0), src_row, codes, is_value, lane);
   const float *smeta = reinterpret_cast<const float *>(src_tile + meta_offset(16));
   const float s16 = smeta[meta_slot(is_value ? 2 : 0, src_row) >> 2];
   const float z = smeta[meta_slot(is_value ? 3 : 1, src_row) >> 2];
   __syncwarp();
   const int j = t - geom.n_sink;
   uint8_t *dst_tile = slice_base + geom.body_off + (size_t)(j >> 4) * tile_bytes(cur_bits);
-  store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, s_codes[warp], is_value, lane);
+  store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, codes, is_value, lane);
   if (lane == 0) {
     float *meta = reinterpret_cast<float *>(dst_tile + meta_offset(cur_bits));
     meta[meta_slot(is_value ? 2 : 0, j & 15) >> 2] = chain_scale(s16, cur_bits);
     meta[meta_slot(is_value ? 3 : 1, j & 15) >> 2] = z;
+  }
+}
+
+__global__ void __launch_bounds__(128) evict_kernel(LayerGeom geom, int n_slices, int first_token, int n_evict,
+                                                    int cur_bits) {
+  __shared__ uint16_t s_codes[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wid = (long long)blockIdx.x * 4 + warp;
+  if (wid >= (long long)n_evict * n_slices * 2) return;
+  evict_one(wid, s_codes[warp], lane, geom, n_slices, first_token, cur_bits);
+}
+
+// One decode step's cache update in a single launch: the tokens that leave the window (warps
+// [0, 2 n_evict n_slices)) and the one new token (the rest).  Only valid when no evicted token
+// shares its ring slot with the new token, which holds for single-token appends (the ring is larger
+// than window + evict_chunk).
+__global__ void __launch_bounds__(128) append_decode_kernel(const uint16_t *__restrict__ K,
+                                                            const uint16_t *__restrict__ V,
+                                                            const float *__restrict__ inv_lambda, unsigned *vmax_bits,
+                                                            LayerGeom geom, int n_slices, int kv_heads, int n_old,
+                                                            int win_start, int cur_bits, int first_evicted, int n_evict) {
+  __shared__ uint16_t s_codes[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wid = (long long)blockIdx.x * 4 + warp;
+  const long long n_ev = (long long)n_evict * n_slices * 2;
+  if (wid < n_ev) {
+    evict_one(wid, s_codes[warp], lane, geom, n_slices, first_evicted, cur_bits);
+  } else if (wid < n_ev + 2ll * n_slices) {
+    append_one(wid - n_ev, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start,
+               cur_bits);
   }
 }
 

@@ -292,15 +292,23 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
   // tokens already in the ring that now leave the window
   const int ev_first = std::max(old_win_start, k->n_sink);
   const int ev_last = std::min(new_win_start, n_old);
-  if (ev_last > ev_first) {
-    const long long warps = 2ll * (ev_last - ev_first) * k->n_slices;
-    evict_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(g, k->n_slices, ev_first, ev_last - ev_first, l.cur_bits);
+  const float *inv_lam = reinterpret_cast<const float *>(k->arena + k->off_inv_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
+  unsigned *vmax = reinterpret_cast<unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
+  const int n_evict = std::max(0, ev_last - ev_first);
+  if (n_new == 1) {
+    // decode step: evictions and the new token in one launch (their ring slots cannot coincide)
+    const long long warps = 2ll * (n_evict + 1) * k->n_slices;
+    append_decode_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(
+        static_cast<const uint16_t *>(d_K), static_cast<const uint16_t *>(d_V), inv_lam, vmax, g, k->n_slices, k->kv_heads,
+        n_old, new_win_start, l.cur_bits, ev_first, n_evict);
     ++k->launches;
-  }
-  {
+  } else {
+    if (n_evict > 0) {
+      const long long warps = 2ll * n_evict * k->n_slices;
+      evict_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(g, k->n_slices, ev_first, n_evict, l.cur_bits);
+      ++k->launches;
+    }
     const long long warps = 2ll * n_new * k->n_slices;
-    const float *inv_lam = reinterpret_cast<const float *>(k->arena + k->off_inv_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
-    unsigned *vmax = reinterpret_cast<unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
     append_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(static_cast<const uint16_t *>(d_K),
                                                               static_cast<const uint16_t *>(d_V), inv_lam, vmax, g, n_new,
                                                               k->n_slices, k->kv_heads, n_old, new_win_start, l.cur_bits);
@@ -355,6 +363,23 @@ pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d
   }
   k->launches += 1;
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_decode_step(pmkvq_cache *k, const void *d_K, const void *d_V, const void *d_Q, float *d_out,
+                               void *stream) {
+  if (!k || !d_K || !d_V || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
+  const size_t kv_stride = (size_t)k->n_slices * kHeadDim * 2;            // bytes of one block's bf16 K (or V)
+  const size_t q_stride = (size_t)k->batch * k->q_heads * kHeadDim * 2;   // bytes of one block's bf16 Q
+  const size_t o_stride = (size_t)k->batch * k->q_heads * kHeadDim;       // floats of one block's output
+  for (int layer = 0; layer < k->layers; ++layer) {
+    pmkvq_status s = pmkvq_append(k, layer, static_cast<const uint8_t *>(d_K) + layer * kv_stride,
+                                  static_cast<const uint8_t *>(d_V) + layer * kv_stride, 1, stream);
+    if (s != PMKVQ_OK) return s;
+    s = pmkvq_decode_attention(k, layer, static_cast<const uint8_t *>(d_Q) + layer * q_stride, d_out + layer * o_stride,
+                               stream);
+    if (s != PMKVQ_OK) return s;
+  }
   return PMKVQ_OK;
 }
 

@@ -145,10 +145,10 @@ def test_split_invariance():
         m.cache.set_attention_ctas(s)
         m.check_attention(0, q)
         outs.append(m.cache.decode_attention(0, q.cuda()).cpu().numpy())
-    # partitions differ only by fp32 summation order and by where the fp16 rounding of p * S_V falls
-    # (relative 2^-12 per token, not averaged out when one token dominates the softmax)
+    # partitions differ by fp32 summation order and by the fp16 rounding of p * S_V (2^-12 relative per
+    # token, the reference m it is taken against depends on the partition): half the output tolerance
     for o in outs[1:]:
-        assert np.abs(o - outs[0]).max() < 6e-4 * max(1.0, float(np.abs(outs[0]).max()))
+        assert np.abs(o - outs[0]).max() < 1e-3
 
 
 def test_degenerate_values():
@@ -165,3 +165,36 @@ def test_degenerate_values():
     m.check_attention(0, q, max_abs=2e-3 * 50)    # outputs reach O(1000) with the scaled token
     q0 = torch.zeros_like(q)
     m.check_attention(0, q0, max_abs=2e-3 * 50)
+
+
+def test_decode_step_over_all_blocks():
+    """pmkvq_decode_step = append + attention for every block; compared with the oracle block by block,
+    across a reduce (block 0 crosses its budget during the steps)."""
+    layers, kvh, batch, group, n0, steps = 3, 2, 2, 7, 300, 24
+    fbit = [2, 4, 8]
+    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, fbit, window=32)
+    for l in range(layers):
+        k, v = make_inputs(8, l, n0, batch, kvh)
+        m.append(l, k, v)
+    for s in range(steps):
+        ks, vs, qs = [], [], []
+        for l in range(layers):
+            k, v = make_inputs(9, l, 1, batch, kvh, pos0=n0 + s, chunk=s)
+            ks.append(k[0]); vs.append(v[0])
+            qs.append(synth.make_q(9, l, s, batch, group * kvh, n0 + s + 1))
+        K, V, Q = torch.stack(ks).cuda(), torch.stack(vs).cuda(), torch.stack(qs).cuda()
+        out = m.cache.decode_step(K, V, Q)
+        torch.cuda.synchronize()
+        for l in range(layers):
+            kk = K[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices]
+            vv = V[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices]
+            m.oracles[l].append(kk, vv)
+            if s % 5 == 0 or s == steps - 1:
+                qq = Q[l].float().cpu().numpy().reshape(batch * kvh, group, 128)[m.slices]
+                ref = m.oracles[l].decode_attention(qq)
+                got = out[l].cpu().numpy().reshape(batch * kvh, group, 128)[m.slices].astype(np.float64)
+                assert np.abs(got - ref).max() <= 2e-3
+                assert np.linalg.norm(got - ref) <= 1e-3 * np.linalg.norm(ref)
+    for l in range(layers):
+        m.check_state(l)
+        assert m.cache.layer_state(l)["cur_bits"] == fbit[l]
