@@ -78,7 +78,7 @@ def make_lambda(wl, seed, device):
     return np.stack(lam)
 
 
-def build_cache(wl, fbit, budgets, lam, n0, device, chunk=2048, seed=0):
+def build_cache(wl, fbit, budgets, lam, n0, device, chunk=8192, seed=0):
     from paper_2505_18610_b200.binding import Cache
     cache = Cache(wl["layers"], wl["q_heads"], wl["kv_heads"], wl["batch"], wl["end_tokens"], fbit,
                   budget_bytes=budgets, lam=lam, n_sink=N_SINK, window=WINDOW, device=device)
