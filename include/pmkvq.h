@@ -41,7 +41,8 @@ typedef enum {
   PMKVQ_ERR_AT_FBIT = 4,         /* progressive_reduce on a block already at its Fbit */
   PMKVQ_ERR_CAPACITY = 5,        /* over budget at Fbit, or past max_tokens */
   PMKVQ_ERR_CUDA = 6,            /* a CUDA runtime call or launch failed */
-  PMKVQ_ERR_STATE = 7            /* internal invariant violated */
+  PMKVQ_ERR_STATE = 7,           /* internal invariant violated */
+  PMKVQ_ERR_SCRATCH_LIMIT = 8    /* pmkvq_decode_attention_static: more slices / CTAs than its fixed scratch holds */
 } pmkvq_status;
 
 typedef struct {
@@ -94,6 +95,26 @@ pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *cache, int32_t layer, void *s
  *   d_Q_bf16: DEVICE bf16 [batch][q_heads][128]; d_out: DEVICE fp32 [batch][q_heads][128]. */
 pmkvq_status pmkvq_decode_attention(pmkvq_cache *cache, int32_t layer, const void *d_Q_bf16, float *d_out,
                                     void *stream);
+
+/* The same computation and the same kernel as pmkvq_decode_attention, for callers that are not
+ * allowed to allocate device memory at the point of the call and have no arena workspace to offer:
+ * code running inside a serving engine's pre-sized memory pool, a plugin called after the host
+ * process has frozen its allocations, a real-time loop in which cudaMalloc's implicit device
+ * synchronisation is not acceptable.  (The paper has no counterpart of this call; it exists for
+ * such hosts.)  The split-K workspace (one ticket per slice, one partial result per CTA and slice)
+ * is a 4 MiB array that is part of the library image: every GPU that loads the library holds it
+ * until the process exits, and the call itself allocates and frees nothing.
+ *   - Limits: batch * kv_heads <= 4096 and (attention CTAs + batch * kv_heads) <= 989; beyond them the
+ *     call returns PMKVQ_ERR_SCRATCH_LIMIT and launches nothing (use pmkvq_decode_attention).
+ *   - The first call on each GPU looks up the array's device address (one runtime query, with that
+ *     GPU current); make that first call outside any stream capture.
+ *   - All calls on a GPU share the one array, whatever cache or stream they use: two such calls that
+ *     overlap on the GPU race and give wrong results.  Keep them on one stream or order them with
+ *     events.  The tickets are cleared on `stream` before every launch; the partials are fully
+ *     rewritten before they are read.
+ * Arguments and results are those of pmkvq_decode_attention. */
+pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *cache, int32_t layer, const void *d_Q_bf16, float *d_out,
+                                           void *stream);
 
 /* One decode step of the whole model's attention path (Sec. 3.4, inference stage): for every block in
  * order, pmkvq_append of one new token followed by pmkvq_decode_attention; everything is enqueued on

@@ -16,13 +16,14 @@ from . import build as _build
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libpmkvq.so")
 
-STATUS_NAMES = ["OK", "INVALID_ARG", "ARENA_TOO_SMALL", "BUDGET_FULL", "AT_FBIT", "CAPACITY", "CUDA", "STATE"]
-OK, INVALID_ARG, ARENA_TOO_SMALL, BUDGET_FULL, AT_FBIT, CAPACITY, CUDA_ERROR, STATE = range(8)
+STATUS_NAMES = ["OK", "INVALID_ARG", "ARENA_TOO_SMALL", "BUDGET_FULL", "AT_FBIT", "CAPACITY", "CUDA", "STATE",
+                "SCRATCH_LIMIT"]
+OK, INVALID_ARG, ARENA_TOO_SMALL, BUDGET_FULL, AT_FBIT, CAPACITY, CUDA_ERROR, STATE, SCRATCH_LIMIT = range(9)
 
 
 class PmkvqError(RuntimeError):
     def __init__(self, status: int, what: str):
-        super().__init__(f"{what}: {STATUS_NAMES[status] if 0 <= status < 8 else status}")
+        super().__init__(f"{what}: {STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}")
         self.status = status
 
 
@@ -55,6 +56,8 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_progressive_reduce.argtypes = [vp, i32, vp]
     lib.pmkvq_decode_attention.restype = i32
     lib.pmkvq_decode_attention.argtypes = [vp, i32, vp, vp, vp]
+    lib.pmkvq_decode_attention_static.restype = i32
+    lib.pmkvq_decode_attention_static.argtypes = [vp, i32, vp, vp, vp]
     lib.pmkvq_decode_step.restype = i32
     lib.pmkvq_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.pmkvq_set_attention_ctas.restype = i32
@@ -171,6 +174,17 @@ class Cache:
         if st != OK:
             raise PmkvqError(st, "pmkvq_decode_attention")
         return out
+
+    def decode_attention_static(self, layer: int, q: torch.Tensor, out: torch.Tensor, stream=None, check: bool = True):
+        """pmkvq_decode_attention_static: same result as decode_attention, split-K workspace inside the
+        library image instead of the arena.  `out` must be supplied (nothing is allocated here either)."""
+        self._check(q, torch.bfloat16, "q"); self._check(out, torch.float32, "out")
+        if q.numel() != self.batch * self.q_heads * 128 or out.numel() != q.numel():
+            raise ValueError("bad Q / out shape")
+        st = lib().pmkvq_decode_attention_static(self._h, layer, q.data_ptr(), out.data_ptr(), _stream_ptr(stream))
+        if check and st != OK:
+            raise PmkvqError(st, "pmkvq_decode_attention_static")
+        return st
 
     def decode_step(self, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, out: Optional[torch.Tensor] = None,
                     stream=None):

@@ -212,6 +212,33 @@ pmkvq_status do_reduce(pmkvq_cache *k, int layer, cudaStream_t st) {
 
 }  // namespace
 
+// ---- scratch of pmkvq_decode_attention_static: lives in the library image, one copy per GPU ----
+constexpr size_t kStaticTicketBytes = 16 * 1024;          // 4096 slice tickets
+constexpr size_t kStaticScratchBytes = 4u * 1024 * 1024;  // tickets + split-K partials
+constexpr size_t kStaticPartialSlots =
+    (kStaticScratchBytes - kStaticTicketBytes) / (kMaxGroup * kPartialStride * sizeof(float));
+constexpr int kMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static void *g_static_scratch_addr[kMaxDevices];  // device address of the array on each GPU, looked up once
+
+// Device address of g_static_scratch on the current GPU (in host code the array's name is only a
+// handle for the runtime, not something a kernel can be given).
+static cudaError_t static_scratch_address(unsigned char **out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_static_scratch_addr[dev]) {
+    void *ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (!ptr) return cudaErrorInvalidSymbol;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = static_cast<unsigned char *>(g_static_scratch_addr[dev]);
+  return cudaSuccess;
+}
+
 extern "C" {
 
 size_t pmkvq_arena_bytes_required(const pmkvq_config *cfg) {
@@ -383,6 +410,59 @@ pmkvq_status pmkvq_decode_step(pmkvq_cache *k, const void *d_K, const void *d_V,
   return PMKVQ_OK;
 }
 
+pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, void *stream) {
+  if (!k || layer < 0 || layer >= k->layers || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
+  const Layer &l = k->L[layer];
+  if (l.n_tokens <= 0) return PMKVQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  AttnParams p;
+  p.geom = k->geom(l);
+  p.Q = static_cast<const uint16_t *>(d_Q);
+  p.lambda = reinterpret_cast<const float *>(k->arena + k->off_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
+  p.vmax_bits = reinterpret_cast<const unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
+  p.out = d_out;
+  p.kv_heads = k->kv_heads; p.group = k->group; p.q_heads = k->q_heads;
+  p.n_tokens = l.n_tokens;
+  p.n_sink_eff = k->sink_at(l.n_tokens);
+  p.n_body = k->body_at(l.n_tokens);
+  p.win_start = p.n_sink_eff + p.n_body;
+  p.cur_bits = l.cur_bits;
+  p.body_tiles = (p.n_body + 15) / 16;
+  p.sink_tiles = k->sink_tiles;
+  p.aux_tiles = k->sink_tiles + k->ring_tiles;
+  p.n_slices = k->n_slices;
+  p.w16 = (tile_bytes(16) + tile_bytes(l.cur_bits) - 1) / tile_bytes(l.cur_bits);
+  p.units_lead = kSegmentCostBytes / tile_bytes(l.cur_bits);
+  p.units_aux = p.units_lead + (long long)p.aux_tiles * p.w16;
+  p.units_slice = p.units_aux + p.body_tiles;
+  p.units_total = p.units_slice * k->n_slices;
+  const int width_idx = l.cur_bits == 16 ? 0 : l.cur_bits == 8 ? 1 : l.cur_bits == 4 ? 2 : 3;
+  const int want = k->user_ctas > 0 ? k->user_ctas : k->resident_ctas[width_idx];
+  const long long per = std::max<long long>((p.units_total + want - 1) / want, k->user_ctas > 0 ? 1 : kMinUnitsPerCta);
+  p.units_per_cta = per;
+  const unsigned n_ctas = (unsigned)((p.units_total + per - 1) / per);
+  p.qk_scale = k->sm_scale * 1.4426950408889634f;
+  // the fixed scratch holds one ticket per slice and one partial per (CTA, slice it touches)
+  if ((size_t)k->n_slices * sizeof(unsigned) > kStaticTicketBytes ||
+      (size_t)n_ctas + (size_t)k->n_slices > kStaticPartialSlots)
+    return PMKVQ_ERR_SCRATCH_LIMIT;
+  unsigned char *scratch = nullptr;
+  if (static_scratch_address(&scratch) != cudaSuccess) return PMKVQ_ERR_CUDA;
+  p.tickets = reinterpret_cast<unsigned *>(scratch);
+  p.partials = reinterpret_cast<float *>(scratch + kStaticTicketBytes);
+  // the array keeps whatever the previous call left: the tickets must start at zero
+  if (cudaMemsetAsync(p.tickets, 0, (size_t)k->n_slices * sizeof(unsigned), st) != cudaSuccess) return PMKVQ_ERR_CUDA;
+  switch (l.cur_bits) {
+    case 16: decode_attn_splitk_kernel<16><<<n_ctas, kAttnThreads, attn_ring_bytes<16>(), st>>>(p); break;
+    case 8: decode_attn_splitk_kernel<8><<<n_ctas, kAttnThreads, attn_ring_bytes<8>(), st>>>(p); break;
+    case 4: decode_attn_splitk_kernel<4><<<n_ctas, kAttnThreads, attn_ring_bytes<4>(), st>>>(p); break;
+    default: decode_attn_splitk_kernel<2><<<n_ctas, kAttnThreads, attn_ring_bytes<2>(), st>>>(p); break;
+  }
+  k->launches += 1;
+  if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  return PMKVQ_OK;
+}
+
 pmkvq_status pmkvq_layer_state(const pmkvq_cache *k, int32_t layer, int32_t *n_tokens, int32_t *cur_bits,
                                uint64_t *bytes_used, uint64_t *budget_bytes) {
   if (!k || layer < 0 || layer >= k->layers) return PMKVQ_ERR_INVALID_ARG;
@@ -474,6 +554,7 @@ const char *pmkvq_status_string(pmkvq_status s) {
     case PMKVQ_ERR_CAPACITY: return "capacity exceeded";
     case PMKVQ_ERR_CUDA: return "CUDA error";
     case PMKVQ_ERR_STATE: return "internal state error";
+    case PMKVQ_ERR_SCRATCH_LIMIT: return "problem too large for the built-in scratch: use pmkvq_decode_attention";
   }
   return "unknown status";
 }
