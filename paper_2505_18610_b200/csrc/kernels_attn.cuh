@@ -45,7 +45,13 @@ constexpr int kMaxGroup = 8;         // query heads per KV head handled by one M
 constexpr int kPartialStride = 132;  // floats per (segment, head): m, l, 2 pad, o[128]
 constexpr float kNegBig = -1.0e30f;
 constexpr float kMaxAhead = 3.0f;    // a score may exceed the reference by this much (log2 units)
-constexpr int kAttnWarps = 16;      // one CTA per SM; its warps share the CTA's tiles dynamically
+#ifndef PMKVQ_WARPS
+#define PMKVQ_WARPS 16
+#endif
+#ifndef PMKVQ_QSMEM
+#define PMKVQ_QSMEM 1
+#endif
+constexpr int kAttnWarps = PMKVQ_WARPS;      // one CTA per SM; its warps share the CTA's tiles dynamically
 constexpr int kAttnThreads = 32 * kAttnWarps;
 
 struct AttnParams {
@@ -169,6 +175,28 @@ template <> struct Fmt<16> {
   __host__ __device__ static constexpr int pos(int) { return 0; }
 };
 
+// The query fragments of a lane (8 k-steps x 4 registers): either kept in registers for the whole
+// segment or fetched from a per-CTA copy in shared memory right before each use (they depend on the
+// lane, not on the warp), which trades 8 shared loads per step for 32 registers.
+struct QRegs {
+  uint32_t v[8][4];
+  __device__ __forceinline__ void load(int s, uint32_t (&q)[4]) const {
+    q[0] = v[s][0]; q[1] = v[s][1]; q[2] = v[s][2]; q[3] = v[s][3];
+  }
+};
+struct QSmem {
+  const uint4 *mine;  // entry (k-step s, this lane) at mine[32 s]
+  __device__ __forceinline__ void load(int s, uint32_t (&q)[4]) const {
+    const uint4 t = mine[32 * s];
+    q[0] = t.x; q[1] = t.y; q[2] = t.z; q[3] = t.w;
+  }
+};
+#if PMKVQ_QSMEM
+using QFrag = QSmem;
+#else
+using QFrag = QRegs;
+#endif
+
 struct WarpState {
   float m, l, zs;   // reference (log2 units), sum of probabilities, sum of p * Z_V, for head g (this lane's quad)
   float acc[8][4];  // O^T accumulators: [m-tile][channel row g / g+8 x head col 2tig / 2tig+1]
@@ -177,7 +205,7 @@ struct WarpState {
 // NT consecutive 16-token tiles.  `mask` (NT == 1 only) has bit r set when token row r is live.
 template <int BITS, int NT, bool MASKED>
 __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mask, WarpState &st,
-                                              const uint32_t (&qa)[8][4], float mu, float sumq, float inv_sigma_e,
+                                              const QFrag &qa, float mu, float sumq, float inv_sigma_e,
                                               int lane) {
   using F = Fmt<BITS>;
   static_assert(!(MASKED && NT != 1), "masked tiles are processed one at a time");
@@ -202,8 +230,10 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
 #pragma unroll
       for (int s = 0; s < 8; ++s) {
         const uint32_t x0 = kw[2 * s], x1 = kw[2 * s + 1];
-        mma_f16(lo, qa[s], x0 & 0x00FF00FFu, x1 & 0x00FF00FFu);
-        mma_f16(hi, qa[s], high_bytes(x0), high_bytes(x1));
+        uint32_t qf[4];
+        qa.load(s, qf);
+        mma_f16(lo, qf, x0 & 0x00FF00FFu, x1 & 0x00FF00FFu);
+        mma_f16(hi, qf, high_bytes(x0), high_bytes(x1));
       }
       dot[2 * r] = fmaf(256.f, hi[0] + hi[2], lo[0] + lo[2]);
       dot[2 * r + 1] = fmaf(256.f, hi[1] + hi[3], lo[1] + lo[3]);
@@ -227,6 +257,9 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
       for (int r = 0; r < 2; ++r) sacc[nt][r][0] = sacc[nt][r][1] = sacc[nt][r][2] = sacc[nt][r][3] = 0.f;
 #pragma unroll
     for (int w = 0; w < BITS; ++w) {
+      uint32_t qf[F::N / 2][4];
+#pragma unroll
+      for (int jj = 0; jj < F::N / 2; ++jj) qa.load((w * F::N) / 2 + jj, qf[jj]);
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -234,7 +267,7 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
           uint32_t e[F::N];
           F::extract(kw[nt][r * BITS + w], e);
 #pragma unroll
-          for (int jj = 0; jj < F::N / 2; ++jj) mma_f16(sacc[nt][r], qa[(w * F::N) / 2 + jj], e[2 * jj], e[2 * jj + 1]);
+          for (int jj = 0; jj < F::N / 2; ++jj) mma_f16(sacc[nt][r], qf[jj], e[2 * jj], e[2 * jj + 1]);
         }
       }
     }
@@ -397,25 +430,48 @@ __device__ __forceinline__ void combine_slice(const AttnParams &p, int slice) {
   }
 }
 
-// Query fragments of head g at the code positions of width BITS, from Q'' in shared memory.
+// Query fragment of head g for k-step s (channels 16 s .. 16 s + 15) at the code positions of width
+// BITS, from Q'' in shared memory: {hi, lo} of channels (c0, c0 + 1) and of (c0 + 8, c0 + 9).
 template <int BITS>
-__device__ __forceinline__ void build_q_fragments(uint32_t (&qa)[8][4], const float (*s_q)[kHeadDim], int e_g, int g,
-                                                  int tig) {
+__device__ __forceinline__ uint4 q_fragment(const float (*s_q)[kHeadDim], int e_g, int g, int tig, int s) {
   using F = Fmt<BITS>;
+  uint32_t r[4];
+#pragma unroll
+  for (int beta = 0; beta < 2; ++beta) {
+    const int W = 2 * s + beta;
+    const float scl = ldexpf(1.0f, F::EQ - F::pos(W % F::N) - e_g);
+    const int c0 = 16 * s + 8 * beta + 2 * tig;
+    const float x0 = s_q[g][c0] * scl, x1 = s_q[g][c0 + 1] * scl;
+    const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+    const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
+    const __half2 hi = __halves2half2(h0, h1), lo = __halves2half2(l0, l1);
+    r[2 * beta] = *reinterpret_cast<const uint32_t *>(&hi);
+    r[2 * beta + 1] = *reinterpret_cast<const uint32_t *>(&lo);
+  }
+  return make_uint4(r[0], r[1], r[2], r[3]);
+}
+
+// The fragments a warp multiplies with at width BITS: in registers, or (shared-memory variant) the
+// CTA's copy `s_frag`, which must have been filled by fill_q_fragments for this width.
+template <int BITS>
+__device__ __forceinline__ void set_q_fragments(QFrag &qa, const float (*s_q)[kHeadDim], const float *s_stat,
+                                                const uint4 *s_frag, int lane) {
+#if PMKVQ_QSMEM
+  qa.mine = s_frag + lane;
+#else
+  const int g = lane >> 2, tig = lane & 3;
 #pragma unroll
   for (int s = 0; s < 8; ++s) {
-#pragma unroll
-    for (int beta = 0; beta < 2; ++beta) {
-      const int W = 2 * s + beta;
-      const float scl = ldexpf(1.0f, F::EQ - F::pos(W % F::N) - e_g);
-      const int c0 = 16 * s + 8 * beta + 2 * tig;
-      const float x0 = s_q[g][c0] * scl, x1 = s_q[g][c0 + 1] * scl;
-      const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
-      const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
-      const __half2 hi = __halves2half2(h0, h1), lo = __halves2half2(l0, l1);
-      qa[s][2 * beta] = *reinterpret_cast<const uint32_t *>(&hi);
-      qa[s][2 * beta + 1] = *reinterpret_cast<const uint32_t *>(&lo);
-    }
+    const uint4 t = q_fragment<BITS>(s_q, (int)s_stat[g], g, tig, s);
+    qa.v[s][0] = t.x; qa.v[s][1] = t.y; qa.v[s][2] = t.z; qa.v[s][3] = t.w;
+  }
+#endif
+}
+template <int BITS>
+__device__ __forceinline__ void fill_q_fragments(uint4 *s_frag, const float (*s_q)[kHeadDim], const float *s_stat) {
+  for (int i = threadIdx.x; i < 256; i += kAttnThreads) {  // entry (k-step i / 32, lane i % 32)
+    const int l = i & 31, g = l >> 2;
+    s_frag[i] = q_fragment<BITS>(s_q, (int)s_stat[g], g, l & 3, i >> 5);
   }
 }
 
@@ -428,7 +484,8 @@ __device__ __forceinline__ void build_q_fragments(uint32_t (&qa)[8][4], const fl
 // tiles stream, then the warps' outputs.
 template <int BITS>
 __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long long u_lo, long long u_hi,
-                                            float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint8_t *ring) {
+                                            float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint4 *s_frag,
+                                            uint8_t *ring) {
   using F = Fmt<BITS>;
   using F16 = Fmt<16>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
@@ -514,6 +571,11 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   __syncthreads();
   const int e_g = (int)s_stat[g];
   const float sumq = s_stat[8 + g];
+#if PMKVQ_QSMEM
+  fill_q_fragments<16>(s_frag, s_q, s_stat);
+  if constexpr (BITS != 16) fill_q_fragments<BITS>(s_frag + 256, s_q, s_stat);
+  __syncthreads();
+#endif
 
   // ---- unit of the V accumulators: a power of two >= every INT16 V scale of this slice; at width b
   //      the scales are at most 2^SIGMA_LOG2 times larger ----
@@ -531,13 +593,13 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   st.m = kNegBig; st.l = 0.f; st.zs = 0.f;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
-  uint32_t qa[8][4];
+  QFrag qa;
 
   // ---- INT16 tiles (sink + window ring) ----
   if (a_hi > a_lo) {
     int it = a_lo + claim(0);
     if (it < a_hi) {
-      build_q_fragments<16>(qa, s_q, e_g, g, tig);
+      set_q_fragments<16>(qa, s_q, s_stat, s_frag, lane);
       const float mu = ldexpf(1.0f, 24 - F16::EQ + e_g);
       const float inv_sigma_e = ldexpf(1.0f, F16::EP) / sigma16;
       const int n_win = p.n_tokens - p.win_start;
@@ -582,7 +644,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   // ---- body tiles ----
   const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
   if (n_steps > 0) {
-    build_q_fragments<BITS>(qa, s_q, e_g, g, tig);
+    set_q_fragments<BITS>(qa, s_q, s_stat, BITS != 16 ? s_frag + 256 : s_frag, lane);
     const float mu = ldexpf(1.0f, 24 - F::EQ + e_g);
     const float inv_sigma_e = ldexpf(1.0f, F::EP) / sigma_u;
     const uint32_t tail_mask = (p.n_body & 15) ? (1u << (p.n_body & 15)) - 1u : 0xFFFFu;
@@ -705,6 +767,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
   __shared__ float s_stat[16 + 2 * kAttnWarps * kMaxGroup];  // head stats, per-warp (m, l)
   __shared__ int s_ctr[4];                                    // work counters (INT16 tiles, body steps), combine flag
+#if PMKVQ_QSMEM
+  __shared__ uint4 s_frag[512];                               // query fragments at INT16 and at the body width
+#else
+  uint4 *s_frag = nullptr;
+#endif
   extern __shared__ __align__(128) uint8_t ring[];
   const long long u_begin = (long long)blockIdx.x * p.units_per_cta;
   const long long u_end = min(u_begin + p.units_per_cta, p.units_total);
@@ -712,7 +779,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
     const int slice = (int)(u / p.units_slice);
     const long long base = (long long)slice * p.units_slice;
     const long long hi = min(u_end - base, p.units_slice);
-    if (hi > p.units_lead) run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, ring);
+    if (hi > p.units_lead) run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
     u = base + hi;
   }
 }

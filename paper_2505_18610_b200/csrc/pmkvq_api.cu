@@ -21,7 +21,9 @@ namespace {
 constexpr size_t kAlign = 256;
 constexpr int kHeadTiles = 8;     // tiles the reduce handles in order before the parallel waves start
 constexpr int kMaxCtas = 2048;      // upper bound on the attention grid (sizes the partials workspace)
-constexpr int kSegmentCostBytes = 40 * 1024;  // set-up + merge + publish of one segment, in streamed bytes
+// Fixed cost of one more segment (set-up, warp merge, publish, its share of the slice combine), in
+// body tiles of each width: about 12 us at the measured per-SM tile rates.
+inline int segment_cost_tiles(int bits) { return bits == 16 ? 48 : bits == 8 ? 96 : bits == 4 ? 176 : 160; }
 constexpr int kMinUnitsPerCta = 32;  // do not cut the work finer than two tiles per warp
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -371,8 +373,8 @@ pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d
   p.n_slices = k->n_slices;
   // one line of work units over all slices: a body tile is one unit, an INT16 tile their byte ratio
   p.w16 = (tile_bytes(16) + tile_bytes(l.cur_bits) - 1) / tile_bytes(l.cur_bits);
-  // a segment costs about as much as streaming 40 KB: every slice starts with that many empty units
-  p.units_lead = kSegmentCostBytes / tile_bytes(l.cur_bits);
+  // every slice starts with empty units that stand for the fixed cost of a segment
+  p.units_lead = segment_cost_tiles(l.cur_bits);
   p.units_aux = p.units_lead + (long long)p.aux_tiles * p.w16;
   p.units_slice = p.units_aux + p.body_tiles;
   p.units_total = p.units_slice * k->n_slices;
@@ -432,7 +434,7 @@ pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *k, int32_t layer, const 
   p.aux_tiles = k->sink_tiles + k->ring_tiles;
   p.n_slices = k->n_slices;
   p.w16 = (tile_bytes(16) + tile_bytes(l.cur_bits) - 1) / tile_bytes(l.cur_bits);
-  p.units_lead = kSegmentCostBytes / tile_bytes(l.cur_bits);
+  p.units_lead = segment_cost_tiles(l.cur_bits);
   p.units_aux = p.units_lead + (long long)p.aux_tiles * p.w16;
   p.units_slice = p.units_aux + p.body_tiles;
   p.units_total = p.units_slice * k->n_slices;
