@@ -122,14 +122,17 @@ pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *cache, int32_t layer, co
  *   d_K_bf16, d_V_bf16: DEVICE bf16 [layers][batch][kv_heads][128]
  *   d_Q_bf16:           DEVICE bf16 [layers][batch][q_heads][128]
  *   d_out:              DEVICE fp32 [layers][batch][q_heads][128]
- * Stops at the first block whose call fails and returns its status; earlier blocks keep their new
- * token.  With auto_reduce = 0 a block whose budget is full returns PMKVQ_ERR_BUDGET_FULL here. */
+ * The budget of every block is tested first (reducing where auto_reduce allows); if a block fails
+ * (PMKVQ_ERR_BUDGET_FULL with auto_reduce = 0, PMKVQ_ERR_CAPACITY) its status is returned and no block has
+ * received its token.  Then one launch appends to all blocks and one attention launch per block
+ * follows; consecutive attention kernels may overlap on the GPU, and all of them have completed
+ * before anything enqueued on `stream` after this call starts. */
 pmkvq_status pmkvq_decode_step(pmkvq_cache *cache, const void *d_K_bf16, const void *d_V_bf16, const void *d_Q_bf16,
                                float *d_out, void *stream);
 
 /* Split-K tuning of pmkvq_decode_attention (flash-decoding partition over the sequence): the tiles
  * of all (batch, kv_head) slices are cut into `n_ctas` equal contiguous pieces, one per CTA
- * (1..2048); 0 restores the default, one wave of resident CTAs on the GPU's SMs. */
+ * (1..1024); 0 restores the default, one wave of resident CTAs on the GPU's SMs. */
 pmkvq_status pmkvq_set_attention_ctas(pmkvq_cache *cache, int32_t n_ctas);
 
 /* Host-side state of a block; any out pointer may be NULL. */

@@ -197,6 +197,14 @@ using QFrag = QSmem;
 using QFrag = QRegs;
 #endif
 
+// 16-byte load of tile data: body tiles sit in shared memory, INT16 tiles are read from global
+// memory past L1 (another kernel may have written them while this SM still holds old lines).
+template <int BITS, class T>
+__device__ __forceinline__ T ld_tile(const void *ptr) {
+  if constexpr (BITS == 16) return __ldcg(reinterpret_cast<const T *>(ptr));
+  else return *reinterpret_cast<const T *>(ptr);
+}
+
 struct WarpState {
   float m, l, zs;   // reference (log2 units), sum of probabilities, sum of p * Z_V, for head g (this lane's quad)
   float acc[8][4];  // O^T accumulators: [m-tile][channel row g / g+8 x head col 2tig / 2tig+1]
@@ -223,7 +231,7 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
       uint32_t kw[16];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const uint4 a = *reinterpret_cast<const uint4 *>(kp + (4 * r + q) * 512);
+        const uint4 a = __ldcg(reinterpret_cast<const uint4 *>(kp + (4 * r + q) * 512));
         kw[4 * q] = a.x; kw[4 * q + 1] = a.y; kw[4 * q + 2] = a.z; kw[4 * q + 3] = a.w;
       }
       float lo[4] = {0.f, 0.f, 0.f, 0.f}, hi[4] = {0.f, 0.f, 0.f, 0.f};
@@ -285,7 +293,8 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const float4 *mp = reinterpret_cast<const float4 *>(tile0 + nt * TB + meta_offset(BITS) + tig * 64);
-    const float4 a = mp[0], b = mp[1], c = mp[2], d = mp[3];
+    const float4 a = ld_tile<BITS, float4>(mp), b = ld_tile<BITS, float4>(mp + 1), c = ld_tile<BITS, float4>(mp + 2),
+                 d = ld_tile<BITS, float4>(mp + 3);
     sk[4 * nt] = a.x; sk[4 * nt + 1] = a.y; sk[4 * nt + 2] = a.z; sk[4 * nt + 3] = a.w;
     zk[4 * nt] = b.x; zk[4 * nt + 1] = b.y; zk[4 * nt + 2] = b.z; zk[4 * nt + 3] = b.w;
     sv[4 * nt] = c.x; sv[4 * nt + 1] = c.y; sv[4 * nt + 2] = c.z; sv[4 * nt + 3] = c.w;
@@ -354,7 +363,7 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
     uint32_t vw[2 * BITS];
 #pragma unroll
     for (int q = 0; q < CHUNKS; ++q) {
-      const uint4 a = *reinterpret_cast<const uint4 *>(vp + q * 512);
+      const uint4 a = ld_tile<BITS, uint4>(vp + q * 512);
       vw[4 * q] = a.x; vw[4 * q + 1] = a.y; vw[4 * q + 2] = a.z; vw[4 * q + 3] = a.w;
     }
     const uint32_t pb0 = pb[2 * nt], pb1 = pb[2 * nt + 1];
@@ -581,7 +590,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   //      the scales are at most 2^SIGMA_LOG2 times larger ----
   float sigma16 = 1.0f;
   {
-    const float s16 = __uint_as_float(p.vmax_bits[slice]);
+    const float s16 = __uint_as_float(__ldcg(p.vmax_bits + slice));
     if (s16 > 0.f) {
       int e;
       frexpf(s16, &e);
@@ -773,6 +782,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
   uint4 *s_frag = nullptr;
 #endif
   extern __shared__ __align__(128) uint8_t ring[];
+  // When launched with programmatic stream serialization (pmkvq_decode_step does that for every block
+  // after the first) the next block's kernel may start as soon as SMs free up; it works on its own
+  // tiles, scratch and output, so nothing of this grid has to be finished for it.  No-op otherwise.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const long long u_begin = (long long)blockIdx.x * p.units_per_cta;
   const long long u_end = min(u_begin + p.units_per_cta, p.units_total);
   for (long long u = u_begin; u < u_end;) {
@@ -782,6 +795,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
     if (hi > p.units_lead) run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
     u = base + hi;
   }
+  // A grid never completes before the grid it was allowed to overlap: kernels complete in launch order,
+  // so whatever follows in the stream sees all of them done.  Returns at once for a normal launch.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace pmkvq

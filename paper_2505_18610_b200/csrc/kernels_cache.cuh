@@ -227,6 +227,48 @@ __global__ void __launch_bounds__(128) append_decode_kernel(const uint16_t *__re
 // a lane at 2B bits become one word at B bits.  Everything is read and transformed before the
 // first store, so the output may overlap this tile's own input.
 // ---------------------------------------------------------------------------------------------
+// ---------------------------------------------------------------------------------------------
+// One decode step's cache update for ALL blocks in a single launch.  The blocks' geometry is a
+// table in device memory (written once when the cache is created); their token counts and widths
+// travel as kernel arguments.  Per block the warps are laid out as in append_decode_kernel, with
+// room for evict_chunk evictions whether or not this step has any.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxStepLayers = 128;
+struct StepParams {
+  int n_old[kMaxStepLayers];               // tokens cached in each block before this step
+  unsigned char cur_bits[kMaxStepLayers];  // body width of each block
+};
+
+__global__ void __launch_bounds__(128) append_step_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
+                                                          const float *__restrict__ inv_lambda, unsigned *vmax_bits,
+                                                          const LayerGeom *__restrict__ geoms, const StepParams sp,
+                                                          int layers, int n_slices, int kv_heads, int n_sink, int window,
+                                                          int evict_chunk) {
+  __shared__ uint16_t s_codes[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long per_layer = 2ll * (evict_chunk + 1) * n_slices;
+  const long long gw = (long long)blockIdx.x * 4 + warp;
+  const int layer = (int)(gw / per_layer);
+  if (layer >= layers) return;
+  const long long w = gw - (long long)layer * per_layer;
+  const LayerGeom geom = geoms[layer];
+  const int n_old = sp.n_old[layer], n_after = n_old + 1, cur_bits = sp.cur_bits[layer];
+  auto body_at = [&](int n) {
+    const int excess = n - n_sink - window;
+    return excess <= 0 ? 0 : excess / evict_chunk * evict_chunk;
+  };
+  const int old_ws = min(n_old, n_sink) + body_at(n_old), new_ws = min(n_after, n_sink) + body_at(n_after);
+  const int ev_first = max(old_ws, n_sink), n_evict = max(0, min(new_ws, n_old) - ev_first);
+  const long long ev_room = 2ll * evict_chunk * n_slices;
+  if (w < ev_room) {
+    if (w < 2ll * n_evict * n_slices) evict_one(w, s_codes[warp], lane, geom, n_slices, ev_first, cur_bits);
+  } else {
+    const size_t in_off = (size_t)layer * n_slices * kHeadDim;
+    append_one(w - ev_room, s_codes[warp], lane, K + in_off, V + in_off, inv_lambda + (size_t)layer * kv_heads * kHeadDim,
+               vmax_bits + (size_t)layer * n_slices, geom, n_slices, kv_heads, n_old, new_ws, cur_bits);
+  }
+}
+
 template <int B>
 __device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1) {
   constexpr int NIN = 8 / B;  // codes per half-word at 2B bits

@@ -20,7 +20,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kHeadTiles = 8;     // tiles the reduce handles in order before the parallel waves start
-constexpr int kMaxCtas = 2048;      // upper bound on the attention grid (sizes the partials workspace)
+constexpr int kMaxCtas = 1024;      // upper bound on the attention grid (sizes the partials workspace)
 // Fixed cost of one more segment (set-up, warp merge, publish, its share of the slice combine), in
 // body tiles of each width: about 12 us at the measured per-SM tile rates.
 inline int segment_cost_tiles(int bits) { return bits == 16 ? 48 : bits == 8 ? 96 : bits == 4 ? 176 : 160; }
@@ -48,7 +48,7 @@ struct pmkvq_cache {
   uint8_t *arena;
   size_t arena_bytes;
   // arena sections
-  size_t off_lambda, off_inv_lambda, off_vmax, off_tickets, off_partials, partial_bytes;
+  size_t off_lambda, off_inv_lambda, off_vmax, off_tickets, off_partials, partial_bytes, off_geoms;  // scratch is per block
   int sink_tiles, ring_tiles, user_ctas;
   int resident_ctas[4];  // one wave of the attention kernel at body width 16, 8, 4, 2
   uint64_t launches = 0;  // kernels launched so far
@@ -122,9 +122,11 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.off_lambda = off; off = align_up(off + lam_bytes, kAlign);
   k.off_inv_lambda = off; off = align_up(off + lam_bytes, kAlign);
   k.off_vmax = off; off = align_up(off + (size_t)k.layers * k.n_slices * sizeof(unsigned), kAlign);
-  k.off_tickets = off; off = align_up(off + (size_t)k.n_slices * sizeof(unsigned), kAlign);
-  k.partial_bytes = ((size_t)kMaxCtas + 2 * (size_t)k.n_slices) * kMaxGroup * kPartialStride * sizeof(float);
-  k.off_partials = off; off = align_up(off + k.partial_bytes, kAlign);
+  // tickets and split-K partials exist once per block: attention kernels of consecutive blocks may overlap
+  k.off_tickets = off; off = align_up(off + (size_t)k.layers * k.n_slices * sizeof(unsigned), kAlign);
+  k.partial_bytes = align_up(((size_t)kMaxCtas + (size_t)k.n_slices) * kMaxGroup * kPartialStride * sizeof(float), kAlign);
+  k.off_partials = off; off = align_up(off + k.partial_bytes * k.layers, kAlign);
+  k.off_geoms = off; off = align_up(off + (size_t)k.layers * sizeof(LayerGeom), kAlign);
 
   k.L.assign(k.layers, Layer());
   for (int i = 0; i < k.layers; ++i) {
@@ -273,7 +275,12 @@ pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
   if (e == cudaSuccess)
     e = cudaMemcpy(k->arena + k->off_inv_lambda, inv.data(), n_lam * sizeof(float), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_vmax, 0, (size_t)k->layers * k->n_slices * sizeof(unsigned));
-  if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_tickets, 0, (size_t)k->n_slices * sizeof(unsigned));
+  if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_tickets, 0, (size_t)k->layers * k->n_slices * sizeof(unsigned));
+  if (e == cudaSuccess) {
+    std::vector<LayerGeom> geoms(k->layers);
+    for (int i = 0; i < k->layers; ++i) geoms[i] = k->geom(k->L[i]);
+    e = cudaMemcpy(k->arena + k->off_geoms, geoms.data(), geoms.size() * sizeof(LayerGeom), cudaMemcpyHostToDevice);
+  }
   if (e == cudaSuccess) e = attention_setup(k);
   if (e != cudaSuccess) {
     delete k;
@@ -291,16 +298,13 @@ pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *k, int32_t layer, void *strea
   return do_reduce(k, layer, static_cast<cudaStream_t>(stream));
 }
 
-pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const void *d_V, int32_t n_new,
-                          void *stream) {
-  if (!k || layer < 0 || layer >= k->layers || !d_K || !d_V || n_new <= 0) return PMKVQ_ERR_INVALID_ARG;
-  if ((reinterpret_cast<uintptr_t>(d_K) | reinterpret_cast<uintptr_t>(d_V)) & 7) return PMKVQ_ERR_INVALID_ARG;
+// Policy part of an append of n_new tokens to one block (Sec. 3.1): capacity and budget tests before
+// anything is mutated, then the reduces the budget asks for.  On PMKVQ_OK the block can take the tokens.
+static pmkvq_status append_prepare(pmkvq_cache *k, int32_t layer, int32_t n_new, cudaStream_t st, int &n_after_out) {
   Layer &l = k->L[layer];
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int64_t n_after64 = (int64_t)l.n_tokens + n_new;
   if (n_after64 > k->max_tokens) return PMKVQ_ERR_CAPACITY;
   const int n_after = (int)n_after64;
-  // budget test before anything is mutated (Sec. 3.1: shrink when the budget is fully used)
   int bits = l.cur_bits, n_reduce = 0;
   while (k->bytes_at(n_after, bits) > l.budget) {
     if (bits <= l.fbit) return PMKVQ_ERR_CAPACITY;
@@ -308,12 +312,25 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
     ++n_reduce;
   }
   if (n_reduce && !k->auto_reduce) return PMKVQ_ERR_BUDGET_FULL;
-  const int new_body = k->body_at(n_after);
-  if ((size_t)((new_body + 15) / 16) * tile_bytes(bits) > l.body_cap) return PMKVQ_ERR_STATE;
+  if ((size_t)((k->body_at(n_after) + 15) / 16) * tile_bytes(bits) > l.body_cap) return PMKVQ_ERR_STATE;
   for (int i = 0; i < n_reduce; ++i) {
     const pmkvq_status s = do_reduce(k, layer, st);
     if (s != PMKVQ_OK) return s;
   }
+  n_after_out = n_after;
+  return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const void *d_V, int32_t n_new,
+                          void *stream) {
+  if (!k || layer < 0 || layer >= k->layers || !d_K || !d_V || n_new <= 0) return PMKVQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_K) | reinterpret_cast<uintptr_t>(d_V)) & 7) return PMKVQ_ERR_INVALID_ARG;
+  Layer &l = k->L[layer];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int n_after = 0;
+  const pmkvq_status ps = append_prepare(k, layer, n_new, st, n_after);
+  if (ps != PMKVQ_OK) return ps;
+  const int new_body = k->body_at(n_after);
   const LayerGeom g = k->geom(l);
   const int n_old = l.n_tokens;
   const int old_win_start = k->sink_at(n_old) + k->body_at(n_old);
@@ -348,19 +365,21 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
   return PMKVQ_OK;
 }
 
-pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, void *stream) {
+}  // extern "C"
+
+// Everything of one attention launch except where its split-K scratch lives.
+static pmkvq_status attn_params(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, AttnParams &p,
+                                unsigned &n_ctas) {
   if (!k || layer < 0 || layer >= k->layers || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
   const Layer &l = k->L[layer];
   if (l.n_tokens <= 0) return PMKVQ_ERR_INVALID_ARG;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  AttnParams p;
   p.geom = k->geom(l);
   p.Q = static_cast<const uint16_t *>(d_Q);
   p.lambda = reinterpret_cast<const float *>(k->arena + k->off_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
   p.vmax_bits = reinterpret_cast<const unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
-  p.partials = reinterpret_cast<float *>(k->arena + k->off_partials);
+  p.partials = nullptr;
+  p.tickets = nullptr;
   p.out = d_out;
-  p.tickets = reinterpret_cast<unsigned *>(k->arena + k->off_tickets);
   p.kv_heads = k->kv_heads; p.group = k->group; p.q_heads = k->q_heads;
   p.n_tokens = l.n_tokens;
   p.n_sink_eff = k->sink_at(l.n_tokens);
@@ -380,70 +399,64 @@ pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d
   p.units_total = p.units_slice * k->n_slices;
   const int width_idx = l.cur_bits == 16 ? 0 : l.cur_bits == 8 ? 1 : l.cur_bits == 4 ? 2 : 3;
   const int want = k->user_ctas > 0 ? k->user_ctas : k->resident_ctas[width_idx];
-  long long per = std::max<long long>((p.units_total + want - 1) / want, k->user_ctas > 0 ? 1 : kMinUnitsPerCta);
+  const long long per = std::max<long long>((p.units_total + want - 1) / want, k->user_ctas > 0 ? 1 : kMinUnitsPerCta);
   p.units_per_cta = per;
-  const unsigned n_ctas = (unsigned)((p.units_total + per - 1) / per);
+  n_ctas = (unsigned)((p.units_total + per - 1) / per);
   p.qk_scale = k->sm_scale * 1.4426950408889634f;
-  switch (l.cur_bits) {
-    case 16: decode_attn_splitk_kernel<16><<<n_ctas, kAttnThreads, attn_ring_bytes<16>(), st>>>(p); break;
-    case 8: decode_attn_splitk_kernel<8><<<n_ctas, kAttnThreads, attn_ring_bytes<8>(), st>>>(p); break;
-    case 4: decode_attn_splitk_kernel<4><<<n_ctas, kAttnThreads, attn_ring_bytes<4>(), st>>>(p); break;
-    default: decode_attn_splitk_kernel<2><<<n_ctas, kAttnThreads, attn_ring_bytes<2>(), st>>>(p); break;
-  }
-  k->launches += 1;
-  if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
   return PMKVQ_OK;
 }
 
-pmkvq_status pmkvq_decode_step(pmkvq_cache *k, const void *d_K, const void *d_V, const void *d_Q, float *d_out,
-                               void *stream) {
-  if (!k || !d_K || !d_V || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
-  const size_t kv_stride = (size_t)k->n_slices * kHeadDim * 2;            // bytes of one block's bf16 K (or V)
-  const size_t q_stride = (size_t)k->batch * k->q_heads * kHeadDim * 2;   // bytes of one block's bf16 Q
-  const size_t o_stride = (size_t)k->batch * k->q_heads * kHeadDim;       // floats of one block's output
-  for (int layer = 0; layer < k->layers; ++layer) {
-    pmkvq_status s = pmkvq_append(k, layer, static_cast<const uint8_t *>(d_K) + layer * kv_stride,
-                                  static_cast<const uint8_t *>(d_V) + layer * kv_stride, 1, stream);
-    if (s != PMKVQ_OK) return s;
-    s = pmkvq_decode_attention(k, layer, static_cast<const uint8_t *>(d_Q) + layer * q_stride, d_out + layer * o_stride,
-                               stream);
-    if (s != PMKVQ_OK) return s;
+template <int BITS>
+static cudaError_t attn_launch_width(const AttnParams &p, unsigned n_ctas, cudaStream_t st, bool overlap_previous) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_ctas);
+  cfg.blockDim = dim3(kAttnThreads);
+  cfg.dynamicSmemBytes = attn_ring_bytes<BITS>();
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap_previous ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, decode_attn_splitk_kernel<BITS>, p);
+}
+
+// overlap_previous: the kernel may start before the previous kernel of the stream has finished (only
+// for launches whose inputs that kernel does not produce).
+static cudaError_t attn_launch(const AttnParams &p, unsigned n_ctas, cudaStream_t st, bool overlap_previous) {
+  switch (p.cur_bits) {
+    case 16: return attn_launch_width<16>(p, n_ctas, st, overlap_previous);
+    case 8: return attn_launch_width<8>(p, n_ctas, st, overlap_previous);
+    case 4: return attn_launch_width<4>(p, n_ctas, st, overlap_previous);
+    default: return attn_launch_width<2>(p, n_ctas, st, overlap_previous);
   }
-  return PMKVQ_OK;
+}
+
+static pmkvq_status attention_on_arena(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, cudaStream_t st,
+                                       bool overlap_previous) {
+  AttnParams p;
+  unsigned n_ctas = 0;
+  const pmkvq_status s = attn_params(k, layer, d_Q, d_out, p, n_ctas);
+  if (s != PMKVQ_OK) return s;
+  p.partials = reinterpret_cast<float *>(k->arena + k->off_partials + (size_t)layer * k->partial_bytes);
+  p.tickets = reinterpret_cast<unsigned *>(k->arena + k->off_tickets) + (size_t)layer * k->n_slices;
+  const cudaError_t e = attn_launch(p, n_ctas, st, overlap_previous);
+  k->launches += 1;
+  return e == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
+}
+
+extern "C" {
+
+pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, void *stream) {
+  return attention_on_arena(k, layer, d_Q, d_out, static_cast<cudaStream_t>(stream), false);
 }
 
 pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, void *stream) {
-  if (!k || layer < 0 || layer >= k->layers || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
-  const Layer &l = k->L[layer];
-  if (l.n_tokens <= 0) return PMKVQ_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   AttnParams p;
-  p.geom = k->geom(l);
-  p.Q = static_cast<const uint16_t *>(d_Q);
-  p.lambda = reinterpret_cast<const float *>(k->arena + k->off_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
-  p.vmax_bits = reinterpret_cast<const unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
-  p.out = d_out;
-  p.kv_heads = k->kv_heads; p.group = k->group; p.q_heads = k->q_heads;
-  p.n_tokens = l.n_tokens;
-  p.n_sink_eff = k->sink_at(l.n_tokens);
-  p.n_body = k->body_at(l.n_tokens);
-  p.win_start = p.n_sink_eff + p.n_body;
-  p.cur_bits = l.cur_bits;
-  p.body_tiles = (p.n_body + 15) / 16;
-  p.sink_tiles = k->sink_tiles;
-  p.aux_tiles = k->sink_tiles + k->ring_tiles;
-  p.n_slices = k->n_slices;
-  p.w16 = (tile_bytes(16) + tile_bytes(l.cur_bits) - 1) / tile_bytes(l.cur_bits);
-  p.units_lead = segment_cost_tiles(l.cur_bits);
-  p.units_aux = p.units_lead + (long long)p.aux_tiles * p.w16;
-  p.units_slice = p.units_aux + p.body_tiles;
-  p.units_total = p.units_slice * k->n_slices;
-  const int width_idx = l.cur_bits == 16 ? 0 : l.cur_bits == 8 ? 1 : l.cur_bits == 4 ? 2 : 3;
-  const int want = k->user_ctas > 0 ? k->user_ctas : k->resident_ctas[width_idx];
-  const long long per = std::max<long long>((p.units_total + want - 1) / want, k->user_ctas > 0 ? 1 : kMinUnitsPerCta);
-  p.units_per_cta = per;
-  const unsigned n_ctas = (unsigned)((p.units_total + per - 1) / per);
-  p.qk_scale = k->sm_scale * 1.4426950408889634f;
+  unsigned n_ctas = 0;
+  const pmkvq_status s = attn_params(k, layer, d_Q, d_out, p, n_ctas);
+  if (s != PMKVQ_OK) return s;
   // the fixed scratch holds one ticket per slice and one partial per (CTA, slice it touches)
   if ((size_t)k->n_slices * sizeof(unsigned) > kStaticTicketBytes ||
       (size_t)n_ctas + (size_t)k->n_slices > kStaticPartialSlots)
@@ -454,14 +467,58 @@ pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *k, int32_t layer, const 
   p.partials = reinterpret_cast<float *>(scratch + kStaticTicketBytes);
   // the array keeps whatever the previous call left: the tickets must start at zero
   if (cudaMemsetAsync(p.tickets, 0, (size_t)k->n_slices * sizeof(unsigned), st) != cudaSuccess) return PMKVQ_ERR_CUDA;
-  switch (l.cur_bits) {
-    case 16: decode_attn_splitk_kernel<16><<<n_ctas, kAttnThreads, attn_ring_bytes<16>(), st>>>(p); break;
-    case 8: decode_attn_splitk_kernel<8><<<n_ctas, kAttnThreads, attn_ring_bytes<8>(), st>>>(p); break;
-    case 4: decode_attn_splitk_kernel<4><<<n_ctas, kAttnThreads, attn_ring_bytes<4>(), st>>>(p); break;
-    default: decode_attn_splitk_kernel<2><<<n_ctas, kAttnThreads, attn_ring_bytes<2>(), st>>>(p); break;
-  }
+  const cudaError_t e = attn_launch(p, n_ctas, st, false);
   k->launches += 1;
+  return e == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
+}
+
+pmkvq_status pmkvq_decode_step(pmkvq_cache *k, const void *d_K, const void *d_V, const void *d_Q, float *d_out,
+                               void *stream) {
+  if (!k || !d_K || !d_V || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_K) | reinterpret_cast<uintptr_t>(d_V)) & 7) return PMKVQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t kv_stride = (size_t)k->n_slices * kHeadDim * 2;            // bytes of one block's bf16 K (or V)
+  const size_t q_stride = (size_t)k->batch * k->q_heads * kHeadDim * 2;   // bytes of one block's bf16 Q
+  const size_t o_stride = (size_t)k->batch * k->q_heads * kHeadDim;       // floats of one block's output
+  if (k->layers > kMaxStepLayers) {  // too many blocks for one argument block: block by block
+    for (int layer = 0; layer < k->layers; ++layer) {
+      pmkvq_status s = pmkvq_append(k, layer, static_cast<const uint8_t *>(d_K) + layer * kv_stride,
+                                    static_cast<const uint8_t *>(d_V) + layer * kv_stride, 1, stream);
+      if (s == PMKVQ_OK)
+        s = pmkvq_decode_attention(k, layer, static_cast<const uint8_t *>(d_Q) + layer * q_stride,
+                                   d_out + layer * o_stride, stream);
+      if (s != PMKVQ_OK) return s;
+    }
+    return PMKVQ_OK;
+  }
+  // 1. policy of every block (budget tests, the reduces they ask for); nothing is appended yet
+  for (int layer = 0; layer < k->layers; ++layer) {
+    int n_after = 0;
+    const pmkvq_status s = append_prepare(k, layer, 1, st, n_after);
+    if (s != PMKVQ_OK) return s;
+  }
+  // 2. quantize-on-append and evictions of all blocks in one launch
+  StepParams sp;
+  for (int layer = 0; layer < k->layers; ++layer) {
+    sp.n_old[layer] = k->L[layer].n_tokens;
+    sp.cur_bits[layer] = (unsigned char)k->L[layer].cur_bits;
+  }
+  const long long warps = 2ll * (k->evict_chunk + 1) * k->n_slices * k->layers;
+  append_step_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(
+      static_cast<const uint16_t *>(d_K), static_cast<const uint16_t *>(d_V),
+      reinterpret_cast<const float *>(k->arena + k->off_inv_lambda), reinterpret_cast<unsigned *>(k->arena + k->off_vmax),
+      reinterpret_cast<const LayerGeom *>(k->arena + k->off_geoms), sp, k->layers, k->n_slices, k->kv_heads, k->n_sink,
+      k->window, k->evict_chunk);
+  ++k->launches;
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  for (int layer = 0; layer < k->layers; ++layer) k->L[layer].n_tokens += 1;
+  // 3. attention block by block; from the second block on a kernel may start while the previous one
+  //    drains (own tiles, own scratch, own output; the append above finished before the first started)
+  for (int layer = 0; layer < k->layers; ++layer) {
+    const pmkvq_status s = attention_on_arena(k, layer, static_cast<const uint8_t *>(d_Q) + layer * q_stride,
+                                              d_out + layer * o_stride, st, layer > 0);
+    if (s != PMKVQ_OK) return s;
+  }
   return PMKVQ_OK;
 }
 
