@@ -58,9 +58,10 @@ __device__ __forceinline__ float chain_scale(float s16, int bits) {
 
 // Write one token's 128 codes (given as INT16 codes in shared memory) into a tile at `bits`,
 // applying the Eq. 3 chain; one warp, every half-word of the token is written by one lane.
-__device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, const uint16_t *codes16, int is_value,
-                                            int lane) {
-  const int n = 16 / bits;
+template <int BITS>
+__device__ __forceinline__ void store_token_w(uint8_t *part, int row, const uint16_t *codes16, int is_value, int lane) {
+  constexpr int bits = BITS;  // a compile-time width turns the index arithmetic below into shifts
+  constexpr int n = 16 / bits;
   const int r = row >> 3;
   for (int hw = lane; hw < 8 * bits; hw += 32) {
     const int w = hw >> 3, sub = hw & 7;
@@ -86,6 +87,16 @@ __device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, co
   }
 }
 
+__device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, const uint16_t *codes16, int is_value,
+                                            int lane) {
+  switch (bits) {
+    case 16: store_token_w<16>(part, row, codes16, is_value, lane); break;
+    case 8: store_token_w<8>(part, row, codes16, is_value, lane); break;
+    case 4: store_token_w<4>(part, row, codes16, is_value, lane); break;
+    default: store_token_w<2>(part, row, codes16, is_value, lane); break;
+  }
+}
+
 // Read one token's INT16 codes from a 16-bit tile into shared memory; one warp.
 __device__ __forceinline__ void load_token16(const uint8_t *part, int row, uint16_t *codes16, int is_value, int lane) {
   for (int ch = lane; ch < kHeadDim; ch += 32) {
@@ -101,23 +112,23 @@ __device__ __forceinline__ void load_token16(const uint8_t *part, int row, uint1
 // channels of the token; Keys are first multiplied by Lambda^-1 (Eq. 9).  The token goes to the
 // sink, straight to the body (bulk appends; Eq. 3 chain to the body width) or to the window ring.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int lane, const uint16_t *__restrict__ K,
-                                           const uint16_t *__restrict__ V, const float *__restrict__ inv_lambda,
-                                           unsigned *vmax_bits, const LayerGeom &geom, int n_slices, int kv_heads,
-                                           int n_old, int win_start, int cur_bits) {
-  const int is_value = (int)(wid & 1);
-  const long long ts = wid >> 1;
-  const int slice = (int)(ts % n_slices);
-  const int i = (int)(ts / n_slices);
-  const uint16_t *src = (is_value ? V : K) + ((size_t)i * n_slices + slice) * kHeadDim + lane * 4;
-  const uint2 raw = *reinterpret_cast<const uint2 *>(src);
+// Eq. 1-2 at 16 bit on one token's 128 channels (Keys first times Lambda^-1, Eq. 9), by one warp: lane l
+// holds channels 4l..4l+3.  Writes the codes to `codes` (shared memory) and returns S; Z goes to `zero`.
+__device__ __forceinline__ float quantize_token16(uint2 raw, const float *__restrict__ inv_lambda_head, uint16_t *codes,
+                                                  int lane, float &zero);
+__device__ __forceinline__ float quantize_token16(const uint16_t *__restrict__ src, const float *__restrict__ inv_lambda_head,
+                                                  uint16_t *codes, int lane, float &zero) {
+  return quantize_token16(*reinterpret_cast<const uint2 *>(src + lane * 4), inv_lambda_head, codes, lane, zero);
+}
+__device__ __forceinline__ float quantize_token16(uint2 raw, const float *__restrict__ inv_lambda_head, uint16_t *codes,
+                                                  int lane, float &zero) {
   float x[4];
   x[0] = __uint_as_float(raw.x << 16);
   x[1] = __uint_as_float(raw.x & 0xFFFF0000u);
   x[2] = __uint_as_float(raw.y << 16);
   x[3] = __uint_as_float(raw.y & 0xFFFF0000u);
-  if (!is_value) {
-    const float4 il = *reinterpret_cast<const float4 *>(inv_lambda + (size_t)(slice % kv_heads) * kHeadDim + lane * 4);
+  if (inv_lambda_head) {
+    const float4 il = *reinterpret_cast<const float4 *>(inv_lambda_head + lane * 4);
     x[0] = __fmul_rn(x[0], il.x);
     x[1] = __fmul_rn(x[1], il.y);
     x[2] = __fmul_rn(x[2], il.z);
@@ -140,6 +151,23 @@ __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int l
     }
     codes[lane * 4 + e] = (uint16_t)c;
   }
+  zero = mn;
+  return scale;
+}
+
+__device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int lane, const uint16_t *__restrict__ K,
+                                           const uint16_t *__restrict__ V, const float *__restrict__ inv_lambda,
+                                           unsigned *vmax_bits, const LayerGeom &geom, int n_slices, int kv_heads,
+                                           int n_old, int win_start, int cur_bits, int skip_lo = 0, int skip_hi = 0) {
+  const int is_value = (int)(wid & 1);
+  const long long ts = wid >> 1;
+  const int slice = (int)(ts % n_slices);
+  const int i = (int)(ts / n_slices);
+  if (n_old + i >= skip_lo && n_old + i < skip_hi) return;  // written tile-wise by append_tiles_kernel
+  const uint16_t *src = (is_value ? V : K) + ((size_t)i * n_slices + slice) * kHeadDim;
+  float mn;
+  const float scale = quantize_token16(src, is_value ? nullptr : inv_lambda + (size_t)(slice % kv_heads) * kHeadDim, codes,
+                                       lane, mn);
   __syncwarp();
   uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
   const TokenDest d = token_dest(geom, slice_base, n_old + i, win_start, cur_bits);
@@ -155,12 +183,66 @@ __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int l
 __global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
                                                      const float *__restrict__ inv_lambda, unsigned *vmax_bits,
                                                      LayerGeom geom, int n_new, int n_slices, int kv_heads,
-                                                     int n_old, int win_start, int cur_bits) {
+                                                     int n_old, int win_start, int cur_bits, int skip_lo, int skip_hi) {
   __shared__ uint16_t s_codes[4][kHeadDim];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wid = (long long)blockIdx.x * 4 + warp;
   if (wid >= (long long)n_new * n_slices * 2) return;
-  append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits);
+  append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits,
+             skip_lo, skip_hi);
+}
+
+// Bulk appends (prefill): body tiles that consist of new tokens only are built whole.  One warp per
+// (tile, slice, K|V) quantizes the tile's 16 tokens, assembles its code part in shared memory in the
+// tile layout (Eq. 3 chain to the body width included) and writes it out with 128-bit stores; a
+// token-at-a-time store would touch every 32-byte sector of the part for 2 bytes.
+__global__ void __launch_bounds__(128) append_tiles_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
+                                                           const float *__restrict__ inv_lambda, unsigned *vmax_bits,
+                                                           LayerGeom geom, int n_slices, int kv_heads, int n_old,
+                                                           int tile_lo, int n_tiles, int bits) {
+  __shared__ __align__(16) uint8_t s_part[4][256 * 16];
+  __shared__ __align__(16) float s_meta[4][32];  // this part's half of the tile's metadata, in tile order
+  __shared__ uint16_t s_codes[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wid = (long long)blockIdx.x * 4 + warp;
+  if (wid >= (long long)n_tiles * n_slices * 2) return;
+  const int is_value = (int)(wid & 1);
+  const int slice = (int)((wid >> 1) % n_slices);
+  const int tile = tile_lo + (int)((wid >> 1) / n_slices);
+  const float *il = is_value ? nullptr : inv_lambda + (size_t)(slice % kv_heads) * kHeadDim;
+  float smax = 0.f;
+  uint2 raw[kTileTokens];  // all 16 tokens in flight at once
+  {
+    const int i0 = geom.n_sink + tile * kTileTokens - n_old;  // index of the tile's first token among the new ones
+    const uint16_t *src = (is_value ? V : K) + ((size_t)i0 * n_slices + slice) * kHeadDim + lane * 4;
+#pragma unroll
+    for (int row = 0; row < kTileTokens; ++row)
+      raw[row] = *reinterpret_cast<const uint2 *>(src + (size_t)row * n_slices * kHeadDim);
+  }
+#pragma unroll
+  for (int row = 0; row < kTileTokens; ++row) {
+    float zero;
+    const float scale = quantize_token16(raw[row], il, s_codes[warp], lane, zero);
+    __syncwarp();
+    store_token(s_part[warp], bits, row, s_codes[warp], is_value, lane);
+    if (lane == 0) {  // meta_slot(kind, row) = tig*64 + kind*16 + i*4; this part keeps kinds {0,1} or {2,3}
+      const int tig = (row & 7) >> 1, idx = (row >> 3) * 2 + (row & 1);
+      s_meta[warp][tig * 8 + idx] = chain_scale(scale, bits);
+      s_meta[warp][tig * 8 + 4 + idx] = zero;
+    }
+    smax = fmaxf(smax, scale);
+    __syncwarp();
+  }
+  uint8_t *dst_tile = geom.base + (size_t)slice * geom.slice_stride + geom.body_off + (size_t)tile * tile_bytes(bits);
+  uint4 *dst = reinterpret_cast<uint4 *>(dst_tile + (is_value ? v_part_offset(bits) : 0));
+  const uint4 *srcp = reinterpret_cast<const uint4 *>(s_part[warp]);
+  for (int c = lane; c < 16 * bits; c += 32) dst[c] = srcp[c];
+  if (lane < 8) {  // 4 records x (S[4], Z[4]) -> byte tig*64 + (is_value ? 32 : 0) + {0, 16}
+    const int tig = lane >> 1, half = lane & 1;
+    *reinterpret_cast<uint4 *>(dst_tile + meta_offset(bits) + tig * 64 + (is_value ? 32 : 0) + half * 16) =
+        *reinterpret_cast<const uint4 *>(&s_meta[warp][tig * 8 + half * 4]);
+  }
+  if (is_value && lane == 0) atomicMax(vmax_bits + slice, __float_as_uint(smax));
 }
 
 // ---------------------------------------------------------------------------------------------
