@@ -66,6 +66,9 @@ typedef struct {
   float sm_scale;         /* softmax scale; 0 => 1/sqrt(head_dim) */
   void *d_arena;          /* DEVICE, 256-byte aligned, caller-owned, must outlive the cache */
   size_t arena_bytes;
+  int32_t shift_variant;  /* how a halving 2b -> b is done (Sec. 4.4.1): 0 Equivalent Right Shift, Eq. 3 (the
+                             method); 1 Direct Right Shift (X >> b, S_b = (2^b+1) S_2b, Z kept); 2 Modified
+                             Right Shift (X >> b, S_b = 2^b S_2b, Z_b = Z_2b + (S_b - S_2b)/2) */
 } pmkvq_config;
 
 /* Bytes of device arena a cache with this configuration needs (d_arena / arena_bytes are

@@ -12,7 +12,9 @@ What it computes, and the passage of the paper each part follows:
 * ``shift_reduce``            - "Equivalent Right Shift" 2b -> b, Eq. 3 (Sec. 3.1),
                                 with ``S_b = (2^b+1) S_2b`` and ``Z_b = Z_2b``.
 * ``direct_right_shift`` /
-  ``modified_right_shift``    - the two ablation variants of Sec. 4.4.1.
+  ``modified_right_shift``    - the two ablation variants of Sec. 4.4.1; ``halve`` /
+                                ``chain_variant`` apply the chosen one, and
+                                ``LayerOracle(shift_variant=...)`` runs the cache with it.
 * ``Policy``                  - progressive policy of Sec. 3.1: 16-bit first,
                                 halve the width of the existing cache when the
                                 block's budget is full, stop at Fbit; first token
@@ -39,6 +41,10 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
   decode_attention     pinned  (N=1, equal scores, brute force loops, library
                                 softmax-attention on the dequantized values,
                                 equalization invariance with power-of-two lambda)
+  direct / modified right shift
+                       pinned  (floor division by 2^b; dequantized value = centre of the
+                                merged bin for the modified variant; half-step error bound
+                                for Equivalent and Modified, 3/4 of a step for Direct)
   pack_canonical       pinned  (hand-written byte examples, round trip)
   accuracy on real models      parity unpinned (needs weights / benchmark items)
 """
@@ -108,6 +114,28 @@ def chain_to(codes16, s16, bits: int):
         w //= 2
         c, s = shift_reduce(c, w), reduce_scale(s, w)
     return c, s
+
+
+SHIFT_EQUIVALENT, SHIFT_DIRECT, SHIFT_MODIFIED = 0, 1, 2
+
+
+def halve(codes_2b, s_2b, z_2b, b: int, variant: int = SHIFT_EQUIVALENT):
+    """One halving 2b -> b of codes, scale and zero-point with the chosen shrinking strategy
+    (Sec. 3.1 for the Equivalent Right Shift, Sec. 4.4.1 for the two ablation variants)."""
+    if variant == SHIFT_DIRECT:
+        return direct_right_shift(codes_2b, s_2b, z_2b, b)
+    if variant == SHIFT_MODIFIED:
+        return modified_right_shift(codes_2b, s_2b, z_2b, b)
+    return shift_reduce(codes_2b, b), reduce_scale(s_2b, b), np.asarray(z_2b, dtype=np.float32)
+
+
+def chain_variant(codes16, s16, z16, bits: int, variant: int = SHIFT_EQUIVALENT):
+    """16 -> 8 -> ... -> ``bits`` with the chosen strategy, one halving after the other."""
+    c, s, z, w = np.asarray(codes16, np.uint16), np.asarray(s16, np.float32), np.asarray(z16, np.float32), 16
+    while w > bits:
+        w //= 2
+        c, s, z = halve(c, s, z, w, variant)
+    return c, s, z
 
 
 def direct_right_shift(codes_2b, s_2b, z_2b, b: int):
@@ -236,8 +264,9 @@ class LayerOracle:
     stored slice, shape [n_stored, 128] (all ones when None).
     """
 
-    def __init__(self, policy: Policy, n_stored: int, lam=None):
+    def __init__(self, policy: Policy, n_stored: int, lam=None, shift_variant: int = SHIFT_EQUIVALENT):
         self.p = policy
+        self.variant = shift_variant
         cap = policy.max_tokens
         self.S = n_stored
         self.lam = (np.ones((n_stored, HEAD_DIM), np.float32) if lam is None
@@ -260,10 +289,10 @@ class LayerOracle:
         b = p.cur_bits // 2
         lo, hi = p.n_sink_at(p.n_tokens), p.n_sink_at(p.n_tokens) + p.n_body_at(p.n_tokens)
         if hi > lo:
-            self.ck[:, lo:hi] = shift_reduce(self.ck[:, lo:hi], b)
-            self.cv[:, lo:hi] = shift_reduce(self.cv[:, lo:hi], b)
-            self.sk[:, lo:hi] = reduce_scale(self.sk[:, lo:hi], b)
-            self.sv[:, lo:hi] = reduce_scale(self.sv[:, lo:hi], b)
+            self.ck[:, lo:hi], self.sk[:, lo:hi], self.zk[:, lo:hi] = halve(
+                self.ck[:, lo:hi], self.sk[:, lo:hi], self.zk[:, lo:hi], b, self.variant)
+            self.cv[:, lo:hi], self.sv[:, lo:hi], self.zv[:, lo:hi] = halve(
+                self.cv[:, lo:hi], self.sv[:, lo:hi], self.zv[:, lo:hi], b, self.variant)
             self.bits[lo:hi] = b
         p.cur_bits = b
         self.n_reduces += 1
@@ -292,8 +321,10 @@ class LayerOracle:
         for e in range(old_body_end, new_body_end):      # tokens leaving the INT16 window
             if e < p.n_sink:
                 continue
-            self.ck[:, e], self.sk[:, e] = chain_to(self.ck[:, e], self.sk[:, e], p.cur_bits)
-            self.cv[:, e], self.sv[:, e] = chain_to(self.cv[:, e], self.sv[:, e], p.cur_bits)
+            self.ck[:, e], self.sk[:, e], self.zk[:, e] = chain_variant(
+                self.ck[:, e], self.sk[:, e], self.zk[:, e], p.cur_bits, self.variant)
+            self.cv[:, e], self.sv[:, e], self.zv[:, e] = chain_variant(
+                self.cv[:, e], self.sv[:, e], self.zv[:, e], p.cur_bits, self.variant)
             self.bits[e] = p.cur_bits
 
     def append(self, k, v, auto_reduce=True):
@@ -329,8 +360,10 @@ class LayerOracle:
         new_body_end = p.n_sink_at(n_after) + p.n_body_at(n_after)
         lo, hi = max(old_body_end, p.n_sink), new_body_end
         if hi > lo:
-            self.ck[:, lo:hi], self.sk[:, lo:hi] = chain_to(self.ck[:, lo:hi], self.sk[:, lo:hi], p.cur_bits)
-            self.cv[:, lo:hi], self.sv[:, lo:hi] = chain_to(self.cv[:, lo:hi], self.sv[:, lo:hi], p.cur_bits)
+            self.ck[:, lo:hi], self.sk[:, lo:hi], self.zk[:, lo:hi] = chain_variant(
+                self.ck[:, lo:hi], self.sk[:, lo:hi], self.zk[:, lo:hi], p.cur_bits, self.variant)
+            self.cv[:, lo:hi], self.sv[:, lo:hi], self.zv[:, lo:hi] = chain_variant(
+                self.cv[:, lo:hi], self.sv[:, lo:hi], self.zv[:, lo:hi], p.cur_bits, self.variant)
             self.bits[lo:hi] = p.cur_bits
 
     # -- Eq. 9 + softmax attention over all cached tokens ------------------------

@@ -18,6 +18,7 @@ struct LayerGeom {
   size_t body_off;      // byte offset of the body inside a slice
   int n_sink;           // leading INT16 tokens (stored in tiles at offset 0)
   int ring_tokens;      // ring capacity in tokens (multiple of 16)
+  int shift_variant;    // ShiftVariant of this cache
 };
 
 struct TokenDest {
@@ -50,16 +51,34 @@ __device__ __forceinline__ TokenDest token_dest(const LayerGeom &g, uint8_t *sli
 }
 
 // Scale after the chain 16 -> ... -> bits: S_b = (2^b + 1) S_2b, one fp32 rounding per step (Sec. 3.1).
-__device__ __forceinline__ float chain_scale(float s16, int bits) {
+__device__ __forceinline__ float chain_scale(float s16, int bits, int variant = kShiftEquivalent) {
   float s = s16;
-  for (int w = 8; w >= bits; w >>= 1) s = __fmul_rn(s, (float)((1 << w) + 1));
+  for (int w = 8; w >= bits; w >>= 1) s = __fmul_rn(s, (float)((1 << w) + (variant == kShiftModified ? 0 : 1)));
   return s;
+}
+// One halving of the metadata of one token: (S_2b, Z_2b) -> (S_b, Z_b), each step one fp32 rounding.
+__device__ __forceinline__ void halve_meta(float &s, float &z, int b, int variant) {
+  if (variant == kShiftModified) {
+    const float sb = __fmul_rn(s, (float)(1 << b));
+    z = __fadd_rn(z, __fmul_rn(__fsub_rn(sb, s), 0.5f));
+    s = sb;
+  } else {
+    s = __fmul_rn(s, (float)((1 << b) + 1));
+  }
+}
+// Zero-point after the chain 16 -> ... -> bits (it only moves under the modified right shift).
+__device__ __forceinline__ float chain_zero(float z16, float s16, int bits, int variant) {
+  float s = s16, z = z16;
+  if (variant == kShiftModified)
+    for (int w = 8; w >= bits; w >>= 1) halve_meta(s, z, w, variant);
+  return z;
 }
 
 // Write one token's 128 codes (given as INT16 codes in shared memory) into a tile at `bits`,
 // applying the Eq. 3 chain; one warp, every half-word of the token is written by one lane.
 template <int BITS>
-__device__ __forceinline__ void store_token_w(uint8_t *part, int row, const uint16_t *codes16, int is_value, int lane) {
+__device__ __forceinline__ void store_token_w(uint8_t *part, int row, const uint16_t *codes16, int is_value, int lane,
+                                              int variant) {
   constexpr int bits = BITS;  // a compile-time width turns the index arithmetic below into shifts
   constexpr int n = 16 / bits;
   const int r = row >> 3;
@@ -79,7 +98,7 @@ __device__ __forceinline__ void store_token_w(uint8_t *part, int row, const uint
     uint32_t val = 0;
     for (int j = 0; j < n; ++j) {
       const int ch = chan_step * (w * n + j) + chan0;
-      val |= shift_chain(codes16[ch], bits) << (j * bits);
+      val |= shift_chain(codes16[ch], bits, variant) << (j * bits);
     }
     int byte_off, bit_off;
     lane_slot(bits, owner, r, w * n, h, byte_off, bit_off);
@@ -88,12 +107,12 @@ __device__ __forceinline__ void store_token_w(uint8_t *part, int row, const uint
 }
 
 __device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, const uint16_t *codes16, int is_value,
-                                            int lane) {
+                                            int lane, int variant) {
   switch (bits) {
-    case 16: store_token_w<16>(part, row, codes16, is_value, lane); break;
-    case 8: store_token_w<8>(part, row, codes16, is_value, lane); break;
-    case 4: store_token_w<4>(part, row, codes16, is_value, lane); break;
-    default: store_token_w<2>(part, row, codes16, is_value, lane); break;
+    case 16: store_token_w<16>(part, row, codes16, is_value, lane, variant); break;
+    case 8: store_token_w<8>(part, row, codes16, is_value, lane, variant); break;
+    case 4: store_token_w<4>(part, row, codes16, is_value, lane, variant); break;
+    default: store_token_w<2>(part, row, codes16, is_value, lane, variant); break;
   }
 }
 
@@ -171,11 +190,11 @@ __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int l
   __syncwarp();
   uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
   const TokenDest d = token_dest(geom, slice_base, n_old + i, win_start, cur_bits);
-  store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, codes, is_value, lane);
+  store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, codes, is_value, lane, geom.shift_variant);
   if (lane == 0) {
     float *meta = reinterpret_cast<float *>(d.tile + meta_offset(d.bits));
-    meta[meta_slot(is_value ? 2 : 0, d.row) >> 2] = chain_scale(scale, d.bits);
-    meta[meta_slot(is_value ? 3 : 1, d.row) >> 2] = mn;
+    meta[meta_slot(is_value ? 2 : 0, d.row) >> 2] = chain_scale(scale, d.bits, geom.shift_variant);
+    meta[meta_slot(is_value ? 3 : 1, d.row) >> 2] = chain_zero(mn, scale, d.bits, geom.shift_variant);
     if (is_value) atomicMax(vmax_bits + slice, __float_as_uint(scale));  // scale >= 0: uint order = float order
   }
 }
@@ -224,11 +243,11 @@ __global__ void __launch_bounds__(128) append_tiles_kernel(const uint16_t *__res
     float zero;
     const float scale = quantize_token16(raw[row], il, s_codes[warp], lane, zero);
     __syncwarp();
-    store_token(s_part[warp], bits, row, s_codes[warp], is_value, lane);
+    store_token(s_part[warp], bits, row, s_codes[warp], is_value, lane, geom.shift_variant);
     if (lane == 0) {  // meta_slot(kind, row) = tig*64 + kind*16 + i*4; this part keeps kinds {0,1} or {2,3}
       const int tig = (row & 7) >> 1, idx = (row >> 3) * 2 + (row & 1);
-      s_meta[warp][tig * 8 + idx] = chain_scale(scale, bits);
-      s_meta[warp][tig * 8 + 4 + idx] = zero;
+      s_meta[warp][tig * 8 + idx] = chain_scale(scale, bits, geom.shift_variant);
+      s_meta[warp][tig * 8 + 4 + idx] = chain_zero(zero, scale, bits, geom.shift_variant);
     }
     smax = fmaxf(smax, scale);
     __syncwarp();
@@ -266,11 +285,12 @@ __device__ __forceinline__ void evict_one(long long wid, uint16_t *codes, int la
   __syncwarp();
   const int j = t - geom.n_sink;
   uint8_t *dst_tile = slice_base + geom.body_off + (size_t)(j >> 4) * tile_bytes(cur_bits);
-  store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, codes, is_value, lane);
+  store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, codes, is_value, lane,
+              geom.shift_variant);
   if (lane == 0) {
     float *meta = reinterpret_cast<float *>(dst_tile + meta_offset(cur_bits));
-    meta[meta_slot(is_value ? 2 : 0, j & 15) >> 2] = chain_scale(s16, cur_bits);
-    meta[meta_slot(is_value ? 3 : 1, j & 15) >> 2] = z;
+    meta[meta_slot(is_value ? 2 : 0, j & 15) >> 2] = chain_scale(s16, cur_bits, geom.shift_variant);
+    meta[meta_slot(is_value ? 3 : 1, j & 15) >> 2] = chain_zero(z, s16, cur_bits, geom.shift_variant);
   }
 }
 
@@ -351,7 +371,7 @@ __global__ void __launch_bounds__(128) append_step_kernel(const uint16_t *__rest
   }
 }
 
-template <int B>
+template <int B, bool SHR>
 __device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1) {
   constexpr int NIN = 8 / B;  // codes per half-word at 2B bits
   constexpr uint32_t MASK = (1u << (2 * B)) - 1u;
@@ -362,15 +382,15 @@ __device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1) {
     for (int j = 0; j < NIN; ++j) {
       const uint32_t c0 = (in0 >> (16 * h + j * 2 * B)) & MASK;
       const uint32_t c1 = (in1 >> (16 * h + j * 2 * B)) & MASK;
-      out |= shift_step(c0, B) << (16 * h + j * B);
-      out |= shift_step(c1, B) << (16 * h + (NIN + j) * B);
+      out |= (SHR ? c0 >> B : shift_step(c0, B)) << (16 * h + j * B);
+      out |= (SHR ? c1 >> B : shift_step(c1, B)) << (16 * h + (NIN + j) * B);
     }
   }
   return out;
 }
 
-template <int B>
-__device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int lane) {
+template <int B, bool SHR>
+__device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, int lane, int variant) {
   constexpr int IN_CHUNKS = B;                          // 16-byte chunks per lane per part at 2B bits
   constexpr int OUT_WORDS = 2 * B;                      // words per lane per part at B bits
   constexpr int OUT_CHUNKS = (OUT_WORDS + 3) / 4;
@@ -388,14 +408,21 @@ __device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int
 #pragma unroll
     for (int lw = 0; lw < OUT_WORDS; ++lw) {
       const int r = lw / B, wp = lw % B;
-      o[part][lw] = merge_words<B>(w[r * 2 * B + 2 * wp], w[r * 2 * B + 2 * wp + 1]);
+      o[part][lw] = merge_words<B, SHR>(w[r * 2 * B + 2 * wp], w[r * 2 * B + 2 * wp + 1]);
     }
   }
   float2 m = *reinterpret_cast<const float2 *>(in + meta_offset(2 * B) + lane * 8);
   const int kind = ((2 * lane) & 15) >> 2;  // 0 S_K, 1 Z_K, 2 S_V, 3 Z_V
+  // a zero-point lane finds the scales of its two tokens two lanes below (16 bytes earlier)
+  const float s_x = __shfl_up_sync(0xffffffffu, m.x, 2), s_y = __shfl_up_sync(0xffffffffu, m.y, 2);
   if ((kind & 1) == 0) {
-    m.x = __fmul_rn(m.x, (float)((1 << B) + 1));
-    m.y = __fmul_rn(m.y, (float)((1 << B) + 1));
+    float unused = 0.f;
+    halve_meta(m.x, unused, B, variant);
+    halve_meta(m.y, unused, B, variant);
+  } else if (variant == kShiftModified) {
+    float sx = s_x, sy = s_y;
+    halve_meta(sx, m.x, B, variant);
+    halve_meta(sy, m.y, B, variant);
   }
   __syncwarp();  // every lane holds its transformed data: the tile's input is dead from here on
 #pragma unroll
@@ -410,13 +437,19 @@ __device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int
   *reinterpret_cast<float2 *>(out + meta_offset(B) + lane * 8) = m;
 }
 
+template <int B>
+__device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int lane, int variant) {
+  if (variant == kShiftEquivalent) reduce_tile_v<B, false>(in, out, lane, variant);
+  else reduce_tile_v<B, true>(in, out, lane, variant);
+}
+
 // First tiles of every slice, one warp per slice, in order (tile i's output overlaps inputs <= i only).
 template <int B>
 __global__ void __launch_bounds__(32) reduce_head_kernel(LayerGeom geom, int n_tiles) {
   uint8_t *body = geom.base + (size_t)blockIdx.x * geom.slice_stride + geom.body_off;
   const int lane = threadIdx.x;
   for (int i = 0; i < n_tiles; ++i) {
-    reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), lane);
+    reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), lane, geom.shift_variant);
     __syncwarp();
   }
 }
@@ -428,7 +461,8 @@ __global__ void __launch_bounds__(128) reduce_wave_kernel(LayerGeom geom, int lo
   const int i = lo + blockIdx.x * 4 + (threadIdx.x >> 5);
   if (i >= hi) return;
   uint8_t *body = geom.base + (size_t)blockIdx.y * geom.slice_stride + geom.body_off;
-  reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), threadIdx.x & 31);
+  reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), threadIdx.x & 31,
+                 geom.shift_variant);
 }
 
 }  // namespace pmkvq

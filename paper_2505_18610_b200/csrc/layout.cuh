@@ -80,8 +80,15 @@ PMKVQ_HD uint32_t shift_step(uint32_t c, int b) {
   return (mult * (c + (1u << (b - 1)))) >> (3 * b);
 }
 
+// How a halving 2b -> b treats codes and metadata (Sec. 4.4.1 compares the three):
+//   kShiftEquivalent  Eq. 3,          S_b = (2^b+1) S_2b, Z unchanged            (the method)
+//   kShiftDirect      X_b = X_2b >> b, S_b = (2^b+1) S_2b, Z unchanged            (ablation 1)
+//   kShiftModified    X_b = X_2b >> b, S_b = 2^b S_2b,     Z_b = Z_2b + (S_b - S_2b)/2  (ablation 2)
+enum ShiftVariant { kShiftEquivalent = 0, kShiftDirect = 1, kShiftModified = 2 };
+
 // 16-bit code -> `bits`-bit code through the chain 16 -> 8 -> 4 -> 2.
-PMKVQ_HD uint32_t shift_chain(uint32_t c16, int bits) {
+PMKVQ_HD uint32_t shift_chain(uint32_t c16, int bits, int variant = kShiftEquivalent) {
+  if (variant != kShiftEquivalent) return c16 >> (16 - bits);  // b right shifts per halving add up
   uint32_t c = c16;
   for (int w = 8; w >= bits; w >>= 1) c = shift_step(c, w);
   return c;

@@ -43,7 +43,7 @@ struct Layer {
 
 struct pmkvq_cache {
   int layers, q_heads, kv_heads, batch, max_tokens, group, n_slices;
-  int n_sink, window, evict_chunk, count_metadata, auto_reduce;
+  int n_sink, window, evict_chunk, count_metadata, auto_reduce, shift_variant;
   float sm_scale;
   uint8_t *arena;
   size_t arena_bytes;
@@ -78,6 +78,7 @@ struct pmkvq_cache {
     g.body_off = g.ring_off + (size_t)ring_tiles * tile_bytes(16);
     g.n_sink = n_sink;
     g.ring_tokens = ring_tiles * 16;
+    g.shift_variant = shift_variant;
     return g;
   }
 };
@@ -95,6 +96,7 @@ bool check_config(const pmkvq_config *c) {
   for (int i = 0; i < c->layers; ++i)
     if (!valid_bits(c->fbit[i])) return false;
   if (c->n_sink < 0 || c->window < 0 || c->evict_chunk < 1) return false;
+  if (c->shift_variant < 0 || c->shift_variant > 2) return false;
   if ((int64_t)c->n_sink + c->window + c->evict_chunk > (1 << 24)) return false;
   if ((int64_t)c->batch * c->kv_heads > 65535) return false;
   if (c->lambda) {
@@ -112,6 +114,7 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.max_tokens = c->max_tokens; k.group = c->q_heads / c->kv_heads; k.n_slices = c->batch * c->kv_heads;
   k.n_sink = c->n_sink; k.window = c->window; k.evict_chunk = c->evict_chunk;
   k.count_metadata = c->count_metadata ? 1 : 0; k.auto_reduce = c->auto_reduce ? 1 : 0;
+  k.shift_variant = c->shift_variant;
   k.sm_scale = c->sm_scale > 0.0f ? c->sm_scale : 1.0f / std::sqrt((float)kHeadDim);
   k.sink_tiles = (k.n_sink + 15) / 16;
   k.ring_tiles = std::max(1, (k.window + k.evict_chunk - 1 + 15) / 16 + 1);

@@ -30,11 +30,12 @@ class Mirror:
         self.cache = Cache(layers, q_heads, kv_heads, batch, max_tokens, fbit, budget_bytes=budget_bytes,
                            lam=self.lam, **kw)
         okw = {k: kw[k] for k in ("n_sink", "window", "evict_chunk", "count_metadata") if k in kw}
+        variant = kw.get("shift_variant", 0)
         self.oracles = []
         for l in range(layers):
             pol = O.Policy(fbit[l], max_tokens, n_slices, None if budget_bytes is None else budget_bytes[l], **okw)
             lam_s = None if self.lam is None else np.stack([self.lam[l, s % kv_heads] for s in self.slices])
-            self.oracles.append(O.LayerOracle(pol, len(self.slices), lam=lam_s))
+            self.oracles.append(O.LayerOracle(pol, len(self.slices), lam=lam_s, shift_variant=variant))
 
     def append(self, layer, k, v, bulk=True):
         """k, v: CPU or CUDA bf16 [n, batch, kv_heads, 128]."""

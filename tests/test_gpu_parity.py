@@ -198,3 +198,20 @@ def test_decode_step_over_all_blocks():
     for l in range(layers):
         m.check_state(l)
         assert m.cache.layer_state(l)["cur_bits"] == fbit[l]
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_shift_variants_direct_and_modified(variant):
+    """The two ablation strategies of Sec. 4.4.1 as cache options: bulk appends, evictions through the
+    chain and progressive reduces down to 2 bit, state bit-exact and attention within tolerance."""
+    layers, kvh, batch, group, n = 2, 2, 2, 4, 900
+    m = Mirror(layers, group * kvh, kvh, batch, n, [2, 4], window=32, shift_variant=variant)
+    for l in range(layers):
+        k, v = make_inputs(10 + variant, l, n, batch, kvh)
+        m.append(l, k[:500], v[:500])
+        for t in range(500, 560):
+            m.append(l, k[t:t + 1], v[t:t + 1], bulk=False)
+        m.append(l, k[560:], v[560:])
+        m.check_state(l)
+        assert m.cache.layer_state(l)["cur_bits"] == [2, 4][l]
+        m.check_attention(l, synth.make_q(10, l, 0, batch, group * kvh, n))

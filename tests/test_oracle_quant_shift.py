@@ -156,6 +156,40 @@ def test_ablation_shift_variants():
         assert np.isclose(sm * q + zm, lv4[4 * q: 4 * q + 4].mean())
 
 
+def test_shift_variant_chains_and_error_ordering():
+    """Chains of the three shrinking strategies (Sec. 4.4.1).  Direct / Modified codes are the upper
+    bits of the INT16 code; Modified dequantizes to the centre of the merged bin; on N(0,1) groups the
+    mean squared reconstruction error after 16 -> 2 orders as Equivalent < Modified < Direct, the
+    mechanics behind the accuracy ordering of Table 4."""
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((512, 128)).astype(np.float32)
+    c16, s16, z16 = O.quantize_asym(x, 16)
+    mse = {}
+    for variant in (O.SHIFT_EQUIVALENT, O.SHIFT_DIRECT, O.SHIFT_MODIFIED):
+        for bits in (8, 4, 2):
+            c, s, z = O.chain_variant(c16, s16, z16, bits, variant)
+            assert c.max() <= (1 << bits) - 1
+            if variant != O.SHIFT_EQUIVALENT:
+                assert np.array_equal(c, c16 >> (16 - bits))
+            if variant == O.SHIFT_MODIFIED:     # level = centre of the 2^(16-bits) fine levels it replaces
+                k = 1 << (16 - bits)
+                centre = s16.astype(np.float64) * (k - 1) / 2 + z16
+                assert np.allclose(z, centre, rtol=1e-5, atol=1e-6)
+                assert np.allclose(s, s16.astype(np.float64) * k, rtol=1e-6)
+            if variant == O.SHIFT_EQUIVALENT:
+                c_ref, s_ref = O.chain_to(c16, s16, bits)
+                assert np.array_equal(c, c_ref) and np.array_equal(s, s_ref) and np.array_equal(z, z16)
+        err = np.abs(O.dequantize(c, s, z) - x)            # c, s, z: the 2-bit end of the chain
+        step = s.astype(np.float64)[:, None]
+        if variant == O.SHIFT_DIRECT:
+            # bins of a quarter of the range, levels a third apart: off by up to 3/4 of a step at the ends
+            assert (err <= step * 0.75 * 1.001 + s16[:, None]).all() and (err > step * 0.6).any()
+        else:
+            assert (err <= step * 0.5 * 1.001 + s16[:, None]).all()
+        mse[variant] = float(np.mean(err ** 2))
+    assert mse[O.SHIFT_EQUIVALENT] < mse[O.SHIFT_DIRECT] and mse[O.SHIFT_MODIFIED] < mse[O.SHIFT_DIRECT]
+
+
 # -------------------------------------------------------------- packing ----
 def test_canonical_packing_hand_and_roundtrip():
     codes = np.zeros(128, np.uint16)
