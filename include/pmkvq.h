@@ -159,6 +159,24 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *cache, int32_t layer, int32_t batch
                                 int32_t is_value, uint16_t *h_codes, float *h_scale, float *h_zero,
                                 uint8_t *h_bits, uint8_t *h_packed);
 
+/* Block-wise bit allocation (Sec. 3.2, Eq. 6-8), host only: choose one bit width per block so that the
+ * summed sensitivity is minimal and the summed memory stays within the budget,
+ *     min  sum_i s[i][c_i]   s.t.  sum_i mem[i][c_i] <= budget,   c_i in {0 .. n_choices-1}.
+ * Solved exactly as a multiple-choice knapsack by dynamic programming over memory in units of the
+ * greatest common divisor of the memory differences (blocks of one model share their shapes, so the
+ * table is tiny); ties are broken towards less memory, then towards the lower choice index in the
+ * earlier block.
+ *   h_widths       HOST [n_choices]           the candidate widths, e.g. {2, 4} (B of Eq. 8)
+ *   h_sensitivity  HOST [layers][n_choices]   s_{i,b} of Eq. 5 (finite, any sign)
+ *   h_mem_bytes    HOST [layers][n_choices]   Mem of block i at width b
+ *   h_fbit_out     HOST [layers]              chosen width per block (a pmkvq_config.fbit array)
+ *   h_cost_out     HOST, may be NULL          the minimal summed sensitivity
+ * Returns PMKVQ_ERR_CAPACITY if even the smallest choice of every block exceeds the budget and
+ * PMKVQ_ERR_INVALID_ARG for bad arguments or a table beyond 2^26 cells. */
+pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_t *h_widths,
+                                 const double *h_sensitivity, const uint64_t *h_mem_bytes, uint64_t budget_bytes,
+                                 uint8_t *h_fbit_out, double *h_cost_out);
+
 const char *pmkvq_status_string(pmkvq_status s);
 
 #ifdef __cplusplus

@@ -45,6 +45,9 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
                        pinned  (floor division by 2^b; dequantized value = centre of the
                                 merged bin for the modified variant; half-step error bound
                                 for Equivalent and Modified, 3/4 of a step for Direct)
+  allocate_bits_brute_force
+                       pinned  (it IS the definition of Eq. 6-8 written out; limits: budget at
+                                the floor / unbounded; hand case)
   pack_canonical       pinned  (hand-written byte examples, round trip)
   accuracy on real models      parity unpinned (needs weights / benchmark items)
 """
@@ -394,3 +397,36 @@ class LayerOracle:
         if is_value:
             return self.cv[s, :n].copy(), self.sv[s, :n].copy(), self.zv[s, :n].copy(), self.bits[:n].copy()
         return self.ck[s, :n].copy(), self.sk[s, :n].copy(), self.zk[s, :n].copy(), self.bits[:n].copy()
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.2: block-wise bit allocation (Eq. 6-8) and the sensitivity stand-in
+# --------------------------------------------------------------------------
+def allocate_bits_brute_force(sensitivity, mem_bytes, budget_bytes):
+    """Eq. 6-8 by exhaustive search: one choice per block, minimal summed sensitivity subject to the
+    summed memory <= budget.  Returns (choice index per block, cost) or (None, inf) if nothing fits.
+    Ties: less memory first, then the lexicographically smallest choice vector.  Small inputs only."""
+    import itertools
+    sens = np.asarray(sensitivity, dtype=np.float64)
+    mem = np.asarray(mem_bytes, dtype=np.int64)
+    layers, c = sens.shape
+    best = (np.inf, np.inf, None)
+    for combo in itertools.product(range(c), repeat=layers):
+        m = int(sum(mem[i, combo[i]] for i in range(layers)))
+        if m > budget_bytes:
+            continue
+        s = float(sum(sens[i, combo[i]] for i in range(layers)))
+        if (s, m, combo) < best:
+            best = (s, m, combo)
+    return (None, np.inf) if best[2] is None else (list(best[2]), best[0])
+
+
+def quantization_sensitivity(k, v, bits: int):
+    """Stand-in for Eq. 5 without the gradient factor (it needs the model): ||K - Q_b(K)||_1 +
+    ||V - Q_b(V)||_1 with the per-token group quantizer of Eq. 1-2 at ``bits``."""
+    total = 0.0
+    for x in (k, v):
+        x = np.asarray(x, dtype=np.float32)
+        c, s, z = quantize_asym(x, bits)
+        total += float(np.abs(dequantize(c, s, z) - x).sum())
+    return total

@@ -70,6 +70,8 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_attention_bytes.argtypes = [vp, i32]
     lib.pmkvq_export_slice.restype = i32
     lib.pmkvq_export_slice.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.pmkvq_allocate_bits.restype = i32
+    lib.pmkvq_allocate_bits.argtypes = [i32, i32, vp, vp, vp, ctypes.c_uint64, vp, vp]
     lib.pmkvq_status_string.restype = ctypes.c_char_p
     lib.pmkvq_status_string.argtypes = [i32]
     return lib
@@ -88,6 +90,24 @@ def lib() -> ctypes.CDLL:
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     s = stream if stream is not None else torch.cuda.current_stream()
     return s.cuda_stream
+
+
+def allocate_bits(widths, sensitivity, mem_bytes, budget_bytes):
+    """Block-wise bit allocation (Eq. 6-8): widths [C], sensitivity and mem_bytes [layers, C] ->
+    (fbit per block as a list, minimal summed sensitivity).  Host only."""
+    sens = np.ascontiguousarray(sensitivity, dtype=np.float64)
+    mem = np.ascontiguousarray(mem_bytes, dtype=np.uint64)
+    w = np.ascontiguousarray(widths, dtype=np.uint8)
+    layers, c = sens.shape
+    if mem.shape != sens.shape or w.shape != (c,):
+        raise ValueError("bad shapes")
+    out = np.zeros(layers, np.uint8)
+    cost = ctypes.c_double()
+    st = lib().pmkvq_allocate_bits(layers, c, w.ctypes.data, sens.ctypes.data, mem.ctypes.data, int(budget_bytes),
+                                   out.ctypes.data, ctypes.addressof(cost))
+    if st != OK:
+        raise PmkvqError(st, "pmkvq_allocate_bits")
+    return out.tolist(), cost.value
 
 
 class Cache:

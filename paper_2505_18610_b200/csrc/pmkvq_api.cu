@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <limits>
 #include <new>
 #include <vector>
 
@@ -618,6 +619,68 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
 pmkvq_status pmkvq_set_attention_ctas(pmkvq_cache *k, int32_t n_ctas) {
   if (!k || n_ctas < 0 || n_ctas > kMaxCtas) return PMKVQ_ERR_INVALID_ARG;
   k->user_ctas = n_ctas;
+  return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_t *h_widths, const double *h_sens,
+                                 const uint64_t *h_mem, uint64_t budget, uint8_t *h_fbit_out, double *h_cost_out) {
+  if (layers <= 0 || n_choices <= 0 || n_choices > 8 || !h_widths || !h_sens || !h_mem || !h_fbit_out)
+    return PMKVQ_ERR_INVALID_ARG;
+  for (int i = 0; i < layers * n_choices; ++i)
+    if (!std::isfinite(h_sens[i])) return PMKVQ_ERR_INVALID_ARG;
+  // memory above each block's smallest choice, in units of the gcd of those differences
+  std::vector<uint64_t> base(layers), extra((size_t)layers * n_choices);
+  uint64_t floor_sum = 0, g = 0;
+  for (int i = 0; i < layers; ++i) {
+    base[i] = *std::min_element(h_mem + (size_t)i * n_choices, h_mem + (size_t)(i + 1) * n_choices);
+    floor_sum += base[i];
+    for (int c = 0; c < n_choices; ++c) {
+      uint64_t d = h_mem[(size_t)i * n_choices + c] - base[i], a = g;
+      extra[(size_t)i * n_choices + c] = d;
+      while (d) { const uint64_t t = a % d; a = d; d = t; }
+      g = a;
+    }
+  }
+  if (floor_sum > budget) return PMKVQ_ERR_CAPACITY;
+  if (g == 0) g = 1;  // all choices of every block cost the same
+  uint64_t max_extra = 0;
+  for (int i = 0; i < layers; ++i) {
+    uint64_t m = 0;
+    for (int c = 0; c < n_choices; ++c) m = std::max(m, extra[(size_t)i * n_choices + c] / g);
+    max_extra += m;
+  }
+  const uint64_t cap = std::min((budget - floor_sum) / g, max_extra);
+  if ((cap + 1) * (uint64_t)layers > (1ull << 26)) return PMKVQ_ERR_INVALID_ARG;
+  const size_t W = (size_t)cap + 1;
+  const double inf = std::numeric_limits<double>::infinity();
+  // best[i][w]: minimal sensitivity of blocks 0..i-1 using exactly w units; pick[i][w]: choice of block i-1
+  std::vector<double> prev(W, inf), cur(W);
+  std::vector<int8_t> pick((size_t)layers * W, -1);
+  prev[0] = 0.0;
+  for (int i = 0; i < layers; ++i) {
+    std::fill(cur.begin(), cur.end(), inf);
+    for (int c = 0; c < n_choices; ++c) {
+      const uint64_t wc = extra[(size_t)i * n_choices + c] / g;
+      const double sc = h_sens[(size_t)i * n_choices + c];
+      for (size_t w = wc; w < W; ++w) {
+        const double v = prev[w - wc] + sc;
+        if (v < cur[w]) { cur[w] = v; pick[(size_t)i * W + w] = (int8_t)c; }  // strict: the lower index wins ties
+      }
+    }
+    prev.swap(cur);
+  }
+  size_t best_w = 0;
+  for (size_t w = 1; w < W; ++w)
+    if (prev[w] < prev[best_w]) best_w = w;  // strict: less memory wins ties
+  if (!(prev[best_w] < inf)) return PMKVQ_ERR_STATE;
+  if (h_cost_out) *h_cost_out = prev[best_w];
+  size_t w = best_w;
+  for (int i = layers - 1; i >= 0; --i) {
+    const int c = pick[(size_t)i * W + w];
+    if (c < 0) return PMKVQ_ERR_STATE;
+    h_fbit_out[i] = h_widths[c];
+    w -= (size_t)(extra[(size_t)i * n_choices + c] / g);
+  }
   return PMKVQ_OK;
 }
 
