@@ -159,6 +159,18 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *cache, int32_t layer, int32_t batch
                                 int32_t is_value, uint16_t *h_codes, float *h_scale, float *h_zero,
                                 uint8_t *h_bits, uint8_t *h_packed);
 
+/* Calibration of the equalization vector with positional interpolation (Sec. 3.3, Eq. 10-12), on the
+ * device: pre-RoPE Keys are rotated with RoPE whose position index is multiplied by pos_scale (Eq. 12;
+ * 1.0 = plain RoPE, Eq. 11; pairs (i, i + 64), theta_i = theta^(-2i/128)), and
+ *     lambda[h][i] = max( max over tokens and sequences |K_rot[.., h, i]| , floor )^alpha      (Eq. 10).
+ *   d_K_pre_bf16  DEVICE bf16 [n_tokens][n_seq][kv_heads][128], token t sits at position t
+ *   d_lambda      DEVICE fp32 [kv_heads][128], written (it also serves as the kernel's only workspace)
+ * The rotation is computed in fp32 from fp64 angles; the result feeds pmkvq_config.lambda after a copy to
+ * the host.  The grid search over alpha of Sec. 4.1.1 is left to the caller (alpha is an argument). */
+pmkvq_status pmkvq_calibrate_lambda(const void *d_K_pre_bf16, int32_t n_tokens, int32_t n_seq, int32_t kv_heads,
+                                    double pos_scale, double theta, float alpha, float floor_value, float *d_lambda,
+                                    void *stream);
+
 /* Block-wise bit allocation (Sec. 3.2, Eq. 6-8), host only: choose one bit width per block so that the
  * summed sensitivity is minimal and the summed memory stays within the budget,
  *     min  sum_i s[i][c_i]   s.t.  sum_i mem[i][c_i] <= budget,   c_i in {0 .. n_choices-1}.

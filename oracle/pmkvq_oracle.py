@@ -45,6 +45,12 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
                        pinned  (floor division by 2^b; dequantized value = centre of the
                                 merged bin for the modified variant; half-step error bound
                                 for Equivalent and Modified, 3/4 of a step for Direct)
+  rope_interpolated / calibrate_lambda
+                       pinned  (norm of every rotated pair is kept; one constant pair sweeps the
+                                closed form r*|cos(m s theta_i + phi)|; s = 4 on n tokens equals
+                                s = 1 at positions 0, 4, 8, ...; with the lowest-frequency pair's
+                                2 pi / theta_i = 54,410-token period (Sec. 3.3) a 2,048-token text
+                                reaches the pair's full amplitude only with interpolation)
   allocate_bits_brute_force
                        pinned  (it IS the definition of Eq. 6-8 written out; limits: budget at
                                 the floor / unbounded; hand case)
@@ -430,3 +436,30 @@ def quantization_sensitivity(k, v, bits: int):
         c, s, z = quantize_asym(x, bits)
         total += float(np.abs(dequantize(c, s, z) - x).sum())
     return total
+
+
+# --------------------------------------------------------------------------
+# Sec. 3.3: calibration of Lambda with positional interpolation (Eq. 10-12)
+# --------------------------------------------------------------------------
+def rope_interpolated(x_pre, positions, pos_scale: float = 1.0, theta: float = 10000.0):
+    """Eq. 12 (Eq. 11 when pos_scale = 1): rotate channel pairs (i, i + d/2) of x_pre [n, ..., d] by the angle
+    pos_scale * m * theta^(-2i/d) of each token's position m.  float64."""
+    x = np.asarray(x_pre, dtype=np.float64)
+    d = x.shape[-1]
+    half = d // 2
+    inv_freq = theta ** (-2.0 * np.arange(half, dtype=np.float64) / d)
+    ang = np.asarray(positions, dtype=np.float64)[:, None] * pos_scale * inv_freq[None, :]
+    shape = (x.shape[0],) + (1,) * (x.ndim - 2) + (half,)
+    c, s = np.cos(ang).reshape(shape), np.sin(ang).reshape(shape)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x1 * s + x2 * c], axis=-1)
+
+
+def calibrate_lambda(k_pre, pos_scale: float = 1.0, theta: float = 10000.0, alpha: float = 0.5, floor: float = 1e-5):
+    """Eq. 10 on Keys rotated per Eq. 12.  k_pre: [n_tokens, n_seq, kv_heads, d], token t at position t.
+    lambda[h, i] = max(max_{t, seq} |K_rot[t, seq, h, i]|, floor)^alpha (absolute maxima, as in the
+    channel-equalization scheme the section builds on)."""
+    k = np.asarray(k_pre, dtype=np.float64)
+    rot = rope_interpolated(k, np.arange(k.shape[0]), pos_scale, theta)
+    amax = np.abs(rot).max(axis=(0, 1))
+    return np.maximum(amax, floor) ** alpha

@@ -70,6 +70,9 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_attention_bytes.argtypes = [vp, i32]
     lib.pmkvq_export_slice.restype = i32
     lib.pmkvq_export_slice.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.pmkvq_calibrate_lambda.restype = i32
+    lib.pmkvq_calibrate_lambda.argtypes = [vp, i32, i32, i32, ctypes.c_double, ctypes.c_double, ctypes.c_float,
+                                           ctypes.c_float, vp, vp]
     lib.pmkvq_allocate_bits.restype = i32
     lib.pmkvq_allocate_bits.argtypes = [i32, i32, vp, vp, vp, ctypes.c_uint64, vp, vp]
     lib.pmkvq_status_string.restype = ctypes.c_char_p
@@ -90,6 +93,22 @@ def lib() -> ctypes.CDLL:
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     s = stream if stream is not None else torch.cuda.current_stream()
     return s.cuda_stream
+
+
+def calibrate_lambda(k_pre: torch.Tensor, pos_scale: float = 1.0, theta: float = 10000.0, alpha: float = 0.5,
+                     floor_value: float = 1e-5, stream=None) -> torch.Tensor:
+    """Eq. 10-12 on the device.  k_pre: CUDA bf16 [n_tokens, n_seq, kv_heads, 128] pre-RoPE Keys, token t at
+    position t -> lambda fp32 [kv_heads, 128] (CUDA)."""
+    if not (k_pre.is_cuda and k_pre.is_contiguous() and k_pre.dtype == torch.bfloat16 and k_pre.dim() == 4
+            and k_pre.shape[3] == 128):
+        raise ValueError("k_pre must be a contiguous CUDA bf16 tensor [n_tokens, n_seq, kv_heads, 128]")
+    n_tokens, n_seq, kv_heads, _ = k_pre.shape
+    lam = torch.empty(kv_heads, 128, dtype=torch.float32, device=k_pre.device)
+    st = lib().pmkvq_calibrate_lambda(k_pre.data_ptr(), n_tokens, n_seq, kv_heads, float(pos_scale), float(theta),
+                                      float(alpha), float(floor_value), lam.data_ptr(), _stream_ptr(stream))
+    if st != OK:
+        raise PmkvqError(st, "pmkvq_calibrate_lambda")
+    return lam
 
 
 def allocate_bits(widths, sensitivity, mem_bytes, budget_bytes):

@@ -13,6 +13,7 @@
 #include "../../include/pmkvq.h"
 #include "kernels_attn.cuh"
 #include "kernels_cache.cuh"
+#include "kernels_calib.cuh"
 #include "layout.cuh"
 
 using namespace pmkvq;
@@ -620,6 +621,23 @@ pmkvq_status pmkvq_set_attention_ctas(pmkvq_cache *k, int32_t n_ctas) {
   if (!k || n_ctas < 0 || n_ctas > kMaxCtas) return PMKVQ_ERR_INVALID_ARG;
   k->user_ctas = n_ctas;
   return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_calibrate_lambda(const void *d_K, int32_t n_tokens, int32_t n_seq, int32_t kv_heads, double pos_scale,
+                                    double theta, float alpha, float floor_value, float *d_lambda, void *stream) {
+  if (!d_K || !d_lambda || n_tokens <= 0 || n_seq <= 0 || kv_heads <= 0 || !(pos_scale > 0.0) || !(theta > 1.0) ||
+      !(floor_value > 0.f) || !std::isfinite(alpha))
+    return PMKVQ_ERR_INVALID_ARG;
+  if ((int64_t)n_seq * kv_heads > (1 << 20)) return PMKVQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n = kv_heads * kHeadDim;
+  if (cudaMemsetAsync(d_lambda, 0, (size_t)n * sizeof(float), st) != cudaSuccess) return PMKVQ_ERR_CUDA;
+  const int tokens_per_cta = std::max(1, (n_tokens + 148 * 8 - 1) / (148 * 8));
+  const unsigned grid = (unsigned)((n_tokens + tokens_per_cta - 1) / tokens_per_cta);
+  calib_absmax_kernel<<<grid, 128, 0, st>>>(static_cast<const uint16_t *>(d_K), reinterpret_cast<unsigned *>(d_lambda),
+                                            n_tokens, n_seq * kv_heads, kv_heads, tokens_per_cta, pos_scale, theta);
+  calib_finish_kernel<<<(n + 255) / 256, 256, 0, st>>>(d_lambda, n, floor_value, alpha);
+  return cudaGetLastError() == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }
 
 pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_t *h_widths, const double *h_sens,
