@@ -177,12 +177,11 @@ __device__ __forceinline__ float quantize_token16(uint2 raw, const float *__rest
 __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int lane, const uint16_t *__restrict__ K,
                                            const uint16_t *__restrict__ V, const float *__restrict__ inv_lambda,
                                            unsigned *vmax_bits, const LayerGeom &geom, int n_slices, int kv_heads,
-                                           int n_old, int win_start, int cur_bits, int skip_lo = 0, int skip_hi = 0) {
+                                           int n_old, int win_start, int cur_bits, int i0 = 0) {
   const int is_value = (int)(wid & 1);
   const long long ts = wid >> 1;
   const int slice = (int)(ts % n_slices);
-  const int i = (int)(ts / n_slices);
-  if (n_old + i >= skip_lo && n_old + i < skip_hi) return;  // written tile-wise by append_tiles_kernel
+  const int i = i0 + (int)(ts / n_slices);  // index among the new tokens
   const uint16_t *src = (is_value ? V : K) + ((size_t)i * n_slices + slice) * kHeadDim;
   float mn;
   const float scale = quantize_token16(src, is_value ? nullptr : inv_lambda + (size_t)(slice % kv_heads) * kHeadDim, codes,
@@ -202,13 +201,13 @@ __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int l
 __global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
                                                      const float *__restrict__ inv_lambda, unsigned *vmax_bits,
                                                      LayerGeom geom, int n_new, int n_slices, int kv_heads,
-                                                     int n_old, int win_start, int cur_bits, int skip_lo, int skip_hi) {
+                                                     int n_old, int win_start, int cur_bits, int i0) {
+  // new tokens i0 .. i0 + n_new - 1 of the K / V arrays, one by one
   __shared__ uint16_t s_codes[4][kHeadDim];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wid = (long long)blockIdx.x * 4 + warp;
   if (wid >= (long long)n_new * n_slices * 2) return;
-  append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits,
-             skip_lo, skip_hi);
+  append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits, i0);
 }
 
 // Bulk appends (prefill): body tiles that consist of new tokens only are built whole.  One warp per

@@ -362,7 +362,7 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
     // new tokens that fill whole body tiles are written tile-wise, the rest (sink, ring, ragged ends) one by one
     const int j_lo = std::max(n_old, k->n_sink) - k->n_sink, j_hi = std::max(new_win_start, k->n_sink) - k->n_sink;
     const int tile_lo = (j_lo + 15) / 16, tile_hi = j_hi / 16;
-    int skip_lo = 0, skip_hi = 0;
+    int skip_lo = n_old, skip_hi = n_old;  // absolute token range written tile-wise
     if (tile_hi > tile_lo) {
       skip_lo = k->n_sink + 16 * tile_lo;
       skip_hi = k->n_sink + 16 * tile_hi;
@@ -373,12 +373,17 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
                                                                    tile_hi - tile_lo, l.cur_bits);
       ++k->launches;
     }
-    const long long warps = 2ll * n_new * k->n_slices;
-    append_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(static_cast<const uint16_t *>(d_K),
-                                                              static_cast<const uint16_t *>(d_V), inv_lam, vmax, g, n_new,
-                                                              k->n_slices, k->kv_heads, n_old, new_win_start, l.cur_bits,
-                                                              skip_lo, skip_hi);
-    ++k->launches;
+    const int ranges[2][2] = {{n_old, skip_lo}, {skip_hi, n_after}};  // what is left, one token per warp
+    for (int r = 0; r < 2; ++r) {
+      const int cnt = ranges[r][1] - ranges[r][0];
+      if (cnt <= 0) continue;
+      const long long warps = 2ll * cnt * k->n_slices;
+      append_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(static_cast<const uint16_t *>(d_K),
+                                                                static_cast<const uint16_t *>(d_V), inv_lam, vmax, g, cnt,
+                                                                k->n_slices, k->kv_heads, n_old, new_win_start, l.cur_bits,
+                                                                ranges[r][0] - n_old);
+      ++k->launches;
+    }
   }
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
   l.n_tokens = n_after;
