@@ -45,13 +45,7 @@ constexpr int kMaxGroup = 8;         // query heads per KV head handled by one M
 constexpr int kPartialStride = 132;  // floats per (segment, head): m, l, 2 pad, o[128]
 constexpr float kNegBig = -1.0e30f;
 constexpr float kMaxAhead = 3.0f;    // a score may exceed the reference by this much (log2 units)
-#ifndef PMKVQ_WARPS
-#define PMKVQ_WARPS 16
-#endif
-#ifndef PMKVQ_QSMEM
-#define PMKVQ_QSMEM 1
-#endif
-constexpr int kAttnWarps = PMKVQ_WARPS;      // one CTA per SM; its warps share the CTA's tiles dynamically
+constexpr int kAttnWarps = 16;       // one CTA per SM; its warps share the CTA's tiles dynamically
 constexpr int kAttnThreads = 32 * kAttnWarps;
 
 struct AttnParams {
@@ -175,27 +169,16 @@ template <> struct Fmt<16> {
   __host__ __device__ static constexpr int pos(int) { return 0; }
 };
 
-// The query fragments of a lane (8 k-steps x 4 registers): either kept in registers for the whole
-// segment or fetched from a per-CTA copy in shared memory right before each use (they depend on the
-// lane, not on the warp), which trades 8 shared loads per step for 32 registers.
-struct QRegs {
-  uint32_t v[8][4];
-  __device__ __forceinline__ void load(int s, uint32_t (&q)[4]) const {
-    q[0] = v[s][0]; q[1] = v[s][1]; q[2] = v[s][2]; q[3] = v[s][3];
-  }
-};
-struct QSmem {
+// The query fragments of a lane (8 k-steps x 4 registers) depend on the lane, not on the warp: the CTA
+// keeps one copy in shared memory and a warp fetches a k-step's fragment right before it uses it
+// (8 shared loads per step instead of 32 registers held for the whole segment).
+struct QFrag {
   const uint4 *mine;  // entry (k-step s, this lane) at mine[32 s]
   __device__ __forceinline__ void load(int s, uint32_t (&q)[4]) const {
     const uint4 t = mine[32 * s];
     q[0] = t.x; q[1] = t.y; q[2] = t.z; q[3] = t.w;
   }
 };
-#if PMKVQ_QSMEM
-using QFrag = QSmem;
-#else
-using QFrag = QRegs;
-#endif
 
 // 16-byte load of tile data: body tiles sit in shared memory, INT16 tiles are read from global
 // memory past L1 (another kernel may have written them while this SM still holds old lines).
@@ -206,7 +189,8 @@ __device__ __forceinline__ T ld_tile(const void *ptr) {
 }
 
 struct WarpState {
-  float m, l, zs;   // reference (log2 units), sum of probabilities, sum of p * Z_V, for head g (this lane's quad)
+  float m;          // reference (log2 units) of head g (this lane's quad)
+  float2 l, zs;     // sum of probabilities and of p * Z_V, two partial sums each (packed arithmetic)
   float acc[8][4];  // O^T accumulators: [m-tile][channel row g / g+8 x head col 2tig / 2tig+1]
 };
 
@@ -223,7 +207,7 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
   const int tig = lane & 3;
 
   // ---- scores: S = Q'' K^T, heads on M (hi rows 0-7, lo rows 8-15), tokens on N ----
-  float dot[NS];
+  float2 dot2[NS / 2];  // pairs of scores: tokens (2tig, 2tig+1) of a token half
   if constexpr (BITS == 16) {
     const uint8_t *kp = tile0 + lane * 16;
 #pragma unroll
@@ -243,8 +227,7 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
         mma_f16(lo, qf, x0 & 0x00FF00FFu, x1 & 0x00FF00FFu);
         mma_f16(hi, qf, high_bytes(x0), high_bytes(x1));
       }
-      dot[2 * r] = fmaf(256.f, hi[0] + hi[2], lo[0] + lo[2]);
-      dot[2 * r + 1] = fmaf(256.f, hi[1] + hi[3], lo[1] + lo[3]);
+      dot2[r] = make_float2(fmaf(256.f, hi[0] + hi[2], lo[0] + lo[2]), fmaf(256.f, hi[1] + hi[3], lo[1] + lo[3]));
     }
   } else {
     // the 2 NT (tile, token half) accumulators advance together: consecutive MMAs are independent
@@ -283,47 +266,46 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
-        dot[4 * nt + 2 * r] = sacc[nt][r][0] + sacc[nt][r][2];
-        dot[4 * nt + 2 * r + 1] = sacc[nt][r][1] + sacc[nt][r][3];
+        dot2[2 * nt + r] = __fadd2_rn(make_float2(sacc[nt][r][0], sacc[nt][r][1]), make_float2(sacc[nt][r][2], sacc[nt][r][3]));
       }
   }
 
   // ---- per-token scale / zero-point of this lane's tokens {2tig, 2tig+1, 8+2tig, 9+2tig} of each tile ----
-  float sk[NS], zk[NS], sv[NS], zv[NS];
+  // (the softmax arithmetic below runs on pairs of scores with the packed fp32x2 instructions)
+  constexpr int NP = NS / 2;
+  float2 sk[NP], zk[NP], sv[NP], zv[NP];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const float4 *mp = reinterpret_cast<const float4 *>(tile0 + nt * TB + meta_offset(BITS) + tig * 64);
     const float4 a = ld_tile<BITS, float4>(mp), b = ld_tile<BITS, float4>(mp + 1), c = ld_tile<BITS, float4>(mp + 2),
                  d = ld_tile<BITS, float4>(mp + 3);
-    sk[4 * nt] = a.x; sk[4 * nt + 1] = a.y; sk[4 * nt + 2] = a.z; sk[4 * nt + 3] = a.w;
-    zk[4 * nt] = b.x; zk[4 * nt + 1] = b.y; zk[4 * nt + 2] = b.z; zk[4 * nt + 3] = b.w;
-    sv[4 * nt] = c.x; sv[4 * nt + 1] = c.y; sv[4 * nt + 2] = c.z; sv[4 * nt + 3] = c.w;
-    zv[4 * nt] = d.x; zv[4 * nt + 1] = d.y; zv[4 * nt + 2] = d.z; zv[4 * nt + 3] = d.w;
+    sk[2 * nt] = make_float2(a.x, a.y); sk[2 * nt + 1] = make_float2(a.z, a.w);
+    zk[2 * nt] = make_float2(b.x, b.y); zk[2 * nt + 1] = make_float2(b.z, b.w);
+    sv[2 * nt] = make_float2(c.x, c.y); sv[2 * nt + 1] = make_float2(c.z, c.w);
+    zv[2 * nt] = make_float2(d.x, d.y); zv[2 * nt + 1] = make_float2(d.z, d.w);
   }
 
   // ---- true scores; the reference moves only when one of them runs ahead of it ----
-  float sc[NS];
+  const float2 mu2 = make_float2(mu, mu), sumq2 = make_float2(sumq, sumq);
+  float2 sc[NP];
   float mx = -INFINITY;
 #pragma unroll
-  for (int i = 0; i < NS; ++i) {
-    sc[i] = fmaf(sk[i] * mu, dot[i], zk[i] * sumq);
+  for (int j = 0; j < NP; ++j) {
+    sc[j] = __ffma2_rn(__fmul2_rn(sk[j], mu2), dot2[j], __fmul2_rn(zk[j], sumq2));
     if constexpr (MASKED) {
-      const bool live = (mask >> (8 * ((i >> 1) & 1) + 2 * tig + (i & 1))) & 1u;
-      if (!live) {
-        sc[i] = -INFINITY;
-        sv[i] = 0.f;
-        zv[i] = 0.f;
-      }
+      const int bit = 8 * (j & 1) + 2 * tig;
+      if (!((mask >> bit) & 1u)) { sc[j].x = -INFINITY; sv[j].x = 0.f; zv[j].x = 0.f; }
+      if (!((mask >> (bit + 1)) & 1u)) { sc[j].y = -INFINITY; sv[j].y = 0.f; zv[j].y = 0.f; }
     }
-    mx = fmaxf(mx, sc[i]);
+    mx = fmaxf(mx, fmaxf(sc[j].x, sc[j].y));
   }
   if (__any_sync(0xffffffffu, mx > st.m + kMaxAhead)) {
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
     const float m_new = fmaxf(st.m, mx);
     const float f = ex2(st.m - m_new);
-    st.l *= f;
-    st.zs *= f;
+    st.l = __fmul2_rn(st.l, make_float2(f, f));
+    st.zs = __fmul2_rn(st.zs, make_float2(f, f));
     const float f0 = __shfl_sync(0xffffffffu, f, (2 * tig) * 4);
     const float f1 = __shfl_sync(0xffffffffu, f, (2 * tig + 1) * 4);
 #pragma unroll
@@ -338,21 +320,18 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
   // when a few tokens carry the whole softmax.
   uint32_t pb[2 * NT];
   {
-    float wv[NS], rs[NS];
+    const float2 neg_m = make_float2(-st.m, -st.m), inv2 = make_float2(inv_sigma_e, inv_sigma_e);
 #pragma unroll
-    for (int i = 0; i < NS; ++i) {
+    for (int j = 0; j < NP; ++j) {
       // a constant V group has S_V = 0 and all codes 0: any finite unit will do for it
-      const float s_e = fmaf(sv[i], inv_sigma_e, sv[i] == 0.f ? 1.f : 0.f);  // S_V / sigma_u * 2^EP
-      rs[i] = rcp_approx(s_e);
-      wv[i] = ex2(sc[i] - st.m) * s_e;
-    }
-#pragma unroll
-    for (int j = 0; j < 2 * NT; ++j) {
-      pb[j] = pack_half2(wv[2 * j], wv[2 * j + 1]);
-      const float2 wf = __half22float2(*reinterpret_cast<const __half2 *>(&pb[j]));
-      const float p0 = wf.x * rs[2 * j], p1 = wf.y * rs[2 * j + 1];
-      st.l += p0 + p1;
-      st.zs = fmaf(p0, zv[2 * j], fmaf(p1, zv[2 * j + 1], st.zs));
+      const float2 s_e = __ffma2_rn(sv[j], inv2, make_float2(sv[j].x == 0.f ? 1.f : 0.f, sv[j].y == 0.f ? 1.f : 0.f));
+      const float2 rs = make_float2(rcp_approx(s_e.x), rcp_approx(s_e.y));
+      const float2 arg = __fadd2_rn(sc[j], neg_m);
+      const float2 w = __fmul2_rn(make_float2(ex2(arg.x), ex2(arg.y)), s_e);  // p * S_V / sigma_u * 2^EP
+      pb[j] = pack_half2(w.x, w.y);
+      const float2 p = __fmul2_rn(__half22float2(*reinterpret_cast<const __half2 *>(&pb[j])), rs);
+      st.l = __fadd2_rn(st.l, p);
+      st.zs = __ffma2_rn(p, zv[j], st.zs);
     }
   }
 
@@ -460,22 +439,7 @@ __device__ __forceinline__ uint4 q_fragment(const float (*s_q)[kHeadDim], int e_
   return make_uint4(r[0], r[1], r[2], r[3]);
 }
 
-// The fragments a warp multiplies with at width BITS: in registers, or (shared-memory variant) the
-// CTA's copy `s_frag`, which must have been filled by fill_q_fragments for this width.
-template <int BITS>
-__device__ __forceinline__ void set_q_fragments(QFrag &qa, const float (*s_q)[kHeadDim], const float *s_stat,
-                                                const uint4 *s_frag, int lane) {
-#if PMKVQ_QSMEM
-  qa.mine = s_frag + lane;
-#else
-  const int g = lane >> 2, tig = lane & 3;
-#pragma unroll
-  for (int s = 0; s < 8; ++s) {
-    const uint4 t = q_fragment<BITS>(s_q, (int)s_stat[g], g, tig, s);
-    qa.v[s][0] = t.x; qa.v[s][1] = t.y; qa.v[s][2] = t.z; qa.v[s][3] = t.w;
-  }
-#endif
-}
+// Fills the CTA's copy of the fragments at width BITS (all threads; a barrier must follow).
 template <int BITS>
 __device__ __forceinline__ void fill_q_fragments(uint4 *s_frag, const float (*s_q)[kHeadDim], const float *s_stat) {
   for (int i = threadIdx.x; i < 256; i += kAttnThreads) {  // entry (k-step i / 32, lane i % 32)
@@ -580,11 +544,9 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   __syncthreads();
   const int e_g = (int)s_stat[g];
   const float sumq = s_stat[8 + g];
-#if PMKVQ_QSMEM
   fill_q_fragments<16>(s_frag, s_q, s_stat);
   if constexpr (BITS != 16) fill_q_fragments<BITS>(s_frag + 256, s_q, s_stat);
   __syncthreads();
-#endif
 
   // ---- unit of the V accumulators: a power of two >= every INT16 V scale of this slice; at width b
   //      the scales are at most 2^SIGMA_LOG2 times larger ----
@@ -599,7 +561,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   }
 
   WarpState st;
-  st.m = kNegBig; st.l = 0.f; st.zs = 0.f;
+  st.m = kNegBig; st.l = make_float2(0.f, 0.f); st.zs = make_float2(0.f, 0.f);
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
   QFrag qa;
@@ -608,7 +570,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   if (a_hi > a_lo) {
     int it = a_lo + claim(0);
     if (it < a_hi) {
-      set_q_fragments<16>(qa, s_q, s_stat, s_frag, lane);
+      qa.mine = s_frag + lane;
       const float mu = ldexpf(1.0f, 24 - F16::EQ + e_g);
       const float inv_sigma_e = ldexpf(1.0f, F16::EP) / sigma16;
       const int n_win = p.n_tokens - p.win_start;
@@ -653,7 +615,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   // ---- body tiles ----
   const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
   if (n_steps > 0) {
-    set_q_fragments<BITS>(qa, s_q, s_stat, BITS != 16 ? s_frag + 256 : s_frag, lane);
+    qa.mine = (BITS != 16 ? s_frag + 256 : s_frag) + lane;
     const float mu = ldexpf(1.0f, 24 - F::EQ + e_g);
     const float inv_sigma_e = ldexpf(1.0f, F::EP) / sigma_u;
     const uint32_t tail_mask = (p.n_body & 15) ? (1u << (p.n_body & 15)) - 1u : 0xFFFFu;
@@ -698,19 +660,20 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   if constexpr (F::SLOTS > 0) cp_async_wait<0>();
 
   // ---- warp epilogue: quad sums, real units, to shared memory (the ring is free now) ----
-  st.l += __shfl_xor_sync(0xffffffffu, st.l, 1);
-  st.l += __shfl_xor_sync(0xffffffffu, st.l, 2);
-  st.zs += __shfl_xor_sync(0xffffffffu, st.zs, 1);
-  st.zs += __shfl_xor_sync(0xffffffffu, st.zs, 2);
+  float l_sum = st.l.x + st.l.y, zs_sum = st.zs.x + st.zs.y;
+  l_sum += __shfl_xor_sync(0xffffffffu, l_sum, 1);
+  l_sum += __shfl_xor_sync(0xffffffffu, l_sum, 2);
+  zs_sum += __shfl_xor_sync(0xffffffffu, zs_sum, 1);
+  zs_sum += __shfl_xor_sync(0xffffffffu, zs_sum, 2);
   __syncthreads();  // every warp is done with its stages
   float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(ring);
   float *s_m = s_stat + 16, *s_l = s_stat + 16 + kAttnWarps * kMaxGroup;
   if (tig == 0) {
     s_m[warp * 8 + g] = st.m;
-    s_l[warp * 8 + g] = st.l;
+    s_l[warp * 8 + g] = l_sum;
   }
-  const float zs0 = __shfl_sync(0xffffffffu, st.zs, (2 * tig) * 4);
-  const float zs1 = __shfl_sync(0xffffffffu, st.zs, (2 * tig + 1) * 4);
+  const float zs0 = __shfl_sync(0xffffffffu, zs_sum, (2 * tig) * 4);
+  const float zs1 = __shfl_sync(0xffffffffu, zs_sum, (2 * tig + 1) * 4);
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
 #pragma unroll
@@ -776,11 +739,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
   __shared__ float s_stat[16 + 2 * kAttnWarps * kMaxGroup];  // head stats, per-warp (m, l)
   __shared__ int s_ctr[4];                                    // work counters (INT16 tiles, body steps), combine flag
-#if PMKVQ_QSMEM
   __shared__ uint4 s_frag[512];                               // query fragments at INT16 and at the body width
-#else
-  uint4 *s_frag = nullptr;
-#endif
   extern __shared__ __align__(128) uint8_t ring[];
   // When launched with programmatic stream serialization (pmkvq_decode_step does that for every block
   // after the first) the next block's kernel may start as soon as SMs free up; it works on its own
