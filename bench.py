@@ -6,7 +6,7 @@ quantize-on-append of one new token per sequence (with window eviction and, when
 budget fills, the progressive reduce) followed by fused dequantize + GQA decode attention over the
 whole mixed-precision cache.  There are no weights / MLP in this path.
 
-Default workload (BASELINE configs[1]): 7B long-CoT shape, 28 blocks, 28 Q / 4 KV heads, head_dim
+Default workload: 7B long-CoT shape, 28 blocks, 28 Q / 4 KV heads, head_dim
 128, batch 16, 32K cached tokens at the end of the run, Fbit 4 in the first/last 4 blocks and 2
 elsewhere; budgets are set so every block's last reduce (2*Fbit -> Fbit) falls inside the run.
 
@@ -34,13 +34,13 @@ from paper_2505_18610_b200 import synth  # noqa: E402
 
 WORKLOADS = {
     # name: layers, q_heads, kv_heads, batch, end tokens, (edge Fbit, inner Fbit, n_edge), outliers, factor
-    "7b": dict(name="7b_longcot_b16_32k (BASELINE configs[1])", layers=28, q_heads=28, kv_heads=4, batch=16,
+    "7b": dict(name="7b_longcot_b16_32k", layers=28, q_heads=28, kv_heads=4, batch=16,
                end_tokens=32768, edge_bits=4, inner_bits=2, n_edge=4, n_outlier=4, factor=15.0),
-    "8b": dict(name="8b_b32_32k_uniform4 (BASELINE configs[2])", layers=32, q_heads=32, kv_heads=8, batch=32,
+    "8b": dict(name="8b_b32_32k_uniform4", layers=32, q_heads=32, kv_heads=8, batch=32,
                end_tokens=32768, edge_bits=4, inner_bits=4, n_edge=4, n_outlier=4, factor=15.0),
-    "32b": dict(name="32b_b8_128k_mixed_2_4 (BASELINE configs[3])", layers=64, q_heads=40, kv_heads=8, batch=8,
+    "32b": dict(name="32b_b8_128k_mixed_2_4", layers=64, q_heads=40, kv_heads=8, batch=8,
                 end_tokens=131072, edge_bits=4, inner_bits=2, n_edge=16, n_outlier=4, factor=15.0),
-    "70b": dict(name="70b_b16_64k_120GB (BASELINE configs[4])", layers=80, q_heads=64, kv_heads=8, batch=16,
+    "70b": dict(name="70b_b16_64k_120GB", layers=80, q_heads=64, kv_heads=8, batch=16,
                 end_tokens=65536, schedule="70b", n_outlier=4, factor=15.0),
     "7b-4l": dict(name="7b_longcot_b16_32k, 4 of 28 blocks (profiling case)", layers=4, q_heads=28, kv_heads=4, batch=16,
                   end_tokens=32768, edge_bits=4, inner_bits=2, n_edge=1, n_outlier=4, factor=15.0),
@@ -190,7 +190,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                       "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -450,8 +450,10 @@ def main():
         "metric": "decode_attention_GBps", "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int2/int4/int16 codes, f16 mma.sync, f32 accumulate", "data": "synthetic",
-        "config": {"workload": wl["name"], "layers": wl["layers"], "q_heads": wl["q_heads"], "kv_heads": wl["kv_heads"],
-                   "batch_per_gpu": wl["batch"], "tokens_at_end": final_tokens, "fbit": fbit,
+        "config": {"workload": wl["name"],
+                   "shape": f"{wl['layers']} blocks x ({wl['q_heads']} Q / {wl['kv_heads']} KV heads, head_dim 128) x batch "
+                            f"{wl['batch']} per GPU x {final_tokens} cached tokens at the end",
+                   "fbit_per_block": fbit,
                    "blocks_reduced_to_fbit_in_run": n_reduced, "n_sink": N_SINK, "window": WINDOW,
                    "l2": "per-step working set (the whole cache) is far larger than L2; no flush needed",
                    "path": "attention path only (no weights / MLP)", "sharding": "batch, no collective"},

@@ -1,4 +1,5 @@
-"""Parity at the full per-block sizes of the BASELINE configs, in the launch configuration bench.py times
+"""Parity at the full per-block sizes of the benchmark workloads (7B / 8B / 32B / 70B long-CoT shapes), in the launch
+configuration bench.py times
 (same batch, heads, context length, default attention grid, pmkvq_decode_step), on sampled (batch,
 kv_head) slices the oracle can compute one by one: cache state bit-exact after the run (it crosses each
 block's last progressive reduce), attention outputs within tolerance at several steps.  Two blocks per

@@ -28,7 +28,7 @@ def test_tiny_token_counts(fbit, n):
 
 
 def test_config1_progressive_16_8_4():
-    """BASELINE config 1: 1 block, batch 1, 4 Q / 1 KV head, 4096 tokens fed one by one, 4 outlier channels
+    """The small progressive case: 1 block, batch 1, 4 Q / 1 KV head, 4096 tokens fed one by one, 4 outlier channels
     x20, default budget for Fbit = 4: the block goes 16 -> 8 -> 4.  Full parity after every reduce."""
     n = 4096
     k, v = make_inputs(0, 0, n, 1, 1, n_outlier=4, factor=20.0)
