@@ -194,20 +194,14 @@ struct WarpState {
   float acc[8][4];  // O^T accumulators: [m-tile][channel row g / g+8 x head col 2tig / 2tig+1]
 };
 
-// NT consecutive 16-token tiles.  `mask` (NT == 1 only) has bit r set when token row r is live.
-template <int BITS, int NT, bool MASKED>
-__device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mask, WarpState &st,
-                                              const QFrag &qa, float mu, float sumq, float inv_sigma_e,
-                                              int lane) {
+// First half of a step: the score dot products of NT consecutive 16-token tiles against the query
+// fragments (no scale / zero-point yet), as pairs: dot2[2 nt + r] = tokens (2tig, 2tig+1) of half r.
+template <int BITS, int NT>
+__device__ __forceinline__ void qk_phase(const uint8_t *tile0, const QFrag &qa, int lane, float2 (&dot2)[2 * NT]) {
   using F = Fmt<BITS>;
-  static_assert(!(MASKED && NT != 1), "masked tiles are processed one at a time");
   constexpr int TB = tile_bytes(BITS);
   constexpr int CHUNKS = BITS / 2;
-  constexpr int NS = 4 * NT;  // scores per lane
-  const int tig = lane & 3;
-
   // ---- scores: S = Q'' K^T, heads on M (hi rows 0-7, lo rows 8-15), tokens on N ----
-  float2 dot2[NS / 2];  // pairs of scores: tokens (2tig, 2tig+1) of a token half
   if constexpr (BITS == 16) {
     const uint8_t *kp = tile0 + lane * 16;
 #pragma unroll
@@ -269,6 +263,20 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
         dot2[2 * nt + r] = __fadd2_rn(make_float2(sacc[nt][r][0], sacc[nt][r][1]), make_float2(sacc[nt][r][2], sacc[nt][r][3]));
       }
   }
+}
+
+// Second half of a step: scale / zero-point, online softmax and O^T += V^T w for the same NT tiles.
+// `mask` (NT == 1 only) has bit r set when token row r is live.
+template <int BITS, int NT, bool MASKED>
+__device__ __forceinline__ void softmax_pv_phase(const uint8_t *tile0, uint32_t mask, WarpState &st,
+                                                 const float2 (&dot2)[2 * NT], float mu, float sumq, float inv_sigma_e,
+                                                 int lane) {
+  using F = Fmt<BITS>;
+  static_assert(!(MASKED && NT != 1), "masked tiles are processed one at a time");
+  constexpr int TB = tile_bytes(BITS);
+  constexpr int CHUNKS = BITS / 2;
+  constexpr int NS = 4 * NT;  // scores per lane
+  const int tig = lane & 3;
 
   // ---- per-token scale / zero-point of this lane's tokens {2tig, 2tig+1, 8+2tig, 9+2tig} of each tile ----
   // (the softmax arithmetic below runs on pairs of scores with the packed fp32x2 instructions)
@@ -367,6 +375,15 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
       }
     }
   }
+}
+
+// A whole step in one go (INT16 tiles, ragged ends).
+template <int BITS, int NT, bool MASKED>
+__device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mask, WarpState &st, const QFrag &qa,
+                                              float mu, float sumq, float inv_sigma_e, int lane) {
+  float2 dot2[2 * NT];
+  qk_phase<BITS, NT>(tile0, qa, lane, dot2);
+  softmax_pv_phase<BITS, NT, MASKED>(tile0, mask, st, dot2, mu, sumq, inv_sigma_e, lane);
 }
 
 // ---- where the partials of a slice live ------------------------------------------------------
