@@ -469,7 +469,12 @@ def main():
                      "algorithmic_bytes_per_launch": attn_bytes / max(1, n_attn),
                      "how": "the timed steps replayed on an identical cache with a CUDA event pair around every "
                             "pmkvq_decode_attention launch (one kernel per call)",
-                     "ms_per_step_with_events": instr_ms / steps},
+                     "ms_per_step_with_events": instr_ms / steps,
+                     "achieved_inside_decode_step": (attn_bytes / max(1, n_attn)) * wl["layers"] * steps / (ms * 1e-3) / 1e9
+                     if n_attn else None,
+                     "achieved_inside_decode_step_note": "attention bytes of a step / whole step time of the device-resident leg "
+                                                         "(appends and reduces included): consecutive blocks' attention kernels "
+                                                         "overlap there, so a per-launch duration does not exist"},
         "e2e": {"value": world * total_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms / steps,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,

@@ -215,3 +215,29 @@ def test_shift_variants_direct_and_modified(variant):
         m.check_state(l)
         assert m.cache.layer_state(l)["cur_bits"] == [2, 4][l]
         m.check_attention(l, synth.make_q(10, l, 0, batch, group * kvh, n))
+
+
+def test_decode_step_budget_full_leaves_every_block_untouched():
+    """With auto_reduce off, a step that would push one block over its budget returns BUDGET_FULL before any
+    block has received its token; after the manual reduce the same step goes through."""
+    from paper_2505_18610_b200 import binding as B
+    layers, kvh, batch, group = 2, 1, 1, 4
+    full = 2 * (16 * 264 + 0)                       # 16 INT16 tokens per (K|V) slice, code + metadata bytes
+    m = Mirror(layers, group * kvh, kvh, batch, 64, [8, 8], n_sink=0, window=0, auto_reduce=False,
+               budget_bytes=[full * 4, full])      # block 1 is full at 16 tokens, block 0 is not
+    k, v = make_inputs(21, 0, 17, batch, kvh)
+    for l in range(layers):
+        m.cache.append(l, k[:16].cuda(), v[:16].cuda())
+    K = torch.stack([k[16], k[16]]).cuda().contiguous(); V = torch.stack([v[16], v[16]]).cuda().contiguous()
+    Q = torch.stack([synth.make_q(21, l, 0, batch, group * kvh, 17) for l in range(layers)]).cuda().contiguous()
+    with pytest.raises(B.PmkvqError) as e:
+        m.cache.decode_step(K, V, Q)
+    assert e.value.status == B.BUDGET_FULL
+    assert [m.cache.layer_state(l)["n_tokens"] for l in range(layers)] == [16, 16]
+    assert [m.cache.layer_state(l)["cur_bits"] for l in range(layers)] == [16, 16]
+    m.cache.progressive_reduce(1)
+    out = m.cache.decode_step(K, V, Q)
+    torch.cuda.synchronize()
+    assert [m.cache.layer_state(l)["n_tokens"] for l in range(layers)] == [17, 17]
+    assert [m.cache.layer_state(l)["cur_bits"] for l in range(layers)] == [16, 8]
+    assert torch.isfinite(out).all()
