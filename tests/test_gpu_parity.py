@@ -241,3 +241,33 @@ def test_decode_step_budget_full_leaves_every_block_untouched():
     assert [m.cache.layer_state(l)["n_tokens"] for l in range(layers)] == [17, 17]
     assert [m.cache.layer_state(l)["cur_bits"] for l in range(layers)] == [16, 8]
     assert torch.isfinite(out).all()
+
+
+@pytest.mark.parametrize("chunk,n_sink,window", [(16, 4, 20), (3, 0, 7), (1, 17, 0)])
+def test_decode_step_with_chunked_eviction(chunk, n_sink, window):
+    """The all-blocks append of pmkvq_decode_step with eviction in chunks, several sink tokens and small
+    windows: blocks at different token counts are not supported by the call, different widths are."""
+    layers, kvh, batch, group, n0, steps = 2, 2, 2, 5, 70, 45
+    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, [2, 8], n_sink=n_sink, window=window, evict_chunk=chunk)
+    for l in range(layers):
+        k, v = make_inputs(30, l, n0, batch, kvh)
+        m.append(l, k, v)
+    for s in range(steps):
+        ks, vs, qs = [], [], []
+        for l in range(layers):
+            k, v = make_inputs(31, l, 1, batch, kvh, pos0=n0 + s, chunk=s)
+            ks.append(k[0]); vs.append(v[0])
+            qs.append(synth.make_q(31, l, s, batch, group * kvh, n0 + s + 1))
+        K, V, Q = torch.stack(ks).cuda(), torch.stack(vs).cuda(), torch.stack(qs).cuda()
+        out = m.cache.decode_step(K, V, Q)
+        torch.cuda.synchronize()
+        for l in range(layers):
+            m.oracles[l].append(K[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices],
+                                V[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices])
+        if s % 11 == 0 or s == steps - 1:
+            for l in range(layers):
+                m.check_state(l)
+                qq = Q[l].float().cpu().numpy().reshape(batch * kvh, group, 128)[m.slices]
+                ref = m.oracles[l].decode_attention(qq)
+                got = out[l].cpu().numpy().reshape(batch * kvh, group, 128)[m.slices].astype(np.float64)
+                assert np.abs(got - ref).max() <= 2e-3 and np.linalg.norm(got - ref) <= 1e-3 * np.linalg.norm(ref)
