@@ -265,17 +265,19 @@ __device__ __forceinline__ void qk_phase(const uint8_t *tile0, const QFrag &qa, 
   }
 }
 
-// Second half of a step: scale / zero-point, online softmax and O^T += V^T w for the same NT tiles.
-// `mask` (NT == 1 only) has bit r set when token row r is live.
+// Second part of a step: scale / zero-point and online softmax of the NT tiles' scores.  Leaves the
+// weights w = p * S_V of this lane's tokens in pb (fp16 pairs, the B fragments of the output MMAs) and
+// returns the factor by which everything accumulated so far for head g must be multiplied (1 unless the
+// reference moved).  `mask` (NT == 1 only) has bit r set when token row r is live.
 template <int BITS, int NT, bool MASKED>
-__device__ __forceinline__ void softmax_pv_phase(const uint8_t *tile0, uint32_t mask, WarpState &st,
-                                                 const float2 (&dot2)[2 * NT], float mu, float sumq, float inv_sigma_e,
-                                                 int lane) {
+__device__ __forceinline__ float softmax_phase(const uint8_t *tile0, uint32_t mask, WarpState &st,
+                                               const float2 (&dot2)[2 * NT], float mu, float sumq, float inv_sigma_e,
+                                               int lane, uint32_t (&pb)[2 * NT]) {
   using F = Fmt<BITS>;
   static_assert(!(MASKED && NT != 1), "masked tiles are processed one at a time");
   constexpr int TB = tile_bytes(BITS);
-  constexpr int CHUNKS = BITS / 2;
   constexpr int NS = 4 * NT;  // scores per lane
+  float rescale = 1.0f;
   const int tig = lane & 3;
 
   // ---- per-token scale / zero-point of this lane's tokens {2tig, 2tig+1, 8+2tig, 9+2tig} of each tile ----
@@ -314,19 +316,13 @@ __device__ __forceinline__ void softmax_pv_phase(const uint8_t *tile0, uint32_t 
     const float f = ex2(st.m - m_new);
     st.l = __fmul2_rn(st.l, make_float2(f, f));
     st.zs = __fmul2_rn(st.zs, make_float2(f, f));
-    const float f0 = __shfl_sync(0xffffffffu, f, (2 * tig) * 4);
-    const float f1 = __shfl_sync(0xffffffffu, f, (2 * tig + 1) * 4);
-#pragma unroll
-    for (int mt = 0; mt < 8; ++mt) {
-      st.acc[mt][0] *= f0; st.acc[mt][1] *= f1; st.acc[mt][2] *= f0; st.acc[mt][3] *= f1;
-    }
+    rescale = f;
     st.m = m_new;
   }
   // w = p * S_V goes to the tensor cores as one fp16; the probability that enters the denominator and
   // the zero-point sum is that rounded w divided by the scale again, so numerator and denominator
   // see the same (slightly perturbed) probabilities and the rounding cancels where it matters most,
   // when a few tokens carry the whole softmax.
-  uint32_t pb[2 * NT];
   {
     const float2 neg_m = make_float2(-st.m, -st.m), inv2 = make_float2(inv_sigma_e, inv_sigma_e);
 #pragma unroll
@@ -342,8 +338,26 @@ __device__ __forceinline__ void softmax_pv_phase(const uint8_t *tile0, uint32_t 
       st.zs = __ffma2_rn(p, zv[j], st.zs);
     }
   }
+  return rescale;
+}
 
-  // ---- output: O^T += V^T w, channels on M, tokens on K, heads on N ----
+// The accumulators of this lane hold heads 2tig and 2tig + 1 (columns): apply the heads' factors.
+__device__ __forceinline__ void rescale_acc(float (&acc)[8][4], float f_of_my_head, int lane) {
+  const int tig = lane & 3;
+  const float f0 = __shfl_sync(0xffffffffu, f_of_my_head, (2 * tig) * 4);
+  const float f1 = __shfl_sync(0xffffffffu, f_of_my_head, (2 * tig + 1) * 4);
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    acc[mt][0] *= f0; acc[mt][1] *= f1; acc[mt][2] *= f0; acc[mt][3] *= f1;
+  }
+}
+
+// Last part of a step: O^T += V^T w for NT tiles, channels on M, tokens on K, heads on N.
+template <int BITS, int NT>
+__device__ __forceinline__ void pv_phase(const uint8_t *tile0, float (&acc)[8][4], const uint32_t (&pb)[2 * NT], int lane) {
+  using F = Fmt<BITS>;
+  constexpr int TB = tile_bytes(BITS);
+  constexpr int CHUNKS = BITS / 2;
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const uint8_t *vp = tile0 + nt * TB + v_part_offset(BITS) + lane * 16;
@@ -359,8 +373,8 @@ __device__ __forceinline__ void softmax_pv_phase(const uint8_t *tile0, uint32_t 
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) {
         const uint32_t a0 = vw[2 * mt], a1 = vw[2 * mt + 1], a2 = vw[16 + 2 * mt], a3 = vw[16 + 2 * mt + 1];
-        mma_f16(st.acc[mt], a0 & 0x00FF00FFu, a1 & 0x00FF00FFu, a2 & 0x00FF00FFu, a3 & 0x00FF00FFu, pb0, pb1);
-        mma_f16(st.acc[mt], (a0 >> 5) & 0x07F807F8u, (a1 >> 5) & 0x07F807F8u, (a2 >> 5) & 0x07F807F8u,
+        mma_f16(acc[mt], a0 & 0x00FF00FFu, a1 & 0x00FF00FFu, a2 & 0x00FF00FFu, a3 & 0x00FF00FFu, pb0, pb1);
+        mma_f16(acc[mt], (a0 >> 5) & 0x07F807F8u, (a1 >> 5) & 0x07F807F8u, (a2 >> 5) & 0x07F807F8u,
                 (a3 >> 5) & 0x07F807F8u, ph0, ph1);
       }
     } else {
@@ -371,10 +385,21 @@ __device__ __forceinline__ void softmax_pv_phase(const uint8_t *tile0, uint32_t 
         F::extract(vw[BITS + w], eb);
 #pragma unroll
         for (int jj = 0; jj < F::N / 2; ++jj)
-          mma_f16(st.acc[(w * F::N) / 2 + jj], ea[2 * jj], ea[2 * jj + 1], eb[2 * jj], eb[2 * jj + 1], pb0, pb1);
+          mma_f16(acc[(w * F::N) / 2 + jj], ea[2 * jj], ea[2 * jj + 1], eb[2 * jj], eb[2 * jj + 1], pb0, pb1);
       }
     }
   }
+}
+
+// Softmax and output of a step in one warp.
+template <int BITS, int NT, bool MASKED>
+__device__ __forceinline__ void softmax_pv_phase(const uint8_t *tile0, uint32_t mask, WarpState &st,
+                                                 const float2 (&dot2)[2 * NT], float mu, float sumq, float inv_sigma_e,
+                                                 int lane) {
+  uint32_t pb[2 * NT];
+  const float f = softmax_phase<BITS, NT, MASKED>(tile0, mask, st, dot2, mu, sumq, inv_sigma_e, lane, pb);
+  if (__any_sync(0xffffffffu, f != 1.0f)) rescale_acc(st.acc, f, lane);
+  pv_phase<BITS, NT>(tile0, st.acc, pb, lane);
 }
 
 // A whole step in one go (INT16 tiles, ragged ends).
