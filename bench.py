@@ -176,8 +176,8 @@ def kernel_source_digest():
 # DRAM read + write bytes per launch of the attention kernel from the ncu capture summarised in
 # profiles/decode_attn_splitk_7b_shape.md (7B shape, body at 4 bit: the launch kind with the largest time
 # share; algorithmic bytes of that launch: 305.5 MB), and the digest of the sources it was taken on.
-NCU_TRAFFIC = {"digest": "6307a3cfc9f539c1", "bytes_per_launch_4bit": 311702784, "algorithmic_4bit": 305485824,
-               "bytes_per_launch_2bit": 178128640, "algorithmic_2bit": 171792384}
+NCU_TRAFFIC = {"digest": "4791df85bfa43836", "bytes_per_launch_4bit": 311378432, "algorithmic_4bit": 305485824,
+               "bytes_per_launch_2bit": 177286912, "algorithmic_2bit": 171792384}
 
 
 class ClockSampler:
@@ -462,8 +462,8 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "decode_attn_splitk (+ combine), per pmkvq_decode_attention call",
                      "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic,
-                     "traffic_source": "ncu dram read+write per launch / algorithmic bytes (4-bit launch: 311.7 / 305.5 MB; "
-                                       "2-bit: 178.1 / 171.8 MB), times this run's average launch; null if the kernel "
+                     "traffic_source": "ncu dram read+write per launch / algorithmic bytes (4-bit launch: 311.4 / 305.5 MB; "
+                                       "2-bit: 177.3 / 171.8 MB), times this run's average launch; null if the kernel "
                                        "sources changed since the capture",
                      "avg_launch_ms": attn_ms / max(1, n_attn), "launches_timed": n_attn,
                      "algorithmic_bytes_per_launch": attn_bytes / max(1, n_attn),
