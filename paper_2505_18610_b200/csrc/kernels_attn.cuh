@@ -62,6 +62,12 @@ struct AttnParams {
   int w16;                    // units of one INT16 tile
   int units_lead;             // empty units at the start of every slice: the fixed cost of one more segment
   long long units_aux, units_slice, units_total, units_per_cta;  // units_aux includes units_lead
+  // Where this block's units sit on the line that is cut into CTA pieces.  A launch for one block has
+  // origin 0 and weight 1; the all-blocks launch strings the blocks together, each unit weighing
+  // `unit_weight` fine units (blocks of different widths cost different time per tile).
+  long long line_origin;      // fine units before this block's first unit
+  int unit_weight;            // fine units per unit
+  int cta_origin;             // first CTA that touches this block (partials are numbered from it)
   float qk_scale;             // sm_scale * log2(e)
 };
 
@@ -412,11 +418,15 @@ __device__ __forceinline__ void process_tiles(const uint8_t *tile0, uint32_t mas
 }
 
 // ---- where the partials of a slice live ------------------------------------------------------
-// Slice s covers units [s U, (s+1) U); the segment of CTA c in it publishes partial number c + s.
+// Slice s covers units [s U, (s+1) U); the segment of CTA c in it publishes partial number (c - cta_origin) + s.
+// A unit belongs to the CTA whose piece holds the unit's first fine unit (units_per_cta counts fine units).
+__device__ __forceinline__ int unit_owner(const AttnParams &p, long long unit) {
+  return (int)((p.line_origin + unit * p.unit_weight) / p.units_per_cta);
+}
 __device__ __forceinline__ void slice_ctas(const AttnParams &p, int slice, int &c_first, int &c_last) {
   const long long lo = (long long)slice * p.units_slice;
-  c_first = (int)((lo + p.units_lead) / p.units_per_cta);  // a CTA that only touches the lead units has no segment
-  c_last = (int)((lo + p.units_slice - 1) / p.units_per_cta);
+  c_first = unit_owner(p, lo + p.units_lead);  // a CTA that only touches the lead units has no segment
+  c_last = unit_owner(p, lo + p.units_slice - 1);
 }
 
 // Log-sum-exp merge of the partials of one slice (all published).  Warp w merges head w;
@@ -427,7 +437,7 @@ __device__ __forceinline__ void combine_slice(const AttnParams &p, int slice) {
   int cf, cl;
   slice_ctas(p, slice, cf, cl);
   const int n_parts = cl - cf + 1;
-  const float *base = p.partials + (size_t)(cf + slice) * kMaxGroup * kPartialStride;
+  const float *base = p.partials + (size_t)(cf - p.cta_origin + slice) * kMaxGroup * kPartialStride;
   for (int h = warp; h < p.group; h += kAttnWarps) {
     const float *ph = base + (size_t)h * kPartialStride;
     float M = kNegBig;
@@ -730,7 +740,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   __syncthreads();
 
   // ---- merge the warps, publish the segment's partial ----
-  float *part = p.partials + (size_t)(blockIdx.x + slice) * kMaxGroup * kPartialStride;
+  float *part = p.partials + (size_t)((int)blockIdx.x - p.cta_origin + slice) * kMaxGroup * kPartialStride;
   for (int i = tid; i < p.group * kHeadDim; i += kAttnThreads) {
     const int h = i >> 7, ch = i & 127;
     float M = kNegBig;
@@ -799,6 +809,108 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
   // A grid never completes before the grid it was allowed to overlap: kernels complete in launch order,
   // so whatever follows in the stream sees all of them done.  Returns at once for a normal launch.
   asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
+// All blocks of a decode step in one launch.  The blocks' units are strung together on one line (a
+// tile of a wider block weighs more fine units, in proportion to the time it takes) and the line is
+// cut into one piece per CTA, so launch ramp, tail and most segment set-ups are paid once per step
+// instead of once per block.  Per-block quantities are derived on the device from the block's token
+// count and width; geometry comes from the table the cache keeps in device memory.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxFusedLayers = 128;
+struct FusedParams {
+  const LayerGeom *geoms;     // [layers]
+  const uint16_t *Q;          // bf16 [layers][batch][q_heads][128]
+  const float *lambda;        // [layers][kv_heads][128]
+  const unsigned *vmax_bits;  // [layers][n_slices]
+  float *partials;            // per block, partial_stride floats apart
+  float *out;                 // fp32 [layers][batch][q_heads][128]
+  unsigned *tickets;          // [layers][n_slices]
+  size_t partial_stride;
+  int layers, kv_heads, group, q_heads, n_slices, batch;
+  int n_sink, window, evict_chunk, sink_tiles, ring_tiles;
+  float qk_scale;
+  long long per_cta, total;              // fine units
+  long long start[kMaxFusedLayers + 1];  // fine units before each block
+  int n_tokens[kMaxFusedLayers];
+  unsigned char bits[kMaxFusedLayers], lead[kMaxFusedLayers], weight[kMaxFusedLayers];
+};
+
+__device__ __forceinline__ void fused_layer_params(const FusedParams &fp, int l, AttnParams &p) {
+  const int n = fp.n_tokens[l], bits = fp.bits[l];
+  p.geom = fp.geoms[l];
+  p.Q = fp.Q + (size_t)l * fp.batch * fp.q_heads * kHeadDim;
+  p.lambda = fp.lambda + (size_t)l * fp.kv_heads * kHeadDim;
+  p.vmax_bits = fp.vmax_bits + (size_t)l * fp.n_slices;
+  p.partials = fp.partials + (size_t)l * fp.partial_stride;
+  p.out = fp.out + (size_t)l * fp.batch * fp.q_heads * kHeadDim;
+  p.tickets = fp.tickets + (size_t)l * fp.n_slices;
+  p.kv_heads = fp.kv_heads; p.group = fp.group; p.q_heads = fp.q_heads; p.n_slices = fp.n_slices;
+  p.n_tokens = n;
+  p.n_sink_eff = min(n, fp.n_sink);
+  const int excess = n - fp.n_sink - fp.window;
+  p.n_body = excess <= 0 ? 0 : excess / fp.evict_chunk * fp.evict_chunk;
+  p.win_start = p.n_sink_eff + p.n_body;
+  p.cur_bits = bits;
+  p.body_tiles = (p.n_body + 15) / 16;
+  p.sink_tiles = fp.sink_tiles;
+  p.aux_tiles = fp.sink_tiles + fp.ring_tiles;
+  p.w16 = (tile_bytes(16) + tile_bytes(bits) - 1) / tile_bytes(bits);
+  p.units_lead = fp.lead[l];
+  p.units_aux = p.units_lead + (long long)p.aux_tiles * p.w16;
+  p.units_slice = p.units_aux + p.body_tiles;
+  p.units_total = p.units_slice * fp.n_slices;
+  p.units_per_cta = fp.per_cta;
+  p.line_origin = fp.start[l];
+  p.unit_weight = fp.weight[l];
+  p.cta_origin = (int)(fp.start[l] / fp.per_cta);
+  p.qk_scale = fp.qk_scale;
+}
+
+__global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_fused_kernel(const __grid_constant__ FusedParams fp) {
+  __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
+  __shared__ float s_stat[16 + 2 * kAttnWarps * kMaxGroup];
+  __shared__ int s_ctr[4];
+  __shared__ uint4 s_frag[512];
+  extern __shared__ __align__(128) uint8_t ring[];
+  const long long f_begin = (long long)blockIdx.x * fp.per_cta;
+  const long long f_end = min(f_begin + fp.per_cta, fp.total);
+  int l = 0;
+  for (long long f = f_begin; f < f_end;) {
+    while (l + 1 < fp.layers && fp.start[l + 1] <= f) ++l;  // the block this fine unit belongs to
+    AttnParams p;
+    fused_layer_params(fp, l, p);
+    const long long f_hi = min(f_end, fp.start[l + 1]);
+    // units of this block whose first fine unit lies in [f, f_hi)
+    const int w = p.unit_weight;
+    long long u = (f - p.line_origin + w - 1) / w;
+    const long long u_end = (f_hi - p.line_origin + w - 1) / w;
+    while (u < u_end) {
+      const int slice = (int)(u / p.units_slice);
+      const long long base = (long long)slice * p.units_slice;
+      const long long hi = min(u_end - base, p.units_slice);
+      if (hi > p.units_lead) {
+        switch (p.cur_bits) {
+          case 16: run_segment<16>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
+          case 8: run_segment<8>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
+          case 4: run_segment<4>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
+          default: run_segment<2>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
+        }
+      }
+      u = base + hi;
+    }
+    f = f_hi;
+  }
+}
+
+// the most dynamic shared memory any width needs
+constexpr int attn_fused_smem_bytes() {
+  int m = attn_ring_bytes<16>();
+  m = attn_ring_bytes<8>() > m ? attn_ring_bytes<8>() : m;
+  m = attn_ring_bytes<4>() > m ? attn_ring_bytes<4>() : m;
+  m = attn_ring_bytes<2>() > m ? attn_ring_bytes<2>() : m;
+  return m;
 }
 
 }  // namespace pmkvq

@@ -53,6 +53,7 @@ struct pmkvq_cache {
   size_t off_lambda, off_inv_lambda, off_vmax, off_tickets, off_partials, partial_bytes, off_geoms;  // scratch is per block
   int sink_tiles, ring_tiles, user_ctas;
   int resident_ctas[4];  // one wave of the attention kernel at body width 16, 8, 4, 2
+  int resident_fused;    // one wave of the all-blocks attention kernel
   uint64_t launches = 0;  // kernels launched so far
   std::vector<Layer> L;
 
@@ -199,6 +200,12 @@ cudaError_t attention_setup(pmkvq_cache *k) {
   if (e == cudaSuccess) e = attention_setup_one<8>(k->resident_ctas[1], sms);
   if (e == cudaSuccess) e = attention_setup_one<4>(k->resident_ctas[2], sms);
   if (e == cudaSuccess) e = attention_setup_one<2>(k->resident_ctas[3], sms);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_attn_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_fused_smem_bytes());
+  int per_sm = 0;
+  if (e == cudaSuccess)
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_fused_kernel, kAttnThreads, attn_fused_smem_bytes());
+  k->resident_fused = std::min(kMaxCtas, std::max(1, per_sm) * sms);
   return e;
 }
 
@@ -426,6 +433,9 @@ static pmkvq_status attn_params(pmkvq_cache *k, int32_t layer, const void *d_Q, 
   const int want = k->user_ctas > 0 ? k->user_ctas : k->resident_ctas[width_idx];
   const long long per = std::max<long long>((p.units_total + want - 1) / want, k->user_ctas > 0 ? 1 : kMinUnitsPerCta);
   p.units_per_cta = per;
+  p.line_origin = 0;
+  p.unit_weight = 1;
+  p.cta_origin = 0;
   n_ctas = (unsigned)((p.units_total + per - 1) / per);
   p.qk_scale = k->sm_scale * 1.4426950408889634f;
   return PMKVQ_OK;
@@ -468,6 +478,51 @@ static pmkvq_status attention_on_arena(pmkvq_cache *k, int32_t layer, const void
   const cudaError_t e = attn_launch(p, n_ctas, st, overlap_previous);
   k->launches += 1;
   return e == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
+}
+
+// Time per 16-token tile at each width, in fiftieths of a 2-bit tile's (measured: 52.6 / 55.4 / 84.1 us per
+// block of 130 560 tiles at 2 / 4 / 8 bit, about 160 us at 16 bit).
+inline int tile_weight(int bits) { return bits == 16 ? 152 : bits == 8 ? 80 : bits == 4 ? 53 : 50; }
+
+static pmkvq_status attention_all_blocks(pmkvq_cache *k, const void *d_Q, float *d_out, cudaStream_t st) {
+  static_assert(kMaxFusedLayers >= kMaxStepLayers, "the step's argument tables share one size");
+  FusedParams fp;
+  fp.geoms = reinterpret_cast<const LayerGeom *>(k->arena + k->off_geoms);
+  fp.Q = static_cast<const uint16_t *>(d_Q);
+  fp.lambda = reinterpret_cast<const float *>(k->arena + k->off_lambda);
+  fp.vmax_bits = reinterpret_cast<const unsigned *>(k->arena + k->off_vmax);
+  fp.partials = reinterpret_cast<float *>(k->arena + k->off_partials);
+  fp.out = d_out;
+  fp.tickets = reinterpret_cast<unsigned *>(k->arena + k->off_tickets);
+  fp.partial_stride = k->partial_bytes / sizeof(float);
+  fp.layers = k->layers; fp.kv_heads = k->kv_heads; fp.group = k->group; fp.q_heads = k->q_heads;
+  fp.n_slices = k->n_slices; fp.batch = k->batch;
+  fp.n_sink = k->n_sink; fp.window = k->window; fp.evict_chunk = k->evict_chunk;
+  fp.sink_tiles = k->sink_tiles; fp.ring_tiles = k->ring_tiles;
+  fp.qk_scale = k->sm_scale * 1.4426950408889634f;
+  long long total = 0;
+  for (int l = 0; l < k->layers; ++l) {
+    const Layer &L = k->L[l];
+    if (L.n_tokens <= 0) return PMKVQ_ERR_INVALID_ARG;
+    const int bits = L.cur_bits;
+    const int w16 = (tile_bytes(16) + tile_bytes(bits) - 1) / tile_bytes(bits);
+    const long long body_tiles = (k->body_at(L.n_tokens) + 15) / 16;
+    const long long units_slice = segment_cost_tiles(bits) + (long long)(k->sink_tiles + k->ring_tiles) * w16 + body_tiles;
+    fp.start[l] = total;
+    fp.n_tokens[l] = L.n_tokens;
+    fp.bits[l] = (unsigned char)bits;
+    fp.lead[l] = (unsigned char)segment_cost_tiles(bits);
+    fp.weight[l] = (unsigned char)tile_weight(bits);
+    total += units_slice * k->n_slices * tile_weight(bits);
+  }
+  fp.start[k->layers] = total;
+  fp.total = total;
+  const int want = k->user_ctas > 0 ? k->user_ctas : k->resident_fused;
+  fp.per_cta = std::max<long long>((total + want - 1) / want, k->user_ctas > 0 ? 1 : 50ll * kMinUnitsPerCta);
+  const unsigned n_ctas = (unsigned)((total + fp.per_cta - 1) / fp.per_cta);
+  decode_attn_fused_kernel<<<n_ctas, kAttnThreads, attn_fused_smem_bytes(), st>>>(fp);
+  k->launches += 1;
+  return cudaGetLastError() == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }
 
 extern "C" {
@@ -537,14 +592,8 @@ pmkvq_status pmkvq_decode_step(pmkvq_cache *k, const void *d_K, const void *d_V,
   ++k->launches;
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
   for (int layer = 0; layer < k->layers; ++layer) k->L[layer].n_tokens += 1;
-  // 3. attention block by block; from the second block on a kernel may start while the previous one
-  //    drains (own tiles, own scratch, own output; the append above finished before the first started)
-  for (int layer = 0; layer < k->layers; ++layer) {
-    const pmkvq_status s = attention_on_arena(k, layer, static_cast<const uint8_t *>(d_Q) + layer * q_stride,
-                                              d_out + layer * o_stride, st, layer > 0);
-    if (s != PMKVQ_OK) return s;
-  }
-  return PMKVQ_OK;
+  // 3. attention of all blocks in one launch: their tiles form one line of work cut into one piece per CTA
+  return attention_all_blocks(k, d_Q, d_out, st);
 }
 
 pmkvq_status pmkvq_layer_state(const pmkvq_cache *k, int32_t layer, int32_t *n_tokens, int32_t *cur_bits,
