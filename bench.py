@@ -173,11 +173,11 @@ def kernel_source_digest():
     return h.hexdigest()[:16]
 
 
-# DRAM read + write bytes per launch of the attention kernel from the ncu capture summarised in
-# profiles/decode_attn_splitk_7b_shape.md (7B shape, body at 4 bit: the launch kind with the largest time
-# share; algorithmic bytes of that launch: 305.5 MB), and the digest of the sources it was taken on.
-NCU_TRAFFIC = {"digest": "4791df85bfa43836", "bytes_per_launch_4bit": 311378432, "algorithmic_4bit": 305485824,
-               "bytes_per_launch_2bit": 177286912, "algorithmic_2bit": 171792384}
+# DRAM read + write bytes of one launch of the all-blocks attention kernel from the ncu capture summarised in
+# profiles/decode_attn_fused_7b_shape.md (4 blocks of the 7B shape: a launch of the 28-block workload moves
+# 7x the bytes, block by block the same way), its algorithmic bytes, and the digest of the sources it was
+# taken on.
+NCU_TRAFFIC = {"digest": "187398695b56c60d", "traffic_bytes": 975_617_536, "algorithmic_bytes": 954_646_528}
 
 
 class ClockSampler:
@@ -240,14 +240,15 @@ def run_steps(cache, wl, pool, steps, first_step, out, host_io=None, attn_events
         elif attn_events is None:
             cache.decode_step(K[i], V[i], Q[i], out=out)
         else:
-            # same launches as decode_step, block by block, with an event pair around each attention call
-            for l in range(L):
-                cache.append(l, K[i, l], V[i, l])
-                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-                e0.record()
-                cache.decode_attention(l, Q[i, l], out=out[l])
-                e1.record()
-                attn_events.append((e0, e1, cache.attention_bytes(l)))
+            # an event pair around the step's launches: the all-blocks attention kernel and the all-blocks
+            # append kernel before it (and, in the few steps where a block's budget fills, its reduce)
+            bits0 = [cache.layer_state(l)["cur_bits"] for l in range(L)]
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            cache.decode_step(K[i], V[i], Q[i], out=out)
+            e1.record()
+            reduced = any(cache.layer_state(l)["cur_bits"] != bits0[l] for l in range(L))
+            attn_events.append((e0, e1, sum(cache.attention_bytes(l) for l in range(L)), reduced))
 
 
 def cpu_oracle_leg(wl, seconds_target=12.0, steps=None, warmup=1, n_sample_slices=4):
@@ -381,7 +382,7 @@ def main():
     cache.close(); del cache
     torch.cuda.empty_cache()
 
-    # ---------------- the same timed region again, with an event pair around every attention launch ----------------
+    # ---------------- the same timed region again, with an event pair around every step ----------------
     attn_ms, attn_bytes, n_attn, instr_ms = float("nan"), 0, 0, float("nan")
     if not args.no_kernel_timing:
         cache = build_cache(wl, fbit, budgets, lam, n0, device)
@@ -396,9 +397,10 @@ def main():
         k1.record()
         barrier()
         instr_ms = k0.elapsed_time(k1)
-        attn_ms = sum(a.elapsed_time(b) for a, b, _ in attn_events)
-        attn_bytes = sum(c for _, _, c in attn_events)
-        n_attn = len(attn_events)
+        plain = [(a, b, c) for a, b, c, reduced in attn_events if not reduced] or [(a, b, c) for a, b, c, _ in attn_events]
+        attn_ms = sum(a.elapsed_time(b) for a, b, _ in plain)
+        attn_bytes = sum(c for _, _, c in plain)
+        n_attn = len(plain)
         cache.close(); del cache
         torch.cuda.empty_cache()
 
@@ -443,7 +445,7 @@ def main():
     traffic = None
     if wl is WORKLOADS["7b"] and kernel_source_digest() == NCU_TRAFFIC["digest"] and n_attn:
         # measured traffic / algorithmic bytes of the captured launches, applied to this run's average launch
-        ratio = NCU_TRAFFIC["bytes_per_launch_4bit"] / NCU_TRAFFIC["algorithmic_4bit"]
+        ratio = NCU_TRAFFIC["traffic_bytes"] / NCU_TRAFFIC["algorithmic_bytes"]
         traffic = ratio * attn_bytes / n_attn
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9 if n_attn else float("nan")
     line = {
@@ -459,22 +461,17 @@ def main():
                    "path": "attention path only (no weights / MLP)", "sharding": "batch, no collective"},
         "tokens_per_s": whole_job_rate(wl["batch"] * steps, world, ms),
         "frac_of_8TBps_nominal": value / world / 8000.0,
-        "roofline": {"bound": "hbm", "kernel": "decode_attn_splitk (+ combine), per pmkvq_decode_attention call",
+        "roofline": {"bound": "hbm", "kernel": "decode_attn_fused_kernel: the attention of all blocks of a step, one launch",
                      "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic,
-                     "traffic_source": "ncu dram read+write per launch / algorithmic bytes (4-bit launch: 311.4 / 305.5 MB; "
-                                       "2-bit: 177.3 / 171.8 MB), times this run's average launch; null if the kernel "
-                                       "sources changed since the capture",
+                     "traffic_source": "ncu dram read+write / algorithmic bytes of a captured 4-block launch of the same kernel, times this "
+                                       "run's average launch; null if the kernel sources changed since the capture",
                      "avg_launch_ms": attn_ms / max(1, n_attn), "launches_timed": n_attn,
                      "algorithmic_bytes_per_launch": attn_bytes / max(1, n_attn),
-                     "how": "the timed steps replayed on an identical cache with a CUDA event pair around every "
-                            "pmkvq_decode_attention launch (one kernel per call)",
-                     "ms_per_step_with_events": instr_ms / steps,
-                     "achieved_inside_decode_step": (attn_bytes / max(1, n_attn)) * wl["layers"] * steps / (ms * 1e-3) / 1e9
-                     if n_attn else None,
-                     "achieved_inside_decode_step_note": "attention bytes of a step / whole step time of the device-resident leg "
-                                                         "(appends and reduces included): consecutive blocks' attention kernels "
-                                                         "overlap there, so a per-launch duration does not exist"},
+                     "how": "the timed steps replayed on an identical cache with a CUDA event pair around every step; "
+                            "the pair also spans the step's append kernel (one launch, under 1 % of the step); steps in "
+                            "which a block was reduced are left out of the average",
+                     "ms_per_step_with_events": instr_ms / steps},
         "e2e": {"value": world * total_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms / steps,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
