@@ -51,6 +51,14 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
                                 s = 1 at positions 0, 4, 8, ...; with the lowest-frequency pair's
                                 2 pi / theta_i = 54,410-token period (Sec. 3.3) a 2,048-token text
                                 reaches the pair's full amplitude only with interpolation)
+  causal_self_attention / attention_reconstruction_losses / grid_search_alpha
+                       pinned  (brute-force loops on a tiny case incl. the head-to-KV-head map;
+                                loss vanishes at 16 bit for every alpha, so Lambda and Lambda^-1 pair
+                                up; one token: loss = the Value quantization error alone, whatever
+                                alpha; the last query row equals decode_attention of a LayerOracle
+                                holding the same tokens; at alpha = 1 the loss is unchanged by
+                                power-of-two rescaling of a channel pair of K against Q; an outlier
+                                channel pair moves the best alpha away from 0)
   allocate_bits_brute_force
                        pinned  (it IS the definition of Eq. 6-8 written out; limits: budget at
                                 the floor / unbounded; hand case)
@@ -463,3 +471,79 @@ def calibrate_lambda(k_pre, pos_scale: float = 1.0, theta: float = 10000.0, alph
     rot = rope_interpolated(k, np.arange(k.shape[0]), pos_scale, theta)
     amax = np.abs(rot).max(axis=(0, 1))
     return np.maximum(amax, floor) ** alpha
+
+
+# --------------------------------------------------------------------------
+# Sec. 4.1.1: alpha of Eq. 10 by grid search on the attention reconstruction loss
+# --------------------------------------------------------------------------
+def causal_self_attention(q, k, v, group: int):
+    """softmax(Q K^T / sqrt(d)) V with a causal mask, per sequence and head, in float64.
+    q: [n, n_seq, kv_heads * group, d]; k, v: [n, n_seq, kv_heads, d]; query head h reads KV head h // group
+    (grouped-query attention); token t attends to tokens 0..t.  Returns [n, n_seq, kv_heads * group, d]."""
+    q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
+    n, n_seq, q_heads, d = q.shape
+    out = np.empty_like(q)
+    mask = np.tril(np.ones((n, n), dtype=bool))
+    for b in range(n_seq):
+        for h in range(q_heads):
+            sc = (q[:, b, h] @ k[:, b, h // group].T) / np.sqrt(float(d))
+            sc = np.where(mask, sc, -np.inf)
+            sc = sc - sc.max(axis=1, keepdims=True)
+            pr = np.exp(sc)
+            pr = pr / pr.sum(axis=1, keepdims=True)
+            out[:, b, h] = pr @ v[:, b, h // group]
+    return out
+
+
+def quantize_progressively(x, bits: int):
+    """What the cache holds for a token that has reached ``bits``: Eq. 1-2 at 16 bit on fp32 values, then
+    the Eq. 3 chain down to ``bits``; returned dequantized (float64)."""
+    c16, s16, z = quantize_asym(np.asarray(x, dtype=np.float32), 16)
+    c, s = chain_to(c16, s16, bits)
+    return dequantize(c, s, z)
+
+
+def attention_reconstruction_losses(k_pre, q_pre, v, group: int, bits: int, alphas, pos_scale: float = 1.0,
+                                    theta: float = 10000.0, floor: float = 1e-5):
+    """Loss of the self-attention operator for each alpha of the grid (Sec. 4.1.1), on one block's calibration
+    tensors: k_pre, v [n, n_seq, kv_heads, d] and q_pre [n, n_seq, kv_heads * group, d], Keys and Queries
+    before RoPE, token t at position t.
+
+    Keys and Queries are rotated with the interpolated RoPE of Eq. 12; lambda(alpha) follows Eq. 10 on the
+    rotated Keys; the quantized operator is Eq. 9, (Q Lambda) . Q_b(K Lambda^-1)^T, with K Lambda^-1 formed
+    in fp32 from the fp32 lambda the cache would be configured with, K and V both quantized the way the cache
+    holds ``bits``-bit tokens.  The loss is the mean squared difference between the causal self-attention
+    output of the unquantized tensors and that of the quantized ones, over all tokens, sequences, heads and
+    channels.  Returns a float64 array, one loss per alpha."""
+    k_pre, q_pre, v = (np.asarray(a, dtype=np.float64) for a in (k_pre, q_pre, v))
+    n = k_pre.shape[0]
+    pos = np.arange(n)
+    k_rot = rope_interpolated(k_pre, pos, pos_scale, theta)
+    q_rot = rope_interpolated(q_pre, pos, pos_scale, theta)
+    amax = np.maximum(np.abs(k_rot).max(axis=(0, 1)), floor)          # [kv_heads, d]
+    ref = causal_self_attention(q_rot, k_rot, v, group)
+    v_hat = quantize_progressively(v, bits)
+    k32 = k_rot.astype(np.float32)
+    losses = []
+    for alpha in alphas:
+        lam = (amax ** float(alpha)).astype(np.float32)              # Eq. 10
+        inv = (np.float32(1.0) / lam).astype(np.float32)
+        k_hat = quantize_progressively((k32 * inv[None, None]).astype(np.float32), bits)
+        q_eq = q_rot * np.repeat(lam.astype(np.float64), group, axis=0)[None, None]
+        got = causal_self_attention(q_eq, k_hat, v_hat, group)
+        losses.append(float(np.mean((got - ref) ** 2)))
+    return np.asarray(losses, dtype=np.float64)
+
+
+def alpha_grid(n_grid: int = 20):
+    """The search grid over [0, 1]: n_grid equally spaced values starting at 0, alpha_j = j / n_grid (the
+    convention of the grid search the section cites; alpha = 1 itself is not visited)."""
+    return np.arange(n_grid, dtype=np.float64) / float(n_grid)
+
+
+def grid_search_alpha(k_pre, q_pre, v, group: int, bits: int, n_grid: int = 20, **kw):
+    """Sec. 4.1.1: the alpha of the grid with the smallest reconstruction loss (the first one on ties).
+    Returns (alpha, losses)."""
+    alphas = alpha_grid(n_grid)
+    losses = attention_reconstruction_losses(k_pre, q_pre, v, group, bits, alphas, **kw)
+    return float(alphas[int(np.argmin(losses))]), losses
