@@ -127,9 +127,9 @@ pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *cache, int32_t layer, co
  *   d_out:              DEVICE fp32 [layers][batch][q_heads][128]
  * The budget of every block is tested first (reducing where auto_reduce allows); if a block fails
  * (PMKVQ_ERR_BUDGET_FULL with auto_reduce = 0, PMKVQ_ERR_CAPACITY) its status is returned and no block has
- * received its token.  Then one launch appends to all blocks and one attention launch per block
- * follows; consecutive attention kernels may overlap on the GPU, and all of them have completed
- * before anything enqueued on `stream` after this call starts. */
+ * received its token.  Then one launch appends to all blocks and one launch computes the attention
+ * of all blocks (up to 128 blocks; beyond that the call falls back to one append and one attention
+ * launch per block). */
 pmkvq_status pmkvq_decode_step(pmkvq_cache *cache, const void *d_K_bf16, const void *d_V_bf16, const void *d_Q_bf16,
                                float *d_out, void *stream);
 
@@ -166,10 +166,36 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *cache, int32_t layer, int32_t batch
  *   d_K_pre_bf16  DEVICE bf16 [n_tokens][n_seq][kv_heads][128], token t sits at position t
  *   d_lambda      DEVICE fp32 [kv_heads][128], written (it also serves as the kernel's only workspace)
  * The rotation is computed in fp32 from fp64 angles; the result feeds pmkvq_config.lambda after a copy to
- * the host.  The grid search over alpha of Sec. 4.1.1 is left to the caller (alpha is an argument). */
+ * the host.  alpha is an argument; pmkvq_alpha_grid_search below picks it as Sec. 4.1.1 does. */
 pmkvq_status pmkvq_calibrate_lambda(const void *d_K_pre_bf16, int32_t n_tokens, int32_t n_seq, int32_t kv_heads,
                                     double pos_scale, double theta, float alpha, float floor_value, float *d_lambda,
                                     void *stream);
+
+/* alpha of Eq. 10 by grid search (Sec. 4.1.1: the alpha that minimises the reconstruction loss of the
+ * self-attention operator), on the device, for one transformer block's calibration tensors.
+ * For every alpha of the grid: lambda = max(amax, floor)^alpha from the Keys rotated per Eq. 12; the
+ * quantized operator is Eq. 9, (Q Lambda) . Q_b(K Lambda^-1)^T, with K Lambda^-1 quantized at 16 bit
+ * (Eq. 1-2, per token and KV head) and taken down the Eq. 3 chain to `bits`, Values quantized the same
+ * way; loss[alpha] = mean squared difference between the causal self-attention output (softmax of
+ * Q K^T / sqrt(128), query head h reads KV head h / group, token t attends to tokens 0..t) of the
+ * unquantized rotated tensors and of the quantized ones, over tokens, sequences, heads and channels.
+ * Arithmetic: fp32 throughout (quantizer decisions as in pmkvq_append), sums of squared errors in fp64.
+ *   d_K_pre_bf16, d_V_bf16  DEVICE bf16 [n_tokens][n_seq][kv_heads][128]; Keys before RoPE, token t at position t
+ *   d_Q_pre_bf16            DEVICE bf16 [n_tokens][n_seq][kv_heads * group][128], before RoPE
+ *   bits                    2, 4, 8 or 16: the width whose loss is minimised (the block's Fbit)
+ *   h_alphas                HOST [n_alphas], 1 <= n_alphas <= 64 (the section's grid: j / 20, j = 0..19)
+ *   d_workspace             DEVICE, 256-byte aligned, pmkvq_alpha_grid_workspace_bytes(n_tokens, kv_heads) bytes
+ *   h_losses                HOST [n_alphas], written
+ *   h_best                  HOST, may be NULL: index of the smallest loss (the first one on ties)
+ * The call synchronises `stream` before it returns (its results are host values).  The paper states
+ * the criterion only; causal masking, the quantization of the Values and the mean-squared form are
+ * this library's reading of it. */
+uint64_t pmkvq_alpha_grid_workspace_bytes(int32_t n_tokens, int32_t kv_heads);
+pmkvq_status pmkvq_alpha_grid_search(const void *d_K_pre_bf16, const void *d_Q_pre_bf16, const void *d_V_bf16,
+                                     int32_t n_tokens, int32_t n_seq, int32_t kv_heads, int32_t group, int32_t bits,
+                                     const float *h_alphas, int32_t n_alphas, double pos_scale, double theta,
+                                     float floor_value, void *d_workspace, double *h_losses, int32_t *h_best,
+                                     void *stream);
 
 /* Block-wise bit allocation (Sec. 3.2, Eq. 6-8), host only: choose one bit width per block so that the
  * summed sensitivity is minimal and the summed memory stays within the budget,

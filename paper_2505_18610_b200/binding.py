@@ -73,6 +73,11 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_calibrate_lambda.restype = i32
     lib.pmkvq_calibrate_lambda.argtypes = [vp, i32, i32, i32, ctypes.c_double, ctypes.c_double, ctypes.c_float,
                                            ctypes.c_float, vp, vp]
+    lib.pmkvq_alpha_grid_workspace_bytes.restype = ctypes.c_uint64
+    lib.pmkvq_alpha_grid_workspace_bytes.argtypes = [i32, i32]
+    lib.pmkvq_alpha_grid_search.restype = i32
+    lib.pmkvq_alpha_grid_search.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, ctypes.c_double, ctypes.c_double,
+                                            ctypes.c_float, vp, vp, vp, vp]
     lib.pmkvq_allocate_bits.restype = i32
     lib.pmkvq_allocate_bits.argtypes = [i32, i32, vp, vp, vp, ctypes.c_uint64, vp, vp]
     lib.pmkvq_status_string.restype = ctypes.c_char_p
@@ -109,6 +114,30 @@ def calibrate_lambda(k_pre: torch.Tensor, pos_scale: float = 1.0, theta: float =
     if st != OK:
         raise PmkvqError(st, "pmkvq_calibrate_lambda")
     return lam
+
+
+def alpha_grid_search(k_pre: torch.Tensor, q_pre: torch.Tensor, v: torch.Tensor, bits: int, alphas=None,
+                      pos_scale: float = 1.0, theta: float = 10000.0, floor_value: float = 1e-5, stream=None):
+    """alpha of Eq. 10 by grid search on the attention reconstruction loss (Sec. 4.1.1), on the device.
+    k_pre, v: CUDA bf16 [n_tokens, n_seq, kv_heads, 128]; q_pre: [n_tokens, n_seq, kv_heads * group, 128];
+    alphas: the grid (default j / 20, j = 0..19).  Returns (best alpha, losses as a float64 array)."""
+    for t in (k_pre, q_pre, v):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16 and t.dim() == 4 and t.shape[3] == 128):
+            raise ValueError("k_pre, q_pre, v must be contiguous CUDA bf16 tensors [n_tokens, n_seq, heads, 128]")
+    n_tokens, n_seq, kv_heads, _ = k_pre.shape
+    if v.shape != k_pre.shape or q_pre.shape[:2] != k_pre.shape[:2] or q_pre.shape[2] % kv_heads:
+        raise ValueError("shapes of k_pre, q_pre, v do not fit together")
+    group = q_pre.shape[2] // kv_heads
+    a = np.ascontiguousarray(np.arange(20) / 20.0 if alphas is None else alphas, dtype=np.float32)
+    ws = torch.empty(int(lib().pmkvq_alpha_grid_workspace_bytes(n_tokens, kv_heads)), dtype=torch.uint8, device=k_pre.device)
+    losses = np.zeros(len(a), np.float64)
+    best = ctypes.c_int32()
+    st = lib().pmkvq_alpha_grid_search(k_pre.data_ptr(), q_pre.data_ptr(), v.data_ptr(), n_tokens, n_seq, kv_heads, group,
+                                       int(bits), a.ctypes.data, len(a), float(pos_scale), float(theta), float(floor_value),
+                                       ws.data_ptr(), losses.ctypes.data, ctypes.addressof(best), _stream_ptr(stream))
+    if st != OK:
+        raise PmkvqError(st, "pmkvq_alpha_grid_search")
+    return float(a[best.value]), losses
 
 
 def allocate_bits(widths, sensitivity, mem_bytes, budget_bytes):

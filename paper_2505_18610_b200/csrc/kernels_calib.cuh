@@ -61,4 +61,213 @@ __global__ void calib_finish_kernel(float *lambda, int n, float floor_value, flo
   if (i < n) lambda[i] = powf(fmaxf(lambda[i], floor_value), alpha);
 }
 
+// ---------------------------------------------------------------------------------------------
+// alpha of Eq. 10 by grid search (Sec. 4.1.1): for every alpha of the grid, the squared error between the
+// causal self-attention of the calibration tensors and the same operator on what the cache would hold
+// at `bits` (Eq. 9: Queries times Lambda, Keys times Lambda^-1 quantized at 16 bit and taken down the
+// Eq. 3 chain; Values quantized likewise).  Keys and Queries are rotated on the fly with the
+// interpolated RoPE of Eq. 12 from a (cos, sin) table.
+// ---------------------------------------------------------------------------------------------
+
+// table[t][pair] = (cos, sin) of pos_scale * t * theta^(-2 pair / 128), rounded from fp64.
+__global__ void rope_table_kernel(float2 *table, int n_tokens, double pos_scale, double theta) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_tokens * 64) return;
+  const int t = i >> 6, pair = i & 63;
+  double s, c;
+  sincos((double)t * pos_scale * pow(theta, -2.0 * pair / (double)kHeadDim), &s, &c);
+  table[i] = make_float2((float)c, (float)s);
+}
+
+constexpr int kGridQueries = 32;  // queries of one CTA (4 threads each)
+constexpr int kGridKeys = 32;     // keys per shared-memory tile
+constexpr int kMaxAlphas = 64;
+
+// One token's 4 channels per lane (channels 4 lane .. 4 lane + 3): rotate by the token's angles.  The
+// partner channel (+-64) sits in lane ^ 16.
+__device__ __forceinline__ void rotate_token(float (&x)[4], const float2 *__restrict__ table_t, int lane) {
+  const int pair0 = (lane & 15) * 4;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float other = __shfl_xor_sync(0xffffffffu, x[e], 16);
+    const float2 cs = table_t[pair0 + e];
+    // lanes 0..15 hold x1 (channel < 64): y1 = x1 c - x2 s;  lanes 16..31 hold x2: y2 = x1 s + x2 c
+    x[e] = lane < 16 ? __fsub_rn(__fmul_rn(x[e], cs.x), __fmul_rn(other, cs.y))
+                     : __fadd_rn(__fmul_rn(other, cs.y), __fmul_rn(x[e], cs.x));
+  }
+}
+
+// Eq. 1-2 at 16 bit on one token's 128 channels spread over a warp, the Eq. 3 chain to `bits`, and back
+// to real values: x <- S_b * code_b + Z.
+__device__ __forceinline__ void quantize_dequantize_token(float (&x)[4], int bits) {
+  float mn = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
+  float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  const float s16 = __fdiv_rn(__fsub_rn(mx, mn), 65535.0f);
+  float sb = s16;
+  for (int w = 8; w >= bits; w >>= 1) sb = __fmul_rn(sb, (float)((1 << w) + 1));
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    int c = 0;
+    if (s16 != 0.0f) {
+      c = __float2int_rn(__fdiv_rn(__fsub_rn(x[e], mn), s16));
+      c = min(max(c, 0), 65535);
+    }
+    x[e] = fmaf((float)shift_chain((uint32_t)c, bits), sb, mn);
+  }
+}
+
+__device__ __forceinline__ void load_bf16x4(const uint16_t *src, float (&x)[4]) {
+  const uint2 raw = *reinterpret_cast<const uint2 *>(src);
+  x[0] = __uint_as_float(raw.x << 16);
+  x[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+  x[2] = __uint_as_float(raw.y << 16);
+  x[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+}
+
+// Grid: (query blocks, query heads, sequences).  K, V: bf16 [n_tokens][n_seq][kv_heads][128];
+// Q: bf16 [n_tokens][n_seq][kv_heads * group][128]; amax [kv_heads][128] from calib_absmax_kernel;
+// loss_sums [n_alphas] (fp64, zero before the launch) receives the summed squared errors.
+// Thread (query, part j) owns channels 16 c + 4 j + e (c < 8, e < 4), so that a rotation pair stays in
+// one thread and the four parts of a query read one 64-byte run of a key row.
+__global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ Q,
+                                                         const uint16_t *__restrict__ V, const float *__restrict__ amax,
+                                                         const float2 *__restrict__ table, const float *__restrict__ alphas,
+                                                         int n_alphas, int n_tokens, int n_seq, int kv_heads, int group,
+                                                         int bits, float floor_value, double *loss_sums) {
+  __shared__ __align__(16) float s_k[kGridKeys][kHeadDim];
+  __shared__ __align__(16) float s_v[kGridKeys][kHeadDim];
+  __shared__ float s_lam[kHeadDim], s_inv[kHeadDim];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;  // long rows first
+  const int q_head = blockIdx.y, seq = blockIdx.z, kv_head = q_head / group, q_heads = kv_heads * group;
+  const int qi = qb * kGridQueries + (tid >> 2), part = tid & 3;
+  const bool q_live = qi < n_tokens;
+  const int q_last = min(n_tokens, (qb + 1) * kGridQueries) - 1;  // last live query of the CTA
+  const size_t kv_row = (size_t)n_seq * kv_heads * kHeadDim;
+  const uint16_t *k_base = K + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
+  const uint16_t *v_base = V + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
+  const float scale_log2 = 1.4426950408889634f * rsqrtf((float)kHeadDim);
+
+  // this thread's rotated query channels, in the order (c, e)
+  float q_rot[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) q_rot[i] = 0.f;
+  if (q_live) {
+    const uint16_t *src = Q + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim;
+    const float2 *tab = table + (size_t)qi * 64;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float x1[4], x2[4];
+      load_bf16x4(src + 16 * c + 4 * part, x1);
+      load_bf16x4(src + 64 + 16 * c + 4 * part, x2);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 cs = tab[16 * c + 4 * part + e];
+        q_rot[4 * c + e] = __fsub_rn(__fmul_rn(x1[e], cs.x), __fmul_rn(x2[e], cs.y));
+        q_rot[4 * (c + 4) + e] = __fadd_rn(__fmul_rn(x1[e], cs.y), __fmul_rn(x2[e], cs.x));
+      }
+    }
+  }
+
+  float ref[32];
+  for (int pass = 0; pass <= n_alphas; ++pass) {
+    __syncthreads();  // the previous pass is done with s_lam / s_inv and the tiles
+    if (pass > 0) {
+      const float lam = powf(fmaxf(amax[(size_t)kv_head * kHeadDim + tid], floor_value), alphas[pass - 1]);
+      s_lam[tid] = lam;
+      s_inv[tid] = __fdiv_rn(1.0f, lam);
+    }
+    __syncthreads();
+    float qe[32], acc[32];
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lam = pass > 0 ? s_lam[16 * c + 4 * part + e] : 1.0f;
+        qe[4 * c + e] = q_rot[4 * c + e] * lam * scale_log2;
+        acc[4 * c + e] = 0.f;
+      }
+    float m = -INFINITY, l = 0.f;
+    for (int k0 = 0; k0 <= q_last; k0 += kGridKeys) {
+      __syncthreads();  // everyone is done with the previous tile
+      // ---- stage the tile: warp w takes keys 8 w .. 8 w + 7 ----
+      for (int r = 0; r < 8; ++r) {
+        const int kk = warp * 8 + r, t = k0 + kk;
+        float xk[4] = {0.f, 0.f, 0.f, 0.f}, xv[4] = {0.f, 0.f, 0.f, 0.f};
+        if (t < n_tokens) {  // warp-uniform
+          load_bf16x4(k_base + (size_t)t * kv_row + 4 * lane, xk);
+          load_bf16x4(v_base + (size_t)t * kv_row + 4 * lane, xv);
+          rotate_token(xk, table + (size_t)t * 64, lane);
+          if (pass > 0) {
+            const float4 inv = *reinterpret_cast<const float4 *>(&s_inv[4 * lane]);
+            xk[0] = __fmul_rn(xk[0], inv.x); xk[1] = __fmul_rn(xk[1], inv.y);
+            xk[2] = __fmul_rn(xk[2], inv.z); xk[3] = __fmul_rn(xk[3], inv.w);
+            quantize_dequantize_token(xk, bits);
+            quantize_dequantize_token(xv, bits);
+          }
+        }
+        *reinterpret_cast<float4 *>(&s_k[kk][4 * lane]) = make_float4(xk[0], xk[1], xk[2], xk[3]);
+        *reinterpret_cast<float4 *>(&s_v[kk][4 * lane]) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+      }
+      __syncthreads();
+      // ---- scores, online softmax, output ----
+      const int k_hi = min(kGridKeys, q_last - k0 + 1);
+      for (int kk = 0; kk < k_hi; ++kk) {
+        float s = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float4 kv = *reinterpret_cast<const float4 *>(&s_k[kk][16 * c + 4 * part]);
+          s = fmaf(qe[4 * c], kv.x, s); s = fmaf(qe[4 * c + 1], kv.y, s);
+          s = fmaf(qe[4 * c + 2], kv.z, s); s = fmaf(qe[4 * c + 3], kv.w, s);
+        }
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        if (k0 + kk <= qi) {  // causal; the four threads of a query agree
+          if (s > m) {
+            const float corr = exp2f(m - s);  // 0 on the first key
+            l *= corr;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] *= corr;
+            m = s;
+          }
+          const float p = exp2f(s - m);
+          l += p;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const float4 vv = *reinterpret_cast<const float4 *>(&s_v[kk][16 * c + 4 * part]);
+            acc[4 * c] = fmaf(p, vv.x, acc[4 * c]); acc[4 * c + 1] = fmaf(p, vv.y, acc[4 * c + 1]);
+            acc[4 * c + 2] = fmaf(p, vv.z, acc[4 * c + 2]); acc[4 * c + 3] = fmaf(p, vv.w, acc[4 * c + 3]);
+          }
+        }
+      }
+    }
+    // ---- the pass's output: keep it (pass 0) or compare with the kept one ----
+    float err = 0.f;
+    if (q_live) {
+      const float inv_l = __fdiv_rn(1.0f, l);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float o = acc[i] * inv_l;
+        if (pass == 0) {
+          ref[i] = o;
+        } else {
+          const float d = o - ref[i];
+          err = fmaf(d, d, err);
+        }
+      }
+    }
+    if (pass > 0) {
+      double e = (double)err;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+      if (lane == 0) atomicAdd(loss_sums + (pass - 1), e);
+    }
+  }
+}
+
 }  // namespace pmkvq

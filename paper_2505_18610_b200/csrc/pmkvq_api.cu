@@ -694,6 +694,64 @@ pmkvq_status pmkvq_calibrate_lambda(const void *d_K, int32_t n_tokens, int32_t n
   return cudaGetLastError() == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }
 
+static size_t grid_ws_round(size_t b) { return (b + 255) / 256 * 256; }
+
+uint64_t pmkvq_alpha_grid_workspace_bytes(int32_t n_tokens, int32_t kv_heads) {
+  if (n_tokens <= 0 || kv_heads <= 0) return 0;
+  return grid_ws_round((size_t)kv_heads * kHeadDim * sizeof(float)) + grid_ws_round((size_t)n_tokens * 64 * sizeof(float2)) +
+         grid_ws_round(kMaxAlphas * sizeof(double)) + grid_ws_round(kMaxAlphas * sizeof(float));
+}
+
+pmkvq_status pmkvq_alpha_grid_search(const void *d_K, const void *d_Q, const void *d_V, int32_t n_tokens, int32_t n_seq,
+                                     int32_t kv_heads, int32_t group, int32_t bits, const float *h_alphas,
+                                     int32_t n_alphas, double pos_scale, double theta, float floor_value,
+                                     void *d_workspace, double *h_losses, int32_t *h_best, void *stream) {
+  if (!d_K || !d_Q || !d_V || !h_alphas || !d_workspace || !h_losses || n_tokens <= 0 || n_seq <= 0 || kv_heads <= 0 ||
+      group <= 0 || n_alphas <= 0 || n_alphas > kMaxAlphas || !(pos_scale > 0.0) || !(theta > 1.0) || !(floor_value > 0.f))
+    return PMKVQ_ERR_INVALID_ARG;
+  if (bits != 2 && bits != 4 && bits != 8 && bits != 16) return PMKVQ_ERR_INVALID_ARG;
+  if ((int64_t)n_seq * kv_heads > (1 << 20) || (int64_t)kv_heads * group > 65535 || n_seq > 65535 ||
+      (reinterpret_cast<uintptr_t>(d_workspace) & 255))
+    return PMKVQ_ERR_INVALID_ARG;
+  for (int i = 0; i < n_alphas; ++i)
+    if (!std::isfinite(h_alphas[i])) return PMKVQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t *ws = static_cast<uint8_t *>(d_workspace);
+  float *d_amax = reinterpret_cast<float *>(ws);
+  ws += grid_ws_round((size_t)kv_heads * kHeadDim * sizeof(float));
+  float2 *d_table = reinterpret_cast<float2 *>(ws);
+  ws += grid_ws_round((size_t)n_tokens * 64 * sizeof(float2));
+  double *d_loss = reinterpret_cast<double *>(ws);
+  ws += grid_ws_round(kMaxAlphas * sizeof(double));
+  float *d_alphas = reinterpret_cast<float *>(ws);
+  if (cudaMemsetAsync(d_amax, 0, (size_t)kv_heads * kHeadDim * sizeof(float), st) != cudaSuccess ||
+      cudaMemsetAsync(d_loss, 0, kMaxAlphas * sizeof(double), st) != cudaSuccess ||
+      cudaMemcpyAsync(d_alphas, h_alphas, (size_t)n_alphas * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return PMKVQ_ERR_CUDA;
+  const int tokens_per_cta = std::max(1, (n_tokens + 148 * 8 - 1) / (148 * 8));
+  calib_absmax_kernel<<<(unsigned)((n_tokens + tokens_per_cta - 1) / tokens_per_cta), 128, 0, st>>>(
+      static_cast<const uint16_t *>(d_K), reinterpret_cast<unsigned *>(d_amax), n_tokens, n_seq * kv_heads, kv_heads,
+      tokens_per_cta, pos_scale, theta);
+  rope_table_kernel<<<(unsigned)((n_tokens * 64 + 255) / 256), 256, 0, st>>>(d_table, n_tokens, pos_scale, theta);
+  const dim3 grid((unsigned)((n_tokens + kGridQueries - 1) / kGridQueries), (unsigned)(kv_heads * group), (unsigned)n_seq);
+  alpha_grid_kernel<<<grid, 128, 0, st>>>(static_cast<const uint16_t *>(d_K), static_cast<const uint16_t *>(d_Q),
+                                          static_cast<const uint16_t *>(d_V), d_amax, d_table, d_alphas, n_alphas, n_tokens,
+                                          n_seq, kv_heads, group, bits, floor_value, d_loss);
+  if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  double sums[kMaxAlphas];
+  if (cudaMemcpyAsync(sums, d_loss, (size_t)n_alphas * sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return PMKVQ_ERR_CUDA;
+  const double count = (double)n_tokens * n_seq * kv_heads * group * kHeadDim;
+  int best = 0;
+  for (int i = 0; i < n_alphas; ++i) {
+    h_losses[i] = sums[i] / count;
+    if (h_losses[i] < h_losses[best]) best = i;  // the first one on ties
+  }
+  if (h_best) *h_best = best;
+  return PMKVQ_OK;
+}
+
 pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_t *h_widths, const double *h_sens,
                                  const uint64_t *h_mem, uint64_t budget, uint8_t *h_fbit_out, double *h_cost_out) {
   if (layers <= 0 || n_choices <= 0 || n_choices > 8 || !h_widths || !h_sens || !h_mem || !h_fbit_out)

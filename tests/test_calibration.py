@@ -178,3 +178,34 @@ def test_device_calibration_matches_oracle(n_tokens, n_seq, kv_heads, scale):
     got = B.calibrate_lambda(k.cuda().contiguous(), pos_scale=scale, alpha=0.5).cpu().numpy()
     assert got.shape == want.shape
     assert np.allclose(got, want, rtol=2e-6 * 8, atol=0)      # fp32 rotation: a few ulp on |K_rot|, halved by the root
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("n_tokens,n_seq,kv_heads,group,bits,scale",
+                         [(1, 1, 1, 1, 2, 1.0), (45, 2, 2, 3, 2, 1.0), (130, 1, 2, 7, 4, 4.0), (97, 2, 1, 2, 8, 2.0)])
+def test_device_alpha_grid_matches_oracle(n_tokens, n_seq, kv_heads, group, bits, scale):
+    from paper_2505_18610_b200 import binding as B
+    k, q, v = _calib_tensors(n_tokens, n_seq, kv_heads, group, seed=100 + n_tokens, outlier=(9, 25.0))
+    alphas = O.alpha_grid(8)
+    want = O.attention_reconstruction_losses(k, q, v, group, bits, alphas, pos_scale=scale)
+    dev = [torch.tensor(t).to(torch.bfloat16).cuda().contiguous() for t in (k, q, v)]
+    best, got = B.alpha_grid_search(dev[0], dev[1], dev[2], bits, alphas=alphas, pos_scale=scale)
+    # fp32 attention on both operators: the loss is a squared difference of two fp32 outputs, so its
+    # relative error grows as the quantization error shrinks (2e-2 covers 8 bit)
+    assert np.allclose(got, want, rtol=2e-2 if bits == 8 else 2e-3, atol=0)
+    order = np.sort(want)
+    if len(order) > 1 and order[1] > 1.05 * order[0]:      # a clear winner must be found
+        assert best == pytest.approx(float(alphas[int(np.argmin(want))]))
+
+
+@pytest.mark.gpu
+def test_device_alpha_grid_argument_checks():
+    from paper_2505_18610_b200 import binding as B
+    k, q, v = (torch.zeros(4, 1, 1, 128, dtype=torch.bfloat16, device="cuda") for _ in range(3))
+    with pytest.raises(B.PmkvqError):
+        B.alpha_grid_search(k, q, v, 3)
+    with pytest.raises(B.PmkvqError):
+        B.alpha_grid_search(k, q, v, 2, alphas=np.zeros(65))
+    # constant tensors: every group has S = 0, nothing is lost, every loss is 0
+    best, losses = B.alpha_grid_search(k, q, v, 2)
+    assert best == 0.0 and np.all(losses == 0.0) and len(losses) == 20
