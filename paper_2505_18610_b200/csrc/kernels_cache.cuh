@@ -131,6 +131,25 @@ __device__ __forceinline__ void load_token16(const uint8_t *part, int row, uint1
 // channels of the token; Keys are first multiplied by Lambda^-1 (Eq. 9).  The token goes to the
 // sink, straight to the body (bulk appends; Eq. 3 chain to the body width) or to the window ring.
 // ---------------------------------------------------------------------------------------------
+// RN(d / s), the correctly rounded fp32 quotient, for 0 <= d and a scale in [2^-60, 2^60], from the
+// correctly rounded reciprocal y = RN(1 / s) that a token computes once.  q0 = RN(d y) is within two units
+// in the last place; the residual d - q s is exact in one fused multiply-add (no underflow in this range
+// unless the quotient is below 2^-20, where any result still rounds to code 0), so the first correction
+// gives a faithful quotient and the second, by Markstein's theorem on correcting a faithful quotient with a
+// correctly rounded reciprocal, the correctly rounded one.  5 instructions against the ~15 of a division.
+__device__ __forceinline__ float quotient_rn(float d, float s, float y) {
+  float q = __fmul_rn(d, y);
+  float r = __fmaf_rn(-q, s, d);
+  q = __fmaf_rn(r, y, q);
+  r = __fmaf_rn(-q, s, d);
+  return __fmaf_rn(r, y, q);
+}
+// round-half-to-even of a quotient in [0, 65536) and the clamp to 16 bits: adding 2^23 leaves the rounded
+// integer in the low mantissa bits.
+__device__ __forceinline__ int code_of_quotient(float q) {
+  return min(__float_as_int(__fadd_rn(q, 8388608.0f)) - 0x4B000000, 65535);
+}
+
 // Eq. 1-2 at 16 bit on one token's 128 channels (Keys first times Lambda^-1, Eq. 9), by one warp: lane l
 // holds channels 4l..4l+3.  Writes the codes to `codes` (shared memory) and returns S; Z goes to `zero`.
 __device__ __forceinline__ float quantize_token16(uint2 raw, const float *__restrict__ inv_lambda_head, uint16_t *codes,
@@ -161,14 +180,14 @@ __device__ __forceinline__ float quantize_token16(uint2 raw, const float *__rest
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   }
   const float scale = __fdiv_rn(__fsub_rn(mx, mn), 65535.0f);
+  if (scale >= 0x1p-60f && scale <= 0x1p60f) {  // one scale per token: the branch is uniform in the warp
+    const float y = __frcp_rn(scale);
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    int c = 0;
-    if (scale != 0.0f) {
-      c = __float2int_rn(__fdiv_rn(__fsub_rn(x[e], mn), scale));
-      c = min(max(c, 0), 65535);
-    }
-    codes[lane * 4 + e] = (uint16_t)c;
+    for (int e = 0; e < 4; ++e) codes[lane * 4 + e] = (uint16_t)code_of_quotient(quotient_rn(__fsub_rn(x[e], mn), scale, y));
+  } else {  // constant tokens (0 / 0 converts to code 0) and scales far outside any real tensor's range
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      codes[lane * 4 + e] = (uint16_t)min(max(__float2int_rn(__fdiv_rn(__fsub_rn(x[e], mn), scale)), 0), 65535);
   }
   zero = mn;
   return scale;
@@ -210,57 +229,168 @@ __global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict_
   append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits, i0);
 }
 
-// Bulk appends (prefill): body tiles that consist of new tokens only are built whole.  One warp per
-// (tile, slice, K|V) quantizes the tile's 16 tokens, assembles its code part in shared memory in the
-// tile layout (Eq. 3 chain to the body width included) and writes it out with 128-bit stores; a
-// token-at-a-time store would touch every 32-byte sector of the part for 2 bytes.
+// Bulk appends (prefill): body tiles that consist of new tokens only are built whole, one warp per
+// (tile, slice, K|V).  Every lane loads exactly the elements whose codes the tile layout makes it own
+// (K part: tokens {g, g+8} x channels {8W + 2 tig + h}; V part: tokens {2 tig + 8r + h} x channels
+// {8J + g}), so a token's minimum and maximum meet inside a quad (K) or across the eight lanes of equal
+// tig (V), the codes are packed in registers (Eq. 3 chain to the body width included) and leave as the
+// lane's own 16-byte chunks: coalesced 128-bit stores, no shared memory.  The strided 2- and 4-byte
+// loads of one warp cover whole 4 KB of input; the sectors they share are served by L1.
+
+// Eq. 1-2 at 16 bit on N values of one token that a lane holds, given the token's min and max; the
+// values are replaced by their codes at `BITS` (Eq. 3 chain).  Returns the INT16 scale.
+template <int BITS, int N>
+__device__ __forceinline__ float quantize_owned(float (&x)[N], float mn, float mx, int variant) {
+  const float scale = __fdiv_rn(__fsub_rn(mx, mn), 65535.0f);
+  if (scale >= 0x1p-60f && scale <= 0x1p60f) {  // one scale per token: the branch is uniform in the warp
+    const float y = __frcp_rn(scale);
+#pragma unroll
+    for (int i = 0; i < N; ++i)
+      x[i] = __uint_as_float(shift_chain((uint32_t)code_of_quotient(quotient_rn(__fsub_rn(x[i], mn), scale, y)), BITS, variant));
+  } else {  // constant tokens (0 / 0 converts to code 0) and scales far outside any real tensor's range
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const int c = min(max(__float2int_rn(__fdiv_rn(__fsub_rn(x[i], mn), scale)), 0), 65535);
+      x[i] = __uint_as_float(shift_chain((uint32_t)c, BITS, variant));
+    }
+  }
+  return scale;
+}
+
+// Lane-words of one token pair: word w holds codes idx = w n + j (n = 16 / BITS) of the token (or
+// channel) in half 0 and of its partner in half 1.  lo / hi: the 16 codes (as bit patterns) of the halves,
+// `step` entries apart.
+template <int BITS>
+__device__ __forceinline__ void pack_words(const float *lo, const float *hi, int step, uint32_t *words) {
+  constexpr int n = 16 / BITS;
+#pragma unroll
+  for (int w = 0; w < BITS; ++w) {
+    uint32_t a = 0, b = 0;
+#pragma unroll
+    for (int j = 0; j < n; ++j) {
+      a |= __float_as_uint(lo[(w * n + j) * step]) << (j * BITS);
+      b |= __float_as_uint(hi[(w * n + j) * step]) << (j * BITS);
+    }
+    words[w] = a | (b << 16);
+  }
+}
+
+// The lane's words lw = r BITS .. r BITS + BITS - 1 (lane-word lw sits in chunk lw / 4 at word lw % 4).
+template <int BITS>
+__device__ __forceinline__ void store_words(uint8_t *part, int r, int lane, const uint32_t *words) {
+  if constexpr (BITS >= 4) {
+#pragma unroll
+    for (int q = 0; q < BITS / 4; ++q)
+      *reinterpret_cast<uint4 *>(part + ((r * (BITS / 4) + q) * 32 + lane) * 16) =
+          make_uint4(words[4 * q], words[4 * q + 1], words[4 * q + 2], words[4 * q + 3]);
+  } else {
+    *reinterpret_cast<uint2 *>(part + lane * 16 + r * 8) = make_uint2(words[0], words[1]);
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ src, size_t row_stride,
+                                                 const float *__restrict__ il, uint8_t *dst_tile, int is_value,
+                                                 unsigned *vmax_slot, int lane, int variant) {
+  const int g = lane >> 2, tig = lane & 3;
+  uint32_t words[BITS];
+  if (!is_value) {
+    float lam[32];  // Lambda^-1 of the lane's channels 8 W + 2 tig + h, at [2 W + h]
+#pragma unroll
+    for (int W = 0; W < 16; ++W) {
+      const float2 l2 = *reinterpret_cast<const float2 *>(il + 8 * W + 2 * tig);
+      lam[2 * W] = l2.x;
+      lam[2 * W + 1] = l2.y;
+    }
+#pragma unroll 1
+    for (int r = 0; r < 2; ++r) {  // token g + 8 r
+      float x[32];                 // [2 W + h]
+      const uint16_t *row = src + (size_t)(g + 8 * r) * row_stride + 2 * tig;
+#pragma unroll
+      for (int W = 0; W < 16; ++W) {
+        const uint32_t raw = *reinterpret_cast<const uint32_t *>(row + 8 * W);
+        x[2 * W] = __fmul_rn(__uint_as_float(raw << 16), lam[2 * W]);
+        x[2 * W + 1] = __fmul_rn(__uint_as_float(raw & 0xFFFF0000u), lam[2 * W + 1]);
+      }
+      float mn = x[0], mx = x[0];
+#pragma unroll
+      for (int i = 1; i < 32; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
+#pragma unroll
+      for (int o = 1; o <= 2; o <<= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+      const float s16 = quantize_owned<BITS>(x, mn, mx, variant);
+      pack_words<BITS>(x, x + 1, 2, words);  // halves of a word: channels h = 0, 1 of the token
+      store_words<BITS>(dst_tile, r, lane, words);
+      // metadata record g / 2 holds tokens {2t, 2t+1, 8+2t, 9+2t} at entries {0, 1, 2, 3}
+      if (tig == 0) {
+        float *rec = reinterpret_cast<float *>(dst_tile + meta_offset(BITS) + (g >> 1) * 64) + 2 * r + (g & 1);
+        rec[0] = chain_scale(s16, BITS, variant);
+        rec[4] = chain_zero(mn, s16, BITS, variant);
+      }
+    }
+  } else {
+    float smax = 0.f;
+#pragma unroll 1
+    for (int r = 0; r < 2; ++r) {  // tokens 2 tig + 8 r + h, h = 0, 1
+      float x[2][16];              // [h][J]
+      const uint16_t *row = src + (size_t)(2 * tig + 8 * r) * row_stride + g;
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int J = 0; J < 16; ++J) x[h][J] = __uint_as_float((uint32_t)row[h * row_stride + 8 * J] << 16);
+      float S[2], Z[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float mn = x[h][0], mx = x[h][0];
+#pragma unroll
+        for (int i = 1; i < 16; ++i) { mn = fminf(mn, x[h][i]); mx = fmaxf(mx, x[h][i]); }
+#pragma unroll
+        for (int o = 4; o <= 16; o <<= 1) {
+          mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        }
+        S[h] = quantize_owned<BITS>(x[h], mn, mx, variant);
+        Z[h] = mn;
+        smax = fmaxf(smax, S[h]);
+      }
+      pack_words<BITS>(x[0], x[1], 1, words);  // halves of a word: tokens h = 0, 1 of one channel
+      store_words<BITS>(dst_tile + v_part_offset(BITS), r, lane, words);
+      if (g == 0) {  // record tig: S_V at bytes 32.., Z_V at 48.., entries 2 r + h
+        float *rec = reinterpret_cast<float *>(dst_tile + meta_offset(BITS) + tig * 64 + 32) + 2 * r;
+        *reinterpret_cast<float2 *>(rec) = make_float2(chain_scale(S[0], BITS, variant), chain_scale(S[1], BITS, variant));
+        *reinterpret_cast<float2 *>(rec + 4) =
+            make_float2(chain_zero(Z[0], S[0], BITS, variant), chain_zero(Z[1], S[1], BITS, variant));
+      }
+    }
+    smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, 1));  // the four tig groups hold different tokens
+    smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, 2));
+    if (lane == 0) atomicMax(vmax_slot, __float_as_uint(smax));  // scale >= 0: uint order = float order
+  }
+}
+
 __global__ void __launch_bounds__(128) append_tiles_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
                                                            const float *__restrict__ inv_lambda, unsigned *vmax_bits,
                                                            LayerGeom geom, int n_slices, int kv_heads, int n_old,
                                                            int tile_lo, int n_tiles, int bits) {
-  __shared__ __align__(16) uint8_t s_part[4][256 * 16];
-  __shared__ __align__(16) float s_meta[4][32];  // this part's half of the tile's metadata, in tile order
-  __shared__ uint16_t s_codes[4][kHeadDim];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wid = (long long)blockIdx.x * 4 + warp;
   if (wid >= (long long)n_tiles * n_slices * 2) return;
   const int is_value = (int)(wid & 1);
   const int slice = (int)((wid >> 1) % n_slices);
   const int tile = tile_lo + (int)((wid >> 1) / n_slices);
-  const float *il = is_value ? nullptr : inv_lambda + (size_t)(slice % kv_heads) * kHeadDim;
-  float smax = 0.f;
-  uint2 raw[kTileTokens];  // all 16 tokens in flight at once
-  {
-    const int i0 = geom.n_sink + tile * kTileTokens - n_old;  // index of the tile's first token among the new ones
-    const uint16_t *src = (is_value ? V : K) + ((size_t)i0 * n_slices + slice) * kHeadDim + lane * 4;
-#pragma unroll
-    for (int row = 0; row < kTileTokens; ++row)
-      raw[row] = *reinterpret_cast<const uint2 *>(src + (size_t)row * n_slices * kHeadDim);
-  }
-#pragma unroll
-  for (int row = 0; row < kTileTokens; ++row) {
-    float zero;
-    const float scale = quantize_token16(raw[row], il, s_codes[warp], lane, zero);
-    __syncwarp();
-    store_token(s_part[warp], bits, row, s_codes[warp], is_value, lane, geom.shift_variant);
-    if (lane == 0) {  // meta_slot(kind, row) = tig*64 + kind*16 + i*4; this part keeps kinds {0,1} or {2,3}
-      const int tig = (row & 7) >> 1, idx = (row >> 3) * 2 + (row & 1);
-      s_meta[warp][tig * 8 + idx] = chain_scale(scale, bits, geom.shift_variant);
-      s_meta[warp][tig * 8 + 4 + idx] = chain_zero(zero, scale, bits, geom.shift_variant);
-    }
-    smax = fmaxf(smax, scale);
-    __syncwarp();
-  }
+  const int i0 = geom.n_sink + tile * kTileTokens - n_old;  // index of the tile's first token among the new ones
+  const size_t row_stride = (size_t)n_slices * kHeadDim;
+  const uint16_t *src = (is_value ? V : K) + ((size_t)i0 * n_slices + slice) * kHeadDim;
+  const float *il = inv_lambda + (size_t)(slice % kv_heads) * kHeadDim;
   uint8_t *dst_tile = geom.base + (size_t)slice * geom.slice_stride + geom.body_off + (size_t)tile * tile_bytes(bits);
-  uint4 *dst = reinterpret_cast<uint4 *>(dst_tile + (is_value ? v_part_offset(bits) : 0));
-  const uint4 *srcp = reinterpret_cast<const uint4 *>(s_part[warp]);
-  for (int c = lane; c < 16 * bits; c += 32) dst[c] = srcp[c];
-  if (lane < 8) {  // 4 records x (S[4], Z[4]) -> byte tig*64 + (is_value ? 32 : 0) + {0, 16}
-    const int tig = lane >> 1, half = lane & 1;
-    *reinterpret_cast<uint4 *>(dst_tile + meta_offset(bits) + tig * 64 + (is_value ? 32 : 0) + half * 16) =
-        *reinterpret_cast<const uint4 *>(&s_meta[warp][tig * 8 + half * 4]);
+  switch (bits) {
+    case 16: append_tile_half<16>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
+    case 8: append_tile_half<8>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
+    case 4: append_tile_half<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
+    default: append_tile_half<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
   }
-  if (is_value && lane == 0) atomicMax(vmax_bits + slice, __float_as_uint(smax));
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 
+#include "kernels_cache.cuh"
 #include "layout.cuh"
 
 namespace pmkvq {
@@ -110,13 +111,12 @@ __device__ __forceinline__ void quantize_dequantize_token(float (&x)[4], int bit
   const float s16 = __fdiv_rn(__fsub_rn(mx, mn), 65535.0f);
   float sb = s16;
   for (int w = 8; w >= bits; w >>= 1) sb = __fmul_rn(sb, (float)((1 << w) + 1));
+  const bool plain = s16 >= 0x1p-60f && s16 <= 0x1p60f;  // else: constant token (0 / 0 converts to code 0) or absurd range
+  const float y = plain ? __frcp_rn(s16) : 0.f;
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
-    int c = 0;
-    if (s16 != 0.0f) {
-      c = __float2int_rn(__fdiv_rn(__fsub_rn(x[e], mn), s16));
-      c = min(max(c, 0), 65535);
-    }
+    const float d = __fsub_rn(x[e], mn);
+    const int c = plain ? code_of_quotient(quotient_rn(d, s16, y)) : min(max(__float2int_rn(__fdiv_rn(d, s16)), 0), 65535);
     x[e] = fmaf((float)shift_chain((uint32_t)c, bits), sb, mn);
   }
 }
