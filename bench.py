@@ -180,6 +180,45 @@ def kernel_source_digest():
 NCU_TRAFFIC = {"digest": "187398695b56c60d", "traffic_bytes": 975_617_536, "algorithmic_bytes": 954_646_528}
 
 
+def aux_leg(wl, device):
+    """The two kernels beside the decode step, timed alone with CUDA events (best of 5 calls after a warm-up):
+    the bulk prefill append of 8192 tokens into one block of the workload's shape, and the alpha grid search
+    of the calibration (512 tokens x 2 sequences of the workload's head counts, 20 alphas, 2 bit)."""
+    from paper_2505_18610_b200 import binding as B
+    n = 8192
+    k, v = synth.make_kv(3, 0, 0, n, wl["batch"], wl["kv_heads"], 0, wl["n_outlier"], wl["factor"], device=device)
+    k, v = k.contiguous(), v.contiguous()
+    n_slices = wl["batch"] * wl["kv_heads"]
+    ts = []
+    for _ in range(6):
+        cache = B.Cache(1, wl["q_heads"], wl["kv_heads"], wl["batch"], 32768, [16], n_sink=N_SINK, window=WINDOW, device=device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(); cache.append(0, k, v); e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+        cache.close(); del cache
+    append_bytes = 2 * n * n_slices * (256 + tokbytes(16))
+    out = {"bulk_append": {"tokens": n, "ms": min(ts[1:]), "GBps": append_bytes / (min(ts[1:]) * 1e-3) / 1e9,
+                           "bytes": append_bytes, "what": "bf16 K, V in, INT16 tiles out, one block"}}
+    g = torch.Generator().manual_seed(5)
+    nt, ns, kvh, grp = 512, 2, wl["kv_heads"], wl["q_heads"] // wl["kv_heads"]
+    kk = torch.randn(nt, ns, kvh, 128, generator=g); kk[..., 9] *= 25.0; kk[..., 73] *= 25.0
+    qq = torch.randn(nt, ns, kvh * grp, 128, generator=g)
+    vv = torch.randn(nt, ns, kvh, 128, generator=g)
+    kk, qq, vv = (t.to(torch.bfloat16).to(device).contiguous() for t in (kk, qq, vv))
+    ts = []
+    for _ in range(4):
+        torch.cuda.synchronize(); t0 = time.perf_counter()
+        best, losses = B.alpha_grid_search(kk, qq, vv, 2, pos_scale=4.0)
+        ts.append((time.perf_counter() - t0) * 1e3)
+    flop = 21 * ns * kvh * grp * (nt * (nt + 1) / 2) * 128 * 4
+    out["alpha_grid_search"] = {"tokens": nt, "sequences": ns, "alphas": 20, "bits": 2, "ms": min(ts[1:]), "best_alpha": best,
+                                "fp32_TFLOPs": flop / (min(ts[1:]) * 1e-3) / 1e12,
+                                "what": "host-timed call (it ends with a synchronize); 21 causal attention passes"}
+    return out
+
+
 class ClockSampler:
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -312,6 +351,7 @@ def main():
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS))
     ap.add_argument("--ctas", type=int, default=0, help="attention grid override (0 = library default: one wave)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-aux", action="store_true", help="skip the prefill-append and calibration timings")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-kernel-timing", action="store_true", help="skip the per-launch event leg (profiling runs)")
     args = ap.parse_args()
@@ -481,6 +521,8 @@ def main():
         gbs, dt, desc, cores, nst, _ = cpu_oracle_leg(wl)
         line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc,
                                 "s_per_oracle_step": dt}
+    if not args.no_aux and world == 1:
+        line["aux"] = aux_leg(wl, device)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

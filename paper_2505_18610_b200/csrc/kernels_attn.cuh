@@ -793,10 +793,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
   __shared__ int s_ctr[4];                                    // work counters (INT16 tiles, body steps), combine flag
   __shared__ uint4 s_frag[512];                               // query fragments at INT16 and at the body width
   extern __shared__ __align__(128) uint8_t ring[];
-  // When launched with programmatic stream serialization (pmkvq_decode_step does that for every block
-  // after the first) the next block's kernel may start as soon as SMs free up; it works on its own
-  // tiles, scratch and output, so nothing of this grid has to be finished for it.  No-op otherwise.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const long long u_begin = (long long)blockIdx.x * p.units_per_cta;
   const long long u_end = min(u_begin + p.units_per_cta, p.units_total);
   for (long long u = u_begin; u < u_end;) {
@@ -806,9 +802,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
     if (hi > p.units_lead) run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
     u = base + hi;
   }
-  // A grid never completes before the grid it was allowed to overlap: kernels complete in launch order,
-  // so whatever follows in the stream sees all of them done.  Returns at once for a normal launch.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------------------------

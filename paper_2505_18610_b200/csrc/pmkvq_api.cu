@@ -128,7 +128,7 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.off_lambda = off; off = align_up(off + lam_bytes, kAlign);
   k.off_inv_lambda = off; off = align_up(off + lam_bytes, kAlign);
   k.off_vmax = off; off = align_up(off + (size_t)k.layers * k.n_slices * sizeof(unsigned), kAlign);
-  // tickets and split-K partials exist once per block: attention kernels of consecutive blocks may overlap
+  // tickets and split-K partials exist once per block: one launch computes the attention of all blocks
   k.off_tickets = off; off = align_up(off + (size_t)k.layers * k.n_slices * sizeof(unsigned), kAlign);
   k.partial_bytes = align_up(((size_t)kMaxCtas + (size_t)k.n_slices) * kMaxGroup * kPartialStride * sizeof(float), kAlign);
   k.off_partials = off; off = align_up(off + k.partial_bytes * k.layers, kAlign);
@@ -442,40 +442,28 @@ static pmkvq_status attn_params(pmkvq_cache *k, int32_t layer, const void *d_Q, 
 }
 
 template <int BITS>
-static cudaError_t attn_launch_width(const AttnParams &p, unsigned n_ctas, cudaStream_t st, bool overlap_previous) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n_ctas);
-  cfg.blockDim = dim3(kAttnThreads);
-  cfg.dynamicSmemBytes = attn_ring_bytes<BITS>();
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = overlap_previous ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, decode_attn_splitk_kernel<BITS>, p);
+static cudaError_t attn_launch_width(const AttnParams &p, unsigned n_ctas, cudaStream_t st) {
+  decode_attn_splitk_kernel<BITS><<<n_ctas, kAttnThreads, attn_ring_bytes<BITS>(), st>>>(p);
+  return cudaGetLastError();
 }
 
-// overlap_previous: the kernel may start before the previous kernel of the stream has finished (only
-// for launches whose inputs that kernel does not produce).
-static cudaError_t attn_launch(const AttnParams &p, unsigned n_ctas, cudaStream_t st, bool overlap_previous) {
+static cudaError_t attn_launch(const AttnParams &p, unsigned n_ctas, cudaStream_t st) {
   switch (p.cur_bits) {
-    case 16: return attn_launch_width<16>(p, n_ctas, st, overlap_previous);
-    case 8: return attn_launch_width<8>(p, n_ctas, st, overlap_previous);
-    case 4: return attn_launch_width<4>(p, n_ctas, st, overlap_previous);
-    default: return attn_launch_width<2>(p, n_ctas, st, overlap_previous);
+    case 16: return attn_launch_width<16>(p, n_ctas, st);
+    case 8: return attn_launch_width<8>(p, n_ctas, st);
+    case 4: return attn_launch_width<4>(p, n_ctas, st);
+    default: return attn_launch_width<2>(p, n_ctas, st);
   }
 }
 
-static pmkvq_status attention_on_arena(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, cudaStream_t st,
-                                       bool overlap_previous) {
+static pmkvq_status attention_on_arena(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, cudaStream_t st) {
   AttnParams p;
   unsigned n_ctas = 0;
   const pmkvq_status s = attn_params(k, layer, d_Q, d_out, p, n_ctas);
   if (s != PMKVQ_OK) return s;
   p.partials = reinterpret_cast<float *>(k->arena + k->off_partials + (size_t)layer * k->partial_bytes);
   p.tickets = reinterpret_cast<unsigned *>(k->arena + k->off_tickets) + (size_t)layer * k->n_slices;
-  const cudaError_t e = attn_launch(p, n_ctas, st, overlap_previous);
+  const cudaError_t e = attn_launch(p, n_ctas, st);
   k->launches += 1;
   return e == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }
@@ -528,7 +516,7 @@ static pmkvq_status attention_all_blocks(pmkvq_cache *k, const void *d_Q, float 
 extern "C" {
 
 pmkvq_status pmkvq_decode_attention(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, void *stream) {
-  return attention_on_arena(k, layer, d_Q, d_out, static_cast<cudaStream_t>(stream), false);
+  return attention_on_arena(k, layer, d_Q, d_out, static_cast<cudaStream_t>(stream));
 }
 
 pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *k, int32_t layer, const void *d_Q, float *d_out, void *stream) {
@@ -547,7 +535,7 @@ pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *k, int32_t layer, const 
   p.partials = reinterpret_cast<float *>(scratch + kStaticTicketBytes);
   // the array keeps whatever the previous call left: the tickets must start at zero
   if (cudaMemsetAsync(p.tickets, 0, (size_t)k->n_slices * sizeof(unsigned), st) != cudaSuccess) return PMKVQ_ERR_CUDA;
-  const cudaError_t e = attn_launch(p, n_ctas, st, false);
+  const cudaError_t e = attn_launch(p, n_ctas, st);
   k->launches += 1;
   return e == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }

@@ -167,6 +167,21 @@ def test_degenerate_values():
     m.check_attention(0, q0, max_abs=2e-3 * 50)
 
 
+@pytest.mark.parametrize("bulk", [True, False])
+def test_quantizer_scale_extremes(bulk):
+    """Tokens whose scale lies outside the range of the reciprocal-based quotient (below 2^-60, above 2^60,
+    exactly 0) take the plain-division path; codes, scales and zero-points stay bit-exact."""
+    n, kvh = 100, 2
+    k, v = make_inputs(11, 0, n, 1, kvh)
+    for t, f in ((3, 1e-30), (20, 1e30), (37, 1e-36), (64, 3e25)):
+        k[t] = (k[t].float() * f).to(k.dtype)
+        v[t] = (v[t].float() * f).to(v.dtype)
+    k[50] = 0.25; v[51] = 0.0
+    m = Mirror(1, 2, kvh, 1, n, [4], window=8)
+    m.append(0, k, v, bulk=bulk)
+    m.check_state(0)
+
+
 def test_decode_step_over_all_blocks():
     """pmkvq_decode_step = append + attention for every block; compared with the oracle block by block,
     across a reduce (block 0 crosses its budget during the steps)."""
