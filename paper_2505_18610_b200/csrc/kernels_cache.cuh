@@ -295,13 +295,6 @@ __device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ sr
   const int g = lane >> 2, tig = lane & 3;
   uint32_t words[BITS];
   if (!is_value) {
-    float lam[32];  // Lambda^-1 of the lane's channels 8 W + 2 tig + h, at [2 W + h]
-#pragma unroll
-    for (int W = 0; W < 16; ++W) {
-      const float2 l2 = *reinterpret_cast<const float2 *>(il + 8 * W + 2 * tig);
-      lam[2 * W] = l2.x;
-      lam[2 * W + 1] = l2.y;
-    }
 #pragma unroll 1
     for (int r = 0; r < 2; ++r) {  // token g + 8 r
       float x[32];                 // [2 W + h]
@@ -309,8 +302,9 @@ __device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ sr
 #pragma unroll
       for (int W = 0; W < 16; ++W) {
         const uint32_t raw = *reinterpret_cast<const uint32_t *>(row + 8 * W);
-        x[2 * W] = __fmul_rn(__uint_as_float(raw << 16), lam[2 * W]);
-        x[2 * W + 1] = __fmul_rn(__uint_as_float(raw & 0xFFFF0000u), lam[2 * W + 1]);
+        const float2 l2 = __ldg(reinterpret_cast<const float2 *>(il + 8 * W + 2 * tig));  // Lambda^-1, L1-resident
+        x[2 * W] = __fmul_rn(__uint_as_float(raw << 16), l2.x);
+        x[2 * W + 1] = __fmul_rn(__uint_as_float(raw & 0xFFFF0000u), l2.y);
       }
       float mn = x[0], mx = x[0];
 #pragma unroll
@@ -370,7 +364,7 @@ __device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ sr
   }
 }
 
-__global__ void __launch_bounds__(128) append_tiles_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
+__global__ void __launch_bounds__(128, 8) append_tiles_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
                                                            const float *__restrict__ inv_lambda, unsigned *vmax_bits,
                                                            LayerGeom geom, int n_slices, int kv_heads, int n_old,
                                                            int tile_lo, int n_tiles, int bits) {

@@ -80,9 +80,10 @@ __global__ void rope_table_kernel(float2 *table, int n_tokens, double pos_scale,
   table[i] = make_float2((float)c, (float)s);
 }
 
-constexpr int kGridQueries = 32;  // queries of one CTA (4 threads each)
+constexpr int kGridQueries = 64;  // queries of one CTA: 16 groups of 4 queries, 8 threads per group
 constexpr int kGridKeys = 32;     // keys per shared-memory tile
 constexpr int kMaxAlphas = 64;
+constexpr int kGridSmemBytes = (2 * kGridKeys + kGridQueries) * kHeadDim * 4;  // K tile, V tile, kept outputs
 
 // One token's 4 channels per lane (channels 4 lane .. 4 lane + 3): rotate by the token's angles.  The
 // partner channel (+-64) sits in lane ^ 16.
@@ -132,49 +133,31 @@ __device__ __forceinline__ void load_bf16x4(const uint16_t *src, float (&x)[4]) 
 // Grid: (query blocks, query heads, sequences).  K, V: bf16 [n_tokens][n_seq][kv_heads][128];
 // Q: bf16 [n_tokens][n_seq][kv_heads * group][128]; amax [kv_heads][128] from calib_absmax_kernel;
 // loss_sums [n_alphas] (fp64, zero before the launch) receives the summed squared errors.
-// Thread (query, part j) owns channels 16 c + 4 j + e (c < 8, e < 4), so that a rotation pair stays in
-// one thread and the four parts of a query read one 64-byte run of a key row.
+// Thread (group, part) works on the group's 4 consecutive queries and on channels 32 c + 4 part + e
+// (c < 4, e < 4): a rotation pair (i, i + 64) stays in one thread, the 8 parts read one 128-byte run of a
+// key row, and every value read from shared memory feeds 4 multiply-adds (one per query), which is what
+// keeps the kernel on the FMA pipe instead of the shared-memory port.
 __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ Q,
                                                          const uint16_t *__restrict__ V, const float *__restrict__ amax,
                                                          const float2 *__restrict__ table, const float *__restrict__ alphas,
                                                          int n_alphas, int n_tokens, int n_seq, int kv_heads, int group,
                                                          int bits, float floor_value, double *loss_sums) {
-  __shared__ __align__(16) float s_k[kGridKeys][kHeadDim];
-  __shared__ __align__(16) float s_v[kGridKeys][kHeadDim];
+  extern __shared__ __align__(16) float s_dyn[];
+  float(*s_k)[kHeadDim] = reinterpret_cast<float(*)[kHeadDim]>(s_dyn);
+  float(*s_v)[kHeadDim] = reinterpret_cast<float(*)[kHeadDim]>(s_dyn + kGridKeys * kHeadDim);
+  float(*s_ref)[kHeadDim] = reinterpret_cast<float(*)[kHeadDim]>(s_dyn + 2 * kGridKeys * kHeadDim);
   __shared__ float s_lam[kHeadDim], s_inv[kHeadDim];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;  // long rows first
   const int q_head = blockIdx.y, seq = blockIdx.z, kv_head = q_head / group, q_heads = kv_heads * group;
-  const int qi = qb * kGridQueries + (tid >> 2), part = tid & 3;
-  const bool q_live = qi < n_tokens;
+  const int ql0 = (tid >> 3) * 4, part = tid & 7;  // first of the thread's 4 queries inside the CTA
+  const int q0 = qb * kGridQueries + ql0;
   const int q_last = min(n_tokens, (qb + 1) * kGridQueries) - 1;  // last live query of the CTA
   const size_t kv_row = (size_t)n_seq * kv_heads * kHeadDim;
   const uint16_t *k_base = K + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
   const uint16_t *v_base = V + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
   const float scale_log2 = 1.4426950408889634f * rsqrtf((float)kHeadDim);
 
-  // this thread's rotated query channels, in the order (c, e)
-  float q_rot[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) q_rot[i] = 0.f;
-  if (q_live) {
-    const uint16_t *src = Q + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim;
-    const float2 *tab = table + (size_t)qi * 64;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float x1[4], x2[4];
-      load_bf16x4(src + 16 * c + 4 * part, x1);
-      load_bf16x4(src + 64 + 16 * c + 4 * part, x2);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 cs = tab[16 * c + 4 * part + e];
-        q_rot[4 * c + e] = __fsub_rn(__fmul_rn(x1[e], cs.x), __fmul_rn(x2[e], cs.y));
-        q_rot[4 * (c + 4) + e] = __fadd_rn(__fmul_rn(x1[e], cs.y), __fmul_rn(x2[e], cs.x));
-      }
-    }
-  }
-
-  float ref[32];
   for (int pass = 0; pass <= n_alphas; ++pass) {
     __syncthreads();  // the previous pass is done with s_lam / s_inv and the tiles
     if (pass > 0) {
@@ -183,19 +166,38 @@ __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restr
       s_inv[tid] = __fdiv_rn(1.0f, lam);
     }
     __syncthreads();
-    float qe[32], acc[32];
+    // the thread's rotated, equalized, pre-scaled query channels: qe[n][4 c + e]
+    float qe[4][16], acc[4][16], m[4], l[4];
 #pragma unroll
-    for (int c = 0; c < 8; ++c)
+    for (int n = 0; n < 4; ++n) {
+      m[n] = -INFINITY;
+      l[n] = 0.f;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float lam = pass > 0 ? s_lam[16 * c + 4 * part + e] : 1.0f;
-        qe[4 * c + e] = q_rot[4 * c + e] * lam * scale_log2;
-        acc[4 * c + e] = 0.f;
+      for (int i = 0; i < 16; ++i) { qe[n][i] = 0.f; acc[n][i] = 0.f; }
+      const int qi = q0 + n;
+      if (qi < n_tokens) {
+        const uint16_t *src = Q + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim;
+        const float2 *tab = table + (size_t)qi * 64;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          float x1[4], x2[4];
+          load_bf16x4(src + 32 * c + 4 * part, x1);
+          load_bf16x4(src + 64 + 32 * c + 4 * part, x2);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int ch = 32 * c + 4 * part + e;
+            const float2 cs = tab[ch];
+            const float y1 = __fsub_rn(__fmul_rn(x1[e], cs.x), __fmul_rn(x2[e], cs.y));
+            const float y2 = __fadd_rn(__fmul_rn(x1[e], cs.y), __fmul_rn(x2[e], cs.x));
+            qe[n][4 * c + e] = y1 * (pass > 0 ? s_lam[ch] : 1.0f) * scale_log2;
+            qe[n][4 * (c + 2) + e] = y2 * (pass > 0 ? s_lam[ch + 64] : 1.0f) * scale_log2;
+          }
+        }
       }
-    float m = -INFINITY, l = 0.f;
+    }
     for (int k0 = 0; k0 <= q_last; k0 += kGridKeys) {
       __syncthreads();  // everyone is done with the previous tile
-      // ---- stage the tile: warp w takes keys 8 w .. 8 w + 7 ----
+      // ---- stage the tile: warp w takes keys 8 w .. 8 w + 7, lane l channels 4 l .. 4 l + 3 ----
       for (int r = 0; r < 8; ++r) {
         const int kk = warp * 8 + r, t = k0 + kk;
         float xk[4] = {0.f, 0.f, 0.f, 0.f}, xv[4] = {0.f, 0.f, 0.f, 0.f};
@@ -218,47 +220,69 @@ __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restr
       // ---- scores, online softmax, output ----
       const int k_hi = min(kGridKeys, q_last - k0 + 1);
       for (int kk = 0; kk < k_hi; ++kk) {
-        float s = 0.f;
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const float4 kv = *reinterpret_cast<const float4 *>(&s_k[kk][16 * c + 4 * part]);
-          s = fmaf(qe[4 * c], kv.x, s); s = fmaf(qe[4 * c + 1], kv.y, s);
-          s = fmaf(qe[4 * c + 2], kv.z, s); s = fmaf(qe[4 * c + 3], kv.w, s);
-        }
-        s += __shfl_xor_sync(0xffffffffu, s, 1);
-        s += __shfl_xor_sync(0xffffffffu, s, 2);
-        if (k0 + kk <= qi) {  // causal; the four threads of a query agree
-          if (s > m) {
-            const float corr = exp2f(m - s);  // 0 on the first key
-            l *= corr;
+        for (int c = 0; c < 4; ++c) {
+          const float4 kv = *reinterpret_cast<const float4 *>(&s_k[kk][32 * c + 4 * part]);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] *= corr;
-            m = s;
+          for (int n = 0; n < 4; ++n) {
+            s[n] = fmaf(qe[n][4 * c], kv.x, s[n]); s[n] = fmaf(qe[n][4 * c + 1], kv.y, s[n]);
+            s[n] = fmaf(qe[n][4 * c + 2], kv.z, s[n]); s[n] = fmaf(qe[n][4 * c + 3], kv.w, s[n]);
           }
-          const float p = exp2f(s - m);
-          l += p;
+        }
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const float4 vv = *reinterpret_cast<const float4 *>(&s_v[kk][16 * c + 4 * part]);
-            acc[4 * c] = fmaf(p, vv.x, acc[4 * c]); acc[4 * c + 1] = fmaf(p, vv.y, acc[4 * c + 1]);
-            acc[4 * c + 2] = fmaf(p, vv.z, acc[4 * c + 2]); acc[4 * c + 3] = fmaf(p, vv.w, acc[4 * c + 3]);
+        for (int n = 0; n < 4; ++n) {
+          s[n] += __shfl_xor_sync(0xffffffffu, s[n], 1);
+          s[n] += __shfl_xor_sync(0xffffffffu, s[n], 2);
+          s[n] += __shfl_xor_sync(0xffffffffu, s[n], 4);
+        }
+        float p[4];
+#pragma unroll
+        for (int n = 0; n < 4; ++n) {
+          p[n] = 0.f;
+          if (k0 + kk <= q0 + n) {  // causal; the eight threads of a group agree
+            if (s[n] > m[n]) {
+              const float corr = exp2f(m[n] - s[n]);  // 0 on the first key
+              l[n] *= corr;
+#pragma unroll
+              for (int i = 0; i < 16; ++i) acc[n][i] *= corr;
+              m[n] = s[n];
+            }
+            p[n] = exp2f(s[n] - m[n]);
+            l[n] += p[n];
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const float4 vv = *reinterpret_cast<const float4 *>(&s_v[kk][32 * c + 4 * part]);
+#pragma unroll
+          for (int n = 0; n < 4; ++n) {
+            acc[n][4 * c] = fmaf(p[n], vv.x, acc[n][4 * c]); acc[n][4 * c + 1] = fmaf(p[n], vv.y, acc[n][4 * c + 1]);
+            acc[n][4 * c + 2] = fmaf(p[n], vv.z, acc[n][4 * c + 2]); acc[n][4 * c + 3] = fmaf(p[n], vv.w, acc[n][4 * c + 3]);
           }
         }
       }
     }
-    // ---- the pass's output: keep it (pass 0) or compare with the kept one ----
+    // ---- the pass's output: keep it (pass 0) or compare with the kept one (only this thread touches
+    // its entries of s_ref, so no barrier is needed around them) ----
     float err = 0.f;
-    if (q_live) {
-      const float inv_l = __fdiv_rn(1.0f, l);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float o = acc[i] * inv_l;
-        if (pass == 0) {
-          ref[i] = o;
-        } else {
-          const float d = o - ref[i];
-          err = fmaf(d, d, err);
-        }
+    for (int n = 0; n < 4; ++n) {
+      if (q0 + n < n_tokens) {
+        const float inv_l = __fdiv_rn(1.0f, l[n]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float o = acc[n][4 * c + e] * inv_l;
+            float &kept = s_ref[ql0 + n][32 * c + 4 * part + e];
+            if (pass == 0) {
+              kept = o;
+            } else {
+              const float d = o - kept;
+              err = fmaf(d, d, err);
+            }
+          }
       }
     }
     if (pass > 0) {

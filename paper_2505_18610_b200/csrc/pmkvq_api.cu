@@ -722,7 +722,9 @@ pmkvq_status pmkvq_alpha_grid_search(const void *d_K, const void *d_Q, const voi
       tokens_per_cta, pos_scale, theta);
   rope_table_kernel<<<(unsigned)((n_tokens * 64 + 255) / 256), 256, 0, st>>>(d_table, n_tokens, pos_scale, theta);
   const dim3 grid((unsigned)((n_tokens + kGridQueries - 1) / kGridQueries), (unsigned)(kv_heads * group), (unsigned)n_seq);
-  alpha_grid_kernel<<<grid, 128, 0, st>>>(static_cast<const uint16_t *>(d_K), static_cast<const uint16_t *>(d_Q),
+  if (cudaFuncSetAttribute(alpha_grid_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGridSmemBytes) != cudaSuccess)
+    return PMKVQ_ERR_CUDA;
+  alpha_grid_kernel<<<grid, 128, kGridSmemBytes, st>>>(static_cast<const uint16_t *>(d_K), static_cast<const uint16_t *>(d_Q),
                                           static_cast<const uint16_t *>(d_V), d_amax, d_table, d_alphas, n_alphas, n_tokens,
                                           n_seq, kv_heads, group, bits, floor_value, d_loss);
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;

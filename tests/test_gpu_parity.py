@@ -215,6 +215,37 @@ def test_decode_step_over_all_blocks():
         assert m.cache.layer_state(l)["cur_bits"] == fbit[l]
 
 
+@pytest.mark.parametrize("layers", [128, 130])
+def test_decode_step_with_many_blocks(layers):
+    """128 blocks fill the argument tables of the one-launch step exactly; 130 take the block-by-block route."""
+    kvh, batch, group, n0, steps = 1, 1, 2, 40, 3
+    fbit = [(2, 4, 8, 16)[l % 4] for l in range(layers)]
+    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, fbit, window=8)
+    for l in range(layers):
+        k, v = make_inputs(21, l, n0, batch, kvh)
+        m.append(l, k, v)
+    for s in range(steps):
+        ks, vs, qs = [], [], []
+        for l in range(layers):
+            k, v = make_inputs(22, l, 1, batch, kvh, pos0=n0 + s, chunk=s)
+            ks.append(k[0]); vs.append(v[0])
+            qs.append(synth.make_q(22, l, s, batch, group * kvh, n0 + s + 1))
+        K, V, Q = torch.stack(ks).cuda(), torch.stack(vs).cuda(), torch.stack(qs).cuda()
+        out = m.cache.decode_step(K, V, Q)
+        torch.cuda.synchronize()
+        for l in range(layers):
+            m.oracles[l].append(K[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices],
+                                V[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices])
+            if s == steps - 1 and l in (0, 1, 2, 3, 63, layers - 2, layers - 1):
+                qq = Q[l].float().cpu().numpy().reshape(batch * kvh, group, 128)[m.slices]
+                ref = m.oracles[l].decode_attention(qq)
+                got = out[l].cpu().numpy().reshape(batch * kvh, group, 128)[m.slices].astype(np.float64)
+                assert np.abs(got - ref).max() <= 2e-3
+                assert np.linalg.norm(got - ref) <= 1e-3 * np.linalg.norm(ref)
+    for l in (0, 5, 127, layers - 1):
+        m.check_state(l)
+
+
 @pytest.mark.parametrize("variant", [1, 2])
 def test_shift_variants_direct_and_modified(variant):
     """The two ablation strategies of Sec. 4.4.1 as cache options: bulk appends, evictions through the
