@@ -512,12 +512,16 @@ __device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1) {
   return out;
 }
 
-template <int B, bool SHR>
-__device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, int lane, int variant) {
+// CTA_WIDE: the warps of a CTA work on consecutive tiles at once; a CTA-wide barrier (reached by every
+// warp, `active` or not) separates all their loads from all their stores.
+template <int B, bool SHR, bool CTA_WIDE>
+__device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, int lane, int variant, bool active) {
   constexpr int IN_CHUNKS = B;                          // 16-byte chunks per lane per part at 2B bits
   constexpr int OUT_WORDS = 2 * B;                      // words per lane per part at B bits
   constexpr int OUT_CHUNKS = (OUT_WORDS + 3) / 4;
   uint32_t o[2][OUT_CHUNKS * 4];
+  float2 m = make_float2(0.f, 0.f);
+  if (active) {
 #pragma unroll
   for (int part = 0; part < 2; ++part) {
     const uint8_t *src = in + part * code_part_bytes(2 * B);
@@ -534,7 +538,7 @@ __device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, i
       o[part][lw] = merge_words<B, SHR>(w[r * 2 * B + 2 * wp], w[r * 2 * B + 2 * wp + 1]);
     }
   }
-  float2 m = *reinterpret_cast<const float2 *>(in + meta_offset(2 * B) + lane * 8);
+  m = *reinterpret_cast<const float2 *>(in + meta_offset(2 * B) + lane * 8);
   const int kind = ((2 * lane) & 15) >> 2;  // 0 S_K, 1 Z_K, 2 S_V, 3 Z_V
   // a zero-point lane finds the scales of its two tokens two lanes below (16 bytes earlier)
   const float s_x = __shfl_up_sync(0xffffffffu, m.x, 2), s_y = __shfl_up_sync(0xffffffffu, m.y, 2);
@@ -547,7 +551,11 @@ __device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, i
     halve_meta(sx, m.x, B, variant);
     halve_meta(sy, m.y, B, variant);
   }
-  __syncwarp();  // every lane holds its transformed data: the tile's input is dead from here on
+  }
+  // every lane (every warp of the CTA) holds its transformed data: the input is dead from here on
+  if constexpr (CTA_WIDE) __syncthreads();
+  else __syncwarp();
+  if (!active) return;
 #pragma unroll
   for (int part = 0; part < 2; ++part) {
     uint8_t *dst = out + part * code_part_bytes(B);
@@ -560,20 +568,25 @@ __device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, i
   *reinterpret_cast<float2 *>(out + meta_offset(B) + lane * 8) = m;
 }
 
-template <int B>
-__device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int lane, int variant) {
-  if (variant == kShiftEquivalent) reduce_tile_v<B, false>(in, out, lane, variant);
-  else reduce_tile_v<B, true>(in, out, lane, variant);
+template <int B, bool CTA_WIDE = false>
+__device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int lane, int variant, bool active = true) {
+  if (variant == kShiftEquivalent) reduce_tile_v<B, false, CTA_WIDE>(in, out, lane, variant, active);
+  else reduce_tile_v<B, true, CTA_WIDE>(in, out, lane, variant, active);
 }
 
-// First tiles of every slice, one warp per slice, in order (tile i's output overlaps inputs <= i only).
+// First tiles of every slice, one CTA per slice, in batches of one tile per warp, batch after batch: the
+// outputs of batch j (tiles [W j, W j + W) at B bits) end at (W j + W) tile_bytes(B), below the first input
+// of batch j + 1, and overlap inputs of batches <= j only, which the barrier inside reduce_tile has seen
+// loaded.
+constexpr int kReduceHeadWarps = 16;
 template <int B>
-__global__ void __launch_bounds__(32) reduce_head_kernel(LayerGeom geom, int n_tiles) {
+__global__ void __launch_bounds__(kReduceHeadWarps * 32) reduce_head_kernel(LayerGeom geom, int n_tiles) {
   uint8_t *body = geom.base + (size_t)blockIdx.x * geom.slice_stride + geom.body_off;
-  const int lane = threadIdx.x;
-  for (int i = 0; i < n_tiles; ++i) {
-    reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), lane, geom.shift_variant);
-    __syncwarp();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int i0 = 0; i0 < n_tiles; i0 += kReduceHeadWarps) {
+    const int i = i0 + warp;
+    reduce_tile<B, true>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), lane, geom.shift_variant,
+                         i < n_tiles);
   }
 }
 

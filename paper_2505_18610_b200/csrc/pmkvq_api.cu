@@ -21,7 +21,7 @@ using namespace pmkvq;
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr int kHeadTiles = 8;     // tiles the reduce handles in order before the parallel waves start
+constexpr int kHeadTiles = 256;   // tiles the reduce handles batch by batch (one CTA per slice) before the parallel waves start
 constexpr int kMaxCtas = 1024;      // upper bound on the attention grid (sizes the partials workspace)
 // Fixed cost of one more segment (set-up, warp merge, publish, its share of the slice combine), in
 // body tiles of each width: about 12 us at the measured per-SM tile rates.
@@ -163,8 +163,8 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
 
 template <int B>
 cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStream_t st, uint64_t &launches) {
-  const int head = std::min(n_tiles, kHeadTiles);
-  if (head > 0) { reduce_head_kernel<B><<<n_slices, 32, 0, st>>>(g, head); ++launches; }
+  const int head = std::min(n_tiles, B == 8 ? kHeadTiles / 2 : kHeadTiles);  // the 16-bit tiles are twice as large
+  if (head > 0) { reduce_head_kernel<B><<<n_slices, kReduceHeadWarps * 32, 0, st>>>(g, head); ++launches; }
   int lo = head;
   while (lo < n_tiles) {
     // outputs of tiles [lo, hi) end at hi * tile_bytes(B); inputs start at lo * tile_bytes(2B)

@@ -134,6 +134,23 @@ def test_manual_reduce_and_error_codes():
         B.Cache(1, 18, 2, 1, 64, [4])          # GQA group of 9 is outside 1..8
 
 
+def test_reduce_head_batches_and_waves():
+    """Bodies of 378, 733 and 1385 tiles cross 16 -> 8 -> 4 -> 2: the in-place reduce runs its CTA-wide head
+    batches (256 tiles) and one, two and three parallel waves behind them."""
+    kvh, n_max = 2, 40000
+    m = Mirror(1, 2 * kvh, kvh, 1, n_max, [2])
+    done, widths = 0, []
+    for upto in (6170, 6200, 11855, 11900, 22279, 22400):
+        k, v = make_inputs(31, 0, upto - done, 1, kvh, pos0=done, chunk=upto)
+        m.append(0, k, v)
+        done = upto
+        widths.append(m.cache.layer_state(0)["cur_bits"])
+        if upto in (6200, 11900, 22400):
+            m.check_state(0)
+    assert widths == [16, 8, 8, 4, 4, 2]
+    m.check_attention(0, synth.make_q(31, 0, 0, 1, 2 * kvh, done))
+
+
 def test_split_invariance():
     kvh, batch, n, group = 2, 2, 5000, 8
     k, v = make_inputs(6, 0, n, batch, kvh)
