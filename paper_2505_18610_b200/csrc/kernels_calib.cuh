@@ -80,9 +80,15 @@ __global__ void rope_table_kernel(float2 *table, int n_tokens, double pos_scale,
   table[i] = make_float2((float)c, (float)s);
 }
 
-constexpr int kGridQueries = 64;  // queries of one CTA: 16 groups of 4 queries, 8 threads per group
+constexpr int kQPT = 2;                     // queries per thread
+constexpr int kGridQueries = 16 * kQPT;     // queries of one CTA: 16 groups of kQPT queries, 8 threads per group
 constexpr int kGridKeys = 32;     // keys per shared-memory tile
 constexpr int kMaxAlphas = 64;
+__device__ __forceinline__ float ex2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 constexpr int kGridSmemBytes = (2 * kGridKeys + kGridQueries) * kHeadDim * 4;  // K tile, V tile, kept outputs
 
 // One token's 4 channels per lane (channels 4 lane .. 4 lane + 3): rotate by the token's angles.  The
@@ -133,10 +139,10 @@ __device__ __forceinline__ void load_bf16x4(const uint16_t *src, float (&x)[4]) 
 // Grid: (query blocks, query heads, sequences).  K, V: bf16 [n_tokens][n_seq][kv_heads][128];
 // Q: bf16 [n_tokens][n_seq][kv_heads * group][128]; amax [kv_heads][128] from calib_absmax_kernel;
 // loss_sums [n_alphas] (fp64, zero before the launch) receives the summed squared errors.
-// Thread (group, part) works on the group's 4 consecutive queries and on channels 32 c + 4 part + e
+// Thread (group, part) works on the group's kQPT consecutive queries and on channels 32 c + 4 part + e
 // (c < 4, e < 4): a rotation pair (i, i + 64) stays in one thread, the 8 parts read one 128-byte run of a
-// key row, and every value read from shared memory feeds 4 multiply-adds (one per query), which is what
-// keeps the kernel on the FMA pipe instead of the shared-memory port.
+// key row, every value read from shared memory feeds kQPT multiply-adds (one per query), and two keys are
+// taken per turn so that their score chains, shuffles and exponentials overlap.
 __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ Q,
                                                          const uint16_t *__restrict__ V, const float *__restrict__ amax,
                                                          const float2 *__restrict__ table, const float *__restrict__ alphas,
@@ -150,7 +156,7 @@ __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restr
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;  // long rows first
   const int q_head = blockIdx.y, seq = blockIdx.z, kv_head = q_head / group, q_heads = kv_heads * group;
-  const int ql0 = (tid >> 3) * 4, part = tid & 7;  // first of the thread's 4 queries inside the CTA
+  const int ql0 = (tid >> 3) * kQPT, part = tid & 7;  // first of the thread's queries inside the CTA
   const int q0 = qb * kGridQueries + ql0;
   const int q_last = min(n_tokens, (qb + 1) * kGridQueries) - 1;  // last live query of the CTA
   const size_t kv_row = (size_t)n_seq * kv_heads * kHeadDim;
@@ -167,9 +173,9 @@ __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restr
     }
     __syncthreads();
     // the thread's rotated, equalized, pre-scaled query channels: qe[n][4 c + e]
-    float qe[4][16], acc[4][16], m[4], l[4];
+    float qe[kQPT][16], acc[kQPT][16], m[kQPT], l[kQPT];
 #pragma unroll
-    for (int n = 0; n < 4; ++n) {
+    for (int n = 0; n < kQPT; ++n) {
       m[n] = -INFINITY;
       l[n] = 0.f;
 #pragma unroll
@@ -219,46 +225,59 @@ __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restr
       __syncthreads();
       // ---- scores, online softmax, output ----
       const int k_hi = min(kGridKeys, q_last - k0 + 1);
-      for (int kk = 0; kk < k_hi; ++kk) {
-        float s[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int kk = 0; kk < k_hi; kk += 2) {  // two keys per turn: their dependent chains overlap
+        // (a second key beyond k_hi lies behind every query of the CTA and is masked below; its row exists)
+        float s[2][kQPT];
+#pragma unroll
+        for (int n = 0; n < kQPT; ++n) s[0][n] = s[1][n] = 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const float4 kv = *reinterpret_cast<const float4 *>(&s_k[kk][32 * c + 4 * part]);
+          const float4 ka = *reinterpret_cast<const float4 *>(&s_k[kk][32 * c + 4 * part]);
+          const float4 kb = *reinterpret_cast<const float4 *>(&s_k[kk + 1][32 * c + 4 * part]);
 #pragma unroll
-          for (int n = 0; n < 4; ++n) {
-            s[n] = fmaf(qe[n][4 * c], kv.x, s[n]); s[n] = fmaf(qe[n][4 * c + 1], kv.y, s[n]);
-            s[n] = fmaf(qe[n][4 * c + 2], kv.z, s[n]); s[n] = fmaf(qe[n][4 * c + 3], kv.w, s[n]);
+          for (int n = 0; n < kQPT; ++n) {
+            s[0][n] = fmaf(qe[n][4 * c], ka.x, s[0][n]); s[1][n] = fmaf(qe[n][4 * c], kb.x, s[1][n]);
+            s[0][n] = fmaf(qe[n][4 * c + 1], ka.y, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 1], kb.y, s[1][n]);
+            s[0][n] = fmaf(qe[n][4 * c + 2], ka.z, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 2], kb.z, s[1][n]);
+            s[0][n] = fmaf(qe[n][4 * c + 3], ka.w, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 3], kb.w, s[1][n]);
           }
         }
 #pragma unroll
-        for (int n = 0; n < 4; ++n) {
-          s[n] += __shfl_xor_sync(0xffffffffu, s[n], 1);
-          s[n] += __shfl_xor_sync(0xffffffffu, s[n], 2);
-          s[n] += __shfl_xor_sync(0xffffffffu, s[n], 4);
-        }
-        float p[4];
+        for (int o = 1; o <= 4; o <<= 1)
 #pragma unroll
-        for (int n = 0; n < 4; ++n) {
-          p[n] = 0.f;
-          if (k0 + kk <= q0 + n) {  // causal; the eight threads of a group agree
-            if (s[n] > m[n]) {
-              const float corr = exp2f(m[n] - s[n]);  // 0 on the first key
-              l[n] *= corr;
-#pragma unroll
-              for (int i = 0; i < 16; ++i) acc[n][i] *= corr;
-              m[n] = s[n];
-            }
-            p[n] = exp2f(s[n] - m[n]);
-            l[n] += p[n];
+          for (int n = 0; n < kQPT; ++n) {
+            s[0][n] += __shfl_xor_sync(0xffffffffu, s[0][n], o);
+            s[1][n] += __shfl_xor_sync(0xffffffffu, s[1][n], o);
           }
+        float p[2][kQPT];
+#pragma unroll
+        for (int n = 0; n < kQPT; ++n) {
+          // causal mask (the eight threads of a group agree); key 0 is live for every query, so m is finite
+          // from the first turn on
+          const float sa = (k0 + kk <= q0 + n) ? s[0][n] : -INFINITY;
+          const float sb = (k0 + kk + 1 <= q0 + n) ? s[1][n] : -INFINITY;
+          const float mx = fmaxf(sa, sb);
+          if (mx > m[n]) {
+            const float corr = ex2_fast(m[n] - mx);  // 0 on the first key
+            l[n] *= corr;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[n][i] *= corr;
+            m[n] = mx;
+          }
+          p[0][n] = ex2_fast(sa - m[n]);
+          p[1][n] = ex2_fast(sb - m[n]);
+          l[n] += p[0][n] + p[1][n];
         }
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          const float4 vv = *reinterpret_cast<const float4 *>(&s_v[kk][32 * c + 4 * part]);
+          const float4 va = *reinterpret_cast<const float4 *>(&s_v[kk][32 * c + 4 * part]);
+          const float4 vb = *reinterpret_cast<const float4 *>(&s_v[kk + 1][32 * c + 4 * part]);
 #pragma unroll
-          for (int n = 0; n < 4; ++n) {
-            acc[n][4 * c] = fmaf(p[n], vv.x, acc[n][4 * c]); acc[n][4 * c + 1] = fmaf(p[n], vv.y, acc[n][4 * c + 1]);
-            acc[n][4 * c + 2] = fmaf(p[n], vv.z, acc[n][4 * c + 2]); acc[n][4 * c + 3] = fmaf(p[n], vv.w, acc[n][4 * c + 3]);
+          for (int n = 0; n < kQPT; ++n) {
+            acc[n][4 * c] = fmaf(p[1][n], vb.x, fmaf(p[0][n], va.x, acc[n][4 * c]));
+            acc[n][4 * c + 1] = fmaf(p[1][n], vb.y, fmaf(p[0][n], va.y, acc[n][4 * c + 1]));
+            acc[n][4 * c + 2] = fmaf(p[1][n], vb.z, fmaf(p[0][n], va.z, acc[n][4 * c + 2]));
+            acc[n][4 * c + 3] = fmaf(p[1][n], vb.w, fmaf(p[0][n], va.w, acc[n][4 * c + 3]));
           }
         }
       }
@@ -267,7 +286,7 @@ __global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restr
     // its entries of s_ref, so no barrier is needed around them) ----
     float err = 0.f;
 #pragma unroll
-    for (int n = 0; n < 4; ++n) {
+    for (int n = 0; n < kQPT; ++n) {
       if (q0 + n < n_tokens) {
         const float inv_l = __fdiv_rn(1.0f, l[n]);
 #pragma unroll
