@@ -32,6 +32,29 @@ def test_binding_mirrors_the_header():
         assert getattr(lib, n).argtypes is not None, f"binding does not marshal {n}"
 
 
+def test_binding_argument_counts_match_the_prototypes():
+    """Every prototype of pmkvq.h has as many parameters as the binding marshals (a drifted signature would
+    otherwise pass garbage in the trailing registers)."""
+    from paper_2505_18610_b200 import binding
+    lib = binding.lib()
+    with open(os.path.join(ROOT, "include", "pmkvq.h")) as f:
+        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    protos = re.findall(r"\b(pmkvq_[a-z0-9_]+)\s*\(([^()]*)\)\s*;", text)
+    assert len(protos) >= 18
+    for name, params in protos:
+        params = params.strip()
+        n = 0 if params in ("", "void") else params.count(",") + 1
+        assert len(getattr(lib, name).argtypes) == n, f"{name}: header has {n} parameters"
+    # alpha grid search: host-side argument errors are answered before anything touches a device
+    a = (ctypes.c_float * 2)(0.0, 0.5)
+    out = (ctypes.c_double * 2)()
+    one = ctypes.c_void_p(256)
+    assert lib.pmkvq_alpha_grid_search(one, one, one, 4, 1, 1, 1, 3, a, 2, 1.0, 10000.0, 1e-5, one, out, None, None) == binding.INVALID_ARG
+    assert lib.pmkvq_alpha_grid_search(one, one, one, 4, 1, 1, 1, 2, a, 65, 1.0, 10000.0, 1e-5, one, out, None, None) == binding.INVALID_ARG
+    assert lib.pmkvq_alpha_grid_search(one, one, one, 4, 1, 1, 1, 2, a, 2, 1.0, 10000.0, 1e-5, ctypes.c_void_p(8), out, None, None) == binding.INVALID_ARG
+    assert lib.pmkvq_alpha_grid_workspace_bytes(0, 1) == 0 and lib.pmkvq_alpha_grid_workspace_bytes(2048, 4) >= 2048 * 64 * 8
+
+
 def test_host_side_validation_without_a_device():
     from paper_2505_18610_b200 import binding
     lib = binding.lib()
