@@ -180,17 +180,20 @@ pmkvq_status pmkvq_calibrate_lambda(const void *d_K_pre_bf16, int32_t n_tokens, 
  * Q K^T / sqrt(128), query head h reads KV head h / group, token t attends to tokens 0..t) of the
  * unquantized rotated tensors and of the quantized ones, over tokens, sequences, heads and channels.
  * Arithmetic: fp32 throughout (quantizer decisions as in pmkvq_append), sums of squared errors in fp64.
+ * 2 + 2 (n_alphas + 1) launches: abs-max, rotation table, then per pass one launch that writes the pass's
+ * Keys (and once the Values) as fp32 into the workspace and one attention launch.
  *   d_K_pre_bf16, d_V_bf16  DEVICE bf16 [n_tokens][n_seq][kv_heads][128]; Keys before RoPE, token t at position t
  *   d_Q_pre_bf16            DEVICE bf16 [n_tokens][n_seq][kv_heads * group][128], before RoPE
  *   bits                    2, 4, 8 or 16: the width whose loss is minimised (the block's Fbit)
  *   h_alphas                HOST [n_alphas], 1 <= n_alphas <= 64 (the section's grid: j / 20, j = 0..19)
- *   d_workspace             DEVICE, 256-byte aligned, pmkvq_alpha_grid_workspace_bytes(n_tokens, kv_heads) bytes
+ *   d_workspace             DEVICE, 256-byte aligned, pmkvq_alpha_grid_workspace_bytes(...) bytes of the same sizes
+ *                           (fp32 copies of each pass's Keys and Values and of the unquantized output)
  *   h_losses                HOST [n_alphas], written
  *   h_best                  HOST, may be NULL: index of the smallest loss (the first one on ties)
  * The call synchronises `stream` before it returns (its results are host values).  The paper states
  * the criterion only; causal masking, the quantization of the Values and the mean-squared form are
  * this library's reading of it. */
-uint64_t pmkvq_alpha_grid_workspace_bytes(int32_t n_tokens, int32_t kv_heads);
+uint64_t pmkvq_alpha_grid_workspace_bytes(int32_t n_tokens, int32_t n_seq, int32_t kv_heads, int32_t group);
 pmkvq_status pmkvq_alpha_grid_search(const void *d_K_pre_bf16, const void *d_Q_pre_bf16, const void *d_V_bf16,
                                      int32_t n_tokens, int32_t n_seq, int32_t kv_heads, int32_t group, int32_t bits,
                                      const float *h_alphas, int32_t n_alphas, double pos_scale, double theta,

@@ -74,7 +74,7 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_calibrate_lambda.argtypes = [vp, i32, i32, i32, ctypes.c_double, ctypes.c_double, ctypes.c_float,
                                            ctypes.c_float, vp, vp]
     lib.pmkvq_alpha_grid_workspace_bytes.restype = ctypes.c_uint64
-    lib.pmkvq_alpha_grid_workspace_bytes.argtypes = [i32, i32]
+    lib.pmkvq_alpha_grid_workspace_bytes.argtypes = [i32, i32, i32, i32]
     lib.pmkvq_alpha_grid_search.restype = i32
     lib.pmkvq_alpha_grid_search.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, ctypes.c_double, ctypes.c_double,
                                             ctypes.c_float, vp, vp, vp, vp]
@@ -129,7 +129,7 @@ def alpha_grid_search(k_pre: torch.Tensor, q_pre: torch.Tensor, v: torch.Tensor,
         raise ValueError("shapes of k_pre, q_pre, v do not fit together")
     group = q_pre.shape[2] // kv_heads
     a = np.ascontiguousarray(np.arange(20) / 20.0 if alphas is None else alphas, dtype=np.float32)
-    ws = torch.empty(int(lib().pmkvq_alpha_grid_workspace_bytes(n_tokens, kv_heads)), dtype=torch.uint8, device=k_pre.device)
+    ws = torch.empty(int(lib().pmkvq_alpha_grid_workspace_bytes(n_tokens, n_seq, kv_heads, group)), dtype=torch.uint8, device=k_pre.device)
     losses = np.zeros(len(a), np.float64)
     best = ctypes.c_int32()
     st = lib().pmkvq_alpha_grid_search(k_pre.data_ptr(), q_pre.data_ptr(), v.data_ptr(), n_tokens, n_seq, kv_heads, group,

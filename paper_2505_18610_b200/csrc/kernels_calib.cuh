@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 
+#include "kernels_attn.cuh"
 #include "kernels_cache.cuh"
 #include "layout.cuh"
 
@@ -80,7 +81,7 @@ __global__ void rope_table_kernel(float2 *table, int n_tokens, double pos_scale,
   table[i] = make_float2((float)c, (float)s);
 }
 
-constexpr int kQPT = 2;                     // queries per thread
+constexpr int kQPT = 4;                     // queries per thread
 constexpr int kGridQueries = 16 * kQPT;     // queries of one CTA: 16 groups of kQPT queries, 8 threads per group
 constexpr int kGridKeys = 32;     // keys per shared-memory tile
 constexpr int kMaxAlphas = 64;
@@ -89,7 +90,7 @@ __device__ __forceinline__ float ex2_fast(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-constexpr int kGridSmemBytes = (2 * kGridKeys + kGridQueries) * kHeadDim * 4;  // K tile, V tile, kept outputs
+constexpr int kGridSmemBytes = 2 * 2 * kGridKeys * kHeadDim * 4;  // two stages of a K tile and a V tile
 
 // One token's 4 channels per lane (channels 4 lane .. 4 lane + 3): rotate by the token's angles.  The
 // partner channel (+-64) sits in lane ^ 16.
@@ -136,180 +137,215 @@ __device__ __forceinline__ void load_bf16x4(const uint16_t *src, float (&x)[4]) 
   x[3] = __uint_as_float(raw.y & 0xFFFF0000u);
 }
 
-// Grid: (query blocks, query heads, sequences).  K, V: bf16 [n_tokens][n_seq][kv_heads][128];
-// Q: bf16 [n_tokens][n_seq][kv_heads * group][128]; amax [kv_heads][128] from calib_absmax_kernel;
-// loss_sums [n_alphas] (fp64, zero before the launch) receives the summed squared errors.
+// One pass's Keys and Values as the attention kernel reads them: fp32 [n_tokens][n_seq][kv_heads][128].
+// One warp per (token, sequence, KV head) vector, lane l on channels 4 l .. 4 l + 3.
+//   alpha_index < 0  (the unquantized operator): k_out = rotated Keys, v_out = Values
+//   alpha_index >= 0: k_out = dequantized Q_bits(rotated Keys * Lambda^-1), lambda = max(amax, floor)^alpha;
+//                     v_out (if not null) = dequantized Q_bits(Values), which no alpha changes
+__global__ void __launch_bounds__(128) alpha_grid_prep_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
+                                                              const float *__restrict__ amax, const float2 *__restrict__ table,
+                                                              const float *__restrict__ alphas, int alpha_index,
+                                                              long long n_vectors, int vec_per_token, int kv_heads, int bits,
+                                                              float floor_value, float *__restrict__ k_out,
+                                                              float *__restrict__ v_out) {
+  const int lane = threadIdx.x & 31;
+  const long long vec = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (vec >= n_vectors) return;
+  const int t = (int)(vec / vec_per_token), kv_head = (int)(vec % kv_heads);
+  float xk[4];
+  load_bf16x4(K + vec * kHeadDim + 4 * lane, xk);
+  rotate_token(xk, table + (size_t)t * 64, lane);
+  if (alpha_index >= 0) {
+    const float alpha = alphas[alpha_index];
+    const float4 am = *reinterpret_cast<const float4 *>(amax + (size_t)kv_head * kHeadDim + 4 * lane);
+    xk[0] = __fmul_rn(xk[0], __fdiv_rn(1.0f, powf(fmaxf(am.x, floor_value), alpha)));
+    xk[1] = __fmul_rn(xk[1], __fdiv_rn(1.0f, powf(fmaxf(am.y, floor_value), alpha)));
+    xk[2] = __fmul_rn(xk[2], __fdiv_rn(1.0f, powf(fmaxf(am.z, floor_value), alpha)));
+    xk[3] = __fmul_rn(xk[3], __fdiv_rn(1.0f, powf(fmaxf(am.w, floor_value), alpha)));
+    quantize_dequantize_token(xk, bits);
+  }
+  *reinterpret_cast<float4 *>(k_out + vec * kHeadDim + 4 * lane) = make_float4(xk[0], xk[1], xk[2], xk[3]);
+  if (v_out) {
+    float xv[4];
+    load_bf16x4(V + vec * kHeadDim + 4 * lane, xv);
+    if (alpha_index >= 0) quantize_dequantize_token(xv, bits);
+    *reinterpret_cast<float4 *>(v_out + vec * kHeadDim + 4 * lane) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+  }
+}
+
+// One pass of causal self-attention in fp32.  Grid: (query blocks, query heads, sequences).
+// Q: bf16 [n_tokens][n_seq][kv_heads * group][128] before RoPE (rotated here, and scaled by lambda(alpha)
+// when alpha_index >= 0, Eq. 9); k_in, v_in: this pass's tensors from alpha_grid_prep_kernel.
+// alpha_index < 0: the outputs go to o_ref [n_tokens][n_seq][q_heads][128]; otherwise the squared
+// differences to o_ref are added to loss_sums[alpha_index] (fp64).
 // Thread (group, part) works on the group's kQPT consecutive queries and on channels 32 c + 4 part + e
 // (c < 4, e < 4): a rotation pair (i, i + 64) stays in one thread, the 8 parts read one 128-byte run of a
 // key row, every value read from shared memory feeds kQPT multiply-adds (one per query), and two keys are
-// taken per turn so that their score chains, shuffles and exponentials overlap.
-__global__ void __launch_bounds__(128) alpha_grid_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ Q,
-                                                         const uint16_t *__restrict__ V, const float *__restrict__ amax,
-                                                         const float2 *__restrict__ table, const float *__restrict__ alphas,
-                                                         int n_alphas, int n_tokens, int n_seq, int kv_heads, int group,
-                                                         int bits, float floor_value, double *loss_sums) {
-  extern __shared__ __align__(16) float s_dyn[];
-  float(*s_k)[kHeadDim] = reinterpret_cast<float(*)[kHeadDim]>(s_dyn);
-  float(*s_v)[kHeadDim] = reinterpret_cast<float(*)[kHeadDim]>(s_dyn + kGridKeys * kHeadDim);
-  float(*s_ref)[kHeadDim] = reinterpret_cast<float(*)[kHeadDim]>(s_dyn + 2 * kGridKeys * kHeadDim);
-  __shared__ float s_lam[kHeadDim], s_inv[kHeadDim];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+// taken per turn so that their score chains, shuffles and exponentials overlap.  Key / Value tiles of 32
+// tokens arrive through a two-stage cp.async ring.
+__global__ void __launch_bounds__(128) alpha_grid_attn_kernel(const uint16_t *__restrict__ Q, const float *__restrict__ k_in,
+                                                              const float *__restrict__ v_in, const float *__restrict__ amax,
+                                                              const float2 *__restrict__ table,
+                                                              const float *__restrict__ alphas, int alpha_index, int n_tokens,
+                                                              int n_seq, int kv_heads, int group, float floor_value,
+                                                              float *__restrict__ o_ref, double *loss_sums) {
+  extern __shared__ __align__(16) float s_dyn[];  // [stage][K | V][32 keys][128]
+  __shared__ float s_lam[kHeadDim];
+  const int tid = threadIdx.x, lane = tid & 31;
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;  // long rows first
   const int q_head = blockIdx.y, seq = blockIdx.z, kv_head = q_head / group, q_heads = kv_heads * group;
   const int ql0 = (tid >> 3) * kQPT, part = tid & 7;  // first of the thread's queries inside the CTA
   const int q0 = qb * kGridQueries + ql0;
   const int q_last = min(n_tokens, (qb + 1) * kGridQueries) - 1;  // last live query of the CTA
   const size_t kv_row = (size_t)n_seq * kv_heads * kHeadDim;
-  const uint16_t *k_base = K + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
-  const uint16_t *v_base = V + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
+  const float *k_base = k_in + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
+  const float *v_base = v_in + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
   const float scale_log2 = 1.4426950408889634f * rsqrtf((float)kHeadDim);
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(s_dyn);
+  constexpr int kStageFloats = 2 * kGridKeys * kHeadDim;
 
-  for (int pass = 0; pass <= n_alphas; ++pass) {
-    __syncthreads();  // the previous pass is done with s_lam / s_inv and the tiles
-    if (pass > 0) {
-      const float lam = powf(fmaxf(amax[(size_t)kv_head * kHeadDim + tid], floor_value), alphas[pass - 1]);
-      s_lam[tid] = lam;
-      s_inv[tid] = __fdiv_rn(1.0f, lam);
+  // tile j -> stage j & 1: thread i copies 16-byte pieces i, i + 128, ... of the 32 x 512-byte rows
+  auto issue = [&](int j) {
+    const uint32_t dst = ring + (uint32_t)((j & 1) * kStageFloats * 4);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const int piece = tid + 128 * c, row = piece >> 5, col = (piece & 31) * 4;
+      const int t = min(j * kGridKeys + row, n_tokens - 1);  // rows behind the last token are masked below
+      cp_async16(dst + (uint32_t)((row * kHeadDim + col) * 4), k_base + (size_t)t * kv_row + col);
+      cp_async16(dst + (uint32_t)(((kGridKeys + row) * kHeadDim + col) * 4), v_base + (size_t)t * kv_row + col);
     }
-    __syncthreads();
-    // the thread's rotated, equalized, pre-scaled query channels: qe[n][4 c + e]
-    float qe[kQPT][16], acc[kQPT][16], m[kQPT], l[kQPT];
+  };
+  const int n_tiles = q_last / kGridKeys + 1;
+  issue(0);
+  cp_async_commit();
+
+  s_lam[tid] = alpha_index >= 0 ? powf(fmaxf(amax[(size_t)kv_head * kHeadDim + tid], floor_value), alphas[alpha_index]) : 1.0f;
+  __syncthreads();
+  // the thread's rotated, equalized, pre-scaled query channels: qe[n][4 c + e]
+  float qe[kQPT][16], acc[kQPT][16], m[kQPT], l[kQPT];
 #pragma unroll
-    for (int n = 0; n < kQPT; ++n) {
-      m[n] = -INFINITY;
-      l[n] = 0.f;
+  for (int n = 0; n < kQPT; ++n) {
+    m[n] = -INFINITY;
+    l[n] = 0.f;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) { qe[n][i] = 0.f; acc[n][i] = 0.f; }
-      const int qi = q0 + n;
-      if (qi < n_tokens) {
-        const uint16_t *src = Q + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim;
-        const float2 *tab = table + (size_t)qi * 64;
+    for (int i = 0; i < 16; ++i) { qe[n][i] = 0.f; acc[n][i] = 0.f; }
+    const int qi = q0 + n;
+    if (qi < n_tokens) {
+      const uint16_t *src = Q + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim;
+      const float2 *tab = table + (size_t)qi * 64;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          float x1[4], x2[4];
-          load_bf16x4(src + 32 * c + 4 * part, x1);
-          load_bf16x4(src + 64 + 32 * c + 4 * part, x2);
+      for (int c = 0; c < 2; ++c) {
+        float x1[4], x2[4];
+        load_bf16x4(src + 32 * c + 4 * part, x1);
+        load_bf16x4(src + 64 + 32 * c + 4 * part, x2);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int ch = 32 * c + 4 * part + e;
-            const float2 cs = tab[ch];
-            const float y1 = __fsub_rn(__fmul_rn(x1[e], cs.x), __fmul_rn(x2[e], cs.y));
-            const float y2 = __fadd_rn(__fmul_rn(x1[e], cs.y), __fmul_rn(x2[e], cs.x));
-            qe[n][4 * c + e] = y1 * (pass > 0 ? s_lam[ch] : 1.0f) * scale_log2;
-            qe[n][4 * (c + 2) + e] = y2 * (pass > 0 ? s_lam[ch + 64] : 1.0f) * scale_log2;
-          }
+        for (int e = 0; e < 4; ++e) {
+          const int ch = 32 * c + 4 * part + e;
+          const float2 cs = tab[ch];
+          const float y1 = __fsub_rn(__fmul_rn(x1[e], cs.x), __fmul_rn(x2[e], cs.y));
+          const float y2 = __fadd_rn(__fmul_rn(x1[e], cs.y), __fmul_rn(x2[e], cs.x));
+          qe[n][4 * c + e] = y1 * s_lam[ch] * scale_log2;
+          qe[n][4 * (c + 2) + e] = y2 * s_lam[ch + 64] * scale_log2;
         }
       }
     }
-    for (int k0 = 0; k0 <= q_last; k0 += kGridKeys) {
-      __syncthreads();  // everyone is done with the previous tile
-      // ---- stage the tile: warp w takes keys 8 w .. 8 w + 7, lane l channels 4 l .. 4 l + 3 ----
-      for (int r = 0; r < 8; ++r) {
-        const int kk = warp * 8 + r, t = k0 + kk;
-        float xk[4] = {0.f, 0.f, 0.f, 0.f}, xv[4] = {0.f, 0.f, 0.f, 0.f};
-        if (t < n_tokens) {  // warp-uniform
-          load_bf16x4(k_base + (size_t)t * kv_row + 4 * lane, xk);
-          load_bf16x4(v_base + (size_t)t * kv_row + 4 * lane, xv);
-          rotate_token(xk, table + (size_t)t * 64, lane);
-          if (pass > 0) {
-            const float4 inv = *reinterpret_cast<const float4 *>(&s_inv[4 * lane]);
-            xk[0] = __fmul_rn(xk[0], inv.x); xk[1] = __fmul_rn(xk[1], inv.y);
-            xk[2] = __fmul_rn(xk[2], inv.z); xk[3] = __fmul_rn(xk[3], inv.w);
-            quantize_dequantize_token(xk, bits);
-            quantize_dequantize_token(xv, bits);
-          }
-        }
-        *reinterpret_cast<float4 *>(&s_k[kk][4 * lane]) = make_float4(xk[0], xk[1], xk[2], xk[3]);
-        *reinterpret_cast<float4 *>(&s_v[kk][4 * lane]) = make_float4(xv[0], xv[1], xv[2], xv[3]);
-      }
-      __syncthreads();
-      // ---- scores, online softmax, output ----
-      const int k_hi = min(kGridKeys, q_last - k0 + 1);
-      for (int kk = 0; kk < k_hi; kk += 2) {  // two keys per turn: their dependent chains overlap
-        // (a second key beyond k_hi lies behind every query of the CTA and is masked below; its row exists)
-        float s[2][kQPT];
+  }
+
+  for (int j = 0; j < n_tiles; ++j) {
+    __syncthreads();  // everyone is done with the stage that tile j + 1 will overwrite
+    if (j + 1 < n_tiles) issue(j + 1);
+    cp_async_commit();
+    cp_async_wait<1>();  // tile j has landed (this thread's pieces)
+    __syncthreads();     // ... and everyone else's
+    const float(*s_k)[kHeadDim] = reinterpret_cast<const float(*)[kHeadDim]>(s_dyn + (j & 1) * kStageFloats);
+    const float(*s_v)[kHeadDim] = s_k + kGridKeys;
+    const int k0 = j * kGridKeys;
+    const int k_hi = min(kGridKeys, q_last - k0 + 1);
+    for (int kk = 0; kk < k_hi; kk += 2) {  // two keys per turn: their dependent chains overlap
+      // (a second key beyond k_hi lies behind every query of the CTA and is masked below; its row exists)
+      float s[2][kQPT];
 #pragma unroll
-        for (int n = 0; n < kQPT; ++n) s[0][n] = s[1][n] = 0.f;
+      for (int n = 0; n < kQPT; ++n) s[0][n] = s[1][n] = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const float4 ka = *reinterpret_cast<const float4 *>(&s_k[kk][32 * c + 4 * part]);
-          const float4 kb = *reinterpret_cast<const float4 *>(&s_k[kk + 1][32 * c + 4 * part]);
-#pragma unroll
-          for (int n = 0; n < kQPT; ++n) {
-            s[0][n] = fmaf(qe[n][4 * c], ka.x, s[0][n]); s[1][n] = fmaf(qe[n][4 * c], kb.x, s[1][n]);
-            s[0][n] = fmaf(qe[n][4 * c + 1], ka.y, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 1], kb.y, s[1][n]);
-            s[0][n] = fmaf(qe[n][4 * c + 2], ka.z, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 2], kb.z, s[1][n]);
-            s[0][n] = fmaf(qe[n][4 * c + 3], ka.w, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 3], kb.w, s[1][n]);
-          }
-        }
-#pragma unroll
-        for (int o = 1; o <= 4; o <<= 1)
-#pragma unroll
-          for (int n = 0; n < kQPT; ++n) {
-            s[0][n] += __shfl_xor_sync(0xffffffffu, s[0][n], o);
-            s[1][n] += __shfl_xor_sync(0xffffffffu, s[1][n], o);
-          }
-        float p[2][kQPT];
+      for (int c = 0; c < 4; ++c) {
+        const float4 ka = *reinterpret_cast<const float4 *>(&s_k[kk][32 * c + 4 * part]);
+        const float4 kb = *reinterpret_cast<const float4 *>(&s_k[kk + 1][32 * c + 4 * part]);
 #pragma unroll
         for (int n = 0; n < kQPT; ++n) {
-          // causal mask (the eight threads of a group agree); key 0 is live for every query, so m is finite
-          // from the first turn on
-          const float sa = (k0 + kk <= q0 + n) ? s[0][n] : -INFINITY;
-          const float sb = (k0 + kk + 1 <= q0 + n) ? s[1][n] : -INFINITY;
-          const float mx = fmaxf(sa, sb);
-          if (mx > m[n]) {
-            const float corr = ex2_fast(m[n] - mx);  // 0 on the first key
-            l[n] *= corr;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[n][i] *= corr;
-            m[n] = mx;
-          }
-          p[0][n] = ex2_fast(sa - m[n]);
-          p[1][n] = ex2_fast(sb - m[n]);
-          l[n] += p[0][n] + p[1][n];
+          s[0][n] = fmaf(qe[n][4 * c], ka.x, s[0][n]); s[1][n] = fmaf(qe[n][4 * c], kb.x, s[1][n]);
+          s[0][n] = fmaf(qe[n][4 * c + 1], ka.y, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 1], kb.y, s[1][n]);
+          s[0][n] = fmaf(qe[n][4 * c + 2], ka.z, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 2], kb.z, s[1][n]);
+          s[0][n] = fmaf(qe[n][4 * c + 3], ka.w, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 3], kb.w, s[1][n]);
         }
+      }
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const float4 va = *reinterpret_cast<const float4 *>(&s_v[kk][32 * c + 4 * part]);
-          const float4 vb = *reinterpret_cast<const float4 *>(&s_v[kk + 1][32 * c + 4 * part]);
+      for (int o = 1; o <= 4; o <<= 1)
 #pragma unroll
-          for (int n = 0; n < kQPT; ++n) {
-            acc[n][4 * c] = fmaf(p[1][n], vb.x, fmaf(p[0][n], va.x, acc[n][4 * c]));
-            acc[n][4 * c + 1] = fmaf(p[1][n], vb.y, fmaf(p[0][n], va.y, acc[n][4 * c + 1]));
-            acc[n][4 * c + 2] = fmaf(p[1][n], vb.z, fmaf(p[0][n], va.z, acc[n][4 * c + 2]));
-            acc[n][4 * c + 3] = fmaf(p[1][n], vb.w, fmaf(p[0][n], va.w, acc[n][4 * c + 3]));
-          }
+        for (int n = 0; n < kQPT; ++n) {
+          s[0][n] += __shfl_xor_sync(0xffffffffu, s[0][n], o);
+          s[1][n] += __shfl_xor_sync(0xffffffffu, s[1][n], o);
+        }
+      float p[2][kQPT];
+#pragma unroll
+      for (int n = 0; n < kQPT; ++n) {
+        // causal mask (the eight threads of a group agree); key 0 is live for every query, so m is finite
+        // from the first turn on
+        const float sa = (k0 + kk <= q0 + n) ? s[0][n] : -INFINITY;
+        const float sb = (k0 + kk + 1 <= q0 + n) ? s[1][n] : -INFINITY;
+        const float mx = fmaxf(sa, sb);
+        if (mx > m[n]) {
+          const float corr = ex2_fast(m[n] - mx);  // 0 on the first key
+          l[n] *= corr;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) acc[n][i] *= corr;
+          m[n] = mx;
+        }
+        p[0][n] = ex2_fast(sa - m[n]);
+        p[1][n] = ex2_fast(sb - m[n]);
+        l[n] += p[0][n] + p[1][n];
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float4 va = *reinterpret_cast<const float4 *>(&s_v[kk][32 * c + 4 * part]);
+        const float4 vb = *reinterpret_cast<const float4 *>(&s_v[kk + 1][32 * c + 4 * part]);
+#pragma unroll
+        for (int n = 0; n < kQPT; ++n) {
+          acc[n][4 * c] = fmaf(p[1][n], vb.x, fmaf(p[0][n], va.x, acc[n][4 * c]));
+          acc[n][4 * c + 1] = fmaf(p[1][n], vb.y, fmaf(p[0][n], va.y, acc[n][4 * c + 1]));
+          acc[n][4 * c + 2] = fmaf(p[1][n], vb.z, fmaf(p[0][n], va.z, acc[n][4 * c + 2]));
+          acc[n][4 * c + 3] = fmaf(p[1][n], vb.w, fmaf(p[0][n], va.w, acc[n][4 * c + 3]));
         }
       }
     }
-    // ---- the pass's output: keep it (pass 0) or compare with the kept one (only this thread touches
-    // its entries of s_ref, so no barrier is needed around them) ----
-    float err = 0.f;
+  }
+  cp_async_wait<0>();
+
+  // ---- the pass's output: keep it (the unquantized pass) or compare with the kept one ----
+  float err = 0.f;
 #pragma unroll
-    for (int n = 0; n < kQPT; ++n) {
-      if (q0 + n < n_tokens) {
-        const float inv_l = __fdiv_rn(1.0f, l[n]);
+  for (int n = 0; n < kQPT; ++n) {
+    if (q0 + n < n_tokens) {
+      const float inv_l = __fdiv_rn(1.0f, l[n]);
+      float *kept = o_ref + (((size_t)(q0 + n) * n_seq + seq) * q_heads + q_head) * kHeadDim + 4 * part;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float o = acc[n][4 * c + e] * inv_l;
-            float &kept = s_ref[ql0 + n][32 * c + 4 * part + e];
-            if (pass == 0) {
-              kept = o;
-            } else {
-              const float d = o - kept;
-              err = fmaf(d, d, err);
-            }
-          }
+      for (int c = 0; c < 4; ++c) {
+        float4 o = make_float4(acc[n][4 * c] * inv_l, acc[n][4 * c + 1] * inv_l, acc[n][4 * c + 2] * inv_l,
+                               acc[n][4 * c + 3] * inv_l);
+        if (alpha_index < 0) {
+          *reinterpret_cast<float4 *>(kept + 32 * c) = o;
+        } else {
+          const float4 r = *reinterpret_cast<const float4 *>(kept + 32 * c);
+          o.x -= r.x; o.y -= r.y; o.z -= r.z; o.w -= r.w;
+          err = fmaf(o.x, o.x, err); err = fmaf(o.y, o.y, err); err = fmaf(o.z, o.z, err); err = fmaf(o.w, o.w, err);
+        }
       }
     }
-    if (pass > 0) {
-      double e = (double)err;
+  }
+  if (alpha_index >= 0) {
+    double e = (double)err;
 #pragma unroll
-      for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
-      if (lane == 0) atomicAdd(loss_sums + (pass - 1), e);
-    }
+    for (int o = 16; o; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+    if (lane == 0) atomicAdd(loss_sums + alpha_index, e);
   }
 }
 

@@ -684,10 +684,30 @@ pmkvq_status pmkvq_calibrate_lambda(const void *d_K, int32_t n_tokens, int32_t n
 
 static size_t grid_ws_round(size_t b) { return (b + 255) / 256 * 256; }
 
-uint64_t pmkvq_alpha_grid_workspace_bytes(int32_t n_tokens, int32_t kv_heads) {
-  if (n_tokens <= 0 || kv_heads <= 0) return 0;
-  return grid_ws_round((size_t)kv_heads * kHeadDim * sizeof(float)) + grid_ws_round((size_t)n_tokens * 64 * sizeof(float2)) +
-         grid_ws_round(kMaxAlphas * sizeof(double)) + grid_ws_round(kMaxAlphas * sizeof(float));
+// workspace of the alpha grid search: abs-max, rotation table, loss sums, alphas, then fp32 copies of this
+// pass's Keys, of the Values (as given and quantized) and the unquantized operator's output
+struct GridWorkspace {
+  size_t amax, table, loss, alphas, k_pass, v_raw, v_hat, o_ref, total;
+};
+static GridWorkspace grid_workspace(int64_t n_tokens, int64_t n_seq, int64_t kv_heads, int64_t group) {
+  GridWorkspace w;
+  size_t off = 0;
+  const size_t kv = (size_t)(n_tokens * n_seq * kv_heads) * kHeadDim * sizeof(float);
+  w.amax = off; off += grid_ws_round((size_t)kv_heads * kHeadDim * sizeof(float));
+  w.table = off; off += grid_ws_round((size_t)n_tokens * 64 * sizeof(float2));
+  w.loss = off; off += grid_ws_round(kMaxAlphas * sizeof(double));
+  w.alphas = off; off += grid_ws_round(kMaxAlphas * sizeof(float));
+  w.k_pass = off; off += grid_ws_round(kv);
+  w.v_raw = off; off += grid_ws_round(kv);
+  w.v_hat = off; off += grid_ws_round(kv);
+  w.o_ref = off; off += grid_ws_round(kv * (size_t)group);
+  w.total = off;
+  return w;
+}
+
+uint64_t pmkvq_alpha_grid_workspace_bytes(int32_t n_tokens, int32_t n_seq, int32_t kv_heads, int32_t group) {
+  if (n_tokens <= 0 || n_seq <= 0 || kv_heads <= 0 || group <= 0) return 0;
+  return grid_workspace(n_tokens, n_seq, kv_heads, group).total;
 }
 
 pmkvq_status pmkvq_alpha_grid_search(const void *d_K, const void *d_Q, const void *d_V, int32_t n_tokens, int32_t n_seq,
@@ -704,29 +724,38 @@ pmkvq_status pmkvq_alpha_grid_search(const void *d_K, const void *d_Q, const voi
   for (int i = 0; i < n_alphas; ++i)
     if (!std::isfinite(h_alphas[i])) return PMKVQ_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const GridWorkspace w = grid_workspace(n_tokens, n_seq, kv_heads, group);
   uint8_t *ws = static_cast<uint8_t *>(d_workspace);
-  float *d_amax = reinterpret_cast<float *>(ws);
-  ws += grid_ws_round((size_t)kv_heads * kHeadDim * sizeof(float));
-  float2 *d_table = reinterpret_cast<float2 *>(ws);
-  ws += grid_ws_round((size_t)n_tokens * 64 * sizeof(float2));
-  double *d_loss = reinterpret_cast<double *>(ws);
-  ws += grid_ws_round(kMaxAlphas * sizeof(double));
-  float *d_alphas = reinterpret_cast<float *>(ws);
+  float *d_amax = reinterpret_cast<float *>(ws + w.amax);
+  float2 *d_table = reinterpret_cast<float2 *>(ws + w.table);
+  double *d_loss = reinterpret_cast<double *>(ws + w.loss);
+  float *d_alphas = reinterpret_cast<float *>(ws + w.alphas);
+  float *d_k = reinterpret_cast<float *>(ws + w.k_pass), *d_v_raw = reinterpret_cast<float *>(ws + w.v_raw);
+  float *d_v_hat = reinterpret_cast<float *>(ws + w.v_hat), *d_o_ref = reinterpret_cast<float *>(ws + w.o_ref);
   if (cudaMemsetAsync(d_amax, 0, (size_t)kv_heads * kHeadDim * sizeof(float), st) != cudaSuccess ||
       cudaMemsetAsync(d_loss, 0, kMaxAlphas * sizeof(double), st) != cudaSuccess ||
       cudaMemcpyAsync(d_alphas, h_alphas, (size_t)n_alphas * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return PMKVQ_ERR_CUDA;
+  const uint16_t *K = static_cast<const uint16_t *>(d_K), *Q = static_cast<const uint16_t *>(d_Q),
+                 *V = static_cast<const uint16_t *>(d_V);
   const int tokens_per_cta = std::max(1, (n_tokens + 148 * 8 - 1) / (148 * 8));
   calib_absmax_kernel<<<(unsigned)((n_tokens + tokens_per_cta - 1) / tokens_per_cta), 128, 0, st>>>(
-      static_cast<const uint16_t *>(d_K), reinterpret_cast<unsigned *>(d_amax), n_tokens, n_seq * kv_heads, kv_heads,
-      tokens_per_cta, pos_scale, theta);
+      K, reinterpret_cast<unsigned *>(d_amax), n_tokens, n_seq * kv_heads, kv_heads, tokens_per_cta, pos_scale, theta);
   rope_table_kernel<<<(unsigned)((n_tokens * 64 + 255) / 256), 256, 0, st>>>(d_table, n_tokens, pos_scale, theta);
-  const dim3 grid((unsigned)((n_tokens + kGridQueries - 1) / kGridQueries), (unsigned)(kv_heads * group), (unsigned)n_seq);
-  if (cudaFuncSetAttribute(alpha_grid_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGridSmemBytes) != cudaSuccess)
+  if (cudaFuncSetAttribute(alpha_grid_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGridSmemBytes) != cudaSuccess)
     return PMKVQ_ERR_CUDA;
-  alpha_grid_kernel<<<grid, 128, kGridSmemBytes, st>>>(static_cast<const uint16_t *>(d_K), static_cast<const uint16_t *>(d_Q),
-                                          static_cast<const uint16_t *>(d_V), d_amax, d_table, d_alphas, n_alphas, n_tokens,
-                                          n_seq, kv_heads, group, bits, floor_value, d_loss);
+  const long long n_vectors = (long long)n_tokens * n_seq * kv_heads;
+  const unsigned prep_grid = (unsigned)((n_vectors + 3) / 4);
+  const dim3 grid((unsigned)((n_tokens + kGridQueries - 1) / kGridQueries), (unsigned)(kv_heads * group), (unsigned)n_seq);
+  // pass -1: the unquantized operator; passes 0 .. n_alphas - 1: Eq. 9 at each alpha
+  for (int pass = -1; pass < n_alphas; ++pass) {
+    float *v_out = pass == -1 ? d_v_raw : pass == 0 ? d_v_hat : nullptr;
+    alpha_grid_prep_kernel<<<prep_grid, 128, 0, st>>>(K, V, d_amax, d_table, d_alphas, pass, n_vectors, n_seq * kv_heads,
+                                                      kv_heads, bits, floor_value, d_k, v_out);
+    alpha_grid_attn_kernel<<<grid, 128, kGridSmemBytes, st>>>(Q, d_k, pass == -1 ? d_v_raw : d_v_hat, d_amax, d_table,
+                                                              d_alphas, pass, n_tokens, n_seq, kv_heads, group, floor_value,
+                                                              d_o_ref, d_loss);
+  }
   if (cudaGetLastError() != cudaSuccess) return PMKVQ_ERR_CUDA;
   double sums[kMaxAlphas];
   if (cudaMemcpyAsync(sums, d_loss, (size_t)n_alphas * sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess ||

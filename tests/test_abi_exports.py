@@ -52,7 +52,8 @@ def test_binding_argument_counts_match_the_prototypes():
     assert lib.pmkvq_alpha_grid_search(one, one, one, 4, 1, 1, 1, 3, a, 2, 1.0, 10000.0, 1e-5, one, out, None, None) == binding.INVALID_ARG
     assert lib.pmkvq_alpha_grid_search(one, one, one, 4, 1, 1, 1, 2, a, 65, 1.0, 10000.0, 1e-5, one, out, None, None) == binding.INVALID_ARG
     assert lib.pmkvq_alpha_grid_search(one, one, one, 4, 1, 1, 1, 2, a, 2, 1.0, 10000.0, 1e-5, ctypes.c_void_p(8), out, None, None) == binding.INVALID_ARG
-    assert lib.pmkvq_alpha_grid_workspace_bytes(0, 1) == 0 and lib.pmkvq_alpha_grid_workspace_bytes(2048, 4) >= 2048 * 64 * 8
+    assert lib.pmkvq_alpha_grid_workspace_bytes(0, 1, 1, 1) == 0
+    assert lib.pmkvq_alpha_grid_workspace_bytes(2048, 8, 4, 7) >= 2048 * 8 * 4 * 512 * (3 + 7)
 
 
 def test_host_side_validation_without_a_device():
