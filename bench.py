@@ -183,7 +183,7 @@ NCU_TRAFFIC = {"digest": "0896cabc2f92bff2", "traffic_bytes": 976_307_200, "algo
 def aux_leg(wl, device):
     """The two kernels beside the decode step, timed alone with CUDA events (best of 5 calls after a warm-up):
     the bulk prefill append of 8192 tokens into one block of the workload's shape, and the alpha grid search
-    of the calibration (512 tokens x 2 sequences of the workload's head counts, 20 alphas, 2 bit)."""
+    of the calibration (2048 tokens x 8 sequences of the workload's head counts, 20 alphas, 2 bit)."""
     from paper_2505_18610_b200 import binding as B
     n = 8192
     k, v = synth.make_kv(3, 0, 0, n, wl["batch"], wl["kv_heads"], 0, wl["n_outlier"], wl["factor"], device=device)
@@ -202,13 +202,13 @@ def aux_leg(wl, device):
     out = {"bulk_append": {"tokens": n, "ms": min(ts[1:]), "GBps": append_bytes / (min(ts[1:]) * 1e-3) / 1e9,
                            "bytes": append_bytes, "what": "bf16 K, V in, INT16 tiles out, one block"}}
     g = torch.Generator().manual_seed(5)
-    nt, ns, kvh, grp = 512, 2, wl["kv_heads"], wl["q_heads"] // wl["kv_heads"]
+    nt, ns, kvh, grp = 2048, 8, wl["kv_heads"], wl["q_heads"] // wl["kv_heads"]    # a 2,048-token calibration text
     kk = torch.randn(nt, ns, kvh, 128, generator=g); kk[..., 9] *= 25.0; kk[..., 73] *= 25.0
     qq = torch.randn(nt, ns, kvh * grp, 128, generator=g)
     vv = torch.randn(nt, ns, kvh, 128, generator=g)
     kk, qq, vv = (t.to(torch.bfloat16).to(device).contiguous() for t in (kk, qq, vv))
     ts = []
-    for _ in range(4):
+    for _ in range(3):
         torch.cuda.synchronize(); t0 = time.perf_counter()
         best, losses = B.alpha_grid_search(kk, qq, vv, 2, pos_scale=4.0)
         ts.append((time.perf_counter() - t0) * 1e3)
