@@ -144,10 +144,11 @@ __device__ __forceinline__ float quotient_rn(float d, float s, float y) {
   r = __fmaf_rn(-q, s, d);
   return __fmaf_rn(r, y, q);
 }
-// round-half-to-even of a quotient in [0, 65536) and the clamp to 16 bits: adding 2^23 leaves the rounded
-// integer in the low mantissa bits.
+// round-half-to-even of a quotient: adding 2^23 leaves the rounded integer in the low mantissa bits.  No
+// clamp is needed: d <= max - min and S = RN((max - min) / 65535) >= (max - min) / 65535 (1 - 2^-24) bound
+// the correctly rounded quotient by 65535 (1 + 2^-23), which is below 65535.5.
 __device__ __forceinline__ int code_of_quotient(float q) {
-  return min(__float_as_int(__fadd_rn(q, 8388608.0f)) - 0x4B000000, 65535);
+  return __float_as_int(__fadd_rn(q, 8388608.0f)) - 0x4B000000;
 }
 
 // Eq. 1-2 at 16 bit on one token's 128 channels (Keys first times Lambda^-1, Eq. 9), by one warp: lane l
