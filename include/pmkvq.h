@@ -85,7 +85,8 @@ void pmkvq_cache_destroy(pmkvq_cache *cache);
  * tokens, then window eviction: tokens leaving the INT16 window are shifted (Eq. 3, repeatedly)
  * to the block's current width.
  *   d_K_bf16, d_V_bf16: DEVICE bf16 [n_new][batch][kv_heads][128], read only.
- * Returns BUDGET_FULL (state unchanged) if the block must be reduced first and auto_reduce is 0. */
+ * Returns BUDGET_FULL (state unchanged) if the block must be reduced first and auto_reduce is 0,
+ * INVALID_ARG for n_new < 1 (an empty append is refused, nothing is launched), CAPACITY beyond max_tokens. */
 pmkvq_status pmkvq_append(pmkvq_cache *cache, int32_t layer, const void *d_K_bf16, const void *d_V_bf16,
                           int32_t n_new, void *stream);
 
@@ -95,7 +96,8 @@ pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *cache, int32_t layer, void *s
 
 /* Decode-step attention of one block over all cached tokens (the one just appended included):
  * out = softmax(sm_scale * (Q Lambda) dequant(K Lambda^-1)^T) dequant(V)  (Eq. 9 with GQA).
- *   d_Q_bf16: DEVICE bf16 [batch][q_heads][128]; d_out: DEVICE fp32 [batch][q_heads][128]. */
+ *   d_Q_bf16: DEVICE bf16 [batch][q_heads][128]; d_out: DEVICE fp32 [batch][q_heads][128].
+ * A block without any cached token has no softmax to take: INVALID_ARG, nothing is launched. */
 pmkvq_status pmkvq_decode_attention(pmkvq_cache *cache, int32_t layer, const void *d_Q_bf16, float *d_out,
                                     void *stream);
 

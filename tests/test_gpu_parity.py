@@ -151,6 +151,30 @@ def test_reduce_head_batches_and_waves():
     m.check_attention(0, synth.make_q(31, 0, 0, 1, 2 * kvh, done))
 
 
+def test_empty_inputs_are_refused_and_empty_bodies_reduce():
+    from paper_2505_18610_b200 import binding as B
+    m = Mirror(2, 4, 1, 1, 64, [4, 4], n_sink=1, window=8, auto_reduce=False)
+    q = synth.make_q(41, 0, 0, 1, 4, 1).cuda()
+    with pytest.raises(B.PmkvqError):                       # no cached token: no softmax to take
+        m.cache.decode_attention(0, q)
+    k, v = make_inputs(41, 0, 3, 1, 1)
+    lib = B.lib()
+    assert lib.pmkvq_append(m.cache._h, 0, k.cuda().data_ptr(), v.cuda().data_ptr(), 0, None) == B.INVALID_ARG
+    assert m.cache.layer_state(0)["n_tokens"] == 0
+    K = torch.zeros(2, 1, 1, 128, dtype=torch.bfloat16, device="cuda")
+    m.append(0, k, v)                                       # block 1 stays empty
+    assert m.cache.progressive_reduce(1, check=False) == B.OK       # an empty body reduces to nothing, the width moves
+    m.oracles[1].reduce()
+    assert m.cache.layer_state(1)["cur_bits"] == 8 and m.cache.layer_state(0)["cur_bits"] == 16
+    m.check_state(0)
+    m.check_attention(0, synth.make_q(41, 0, 1, 1, 4, 3))
+    # a step needs every block's token: it appends to both and attends over 4 and 1 tokens
+    out = m.cache.decode_step(K, K, torch.stack([q, q]))
+    torch.cuda.synchronize()
+    assert m.cache.layer_state(1)["n_tokens"] == 1 and m.cache.layer_state(0)["n_tokens"] == 4
+    assert torch.isfinite(out).all()
+
+
 def test_split_invariance():
     kvh, batch, n, group = 2, 2, 5000, 8
     k, v = make_inputs(6, 0, n, batch, kvh)
