@@ -42,7 +42,8 @@ typedef enum {
   PMKVQ_ERR_CAPACITY = 5,        /* over budget at Fbit, or past max_tokens */
   PMKVQ_ERR_CUDA = 6,            /* a CUDA runtime call or launch failed */
   PMKVQ_ERR_STATE = 7,           /* internal invariant violated */
-  PMKVQ_ERR_SCRATCH_LIMIT = 8    /* pmkvq_decode_attention_static: more slices / CTAs than its fixed scratch holds */
+  PMKVQ_ERR_SCRATCH_LIMIT = 8,   /* pmkvq_decode_attention_static: more slices / CTAs than its fixed scratch holds */
+  PMKVQ_ERR_DEVICE_WAIT = 9      /* pmkvq_device_status: a bounded wait inside a kernel ran out */
 } pmkvq_status;
 
 typedef struct {
@@ -127,13 +128,33 @@ pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *cache, int32_t layer, co
  *   d_K_bf16, d_V_bf16: DEVICE bf16 [layers][batch][kv_heads][128]
  *   d_Q_bf16:           DEVICE bf16 [layers][batch][q_heads][128]
  *   d_out:              DEVICE fp32 [layers][batch][q_heads][128]
- * The budget of every block is tested first (reducing where auto_reduce allows); if a block fails
- * (PMKVQ_ERR_BUDGET_FULL with auto_reduce = 0, PMKVQ_ERR_CAPACITY) its status is returned and no block has
- * received its token.  Then one launch appends to all blocks and one launch computes the attention
- * of all blocks (up to 128 blocks; beyond that the call falls back to one append and one attention
- * launch per block). */
+ * The budget of every block is tested first, without touching anything: if a block fails
+ * (PMKVQ_ERR_BUDGET_FULL with auto_reduce = 0, PMKVQ_ERR_CAPACITY) its status is returned and the whole
+ * cache is as it was: no block has been reduced and no block has received its token.  Only then are
+ * the reduces run that the budgets ask for (auto_reduce = 1), one launch appends to all blocks and one
+ * launch computes the attention of all blocks (up to 128 blocks; beyond that the call falls back to
+ * one append and one attention launch per block). */
 pmkvq_status pmkvq_decode_step(pmkvq_cache *cache, const void *d_K_bf16, const void *d_V_bf16, const void *d_Q_bf16,
                                float *d_out, void *stream);
+
+/* The attention half of pmkvq_decode_step alone: decode attention of every block over its cached tokens
+ * in one launch (Eq. 9 with GQA, Sec. 3.4), nothing appended.  Up to 128 blocks, every block non-empty.
+ *   d_Q_bf16: DEVICE bf16 [layers][batch][q_heads][128]; d_out: DEVICE fp32 [layers][batch][q_heads][128]. */
+pmkvq_status pmkvq_decode_attention_all(pmkvq_cache *cache, const void *d_Q_bf16, float *d_out, void *stream);
+
+/* The attention kernels wait on hardware barriers (copies into shared memory, tensor-core completion); every
+ * such wait has an iteration limit instead of spinning for ever.  A wait that runs out makes its CTA
+ * skip the rest of its waits and return, and sets a bit in a word of the arena (1: tile copy, 2: score
+ * MMAs, 4: output MMAs).  This call synchronises the device and returns PMKVQ_ERR_DEVICE_WAIT if any bit is
+ * set (the outputs of the affected launch are then meaningless), PMKVQ_OK otherwise; *h_wait_bits (may be
+ * NULL) receives the word.  The word is never cleared: create a new cache after a failure. */
+pmkvq_status pmkvq_device_status(pmkvq_cache *cache, uint32_t *h_wait_bits);
+
+/* Checkpoint / restore of a block's host-side state.  The device-side state of a cache is the arena; a
+ * caller that saved a copy of the arena together with pmkvq_layer_state()'s (n_tokens, cur_bits) of every
+ * block puts the bytes back and then calls this for every block.  INVALID_ARG if the pair cannot be a state
+ * of this block (width below Fbit, over budget, beyond capacity); nothing on the device is touched. */
+pmkvq_status pmkvq_restore_layer_state(pmkvq_cache *cache, int32_t layer, int32_t n_tokens, int32_t cur_bits);
 
 /* Split-K tuning of pmkvq_decode_attention (flash-decoding partition over the sequence): the tiles
  * of all (batch, kv_head) slices are cut into `n_ctas` equal contiguous pieces, one per CTA

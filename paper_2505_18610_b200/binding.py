@@ -17,8 +17,9 @@ from . import build as _build
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libpmkvq.so")
 
 STATUS_NAMES = ["OK", "INVALID_ARG", "ARENA_TOO_SMALL", "BUDGET_FULL", "AT_FBIT", "CAPACITY", "CUDA", "STATE",
-                "SCRATCH_LIMIT"]
-OK, INVALID_ARG, ARENA_TOO_SMALL, BUDGET_FULL, AT_FBIT, CAPACITY, CUDA_ERROR, STATE, SCRATCH_LIMIT = range(9)
+                "SCRATCH_LIMIT", "DEVICE_WAIT"]
+(OK, INVALID_ARG, ARENA_TOO_SMALL, BUDGET_FULL, AT_FBIT, CAPACITY, CUDA_ERROR, STATE, SCRATCH_LIMIT,
+ DEVICE_WAIT) = range(10)
 
 
 class PmkvqError(RuntimeError):
@@ -60,6 +61,12 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_decode_attention_static.argtypes = [vp, i32, vp, vp, vp]
     lib.pmkvq_decode_step.restype = i32
     lib.pmkvq_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.pmkvq_decode_attention_all.restype = i32
+    lib.pmkvq_decode_attention_all.argtypes = [vp, vp, vp, vp]
+    lib.pmkvq_device_status.restype = i32
+    lib.pmkvq_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.pmkvq_restore_layer_state.restype = i32
+    lib.pmkvq_restore_layer_state.argtypes = [vp, i32, i32, i32]
     lib.pmkvq_set_attention_ctas.restype = i32
     lib.pmkvq_set_attention_ctas.argtypes = [vp, i32]
     lib.pmkvq_layer_state.restype = i32
@@ -272,6 +279,35 @@ class Cache:
         if st != OK:
             raise PmkvqError(st, "pmkvq_decode_step")
         return out
+
+    def decode_attention_all(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None):
+        """Attention of all blocks in one launch, nothing appended.  q: bf16 [layers, batch, q_heads, 128]
+        -> fp32 [layers, batch, q_heads, 128]."""
+        self._check(q, torch.bfloat16, "q")
+        if q.numel() != self.layers * self.batch * self.q_heads * 128:
+            raise ValueError("bad Q shape")
+        if out is None:
+            out = torch.empty(self.layers, self.batch, self.q_heads, 128, dtype=torch.float32, device=q.device)
+        self._check(out, torch.float32, "out")
+        if out.numel() != q.numel():
+            raise ValueError("bad out shape")
+        st = lib().pmkvq_decode_attention_all(self._h, q.data_ptr(), out.data_ptr(), _stream_ptr(stream))
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_decode_attention_all")
+        return out
+
+    def device_status(self, check: bool = True) -> int:
+        """Synchronises; returns the word of device-side waits that ran out (0 = none)."""
+        word = ctypes.c_uint32()
+        st = lib().pmkvq_device_status(self._h, ctypes.byref(word))
+        if check and st != OK:
+            raise PmkvqError(st, f"pmkvq_device_status (bits {word.value:#x})")
+        return int(word.value)
+
+    def restore_layer_state(self, layer: int, n_tokens: int, cur_bits: int):
+        st = lib().pmkvq_restore_layer_state(self._h, layer, int(n_tokens), int(cur_bits))
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_restore_layer_state")
 
     def set_attention_ctas(self, n_ctas: int):
         st = lib().pmkvq_set_attention_ctas(self._h, n_ctas)

@@ -14,14 +14,14 @@
 // publishes one partial (m, l, o[128]) per head.  The CTA that publishes the
 // last partial of a slice (atomic ticket, nobody waits) merges the slice and writes the output.
 //
-// Body tiles are staged through a per-warp cp.async ring in shared memory (a tile is one
-// contiguous run of bytes); tiles are consumed two at a time at 2 and 4 bit so that the softmax
-// bookkeeping is paid once per 32 tokens.
-//
-// The contraction runs on the tensor cores with mma.sync.m16n8k16 (f16 inputs, f32 accumulate) and
-// register operands: packed codes go from 128-bit loads to MMA fragments with one AND per pair of
-// codes - a code field left in place inside an fp16 bit pattern below bit 11 is the exact value
-// code * 2^(pos-24) (fp16 subnormals and the first binade are linear in the bit pattern).
+// Two contraction paths share this decomposition.  The 4- and 2-bit body, which holds most bytes of a
+// cache in its steady state, runs on tcgen05.mma with its code operands in tensor memory
+// (kernels_attn_tc.cuh).  INT16 tiles (sink, window) and an 8- or 16-bit body run on warp-level
+// mma.sync.m16n8k16 (f16 inputs, f32 accumulate) with register operands, the body tiles staged through a
+// per-warp cp.async ring in shared memory (a tile is one contiguous run of bytes); in both paths packed
+// codes become MMA operands with one logic operation per pair of codes - a code field left in place
+// inside an fp16 bit pattern below bit 11 is the exact value code * 2^(pos-24) (fp16 subnormals and the
+// first binade are linear in the bit pattern).
 //   scores:  S[h, t]  = sum_i Q''[h, i] * c_K[t, i]      A = Q'' (rows 0-7: fp16 "hi" part of the 8 heads,
 //                                                        rows 8-15: the "lo" remainder), B = K codes
 //   output:  O^T[i,h] = sum_t c_V[t, i] * w[t, h]        A = V codes, B = w = p * S_V (one fp16)
@@ -38,6 +38,7 @@
 
 #include "kernels_cache.cuh"
 #include "layout.cuh"
+#include "tc05.cuh"
 
 namespace pmkvq {
 
@@ -45,8 +46,9 @@ constexpr int kMaxGroup = 8;         // query heads per KV head handled by one M
 constexpr int kPartialStride = 132;  // floats per (segment, head): m, l, 2 pad, o[128]
 constexpr float kNegBig = -1.0e30f;
 constexpr float kMaxAhead = 3.0f;    // a score may exceed the reference by this much (log2 units)
-constexpr int kAttnWarps = 16;       // one CTA per SM; its warps share the CTA's tiles dynamically
+constexpr int kAttnWarps = 12;       // one CTA per SM: three warpgroups; its warps share the CTA's INT16 / 8-bit tiles dynamically
 constexpr int kAttnThreads = 32 * kAttnWarps;
+constexpr int kParts = kAttnWarps + 3;  // partial results a segment merges: one per warp, one per warpgroup
 
 struct AttnParams {
   LayerGeom geom;
@@ -140,25 +142,6 @@ __device__ __forceinline__ uint32_t high_bytes(uint32_t x) { return __byte_perm(
 // is also how far apart the warps of a CTA can finish, so the ring is kept shallow: 16 warps per SM
 // already keep about 70 KB in flight).
 template <int BITS> struct Fmt;
-template <> struct Fmt<2> {
-    static constexpr int N = 8, EQ = 14, EP = 12, SIGMA_LOG2 = 15, NT = 2, SLOTS = 2;
-  __host__ __device__ static constexpr int pos(int j) { return j < 5 ? 2 * j : 2 * j - 5; }
-  __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[8]) {
-    const uint32_t xr = x >> 5;
-    e[0] = x & 0x00030003u; e[1] = x & 0x000C000Cu; e[2] = x & 0x00300030u; e[3] = x & 0x00C000C0u;
-    e[4] = x & 0x03000300u;
-    e[5] = xr & 0x00600060u; e[6] = xr & 0x01800180u; e[7] = xr & 0x06000600u;
-  }
-};
-template <> struct Fmt<4> {
-  static constexpr int N = 4, EQ = 14, EP = 12, SIGMA_LOG2 = 13, NT = 2, SLOTS = 2;
-  __host__ __device__ static constexpr int pos(int j) { return (j & 1) ? 4 : 0; }
-  __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[4]) {
-    const uint32_t xr = x >> 8;
-    e[0] = x & 0x000F000Fu; e[1] = x & 0x00F000F0u;
-    e[2] = xr & 0x000F000Fu; e[3] = xr & 0x00F000F0u;
-  }
-};
 template <> struct Fmt<8> {
   static constexpr int N = 2, EQ = 14, EP = 12, SIGMA_LOG2 = 9, NT = 1, SLOTS = 2;
   __host__ __device__ static constexpr int pos(int) { return 0; }
@@ -337,9 +320,14 @@ __device__ __forceinline__ float softmax_phase(const uint8_t *tile0, uint32_t ma
       const float2 s_e = __ffma2_rn(sv[j], inv2, make_float2(sv[j].x == 0.f ? 1.f : 0.f, sv[j].y == 0.f ? 1.f : 0.f));
       const float2 rs = make_float2(rcp_approx(s_e.x), rcp_approx(s_e.y));
       const float2 arg = __fadd2_rn(sc[j], neg_m);
-      const float2 w = __fmul2_rn(make_float2(ex2(arg.x), ex2(arg.y)), s_e);  // p * S_V / sigma_u * 2^EP
+      const float2 e = make_float2(ex2(arg.x), ex2(arg.y));
+      const float2 w = __fmul2_rn(e, s_e);  // p * S_V / sigma_u * 2^EP
       pb[j] = pack_half2(w.x, w.y);
-      const float2 p = __fmul2_rn(__half22float2(*reinterpret_cast<const __half2 *>(&pb[j])), rs);
+      float2 p = __fmul2_rn(__half22float2(*reinterpret_cast<const __half2 *>(&pb[j])), rs);
+      // a V scale far below the slice's largest takes w out of fp16's normal range (the token's codes then
+      // carry next to nothing): its probability enters the sums as it is
+      if (s_e.x < 0x1p-10f) p.x = e.x;
+      if (s_e.y < 0x1p-10f) p.y = e.y;
       st.l = __fadd2_rn(st.l, p);
       st.zs = __ffma2_rn(p, zv[j], st.zs);
     }
@@ -500,72 +488,12 @@ __device__ __forceinline__ void fill_q_fragments(uint4 *s_frag, const float (*s_
   }
 }
 
-// One segment: the part [u_lo, u_hi) (units relative to the slice) of one slice that this CTA owns.
-// Builds the slice's query, runs the INT16 tiles and then the body tiles (width BITS) of the range,
-// merges the warps and publishes one partial per head; the CTA that publishes the slice's last
-// partial merges the slice.  The warps of the CTA draw work from two shared counters (INT16 tiles,
-// then body steps of NT tiles), so they all finish together whatever share of the issue slots
-// each of them gets.  `ring` is the CTA's dynamic shared memory: the per-warp cp.async stages while
-// tiles stream, then the warps' outputs.
-template <int BITS>
-__device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long long u_lo, long long u_hi,
-                                            float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint4 *s_frag,
-                                            uint8_t *ring) {
-  using F = Fmt<BITS>;
-  using F16 = Fmt<16>;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
-  const int b = slice / p.kv_heads, hkv = slice % p.kv_heads;
+// ---- pieces of a segment that both contraction paths share --------------------------------------
 
-  // (the previous segment ended with a CTA-wide barrier after its last use of s_q / s_stat / s_ctr / ring)
-  if (tid == 0) s_ctr[0] = s_ctr[1] = 0;
-  __syncthreads();
-
-  // ranges of this segment: INT16 tiles [a_lo, a_hi) (a tile belongs to the segment that holds its
-  // first unit) and body tiles [t_lo, t_hi)
-  int a_lo = 0, a_hi = 0, t_lo = 0, t_hi = 0;
-  if (u_lo < p.units_aux) {
-    a_lo = (int)((max(u_lo - p.units_lead, 0ll) + p.w16 - 1) / p.w16);
-    a_hi = (int)((min(u_hi, p.units_aux) - p.units_lead + p.w16 - 1) / p.w16);
-  }
-  if (u_hi > p.units_aux) {
-    t_lo = (int)(max(u_lo, p.units_aux) - p.units_aux);
-    t_hi = (int)(u_hi - p.units_aux);
-  }
-  const uint8_t *slice_base = p.geom.base + (size_t)slice * p.geom.slice_stride;
-
-  // ---- body stream set-up: claim the first steps and start their copies before anything else ----
-  constexpr int TB = tile_bytes(BITS);
-  constexpr int NT = F::NT, S = F::SLOTS > 0 ? F::SLOTS : 1, SB = NT * TB;
-  const int n_steps = (t_hi - t_lo + NT - 1) / NT;
-  const uint8_t *body = slice_base + p.geom.body_off;
-  uint8_t *my_ring = ring + (size_t)warp * S * SB;
-  const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
-  auto claim = [&](int which) { return claim_next(s_ctr + which, lane); };
-  auto issue = [&](int j, int slot) {
-    const int t = t_lo + NT * j;
-    const uint8_t *src = body + (size_t)t * TB + lane * 16;
-    const uint32_t dst = ring_addr + slot * SB + lane * 16;
-    const int n_tiles = t_hi - t;
-    if ((SB / 16) % 32 == 0 && n_tiles >= NT) {  // whole step, every lane copies the same number of chunks
-      cp_async_run<SB / 512>(dst, src);
-    } else {
-      const int n_chunks = min(NT, n_tiles) * (TB / 16);
-#pragma unroll
-      for (int c = 0; c < (SB / 16 + 31) / 32; ++c)
-        if (c * 32 + lane < n_chunks) cp_async16(dst + c * 512, src + c * 512);
-    }
-  };
-  int pending[S];  // steps claimed and in flight, oldest first (>= n_steps: none)
-  if constexpr (F::SLOTS > 0) {
-#pragma unroll
-    for (int i = 0; i < S - 1; ++i) {
-      pending[i] = n_steps > 0 ? claim(1) : 0;
-      if (pending[i] < n_steps) issue(pending[i], i);
-      cp_async_commit();
-    }
-  }
-
-  // ---- Q'' = Q * lambda * sm_scale * log2(e)  (Eq. 9: the equalization scale migrates into Q) ----
+// Q'' = Q * lambda * sm_scale * log2(e)  (Eq. 9: the equalization scale migrates into Q), per-head
+// exponent of max |q''| and sum of q''.  Ends with a CTA-wide barrier.
+__device__ __forceinline__ void build_query(const AttnParams &p, int b, int hkv, float (*s_q)[kHeadDim], float *s_stat) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   for (int i = tid; i < kMaxGroup * kHeadDim; i += kAttnThreads) {
     const int h = i >> 7, ch = i & 127;
     float v = 0.f;
@@ -576,7 +504,6 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
     s_q[h][ch] = v;
   }
   __syncthreads();
-
   if (warp < kMaxGroup) {  // per-head max |q''| and sum q''
     const float4 v = *reinterpret_cast<const float4 *>(&s_q[warp][lane * 4]);
     float mx = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
@@ -594,135 +521,71 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
     }
   }
   __syncthreads();
-  const int e_g = (int)s_stat[g];
-  const float sumq = s_stat[8 + g];
-  fill_q_fragments<16>(s_frag, s_q, s_stat);
-  if constexpr (BITS != 16) fill_q_fragments<BITS>(s_frag + 256, s_q, s_stat);
-  __syncthreads();
+}
 
-  // ---- unit of the V accumulators: a power of two >= every INT16 V scale of this slice; at width b
-  //      the scales are at most 2^SIGMA_LOG2 times larger ----
-  float sigma16 = 1.0f;
-  {
-    const float s16 = __uint_as_float(__ldcg(p.vmax_bits + slice));
-    if (s16 > 0.f) {
-      int e;
-      frexpf(s16, &e);
-      sigma16 = ldexpf(1.0f, e);
-    }
+// unit of the V accumulators: a power of two >= every INT16 V scale of this slice
+__device__ __forceinline__ float slice_sigma16(const AttnParams &p, int slice) {
+  const float s16 = __uint_as_float(__ldcg(p.vmax_bits + slice));
+  if (s16 > 0.f) {
+    int e;
+    frexpf(s16, &e);
+    return ldexpf(1.0f, e);
   }
+  return 1.0f;
+}
 
-  WarpState st;
-  st.m = kNegBig; st.l = make_float2(0.f, 0.f); st.zs = make_float2(0.f, 0.f);
-#pragma unroll
-  for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
+// The INT16 tiles [a_lo, a_hi) of a slice (sink tiles, then the window ring), drawn from the shared
+// counter s_ctr[0] by the warps of the CTA.
+__device__ __forceinline__ void run_int16_tiles(const AttnParams &p, const uint8_t *slice_base, int a_lo, int a_hi,
+                                                WarpState &st, const uint4 *s_frag, int *s_ctr, int e_g, float sumq,
+                                                float sigma16, int lane) {
+  using F16 = Fmt<16>;
+  int it = a_lo + claim_next(s_ctr, lane);
+  if (it >= a_hi) return;
   QFrag qa;
-
-  // ---- INT16 tiles (sink + window ring) ----
-  if (a_hi > a_lo) {
-    int it = a_lo + claim(0);
-    if (it < a_hi) {
-      qa.mine = s_frag + lane;
-      const float mu = ldexpf(1.0f, 24 - F16::EQ + e_g);
-      const float inv_sigma_e = ldexpf(1.0f, F16::EP) / sigma16;
-      const int n_win = p.n_tokens - p.win_start;
-      const int first_slot = n_win > 0 ? (p.win_start - p.geom.n_sink) % p.geom.ring_tokens : 0;
-      do {
-        uint32_t mask = 0;
-        const uint8_t *tile;
-        if (it < p.sink_tiles) {
-          const int live = max(0, min(16, p.n_sink_eff - 16 * it));
-          mask = (1u << live) - 1u;
-          tile = slice_base + (size_t)it * tile_bytes(16);
-        } else {
-          const int rt = it - p.sink_tiles;
-          tile = slice_base + p.geom.ring_off + (size_t)rt * tile_bytes(16);
-          if (n_win > 0) {
-            for (int r = 0; r < 16; ++r) {
-              int d = rt * 16 + r - first_slot;
-              if (d < 0) d += p.geom.ring_tokens;
-              if (d < n_win) mask |= 1u << r;
-            }
-          }
-        }
-        if (mask == 0xFFFFu) process_tiles<16, 1, false>(tile, mask, st, qa, mu, sumq, inv_sigma_e, lane);
-        else if (mask) process_tiles<16, 1, true>(tile, mask, st, qa, mu, sumq, inv_sigma_e, lane);
-        it = a_lo + claim(0);
-      } while (it < a_hi);
-      if constexpr (BITS != 16) {
-        // accumulator units change with the width: INT16 units -> body units (exact powers of two)
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-#pragma unroll
-          for (int rr = 0; rr < 2; ++rr) {
-            const float f = ldexpf(1.0f, F::EP - F16::EP + F::pos((2 * mt + rr) % F::N) - F::SIGMA_LOG2);
-            st.acc[mt][2 * rr] *= f;
-            st.acc[mt][2 * rr + 1] *= f;
-          }
-        }
-      }
-    }
-  }
-
-  // ---- body tiles ----
-  const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
-  if (n_steps > 0) {
-    qa.mine = (BITS != 16 ? s_frag + 256 : s_frag) + lane;
-    const float mu = ldexpf(1.0f, 24 - F::EQ + e_g);
-    const float inv_sigma_e = ldexpf(1.0f, F::EP) / sigma_u;
-    const uint32_t tail_mask = (p.n_body & 15) ? (1u << (p.n_body & 15)) - 1u : 0xFFFFu;
-    const int tail_tile = tail_mask != 0xFFFFu ? p.body_tiles - 1 : -1;  // the one tile with dead rows
-    if constexpr (F::SLOTS == 0) {
-      for (int t = t_lo + claim(1); t < t_hi; t = t_lo + claim(1)) {
-        const uint8_t *tile = body + (size_t)t * TB;
-        if (t == tail_tile) process_tiles<BITS, 1, true>(tile, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
-        else process_tiles<BITS, 1, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
-      }
+  qa.mine = s_frag + lane;
+  const float mu = ldexpf(1.0f, 24 - F16::EQ + e_g);
+  const float inv_sigma_e = ldexpf(1.0f, F16::EP) / sigma16;
+  const int n_win = p.n_tokens - p.win_start;
+  const int first_slot = n_win > 0 ? (p.win_start - p.geom.n_sink) % p.geom.ring_tokens : 0;
+  do {
+    uint32_t mask = 0;
+    const uint8_t *tile;
+    if (it < p.sink_tiles) {
+      const int live = max(0, min(16, p.n_sink_eff - 16 * it));
+      mask = (1u << live) - 1u;
+      tile = slice_base + (size_t)it * tile_bytes(16);
     } else {
-      int slot = 0, fill = S - 1;
-      while (pending[0] < n_steps) {
-        const int nxt = claim(1);
-        if (nxt < n_steps) issue(nxt, fill);
-        cp_async_commit();
-        cp_async_wait<S - 1>();
-        __syncwarp();
-        const uint8_t *tile = my_ring + slot * SB;
-        const int t = t_lo + NT * pending[0];
-        if (NT == 2 && t + 1 < t_hi && t + 1 != tail_tile) {
-          process_tiles<BITS, NT, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
-        } else {
-#pragma unroll
-          for (int k = 0; k < NT; ++k) {
-            if (t + k >= t_hi) break;
-            if (t + k == tail_tile)
-              process_tiles<BITS, 1, true>(tile + k * TB, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
-            else
-              process_tiles<BITS, 1, false>(tile + k * TB, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
-          }
+      const int rt = it - p.sink_tiles;
+      tile = slice_base + p.geom.ring_off + (size_t)rt * tile_bytes(16);
+      if (n_win > 0) {
+        for (int r = 0; r < 16; ++r) {
+          int d = rt * 16 + r - first_slot;
+          if (d < 0) d += p.geom.ring_tokens;
+          if (d < n_win) mask |= 1u << r;
         }
-        __syncwarp();
-#pragma unroll
-        for (int i = 0; i + 2 < S; ++i) pending[i] = pending[i + 1];
-        pending[S - 2] = nxt;
-        fill = slot;
-        slot = (slot + 1 == S) ? 0 : slot + 1;
       }
     }
-  }
-  if constexpr (F::SLOTS > 0) cp_async_wait<0>();
+    if (mask == 0xFFFFu) process_tiles<16, 1, false>(tile, mask, st, qa, mu, sumq, inv_sigma_e, lane);
+    else if (mask) process_tiles<16, 1, true>(tile, mask, st, qa, mu, sumq, inv_sigma_e, lane);
+    it = a_lo + claim_next(s_ctr, lane);
+  } while (it < a_hi);
+}
 
-  // ---- warp epilogue: quad sums, real units, to shared memory (the ring is free now) ----
+// A warp's running state -> its partial (m, l, o[128]) per head in real units, slot `slot`.
+// f_of(J) is the factor of accumulator column block J (channels 8 J + g).
+template <class FactorOf>
+__device__ __forceinline__ void store_warp_partial(const WarpState &st, FactorOf f_of, float (*s_o)[kMaxGroup][kHeadDim],
+                                                   float *s_m, float *s_l, int slot, int lane) {
+  const int g = lane >> 2, tig = lane & 3;
   float l_sum = st.l.x + st.l.y, zs_sum = st.zs.x + st.zs.y;
   l_sum += __shfl_xor_sync(0xffffffffu, l_sum, 1);
   l_sum += __shfl_xor_sync(0xffffffffu, l_sum, 2);
   zs_sum += __shfl_xor_sync(0xffffffffu, zs_sum, 1);
   zs_sum += __shfl_xor_sync(0xffffffffu, zs_sum, 2);
-  __syncthreads();  // every warp is done with its stages
-  float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(ring);
-  float *s_m = s_stat + 16, *s_l = s_stat + 16 + kAttnWarps * kMaxGroup;
   if (tig == 0) {
-    s_m[warp * 8 + g] = st.m;
-    s_l[warp * 8 + g] = l_sum;
+    s_m[slot * 8 + g] = st.m;
+    s_l[slot * 8 + g] = l_sum;
   }
   const float zs0 = __shfl_sync(0xffffffffu, zs_sum, (2 * tig) * 4);
   const float zs1 = __shfl_sync(0xffffffffu, zs_sum, (2 * tig + 1) * 4);
@@ -730,25 +593,27 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   for (int mt = 0; mt < 8; ++mt) {
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
-      const int J = 2 * mt + rr;
-      const float f = ldexpf(sigma_u, 24 - F::EP - F::pos(J % F::N));
+      const float f = f_of(2 * mt + rr);
       const int ch = 16 * mt + 8 * rr + g;
-      s_o[warp][2 * tig][ch] = fmaf(st.acc[mt][2 * rr], f, zs0);
-      s_o[warp][2 * tig + 1][ch] = fmaf(st.acc[mt][2 * rr + 1], f, zs1);
+      s_o[slot][2 * tig][ch] = fmaf(st.acc[mt][2 * rr], f, zs0);
+      s_o[slot][2 * tig + 1][ch] = fmaf(st.acc[mt][2 * rr + 1], f, zs1);
     }
   }
-  __syncthreads();
+}
 
-  // ---- merge the warps, publish the segment's partial ----
+// Merges the segment's n_parts partials (all written, a CTA-wide barrier passed), publishes the segment's
+// partial, and lets the CTA that publishes the slice's last partial merge the slice (nobody waits).
+__device__ __forceinline__ void publish_segment(const AttnParams &p, int slice, int n_parts,
+                                                const float (*s_o)[kMaxGroup][kHeadDim], const float *s_m, const float *s_l,
+                                                int *s_ctr) {
+  const int tid = threadIdx.x;
   float *part = p.partials + (size_t)((int)blockIdx.x - p.cta_origin + slice) * kMaxGroup * kPartialStride;
   for (int i = tid; i < p.group * kHeadDim; i += kAttnThreads) {
     const int h = i >> 7, ch = i & 127;
     float M = kNegBig;
-#pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, s_m[w * 8 + h]);
+    for (int w = 0; w < n_parts; ++w) M = fmaxf(M, s_m[w * 8 + h]);
     float o = 0.f, l = 0.f;
-#pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) {
+    for (int w = 0; w < n_parts; ++w) {
       const float wt = ex2(s_m[w * 8 + h] - M);
       o = fmaf(wt, s_o[w][h][ch], o);
       l = fmaf(wt, s_l[w * 8 + h], l);
@@ -759,8 +624,6 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
       __stcg(part + h * kPartialStride + 1, l);
     }
   }
-
-  // ---- the segment that publishes the slice's last partial merges the slice (nobody waits) ----
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -775,33 +638,278 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
     combine_slice(p, slice);
     if (tid == 0) p.tickets[slice] = 0u;  // ready for the next launch (stream order)
   }
-  __syncthreads();  // s_q, s_stat, s_ctr and the ring may be reused
+  __syncthreads();  // the segment's shared memory may be reused
+}
+
+// Ranges of a segment [u_lo, u_hi) (units relative to the slice): INT16 tiles [a_lo, a_hi) (a tile belongs to
+// the segment that holds its first unit) and body tiles [t_lo, t_hi).
+__device__ __forceinline__ void segment_ranges(const AttnParams &p, long long u_lo, long long u_hi, int &a_lo, int &a_hi,
+                                               int &t_lo, int &t_hi) {
+  a_lo = a_hi = t_lo = t_hi = 0;
+  if (u_lo < p.units_aux) {
+    a_lo = (int)((max(u_lo - p.units_lead, 0ll) + p.w16 - 1) / p.w16);
+    a_hi = (int)((min(u_hi, p.units_aux) - p.units_lead + p.w16 - 1) / p.w16);
+  }
+  if (u_hi > p.units_aux) {
+    t_lo = (int)(max(u_lo, p.units_aux) - p.units_aux);
+    t_hi = (int)(u_hi - p.units_aux);
+  }
+}
+
+// One segment with a 16- or 8-bit body: the part [u_lo, u_hi) (units relative to the slice) of one slice
+// that this CTA owns.  Builds the slice's query, runs the INT16 tiles and then the body tiles (width
+// BITS) of the range, merges the warps and publishes one partial per head.  The warps of the CTA draw
+// work from two shared counters (INT16 tiles, then body tiles), so they all finish together whatever share
+// of the issue slots each of them gets.  `ring` is the CTA's dynamic shared memory: the per-warp cp.async
+// stages while tiles stream, then the warps' outputs.
+template <int BITS>
+__device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long long u_lo, long long u_hi,
+                                            float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint4 *s_frag,
+                                            uint8_t *ring) {
+  static_assert(BITS == 16 || BITS == 8, "narrower bodies take the tensor-memory path");
+  using F = Fmt<BITS>;
+  using F16 = Fmt<16>;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2;
+  const int b = slice / p.kv_heads, hkv = slice % p.kv_heads;
+
+  // (the previous segment ended with a CTA-wide barrier after its last use of s_q / s_stat / s_ctr / ring)
+  if (tid == 0) s_ctr[0] = s_ctr[1] = 0;
+  __syncthreads();
+  int a_lo, a_hi, t_lo, t_hi;
+  segment_ranges(p, u_lo, u_hi, a_lo, a_hi, t_lo, t_hi);
+  const uint8_t *slice_base = p.geom.base + (size_t)slice * p.geom.slice_stride;
+
+  // ---- body stream set-up: claim the first tiles and start their copies before anything else ----
+  constexpr int TB = tile_bytes(BITS);
+  constexpr int S = F::SLOTS > 0 ? F::SLOTS : 1;
+  const int n_steps = t_hi - t_lo;
+  const uint8_t *body = slice_base + p.geom.body_off;
+  const size_t stream_stride = p.geom.stream_stride;
+  uint8_t *my_ring = ring + (size_t)warp * S * TB;
+  const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
+  auto claim = [&](int which) { return claim_next(s_ctr + which, lane); };
+  auto issue = [&](int j, int slot) {
+    const uint8_t *src = body + body_tile_offset(t_lo + j, BITS, stream_stride) + lane * 16;
+    const uint32_t dst = ring_addr + slot * TB + lane * 16;
+#pragma unroll
+    for (int c = 0; c < (TB / 16 + 31) / 32; ++c)
+      if (c * 32 + lane < TB / 16) cp_async16(dst + c * 512, src + c * 512);
+  };
+  int pending[S];  // tiles claimed and in flight, oldest first (>= n_steps: none)
+  if constexpr (F::SLOTS > 0) {
+#pragma unroll
+    for (int i = 0; i < S - 1; ++i) {
+      pending[i] = n_steps > 0 ? claim(1) : 0;
+      if (pending[i] < n_steps) issue(pending[i], i);
+      cp_async_commit();
+    }
+  }
+
+  build_query(p, b, hkv, s_q, s_stat);
+  const int e_g = (int)s_stat[g];
+  const float sumq = s_stat[8 + g];
+  fill_q_fragments<16>(s_frag, s_q, s_stat);
+  if constexpr (BITS != 16) fill_q_fragments<BITS>(s_frag + 256, s_q, s_stat);
+  __syncthreads();
+  const float sigma16 = slice_sigma16(p, slice);
+
+  WarpState st;
+  st.m = kNegBig; st.l = make_float2(0.f, 0.f); st.zs = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
+
+  // ---- INT16 tiles (sink + window ring) ----
+  if (a_hi > a_lo) {
+    run_int16_tiles(p, slice_base, a_lo, a_hi, st, s_frag, s_ctr, e_g, sumq, sigma16, lane);
+    if constexpr (BITS != 16) {
+      // accumulator units change with the width: INT16 units -> body units (exact powers of two)
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          const float f = ldexpf(1.0f, F::EP - F16::EP + F::pos((2 * mt + rr) % F::N) - F::SIGMA_LOG2);
+          st.acc[mt][2 * rr] *= f;
+          st.acc[mt][2 * rr + 1] *= f;
+        }
+      }
+    }
+  }
+
+  // ---- body tiles ----
+  const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
+  if (n_steps > 0) {
+    QFrag qa;
+    qa.mine = (BITS != 16 ? s_frag + 256 : s_frag) + lane;
+    const float mu = ldexpf(1.0f, 24 - F::EQ + e_g);
+    const float inv_sigma_e = ldexpf(1.0f, F::EP) / sigma_u;
+    const uint32_t tail_mask = (p.n_body & 15) ? (1u << (p.n_body & 15)) - 1u : 0xFFFFu;
+    const int tail_tile = tail_mask != 0xFFFFu ? p.body_tiles - 1 : -1;  // the one tile with dead rows
+    if constexpr (F::SLOTS == 0) {
+      for (int t = t_lo + claim(1); t < t_hi; t = t_lo + claim(1)) {
+        const uint8_t *tile = body + body_tile_offset(t, BITS, stream_stride);
+        if (t == tail_tile) process_tiles<BITS, 1, true>(tile, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
+        else process_tiles<BITS, 1, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+      }
+    } else {
+      int slot = 0, fill = S - 1;
+      while (pending[0] < n_steps) {
+        const int nxt = claim(1);
+        if (nxt < n_steps) issue(nxt, fill);
+        cp_async_commit();
+        cp_async_wait<S - 1>();
+        __syncwarp();
+        const uint8_t *tile = my_ring + slot * TB;
+        const int t = t_lo + pending[0];
+        if (t == tail_tile) process_tiles<BITS, 1, true>(tile, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
+        else process_tiles<BITS, 1, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i + 2 < S; ++i) pending[i] = pending[i + 1];
+        pending[S - 2] = nxt;
+        fill = slot;
+        slot = (slot + 1 == S) ? 0 : slot + 1;
+      }
+    }
+  }
+  if constexpr (F::SLOTS > 0) cp_async_wait<0>();
+
+  // ---- warp epilogue: quad sums, real units, to shared memory (the ring is free now) ----
+  __syncthreads();  // every warp is done with its stages
+  float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(ring);
+  float *s_m = s_stat + 16, *s_l = s_stat + 16 + kParts * kMaxGroup;
+  store_warp_partial(st, [&](int J) { return ldexpf(sigma_u, 24 - F::EP - F::pos(J % F::N)); }, s_o, s_m, s_l, warp, lane);
+  __syncthreads();
+  publish_segment(p, slice, kAttnWarps, s_o, s_m, s_l, s_ctr);
+}
+
+}  // namespace pmkvq
+#include "kernels_attn_tc.cuh"
+namespace pmkvq {
+
+// Dynamic shared memory of a CTA that may run the tensor-memory path.
+constexpr int kSmemStages = kWarpgroups * kStagesPerWg * kStageBytes;   // also the cp.async ring / outputs of the 8- and 16-bit path
+constexpr int kSmemQOperand = kSmemStages;
+constexpr int kSmemWBuf = kSmemQOperand + kQOperandBytes;
+constexpr int kSmemParts = kSmemWBuf + kWarpgroups * kWBufBytes;
+constexpr int kSmemTcTotal = kSmemParts + kParts * kMaxGroup * kHeadDim * 4;
+
+// One segment with a 4- or 2-bit body.  The INT16 tiles run as above, on the warps' own accumulators, and
+// every warp parks its partial in shared memory; the body runs on the tensor-memory path, one partial per
+// warpgroup.
+template <int BITS>
+__device__ __forceinline__ void run_segment_tc(const AttnParams &p, int slice, long long u_lo, long long u_hi,
+                                               float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint4 *s_frag,
+                                               TcCtx &tc) {
+  using F16 = Fmt<16>;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2;
+  const int b = slice / p.kv_heads, hkv = slice % p.kv_heads;
+  if (tid == 0) s_ctr[0] = s_ctr[1] = 0;
+  __syncthreads();
+  int a_lo, a_hi, t_lo, t_hi;
+  segment_ranges(p, u_lo, u_hi, a_lo, a_hi, t_lo, t_hi);
+  const uint8_t *slice_base = p.geom.base + (size_t)slice * p.geom.slice_stride;
+
+  build_query(p, b, hkv, s_q, s_stat);
+  if (a_hi > a_lo) fill_q_fragments<16>(s_frag, s_q, s_stat);
+  if (t_hi > t_lo) {
+    fill_q_operand<BITS>(tc.q_operand, s_q, s_stat);
+    tc05::fence_async_smem();
+  }
+  __syncthreads();
+  const float sigma16 = slice_sigma16(p, slice);
+  float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(tc.part_o);
+  float *s_m = s_stat + 16, *s_l = s_stat + 16 + kParts * kMaxGroup;
+
+  {
+    WarpState st;
+    st.m = kNegBig; st.l = make_float2(0.f, 0.f); st.zs = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
+    if (a_hi > a_lo) run_int16_tiles(p, slice_base, a_lo, a_hi, st, s_frag, s_ctr, (int)s_stat[g], s_stat[8 + g], sigma16, lane);
+    store_warp_partial(st, [&](int J) { return ldexpf(sigma16, 24 - F16::EP - F16::pos(J % F16::N)); }, s_o, s_m, s_l, warp, lane);
+  }
+  if (t_hi > t_lo) {
+    tc_body<BITS>(p, tc, slice_base + p.geom.body_off, t_lo, t_hi, s_stat, sigma16, s_m, s_l, kAttnWarps + (warp >> 2));
+  } else {
+    const int slot = kAttnWarps + (warp >> 2), tw = tid & 127;
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) s_o[slot][h][tw] = 0.f;
+    if (tw < kMaxGroup) { s_m[slot * 8 + tw] = kNegBig; s_l[slot * 8 + tw] = 0.f; }
+  }
+  __syncthreads();
+  publish_segment(p, slice, kParts, s_o, s_m, s_l, s_ctr);
 }
 
 template <int BITS>
-constexpr int attn_ring_bytes() {
-  // per-warp stages while streaming; at least the warps' outputs they are reused for
-  constexpr int out_bytes = kAttnWarps * kMaxGroup * kHeadDim * 4;
-  constexpr int ring = kAttnWarps * Fmt<BITS>::SLOTS * Fmt<BITS>::NT * tile_bytes(BITS);
-  return ring > out_bytes ? ring : out_bytes;
+constexpr int attn_smem_bytes() {
+  if constexpr (BITS <= 4) {
+    return kSmemTcTotal;
+  } else {
+    // per-warp stages while streaming; at least the warps' outputs they are reused for
+    constexpr int out_bytes = kAttnWarps * kMaxGroup * kHeadDim * 4;
+    constexpr int ring = kAttnWarps * Fmt<BITS>::SLOTS * tile_bytes(BITS);
+    return ring > out_bytes ? ring : out_bytes;
+  }
+}
+
+// CTA set-up of the tensor-memory path: barriers, tensor memory, the zero half of the weight operands.
+// Ends with a CTA-wide barrier.
+__device__ __forceinline__ void tc_setup(TcShared *sh, TcCtx &tc, uint8_t *ring, unsigned *error_word) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  tc.sh = sh;
+  tc.stages = ring;
+  tc.q_operand = ring + kSmemQOperand;
+  tc.wbuf = ring + kSmemWBuf;
+  tc.part_o = reinterpret_cast<float *>(ring + kSmemParts);
+  tc.error_word = error_word;
+  tc.ph_full = 0; tc.ph_s = 0; tc.ph_o = 0;
+  if (tid == 0) {
+    for (int w = 0; w < kWarpgroups; ++w) {
+      for (int s = 0; s < kStagesPerWg; ++s) tc05::mbar_init(tc05::smem_u32(&sh->bar_full[w][s]), 1);
+      tc05::mbar_init(tc05::smem_u32(&sh->bar_s[w]), 1);
+      tc05::mbar_init(tc05::smem_u32(&sh->bar_o[w]), 1);
+    }
+    sh->abort = 0;
+    tc05::mbar_init_fence();
+  }
+  if (warp == 0) tc05::tmem_alloc(tc05::smem_u32(&sh->tmem_base), kTmemCols);
+  for (int i = tid; i < kWarpgroups * kWBufBytes / 16; i += kAttnThreads)
+    reinterpret_cast<uint4 *>(tc.wbuf)[i] = make_uint4(0u, 0u, 0u, 0u);
+  tc05::fence_async_smem();
+  tc05::fence_before_sync();
+  __syncthreads();
+  tc05::fence_after_sync();
+  tc.tmem_base = sh->tmem_base;
+}
+__device__ __forceinline__ void tc_teardown(TcCtx &tc) {
+  tc05::fence_before_sync();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 0) tc05::tmem_dealloc(tc.tmem_base, kTmemCols);
 }
 
 template <int BODY_BITS>
-__global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(const AttnParams p, unsigned *error_word) {
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
-  __shared__ float s_stat[16 + 2 * kAttnWarps * kMaxGroup];  // head stats, per-warp (m, l)
-  __shared__ int s_ctr[4];                                    // work counters (INT16 tiles, body steps), combine flag
-  __shared__ uint4 s_frag[512];                               // query fragments at INT16 and at the body width
+  __shared__ float s_stat[16 + 2 * kParts * kMaxGroup];  // head stats, per-partial (m, l)
+  __shared__ int s_ctr[4];                                // work counters (INT16 tiles, body tiles), combine flag
+  __shared__ uint4 s_frag[512];                           // query fragments at INT16 and at the body width
+  __shared__ TcShared s_tc;
   extern __shared__ __align__(128) uint8_t ring[];
+  TcCtx tc;
+  if constexpr (BODY_BITS <= 4) tc_setup(&s_tc, tc, ring, error_word);
   const long long u_begin = (long long)blockIdx.x * p.units_per_cta;
   const long long u_end = min(u_begin + p.units_per_cta, p.units_total);
   for (long long u = u_begin; u < u_end;) {
     const int slice = (int)(u / p.units_slice);
     const long long base = (long long)slice * p.units_slice;
     const long long hi = min(u_end - base, p.units_slice);
-    if (hi > p.units_lead) run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
+    if (hi > p.units_lead) {
+      if constexpr (BODY_BITS <= 4) run_segment_tc<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc);
+      else run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
+    }
     u = base + hi;
   }
+  if constexpr (BODY_BITS <= 4) tc_teardown(tc);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -820,6 +928,7 @@ struct FusedParams {
   float *partials;            // per block, partial_stride floats apart
   float *out;                 // fp32 [layers][batch][q_heads][128]
   unsigned *tickets;          // [layers][n_slices]
+  unsigned *error_word;       // bits set by a wait that ran out
   size_t partial_stride;
   int layers, kv_heads, group, q_heads, n_slices, batch;
   int n_sink, window, evict_chunk, sink_tiles, ring_tiles;
@@ -863,10 +972,13 @@ __device__ __forceinline__ void fused_layer_params(const FusedParams &fp, int l,
 
 __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_fused_kernel(const __grid_constant__ FusedParams fp) {
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
-  __shared__ float s_stat[16 + 2 * kAttnWarps * kMaxGroup];
+  __shared__ float s_stat[16 + 2 * kParts * kMaxGroup];
   __shared__ int s_ctr[4];
   __shared__ uint4 s_frag[512];
+  __shared__ TcShared s_tc;
   extern __shared__ __align__(128) uint8_t ring[];
+  TcCtx tc;
+  tc_setup(&s_tc, tc, ring, fp.error_word);
   const long long f_begin = (long long)blockIdx.x * fp.per_cta;
   const long long f_end = min(f_begin + fp.per_cta, fp.total);
   int l = 0;
@@ -887,23 +999,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_fused_kernel(cons
         switch (p.cur_bits) {
           case 16: run_segment<16>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
           case 8: run_segment<8>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
-          case 4: run_segment<4>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
-          default: run_segment<2>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
+          case 4: run_segment_tc<4>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc); break;
+          default: run_segment_tc<2>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc); break;
         }
       }
       u = base + hi;
     }
     f = f_hi;
   }
+  tc_teardown(tc);
 }
 
-// the most dynamic shared memory any width needs
-constexpr int attn_fused_smem_bytes() {
-  int m = attn_ring_bytes<16>();
-  m = attn_ring_bytes<8>() > m ? attn_ring_bytes<8>() : m;
-  m = attn_ring_bytes<4>() > m ? attn_ring_bytes<4>() : m;
-  m = attn_ring_bytes<2>() > m ? attn_ring_bytes<2>() : m;
-  return m;
-}
+constexpr int attn_fused_smem_bytes() { return kSmemTcTotal; }
 
 }  // namespace pmkvq

@@ -16,6 +16,7 @@ struct LayerGeom {
   size_t slice_stride;  // bytes between (batch, kv_head) slices
   size_t ring_off;      // byte offset of the INT16 window ring inside a slice
   size_t body_off;      // byte offset of the body inside a slice
+  size_t stream_stride; // bytes between the eight interleaved streams of the body
   int n_sink;           // leading INT16 tokens (stored in tiles at offset 0)
   int ring_tokens;      // ring capacity in tokens (multiple of 16)
   int shift_variant;    // ShiftVariant of this cache
@@ -38,7 +39,7 @@ __device__ __forceinline__ TokenDest token_dest(const LayerGeom &g, uint8_t *sli
     d.bits = 16;
   } else if (t < win_start) {
     const int j = t - g.n_sink;
-    d.tile = slice + g.body_off + (size_t)(j >> 4) * tile_bytes(cur_bits);
+    d.tile = slice + g.body_off + body_tile_offset(j >> 4, cur_bits, g.stream_stride);
     d.row = j & 15;
     d.bits = cur_bits;
   } else {
@@ -106,13 +107,48 @@ __device__ __forceinline__ void store_token_w(uint8_t *part, int row, const uint
   }
 }
 
+// Row tiles (4 and 2 bit), K part: the token's 16*BITS bytes are its own; lane w builds word w.
+template <int BITS>
+__device__ __forceinline__ void store_key_row(uint8_t *k_part, int row, const uint16_t *codes16, int lane, int variant) {
+  constexpr int per_word = 32 / BITS, n_words = 4 * BITS;
+  if (lane < n_words) {
+    uint32_t val = 0;
+#pragma unroll
+    for (int i = 0; i < per_word; ++i)
+      val |= shift_chain(codes16[per_word * lane + i], BITS, variant) << (16 * (i & 1) + BITS * (i >> 1));
+    *reinterpret_cast<uint32_t *>(k_part + row * 16 * BITS + 4 * lane) = val;
+  }
+}
+// Row tiles, V part: a half-word of a channel's row holds the codes of 16/BITS tokens, so a token is
+// inserted by read-modify-write; lane l handles channels l, l+32, l+64, l+96.  Only ONE warp at a time may
+// insert tokens into a given tile (the callers below let the first token of a tile do the tile's others).
+template <int BITS>
+__device__ __forceinline__ void insert_value_row(uint8_t *v_part, int row, const uint16_t *codes16, int lane, int variant) {
+  int bo, sh;
+  row_slot(BITS, row, bo, sh);
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int ch = lane + 32 * j;
+    uint16_t *hw = reinterpret_cast<uint16_t *>(v_part + ch * 2 * BITS + bo);
+    const uint32_t v = *hw;
+    *hw = (uint16_t)((v & ~(mask << sh)) | (shift_chain(codes16[ch], BITS, variant) << sh));
+  }
+}
+
 __device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, const uint16_t *codes16, int is_value,
                                             int lane, int variant) {
   switch (bits) {
     case 16: store_token_w<16>(part, row, codes16, is_value, lane, variant); break;
     case 8: store_token_w<8>(part, row, codes16, is_value, lane, variant); break;
-    case 4: store_token_w<4>(part, row, codes16, is_value, lane, variant); break;
-    default: store_token_w<2>(part, row, codes16, is_value, lane, variant); break;
+    case 4:
+      if (is_value) insert_value_row<4>(part, row, codes16, lane, variant);
+      else store_key_row<4>(part, row, codes16, lane, variant);
+      break;
+    default:
+      if (is_value) insert_value_row<2>(part, row, codes16, lane, variant);
+      else store_key_row<2>(part, row, codes16, lane, variant);
+      break;
   }
 }
 
@@ -194,27 +230,46 @@ __device__ __forceinline__ float quantize_token16(uint2 raw, const float *__rest
   return scale;
 }
 
+// Writes the metadata of one stored token (S, Z of K or of V after the chain to `bits`).
+__device__ __forceinline__ void store_meta(uint8_t *tile, int bits, int row, int is_value, float s16, float z16, int variant) {
+  float *meta = reinterpret_cast<float *>(tile + meta_offset(bits));
+  meta[meta_slot(bits, is_value ? 2 : 0, row) >> 2] = chain_scale(s16, bits, variant);
+  meta[meta_slot(bits, is_value ? 3 : 1, row) >> 2] = chain_zero(z16, s16, bits, variant);
+}
+
+// One warp per (new token, slice, K|V) of the new tokens i0 .. i0 + n_cnt - 1.  Values that go straight
+// into a row tile of the body (4 and 2 bit) are inserted by read-modify-write of half-words that the
+// tile's tokens share, so the first such token of a tile inside the launch's range does the tile's
+// other tokens of the range too, one after the other, and their own warps leave.
 __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int lane, const uint16_t *__restrict__ K,
                                            const uint16_t *__restrict__ V, const float *__restrict__ inv_lambda,
                                            unsigned *vmax_bits, const LayerGeom &geom, int n_slices, int kv_heads,
-                                           int n_old, int win_start, int cur_bits, int i0 = 0) {
+                                           int n_old, int win_start, int cur_bits, int i0 = 0, int n_cnt = 1) {
   const int is_value = (int)(wid & 1);
   const long long ts = wid >> 1;
   const int slice = (int)(ts % n_slices);
-  const int i = i0 + (int)(ts / n_slices);  // index among the new tokens
-  const uint16_t *src = (is_value ? V : K) + ((size_t)i * n_slices + slice) * kHeadDim;
-  float mn;
-  const float scale = quantize_token16(src, is_value ? nullptr : inv_lambda + (size_t)(slice % kv_heads) * kHeadDim, codes,
-                                       lane, mn);
-  __syncwarp();
+  int i = i0 + (int)(ts / n_slices);  // index among the new tokens
   uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
-  const TokenDest d = token_dest(geom, slice_base, n_old + i, win_start, cur_bits);
-  store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, codes, is_value, lane, geom.shift_variant);
-  if (lane == 0) {
-    float *meta = reinterpret_cast<float *>(d.tile + meta_offset(d.bits));
-    meta[meta_slot(is_value ? 2 : 0, d.row) >> 2] = chain_scale(scale, d.bits, geom.shift_variant);
-    meta[meta_slot(is_value ? 3 : 1, d.row) >> 2] = chain_zero(mn, scale, d.bits, geom.shift_variant);
-    if (is_value) atomicMax(vmax_bits + slice, __float_as_uint(scale));  // scale >= 0: uint order = float order
+  int t = n_old + i, last = t;
+  const bool shared_rows = is_value && t >= geom.n_sink && t < win_start && row_layout(cur_bits);
+  if (shared_rows) {
+    const int j = t - geom.n_sink;
+    if (i != i0 && (j & 15) != 0) return;  // an earlier token of this tile does this one
+    last = min(min(n_old + i0 + n_cnt, win_start), geom.n_sink + (j | 15) + 1) - 1;
+  }
+  for (; t <= last; ++t, ++i) {
+    const uint16_t *src = (is_value ? V : K) + ((size_t)i * n_slices + slice) * kHeadDim;
+    float mn;
+    const float scale = quantize_token16(src, is_value ? nullptr : inv_lambda + (size_t)(slice % kv_heads) * kHeadDim,
+                                         codes, lane, mn);
+    __syncwarp();
+    const TokenDest d = token_dest(geom, slice_base, t, win_start, cur_bits);
+    store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, codes, is_value, lane, geom.shift_variant);
+    if (lane == 0) {
+      store_meta(d.tile, d.bits, d.row, is_value, scale, mn, geom.shift_variant);
+      if (is_value) atomicMax(vmax_bits + slice, __float_as_uint(scale));  // scale >= 0: uint order = float order
+    }
+    __syncwarp();
   }
 }
 
@@ -227,7 +282,8 @@ __global__ void __launch_bounds__(128) append_kernel(const uint16_t *__restrict_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wid = (long long)blockIdx.x * 4 + warp;
   if (wid >= (long long)n_new * n_slices * 2) return;
-  append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits, i0);
+  append_one(wid, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start, cur_bits, i0,
+             n_new);
 }
 
 // Bulk appends (prefill): body tiles that consist of new tokens only are built whole, one warp per
@@ -365,10 +421,108 @@ __device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ sr
   }
 }
 
+// The same for row tiles (4 and 2 bit).  Lane 4 r' + q quantizes channels [32 q, 32 q + 32) of token
+// 8 rr + r' (two rounds rr); a token's minimum and maximum meet inside a quad.  Keys leave as the token's own
+// words.  Values are transposed through `scratch` (16 x 128 code bytes of this warp): afterwards lane l
+// builds the words of channels l, l + 32, l + 64, l + 96, whose halves interleave the tile's tokens.
+template <int BITS>
+__device__ __forceinline__ void append_tile_half_row(const uint16_t *__restrict__ src, size_t row_stride,
+                                                     const float *__restrict__ il, uint8_t *dst_tile, int is_value,
+                                                     unsigned *vmax_slot, int lane, int variant, uint8_t *scratch) {
+  constexpr int per_word = 32 / BITS, words_per_lane = 32 / per_word;
+  const int rq = lane >> 2, q = lane & 3;
+  float smax = 0.f;
+#pragma unroll 1
+  for (int rr = 0; rr < 2; ++rr) {
+    const int row = 8 * rr + rq;
+    float x[32];
+    const uint4 *rp = reinterpret_cast<const uint4 *>(src + (size_t)row * row_stride + 32 * q);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint4 raw = rp[c];
+      const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        x[8 * c + 2 * e] = __uint_as_float(w4[e] << 16);
+        x[8 * c + 2 * e + 1] = __uint_as_float(w4[e] & 0xFFFF0000u);
+      }
+    }
+    if (!is_value) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float4 l4 = __ldg(reinterpret_cast<const float4 *>(il + 32 * q) + c);  // Lambda^-1, L1-resident
+        x[4 * c] = __fmul_rn(x[4 * c], l4.x); x[4 * c + 1] = __fmul_rn(x[4 * c + 1], l4.y);
+        x[4 * c + 2] = __fmul_rn(x[4 * c + 2], l4.z); x[4 * c + 3] = __fmul_rn(x[4 * c + 3], l4.w);
+      }
+    }
+    float mn = x[0], mx = x[0];
+#pragma unroll
+    for (int i = 1; i < 32; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    const float s16 = quantize_owned<BITS>(x, mn, mx, variant);
+    if (!is_value) {
+      uint32_t words[words_per_lane];
+#pragma unroll
+      for (int w = 0; w < words_per_lane; ++w) {
+        uint32_t a = 0;
+#pragma unroll
+        for (int i = 0; i < per_word; ++i) a |= __float_as_uint(x[per_word * w + i]) << (16 * (i & 1) + BITS * (i >> 1));
+        words[w] = a;
+      }
+      uint8_t *dst = dst_tile + row * 16 * BITS + q * 4 * words_per_lane;
+      if constexpr (words_per_lane == 2) *reinterpret_cast<uint2 *>(dst) = make_uint2(words[0], words[1]);
+      else *reinterpret_cast<uint4 *>(dst) = make_uint4(words[0], words[1], words[2], words[3]);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t b4[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          b4[e] = __float_as_uint(x[16 * c + 4 * e]) | (__float_as_uint(x[16 * c + 4 * e + 1]) << 8) |
+                  (__float_as_uint(x[16 * c + 4 * e + 2]) << 16) | (__float_as_uint(x[16 * c + 4 * e + 3]) << 24);
+        *reinterpret_cast<uint4 *>(scratch + row * kHeadDim + 32 * q + 16 * c) = make_uint4(b4[0], b4[1], b4[2], b4[3]);
+      }
+      smax = fmaxf(smax, s16);
+    }
+    if (q == 0) {
+      float *rec = reinterpret_cast<float *>(dst_tile + meta_offset(BITS) + row * 16) + (is_value ? 2 : 0);
+      *reinterpret_cast<float2 *>(rec) = make_float2(chain_scale(s16, BITS, variant), chain_zero(mn, s16, BITS, variant));
+    }
+  }
+  if (is_value) {
+    __syncwarp();
+    constexpr int words_per_ch = BITS / 2;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int ch = lane + 32 * j;
+      uint32_t words[words_per_ch];
+#pragma unroll
+      for (int w = 0; w < words_per_ch; ++w) {
+        uint32_t a = 0;
+#pragma unroll
+        for (int i = 0; i < per_word; ++i) a |= (uint32_t)scratch[(per_word * w + i) * kHeadDim + ch] << (16 * (i & 1) + BITS * (i >> 1));
+        words[w] = a;
+      }
+      uint8_t *dst = dst_tile + v_part_offset(BITS) + ch * 2 * BITS;
+      if constexpr (words_per_ch == 1) *reinterpret_cast<uint32_t *>(dst) = words[0];
+      else *reinterpret_cast<uint2 *>(dst) = make_uint2(words[0], words[1]);
+    }
+#pragma unroll
+    for (int o = 1; o <= 16; o <<= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+    if (lane == 0) atomicMax(vmax_slot, __float_as_uint(smax));  // scale >= 0: uint order = float order
+    __syncwarp();
+  }
+}
+
 __global__ void __launch_bounds__(128, 8) append_tiles_kernel(const uint16_t *__restrict__ K, const uint16_t *__restrict__ V,
                                                            const float *__restrict__ inv_lambda, unsigned *vmax_bits,
                                                            LayerGeom geom, int n_slices, int kv_heads, int n_old,
                                                            int tile_lo, int n_tiles, int bits) {
+  __shared__ __align__(16) uint8_t s_scratch[4][kTileTokens * kHeadDim];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wid = (long long)blockIdx.x * 4 + warp;
   if (wid >= (long long)n_tiles * n_slices * 2) return;
@@ -379,42 +533,48 @@ __global__ void __launch_bounds__(128, 8) append_tiles_kernel(const uint16_t *__
   const size_t row_stride = (size_t)n_slices * kHeadDim;
   const uint16_t *src = (is_value ? V : K) + ((size_t)i0 * n_slices + slice) * kHeadDim;
   const float *il = inv_lambda + (size_t)(slice % kv_heads) * kHeadDim;
-  uint8_t *dst_tile = geom.base + (size_t)slice * geom.slice_stride + geom.body_off + (size_t)tile * tile_bytes(bits);
+  uint8_t *dst_tile = geom.base + (size_t)slice * geom.slice_stride + geom.body_off + body_tile_offset(tile, bits, geom.stream_stride);
   switch (bits) {
     case 16: append_tile_half<16>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
     case 8: append_tile_half<8>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
-    case 4: append_tile_half<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
-    default: append_tile_half<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
+    case 4: append_tile_half_row<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]); break;
+    default: append_tile_half_row<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]); break;
   }
 }
 
 // ---------------------------------------------------------------------------------------------
 // Window eviction.  One warp per (evicted token, slice, K|V): the INT16 token leaves the ring and
-// enters the body at the body width through the Eq. 3 chain (16 -> 8 -> ... -> cur_bits).
+// enters the body at the body width through the Eq. 3 chain (16 -> 8 -> ... -> cur_bits).  Values that
+// enter a row tile share half-words with the tile's other tokens: the first evicted token of a tile does
+// the tile's other evicted tokens too, and their own warps leave (see append_one).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void evict_one(long long wid, uint16_t *codes, int lane, const LayerGeom &geom, int n_slices,
-                                          int first_token, int cur_bits) {
+                                          int first_token, int n_evict, int cur_bits) {
   const int is_value = (int)(wid & 1);
   const long long ts = wid >> 1;
   const int slice = (int)(ts % n_slices);
-  const int t = first_token + (int)(ts / n_slices);
+  int t = first_token + (int)(ts / n_slices), last = t;
   uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
-  const int rp = (t - geom.n_sink) % geom.ring_tokens;
-  const uint8_t *src_tile = slice_base + geom.ring_off + (size_t)(rp >> 4) * tile_bytes(16);
-  const int src_row = rp & 15;
-  load_token16(src_tile + (is_value ? v_part_offset(16) : 0), src_row, codes, is_value, lane);
-  const float *smeta = reinterpret_cast<const float *>(src_tile + meta_offset(16));
-  const float s16 = smeta[meta_slot(is_value ? 2 : 0, src_row) >> 2];
-  const float z = smeta[meta_slot(is_value ? 3 : 1, src_row) >> 2];
-  __syncwarp();
-  const int j = t - geom.n_sink;
-  uint8_t *dst_tile = slice_base + geom.body_off + (size_t)(j >> 4) * tile_bytes(cur_bits);
-  store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, codes, is_value, lane,
-              geom.shift_variant);
-  if (lane == 0) {
-    float *meta = reinterpret_cast<float *>(dst_tile + meta_offset(cur_bits));
-    meta[meta_slot(is_value ? 2 : 0, j & 15) >> 2] = chain_scale(s16, cur_bits, geom.shift_variant);
-    meta[meta_slot(is_value ? 3 : 1, j & 15) >> 2] = chain_zero(z, s16, cur_bits, geom.shift_variant);
+  if (is_value && row_layout(cur_bits)) {
+    const int j = t - geom.n_sink;
+    if (t != first_token && (j & 15) != 0) return;
+    last = min(first_token + n_evict, geom.n_sink + (j | 15) + 1) - 1;
+  }
+  for (; t <= last; ++t) {
+    const int rp = (t - geom.n_sink) % geom.ring_tokens;
+    const uint8_t *src_tile = slice_base + geom.ring_off + (size_t)(rp >> 4) * tile_bytes(16);
+    const int src_row = rp & 15;
+    load_token16(src_tile + (is_value ? v_part_offset(16) : 0), src_row, codes, is_value, lane);
+    const float *smeta = reinterpret_cast<const float *>(src_tile + meta_offset(16));
+    const float s16 = smeta[meta_slot(16, is_value ? 2 : 0, src_row) >> 2];
+    const float z = smeta[meta_slot(16, is_value ? 3 : 1, src_row) >> 2];
+    __syncwarp();
+    const int j = t - geom.n_sink;
+    uint8_t *dst_tile = slice_base + geom.body_off + body_tile_offset(j >> 4, cur_bits, geom.stream_stride);
+    store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, codes, is_value, lane,
+                geom.shift_variant);
+    if (lane == 0) store_meta(dst_tile, cur_bits, j & 15, is_value, s16, z, geom.shift_variant);
+    __syncwarp();
   }
 }
 
@@ -424,13 +584,14 @@ __global__ void __launch_bounds__(128) evict_kernel(LayerGeom geom, int n_slices
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wid = (long long)blockIdx.x * 4 + warp;
   if (wid >= (long long)n_evict * n_slices * 2) return;
-  evict_one(wid, s_codes[warp], lane, geom, n_slices, first_token, cur_bits);
+  evict_one(wid, s_codes[warp], lane, geom, n_slices, first_token, n_evict, cur_bits);
 }
 
 // One decode step's cache update in a single launch: the tokens that leave the window (warps
 // [0, 2 n_evict n_slices)) and the one new token (the rest).  Only valid when no evicted token
-// shares its ring slot with the new token, which holds for single-token appends (the ring is larger
-// than window + evict_chunk).
+// shares its ring slot with the new token (single-token appends: the ring is larger than window +
+// evict_chunk) and the new token does not enter a body tile that an evicted token enters too (the host
+// sends the one configuration where that happens, window = 0 with evict_chunk > 1, through two launches).
 __global__ void __launch_bounds__(128) append_decode_kernel(const uint16_t *__restrict__ K,
                                                             const uint16_t *__restrict__ V,
                                                             const float *__restrict__ inv_lambda, unsigned *vmax_bits,
@@ -441,18 +602,13 @@ __global__ void __launch_bounds__(128) append_decode_kernel(const uint16_t *__re
   const long long wid = (long long)blockIdx.x * 4 + warp;
   const long long n_ev = (long long)n_evict * n_slices * 2;
   if (wid < n_ev) {
-    evict_one(wid, s_codes[warp], lane, geom, n_slices, first_evicted, cur_bits);
+    evict_one(wid, s_codes[warp], lane, geom, n_slices, first_evicted, n_evict, cur_bits);
   } else if (wid < n_ev + 2ll * n_slices) {
     append_one(wid - n_ev, s_codes[warp], lane, K, V, inv_lambda, vmax_bits, geom, n_slices, kv_heads, n_old, win_start,
                cur_bits);
   }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Progressive reduce 2B -> B (Eq. 3) of one tile, by one warp.  Lane-local: two adjacent words of
-// a lane at 2B bits become one word at B bits.  Everything is read and transformed before the
-// first store, so the output may overlap this tile's own input.
-// ---------------------------------------------------------------------------------------------
 // ---------------------------------------------------------------------------------------------
 // One decode step's cache update for ALL blocks in a single launch.  The blocks' geometry is a
 // table in device memory (written once when the cache is created); their token counts and widths
@@ -487,7 +643,7 @@ __global__ void __launch_bounds__(128) append_step_kernel(const uint16_t *__rest
   const int ev_first = max(old_ws, n_sink), n_evict = max(0, min(new_ws, n_old) - ev_first);
   const long long ev_room = 2ll * evict_chunk * n_slices;
   if (w < ev_room) {
-    if (w < 2ll * n_evict * n_slices) evict_one(w, s_codes[warp], lane, geom, n_slices, ev_first, cur_bits);
+    if (w < 2ll * n_evict * n_slices) evict_one(w, s_codes[warp], lane, geom, n_slices, ev_first, n_evict, cur_bits);
   } else {
     const size_t in_off = (size_t)layer * n_slices * kHeadDim;
     append_one(w - ev_room, s_codes[warp], lane, K + in_off, V + in_off, inv_lambda + (size_t)layer * kv_heads * kHeadDim,
@@ -495,6 +651,11 @@ __global__ void __launch_bounds__(128) append_step_kernel(const uint16_t *__rest
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Progressive reduce 2B -> B (Eq. 3) of one tile, by one warp: two adjacent words at 2B bits become
+// one word at B bits.  Everything is read and transformed before the first store, so the output may
+// overlap this tile's own input.
+// ---------------------------------------------------------------------------------------------
 template <int B, bool SHR>
 __device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1) {
   constexpr int NIN = 8 / B;  // codes per half-word at 2B bits
@@ -575,31 +736,151 @@ __device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int
   else reduce_tile_v<B, true, CTA_WIDE>(in, out, lane, variant, active);
 }
 
-// First tiles of every slice, one CTA per slice, in batches of one tile per warp, batch after batch: the
-// outputs of batch j (tiles [W j, W j + W) at B bits) end at (W j + W) tile_bytes(B), below the first input
-// of batch j + 1, and overlap inputs of batches <= j only, which the barrier inside reduce_tile has seen
-// loaded.
-constexpr int kReduceHeadWarps = 16;
-template <int B>
-__global__ void __launch_bounds__(kReduceHeadWarps * 32) reduce_head_kernel(LayerGeom geom, int n_tiles) {
-  uint8_t *body = geom.base + (size_t)blockIdx.x * geom.slice_stride + geom.body_off;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int i0 = 0; i0 < n_tiles; i0 += kReduceHeadWarps) {
-    const int i = i0 + warp;
-    reduce_tile<B, true>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), lane, geom.shift_variant,
-                         i < n_tiles);
+// Row tile at 4 bit -> row tile at 2 bit: in both parts the words of a row pair up (a token row has 16
+// words, a channel row 2), so the tile is a flat array of word pairs; a lane takes four words at a time.
+template <bool SHR>
+__device__ __forceinline__ void reduce_tile_row(const uint8_t *in, uint8_t *out, int lane, int variant, bool active) {
+  uint2 o[2][2];
+  float4 m = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (active) {
+#pragma unroll
+    for (int part = 0; part < 2; ++part)
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const uint4 v = *reinterpret_cast<const uint4 *>(in + part * code_part_bytes(4) + (q * 32 + lane) * 16);
+        o[part][q] = make_uint2(merge_words<2, SHR>(v.x, v.y), merge_words<2, SHR>(v.z, v.w));
+      }
+    if (lane < 16) {
+      m = *reinterpret_cast<const float4 *>(in + meta_offset(4) + lane * 16);
+      halve_meta(m.x, m.y, 2, variant);
+      halve_meta(m.z, m.w, 2, variant);
+    }
   }
+  __syncthreads();  // every warp of the CTA holds its transformed tile: the inputs are dead from here on
+  if (!active) return;
+#pragma unroll
+  for (int part = 0; part < 2; ++part)
+#pragma unroll
+    for (int q = 0; q < 2; ++q) *reinterpret_cast<uint2 *>(out + part * code_part_bytes(2) + (q * 32 + lane) * 8) = o[part][q];
+  if (lane < 16) *reinterpret_cast<float4 *>(out + meta_offset(2) + lane * 16) = m;
 }
 
-// One wave: tiles [lo, hi) of every slice, one warp per tile.  The host picks the waves so that
-// hi * tile_bytes(B) <= lo * tile_bytes(2B): no output of the wave lands on an input of the wave.
+// Lane-owned tile at 8 bit -> row tile at 4 bit.  The 4-bit codes go through `scratch` (16 x 128 code
+// bytes of this warp, one part at a time), from which the lanes gather the row words.
+template <bool SHR>
+__device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *out, int lane, int variant, bool active,
+                                                   uint8_t *scratch) {
+  const int g = lane >> 2, tig = lane & 3;
+  uint4 ko[4];       // K part: this lane's 16 bytes of rows lane / 2 (+ 0, 1 ... see below)
+  uint2 vo[4];       // V part: channels lane, lane + 32, ...
+  float m[8];        // metadata records
+  if (active) {
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+      const uint8_t *src = in + part * code_part_bytes(8);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 v = *reinterpret_cast<const uint4 *>(src + (q * 32 + lane) * 16);
+        const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int lw = 4 * q + e, r = lw >> 3, w = lw & 7;
+#pragma unroll
+          for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              const uint32_t c8 = (w4[e] >> (16 * h + 8 * j)) & 0xFFu;
+              const uint32_t c4 = SHR ? c8 >> 4 : shift_step(c8, 4);
+              const int idx = 2 * w + j;
+              const int row = part == 0 ? g + 8 * r : 2 * tig + 8 * r + h;
+              const int ch = part == 0 ? 8 * idx + 2 * tig + h : 8 * idx + g;
+              scratch[row * kHeadDim + ch] = (uint8_t)c4;
+            }
+        }
+      }
+      __syncwarp();
+      if (part == 0) {
+        // K rows: 16 rows x 16 words; lane l builds words 4 (l & 3) .. + 3 of rows (l >> 2) and (l >> 2) + 8
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          const int row = (lane >> 2) + 8 * rr;
+          uint32_t wd[4];
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            const uint2 b = *reinterpret_cast<const uint2 *>(scratch + row * kHeadDim + 8 * (4 * (lane & 3) + w));
+            uint32_t a = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint32_t c = ((i < 4 ? b.x : b.y) >> (8 * (i & 3))) & 0xFu;
+              a |= c << (16 * (i & 1) + 4 * (i >> 1));
+            }
+            wd[w] = a;
+          }
+          ko[rr] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int ch = lane + 32 * j;
+          uint32_t wd[2];
+#pragma unroll
+          for (int w = 0; w < 2; ++w) {
+            uint32_t a = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) a |= (uint32_t)scratch[(8 * w + i) * kHeadDim + ch] << (16 * (i & 1) + 4 * (i >> 1));
+            wd[w] = a;
+          }
+          vo[j] = make_uint2(wd[0], wd[1]);
+        }
+      }
+      __syncwarp();
+    }
+    // metadata: lane-owned records {S_K[4], Z_K[4], S_V[4], Z_V[4]} per tig -> rows; lane l < 16 takes token row l
+    if (lane < 16) {
+      const float *mi = reinterpret_cast<const float *>(in + meta_offset(8));
+#pragma unroll
+      for (int kind = 0; kind < 4; ++kind) m[kind] = mi[meta_slot(8, kind, lane) >> 2];
+      halve_meta(m[0], m[1], 4, variant);
+      halve_meta(m[2], m[3], 4, variant);
+    }
+  }
+  __syncthreads();  // every warp of the CTA holds its transformed tile: the inputs are dead from here on
+  if (!active) return;
+#pragma unroll
+  for (int rr = 0; rr < 2; ++rr)
+    *reinterpret_cast<uint4 *>(out + ((lane >> 2) + 8 * rr) * 64 + 16 * (lane & 3)) = ko[rr];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) *reinterpret_cast<uint2 *>(out + v_part_offset(4) + (lane + 32 * j) * 8) = vo[j];
+  if (lane < 16) *reinterpret_cast<float4 *>(out + meta_offset(4) + lane * 16) = make_float4(m[0], m[1], m[2], m[3]);
+}
+
+// The whole body of a block in one launch: one CTA per (stream, slice) walks its stream front to back in
+// batches of one tile per warp.  Inside a stream tile j moves from j tile_bytes(2B) to j tile_bytes(B):
+// the outputs of a batch end below the inputs of every later batch and overlap inputs of this and earlier
+// batches only, which the CTA-wide barrier between a batch's loads and its stores has seen loaded.
+constexpr int kReduceWarps = 8;
 template <int B>
-__global__ void __launch_bounds__(128) reduce_wave_kernel(LayerGeom geom, int lo, int hi) {
-  const int i = lo + blockIdx.x * 4 + (threadIdx.x >> 5);
-  if (i >= hi) return;
-  uint8_t *body = geom.base + (size_t)blockIdx.y * geom.slice_stride + geom.body_off;
-  reduce_tile<B>(body + (size_t)i * tile_bytes(2 * B), body + (size_t)i * tile_bytes(B), threadIdx.x & 31,
-                 geom.shift_variant);
+__global__ void __launch_bounds__(kReduceWarps * 32) reduce_stream_kernel(LayerGeom geom, int n_tiles) {
+  __shared__ __align__(16) uint8_t s_scratch[B == 4 ? kReduceWarps : 1][B == 4 ? kTileTokens * kHeadDim : 16];
+  const int stream = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint8_t *base = geom.base + (size_t)blockIdx.y * geom.slice_stride + geom.body_off + (size_t)stream * geom.stream_stride;
+  const int cnt = (n_tiles - stream + kStreams - 1) / kStreams;  // tiles of this stream
+  const bool shr = geom.shift_variant != kShiftEquivalent;
+  for (int j0 = 0; j0 < cnt; j0 += kReduceWarps) {
+    const int j = j0 + warp;
+    const bool active = j < cnt;
+    const uint8_t *in = base + (size_t)j * tile_bytes(2 * B);
+    uint8_t *out = base + (size_t)j * tile_bytes(B);
+    if constexpr (B == 8) {
+      reduce_tile<8, true>(in, out, lane, geom.shift_variant, active);
+    } else if constexpr (B == 4) {
+      if (shr) reduce_tile_to_row<true>(in, out, lane, geom.shift_variant, active, s_scratch[warp]);
+      else reduce_tile_to_row<false>(in, out, lane, geom.shift_variant, active, s_scratch[warp]);
+    } else {
+      if (shr) reduce_tile_row<true>(in, out, lane, geom.shift_variant, active);
+      else reduce_tile_row<false>(in, out, lane, geom.shift_variant, active);
+    }
+  }
 }
 
 }  // namespace pmkvq

@@ -21,7 +21,6 @@ using namespace pmkvq;
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr int kHeadTiles = 256;   // tiles the reduce handles batch by batch (one CTA per slice) before the parallel waves start
 constexpr int kMaxCtas = 1024;      // upper bound on the attention grid (sizes the partials workspace)
 // Fixed cost of one more segment (set-up, warp merge, publish, its share of the slice combine), in
 // body tiles of each width: about 12 us at the measured per-SM tile rates.
@@ -38,7 +37,7 @@ struct Layer {
   uint64_t budget = 0;
   size_t offset = 0;        // of the first slice inside the arena
   size_t slice_stride = 0;
-  size_t body_cap = 0;      // bytes of body per slice
+  size_t stream_stride = 0; // bytes of each of the body's eight interleaved streams (capacity of a stream)
 };
 
 }  // namespace
@@ -51,6 +50,7 @@ struct pmkvq_cache {
   size_t arena_bytes;
   // arena sections
   size_t off_lambda, off_inv_lambda, off_vmax, off_tickets, off_partials, partial_bytes, off_geoms;  // scratch is per block
+  size_t off_error;  // one word: bits set by a device-side wait that ran out
   int sink_tiles, ring_tiles, user_ctas;
   int resident_ctas[4];  // one wave of the attention kernel at body width 16, 8, 4, 2
   int resident_fused;    // one wave of the all-blocks attention kernel
@@ -79,6 +79,7 @@ struct pmkvq_cache {
     g.slice_stride = l.slice_stride;
     g.ring_off = (size_t)sink_tiles * tile_bytes(16);
     g.body_off = g.ring_off + (size_t)ring_tiles * tile_bytes(16);
+    g.stream_stride = l.stream_stride;
     g.n_sink = n_sink;
     g.ring_tokens = ring_tiles * 16;
     g.shift_variant = shift_variant;
@@ -133,13 +134,15 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.partial_bytes = align_up(((size_t)kMaxCtas + (size_t)k.n_slices) * kMaxGroup * kPartialStride * sizeof(float), kAlign);
   k.off_partials = off; off = align_up(off + k.partial_bytes * k.layers, kAlign);
   k.off_geoms = off; off = align_up(off + (size_t)k.layers * sizeof(LayerGeom), kAlign);
+  k.off_error = off; off = align_up(off + sizeof(unsigned), kAlign);
 
   k.L.assign(k.layers, Layer());
   for (int i = 0; i < k.layers; ++i) {
     Layer &l = k.L[i];
     l.fbit = c->fbit[i];
     l.budget = c->budget_bytes ? c->budget_bytes[i] : k.default_budget(l.fbit);
-    // body capacity: the most tiles the policy can ever ask for at any width of the chain
+    // body capacity: the most tiles the policy can ever ask for at any width of the chain, dealt out
+    // over the eight streams (tile i sits in stream i mod 8)
     size_t cap = 0;
     for (int b = 16; b >= l.fbit; b >>= 1) {
       int lo = 0, hi = k.max_tokens;  // largest n with bytes_at(n, b) <= budget (bytes_at is monotone enough
@@ -151,10 +154,11 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
       int nb = 0;
       for (int n = std::max(0, lo - 2 * k.evict_chunk); n <= std::min(k.max_tokens, lo + 2 * k.evict_chunk); ++n)
         if (k.bytes_at(n, b) <= l.budget) nb = std::max(nb, k.body_at(n));
-      cap = std::max(cap, (size_t)((nb + 15) / 16) * tile_bytes(b));
+      const size_t tiles = (size_t)((nb + 15) / 16);
+      cap = std::max(cap, (tiles + kStreams - 1) / kStreams * tile_bytes(b));
     }
-    l.body_cap = cap;
-    l.slice_stride = align_up((size_t)(k.sink_tiles + k.ring_tiles) * tile_bytes(16) + cap, kAlign);
+    l.stream_stride = align_up(cap, kAlign);
+    l.slice_stride = align_up((size_t)(k.sink_tiles + k.ring_tiles) * tile_bytes(16) + l.stream_stride * kStreams, kAlign);
     l.offset = off;
     off = align_up(off + l.slice_stride * k.n_slices, kAlign);
   }
@@ -163,30 +167,20 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
 
 template <int B>
 cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStream_t st, uint64_t &launches) {
-  const int head = std::min(n_tiles, B == 8 ? kHeadTiles / 2 : kHeadTiles);  // the 16-bit tiles are twice as large
-  if (head > 0) { reduce_head_kernel<B><<<n_slices, kReduceHeadWarps * 32, 0, st>>>(g, head); ++launches; }
-  int lo = head;
-  while (lo < n_tiles) {
-    // outputs of tiles [lo, hi) end at hi * tile_bytes(B); inputs start at lo * tile_bytes(2B)
-    long long hi = (long long)lo * tile_bytes(2 * B) / tile_bytes(B);
-    hi = std::min<long long>(hi, n_tiles);
-    if (hi <= lo) return cudaErrorUnknown;
-    dim3 grid((unsigned)((hi - lo + 3) / 4), (unsigned)n_slices);
-    reduce_wave_kernel<B><<<grid, 128, 0, st>>>(g, lo, (int)hi);
-    ++launches;
-    lo = (int)hi;
-  }
+  // one CTA per (stream, slice): the streams compact in place independently of one another
+  reduce_stream_kernel<B><<<dim3(kStreams, (unsigned)n_slices), kReduceWarps * 32, 0, st>>>(g, n_tiles);
+  ++launches;
   return cudaGetLastError();
 }
 
 template <int BITS>
 cudaError_t attention_setup_one(int &resident, int sms) {
   cudaError_t e = cudaFuncSetAttribute(decode_attn_splitk_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       attn_ring_bytes<BITS>());
+                                       attn_smem_bytes<BITS>());
   int per_sm = 0;
   if (e == cudaSuccess)
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_splitk_kernel<BITS>, kAttnThreads,
-                                                      attn_ring_bytes<BITS>());
+                                                      attn_smem_bytes<BITS>());
   resident = std::min(kMaxCtas, std::max(1, per_sm) * sms);
   return e;
 }
@@ -288,6 +282,7 @@ pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
     e = cudaMemcpy(k->arena + k->off_inv_lambda, inv.data(), n_lam * sizeof(float), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_vmax, 0, (size_t)k->layers * k->n_slices * sizeof(unsigned));
   if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_tickets, 0, (size_t)k->layers * k->n_slices * sizeof(unsigned));
+  if (e == cudaSuccess) e = cudaMemset(k->arena + k->off_error, 0, sizeof(unsigned));
   if (e == cudaSuccess) {
     std::vector<LayerGeom> geoms(k->layers);
     for (int i = 0; i < k->layers; ++i) geoms[i] = k->geom(k->L[i]);
@@ -310,10 +305,10 @@ pmkvq_status pmkvq_progressive_reduce(pmkvq_cache *k, int32_t layer, void *strea
   return do_reduce(k, layer, static_cast<cudaStream_t>(stream));
 }
 
-// Policy part of an append of n_new tokens to one block (Sec. 3.1): capacity and budget tests before
-// anything is mutated, then the reduces the budget asks for.  On PMKVQ_OK the block can take the tokens.
-static pmkvq_status append_prepare(pmkvq_cache *k, int32_t layer, int32_t n_new, cudaStream_t st, int &n_after_out) {
-  Layer &l = k->L[layer];
+// Policy part of an append of n_new tokens to one block (Sec. 3.1), without side effects: capacity and
+// budget tests; on PMKVQ_OK `n_reduce` is the number of halvings the budget asks for first.
+static pmkvq_status append_check(const pmkvq_cache *k, int32_t layer, int32_t n_new, int &n_after_out, int &n_reduce_out) {
+  const Layer &l = k->L[layer];
   const int64_t n_after64 = (int64_t)l.n_tokens + n_new;
   if (n_after64 > k->max_tokens) return PMKVQ_ERR_CAPACITY;
   const int n_after = (int)n_after64;
@@ -324,12 +319,22 @@ static pmkvq_status append_prepare(pmkvq_cache *k, int32_t layer, int32_t n_new,
     ++n_reduce;
   }
   if (n_reduce && !k->auto_reduce) return PMKVQ_ERR_BUDGET_FULL;
-  if ((size_t)((k->body_at(n_after) + 15) / 16) * tile_bytes(bits) > l.body_cap) return PMKVQ_ERR_STATE;
+  if ((size_t)(((k->body_at(n_after) + 15) / 16 + kStreams - 1) / kStreams) * tile_bytes(bits) > l.stream_stride)
+    return PMKVQ_ERR_STATE;
+  n_after_out = n_after;
+  n_reduce_out = n_reduce;
+  return PMKVQ_OK;
+}
+
+// The same, followed by the reduces.  On PMKVQ_OK the block can take the tokens.
+static pmkvq_status append_prepare(pmkvq_cache *k, int32_t layer, int32_t n_new, cudaStream_t st, int &n_after_out) {
+  int n_reduce = 0;
+  const pmkvq_status c = append_check(k, layer, n_new, n_after_out, n_reduce);
+  if (c != PMKVQ_OK) return c;
   for (int i = 0; i < n_reduce; ++i) {
     const pmkvq_status s = do_reduce(k, layer, st);
     if (s != PMKVQ_OK) return s;
   }
-  n_after_out = n_after;
   return PMKVQ_OK;
 }
 
@@ -353,7 +358,10 @@ pmkvq_status pmkvq_append(pmkvq_cache *k, int32_t layer, const void *d_K, const 
   const float *inv_lam = reinterpret_cast<const float *>(k->arena + k->off_inv_lambda) + (size_t)layer * k->kv_heads * kHeadDim;
   unsigned *vmax = reinterpret_cast<unsigned *>(k->arena + k->off_vmax) + (size_t)layer * k->n_slices;
   const int n_evict = std::max(0, ev_last - ev_first);
-  if (n_new == 1) {
+  // With window = 0 and chunked eviction the new token enters the body together with the chunk's other
+  // tokens, possibly in one tile: they then go through separate launches (see append_decode_kernel).
+  const bool shares_tile = k->window == 0 && k->evict_chunk > 1;
+  if (n_new == 1 && !shares_tile) {
     // decode step: evictions and the new token in one launch (their ring slots cannot coincide)
     const long long warps = 2ll * (n_evict + 1) * k->n_slices;
     append_decode_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(
@@ -442,17 +450,17 @@ static pmkvq_status attn_params(pmkvq_cache *k, int32_t layer, const void *d_Q, 
 }
 
 template <int BITS>
-static cudaError_t attn_launch_width(const AttnParams &p, unsigned n_ctas, cudaStream_t st) {
-  decode_attn_splitk_kernel<BITS><<<n_ctas, kAttnThreads, attn_ring_bytes<BITS>(), st>>>(p);
+static cudaError_t attn_launch_width(const AttnParams &p, unsigned n_ctas, cudaStream_t st, unsigned *error_word) {
+  decode_attn_splitk_kernel<BITS><<<n_ctas, kAttnThreads, attn_smem_bytes<BITS>(), st>>>(p, error_word);
   return cudaGetLastError();
 }
 
-static cudaError_t attn_launch(const AttnParams &p, unsigned n_ctas, cudaStream_t st) {
+static cudaError_t attn_launch(const AttnParams &p, unsigned n_ctas, cudaStream_t st, unsigned *error_word) {
   switch (p.cur_bits) {
-    case 16: return attn_launch_width<16>(p, n_ctas, st);
-    case 8: return attn_launch_width<8>(p, n_ctas, st);
-    case 4: return attn_launch_width<4>(p, n_ctas, st);
-    default: return attn_launch_width<2>(p, n_ctas, st);
+    case 16: return attn_launch_width<16>(p, n_ctas, st, error_word);
+    case 8: return attn_launch_width<8>(p, n_ctas, st, error_word);
+    case 4: return attn_launch_width<4>(p, n_ctas, st, error_word);
+    default: return attn_launch_width<2>(p, n_ctas, st, error_word);
   }
 }
 
@@ -463,7 +471,7 @@ static pmkvq_status attention_on_arena(pmkvq_cache *k, int32_t layer, const void
   if (s != PMKVQ_OK) return s;
   p.partials = reinterpret_cast<float *>(k->arena + k->off_partials + (size_t)layer * k->partial_bytes);
   p.tickets = reinterpret_cast<unsigned *>(k->arena + k->off_tickets) + (size_t)layer * k->n_slices;
-  const cudaError_t e = attn_launch(p, n_ctas, st);
+  const cudaError_t e = attn_launch(p, n_ctas, st, reinterpret_cast<unsigned *>(k->arena + k->off_error));
   k->launches += 1;
   return e == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }
@@ -482,6 +490,7 @@ static pmkvq_status attention_all_blocks(pmkvq_cache *k, const void *d_Q, float 
   fp.partials = reinterpret_cast<float *>(k->arena + k->off_partials);
   fp.out = d_out;
   fp.tickets = reinterpret_cast<unsigned *>(k->arena + k->off_tickets);
+  fp.error_word = reinterpret_cast<unsigned *>(k->arena + k->off_error);
   fp.partial_stride = k->partial_bytes / sizeof(float);
   fp.layers = k->layers; fp.kv_heads = k->kv_heads; fp.group = k->group; fp.q_heads = k->q_heads;
   fp.n_slices = k->n_slices; fp.batch = k->batch;
@@ -506,7 +515,11 @@ static pmkvq_status attention_all_blocks(pmkvq_cache *k, const void *d_Q, float 
   fp.start[k->layers] = total;
   fp.total = total;
   const int want = k->user_ctas > 0 ? k->user_ctas : k->resident_fused;
-  fp.per_cta = std::max<long long>((total + want - 1) / want, k->user_ctas > 0 ? 1 : 50ll * kMinUnitsPerCta);
+  // A piece must never be shorter than the heaviest unit: then every CTA between the owners of a slice's
+  // first and last unit holds the first fine unit of at least one unit of that slice and publishes a
+  // partial, which is what the slice's ticket count expects.
+  fp.per_cta = std::max<long long>((total + want - 1) / want,
+                                   k->user_ctas > 0 ? (long long)tile_weight(16) : 50ll * kMinUnitsPerCta);
   const unsigned n_ctas = (unsigned)((total + fp.per_cta - 1) / fp.per_cta);
   decode_attn_fused_kernel<<<n_ctas, kAttnThreads, attn_fused_smem_bytes(), st>>>(fp);
   k->launches += 1;
@@ -535,7 +548,7 @@ pmkvq_status pmkvq_decode_attention_static(pmkvq_cache *k, int32_t layer, const 
   p.partials = reinterpret_cast<float *>(scratch + kStaticTicketBytes);
   // the array keeps whatever the previous call left: the tickets must start at zero
   if (cudaMemsetAsync(p.tickets, 0, (size_t)k->n_slices * sizeof(unsigned), st) != cudaSuccess) return PMKVQ_ERR_CUDA;
-  const cudaError_t e = attn_launch(p, n_ctas, st);
+  const cudaError_t e = attn_launch(p, n_ctas, st, reinterpret_cast<unsigned *>(k->arena + k->off_error));
   k->launches += 1;
   return e == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }
@@ -548,22 +561,30 @@ pmkvq_status pmkvq_decode_step(pmkvq_cache *k, const void *d_K, const void *d_V,
   const size_t kv_stride = (size_t)k->n_slices * kHeadDim * 2;            // bytes of one block's bf16 K (or V)
   const size_t q_stride = (size_t)k->batch * k->q_heads * kHeadDim * 2;   // bytes of one block's bf16 Q
   const size_t o_stride = (size_t)k->batch * k->q_heads * kHeadDim;       // floats of one block's output
-  if (k->layers > kMaxStepLayers) {  // too many blocks for one argument block: block by block
+  // 1. policy of every block, first without side effects: if any block cannot take its token (capacity, or a
+  //    full budget without auto_reduce) the call fails here and no block has been reduced or appended to
+  for (int layer = 0; layer < k->layers; ++layer) {
+    int n_after = 0, n_reduce = 0;
+    const pmkvq_status s = append_check(k, layer, 1, n_after, n_reduce);
+    if (s != PMKVQ_OK) return s;
+  }
+  if (k->layers > kMaxStepLayers || (k->window == 0 && k->evict_chunk > 1)) {
+    // too many blocks for one argument block, or appends that need two launches per block: block by block
     for (int layer = 0; layer < k->layers; ++layer) {
       pmkvq_status s = pmkvq_append(k, layer, static_cast<const uint8_t *>(d_K) + layer * kv_stride,
                                     static_cast<const uint8_t *>(d_V) + layer * kv_stride, 1, stream);
       if (s == PMKVQ_OK)
         s = pmkvq_decode_attention(k, layer, static_cast<const uint8_t *>(d_Q) + layer * q_stride,
                                    d_out + layer * o_stride, stream);
-      if (s != PMKVQ_OK) return s;
+      if (s != PMKVQ_OK) return s;  // only a CUDA launch error can get here
     }
     return PMKVQ_OK;
   }
-  // 1. policy of every block (budget tests, the reduces they ask for); nothing is appended yet
+  //    then the reduces the budgets ask for; nothing is appended yet
   for (int layer = 0; layer < k->layers; ++layer) {
     int n_after = 0;
     const pmkvq_status s = append_prepare(k, layer, 1, st, n_after);
-    if (s != PMKVQ_OK) return s;
+    if (s != PMKVQ_OK) return s;  // only a CUDA launch error can get here
   }
   // 2. quantize-on-append and evictions of all blocks in one launch
   StepParams sp;
@@ -582,6 +603,34 @@ pmkvq_status pmkvq_decode_step(pmkvq_cache *k, const void *d_K, const void *d_V,
   for (int layer = 0; layer < k->layers; ++layer) k->L[layer].n_tokens += 1;
   // 3. attention of all blocks in one launch: their tiles form one line of work cut into one piece per CTA
   return attention_all_blocks(k, d_Q, d_out, st);
+}
+
+pmkvq_status pmkvq_decode_attention_all(pmkvq_cache *k, const void *d_Q, float *d_out, void *stream) {
+  if (!k || !d_Q || !d_out) return PMKVQ_ERR_INVALID_ARG;
+  if (k->layers > kMaxFusedLayers) return PMKVQ_ERR_INVALID_ARG;
+  return attention_all_blocks(k, d_Q, d_out, static_cast<cudaStream_t>(stream));
+}
+
+pmkvq_status pmkvq_device_status(pmkvq_cache *k, uint32_t *h_wait_bits) {
+  if (!k) return PMKVQ_ERR_INVALID_ARG;
+  unsigned word = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return PMKVQ_ERR_CUDA;
+  if (cudaMemcpy(&word, k->arena + k->off_error, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return PMKVQ_ERR_CUDA;
+  if (h_wait_bits) *h_wait_bits = word;
+  return word ? PMKVQ_ERR_DEVICE_WAIT : PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_restore_layer_state(pmkvq_cache *k, int32_t layer, int32_t n_tokens, int32_t cur_bits) {
+  if (!k || layer < 0 || layer >= k->layers || n_tokens < 0 || n_tokens > k->max_tokens || !valid_bits(cur_bits))
+    return PMKVQ_ERR_INVALID_ARG;
+  Layer &l = k->L[layer];
+  if (cur_bits < l.fbit) return PMKVQ_ERR_INVALID_ARG;
+  if (k->bytes_at(n_tokens, cur_bits) > l.budget) return PMKVQ_ERR_INVALID_ARG;
+  if ((size_t)(((k->body_at(n_tokens) + 15) / 16 + kStreams - 1) / kStreams) * tile_bytes(cur_bits) > l.stream_stride)
+    return PMKVQ_ERR_INVALID_ARG;
+  l.n_tokens = n_tokens;
+  l.cur_bits = cur_bits;
+  return PMKVQ_OK;
 }
 
 pmkvq_status pmkvq_layer_state(const pmkvq_cache *k, int32_t layer, int32_t *n_tokens, int32_t *cur_bits,
@@ -616,7 +665,7 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
   const LayerGeom g = k->geom(l);
   const int n = l.n_tokens, n_sink_eff = k->sink_at(n), n_body = k->body_at(n), win_start = n_sink_eff + n_body;
   const size_t fixed = g.body_off;
-  const size_t body_bytes = (size_t)((n_body + 15) / 16) * tile_bytes(l.cur_bits);
+  const size_t body_bytes = n_body > 0 ? g.stream_stride * kStreams : 0;
   std::vector<uint8_t> host(fixed + body_bytes);
   const uint8_t *src = g.base + (size_t)(batch_idx * k->kv_heads + kv_head) * g.slice_stride;
   if (cudaMemcpy(host.data(), src, host.size(), cudaMemcpyDeviceToHost) != cudaSuccess) return PMKVQ_ERR_CUDA;
@@ -628,7 +677,7 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
       tile = host.data() + (size_t)(t >> 4) * tile_bytes(16); row = t & 15; bits = 16;
     } else if (t < win_start) {
       const int j = t - k->n_sink;
-      tile = host.data() + g.body_off + (size_t)(j >> 4) * tile_bytes(l.cur_bits); row = j & 15; bits = l.cur_bits;
+      tile = host.data() + g.body_off + body_tile_offset(j >> 4, l.cur_bits, g.stream_stride); row = j & 15; bits = l.cur_bits;
     } else {
       const int rp = (t - k->n_sink) % g.ring_tokens;
       tile = host.data() + g.ring_off + (size_t)(rp >> 4) * tile_bytes(16); row = rp & 15; bits = 16;
@@ -648,8 +697,8 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
       else packed[(ch * bits) >> 3] |= (uint8_t)(c << ((ch * bits) & 7));
     }
     float sc, ze;
-    std::memcpy(&sc, tile + meta_offset(bits) + meta_slot(is_value ? 2 : 0, row), 4);
-    std::memcpy(&ze, tile + meta_offset(bits) + meta_slot(is_value ? 3 : 1, row), 4);
+    std::memcpy(&sc, tile + meta_offset(bits) + meta_slot(bits, is_value ? 2 : 0, row), 4);
+    std::memcpy(&ze, tile + meta_offset(bits) + meta_slot(bits, is_value ? 3 : 1, row), 4);
     if (h_scale) h_scale[t] = sc;
     if (h_zero) h_zero[t] = ze;
     if (h_bits) h_bits[t] = (uint8_t)bits;
@@ -844,6 +893,7 @@ const char *pmkvq_status_string(pmkvq_status s) {
     case PMKVQ_ERR_CUDA: return "CUDA error";
     case PMKVQ_ERR_STATE: return "internal state error";
     case PMKVQ_ERR_SCRATCH_LIMIT: return "problem too large for the built-in scratch: use pmkvq_decode_attention";
+    case PMKVQ_ERR_DEVICE_WAIT: return "a device-side wait ran out: the results of the affected launch are invalid";
   }
   return "unknown status";
 }
