@@ -16,7 +16,7 @@
 //      the score MMAs run;
 //   5. thread t reads its token's 16 score sums (tcgen05.ld), applies scale and zero-point
 //      (q.k = S_K (q.c) + Z_K sum(q)), takes p = 2^(s - m) against the warpgroup's reference m and writes
-//      w = p * S_V (one fp16 per head) as row t of the MN-major B operand of the output MMA;
+//      w = p * S_V (fp16 hi + lo per head) as row t of the MN-major B operand of the output MMA;
 //   6. one thread issues O^T[channel, head] += A_V . w: one tcgen05.mma per live tile of the block.
 //
 // The reference m only moves when some score of a block exceeds it by more than kMaxAhead (found with one
@@ -37,7 +37,7 @@ constexpr int kTmemCols = 512;
 constexpr int kTmemColsPerWg = 160;        // A_K 64 | A_V 64 | D_S 16 | D_O 16
 constexpr int kStageTiles = kBlockTiles;   // one block per stage
 constexpr int kStagesPerWg = 2;
-constexpr int kWBufBytes = 4096;           // [n-group 2][128 tokens][8 heads] fp16; group 1 stays zero
+constexpr int kWBufBytes = 4096;           // [hi | lo][128 tokens][8 heads] fp16: columns h and 8 + h of the weights
 constexpr int kQOperandBytes = 4096;       // [n-group 2][k-chunk 16][8 rows][8 channels] fp16
 constexpr int kEPV = 12;                   // w = p * S_V / sigma_u * 2^(kEPV - pos) stays below 2^16
 
@@ -91,14 +91,13 @@ __device__ __forceinline__ void tc_wait(TcCtx &tc, uint32_t bar, uint32_t parity
 template <int BITS> struct RowFmt;
 template <> struct RowFmt<2> {
   static constexpr int SIGMA_LOG2 = 15;
-  __host__ __device__ static constexpr int pos(int f) { return f < 5 ? 2 * f : 2 * f - 5; }  // f = field 0..7
+  __host__ __device__ static constexpr int pos(int f) { return 2 * (f & 3); }                // f = field 0..7
   __host__ __device__ static constexpr int field(int idx) { return (idx & 15) >> 1; }        // of channel / token index
   // one word (16 codes) -> 8 tensor-memory columns (column f = fields f of the two halves)
   __device__ static __forceinline__ void extract(uint32_t x, uint32_t *e) {
-    const uint32_t xr = x >> 5;
+    const uint32_t xr = x >> 8;
     e[0] = x & 0x00030003u; e[1] = x & 0x000C000Cu; e[2] = x & 0x00300030u; e[3] = x & 0x00C000C0u;
-    e[4] = x & 0x03000300u;
-    e[5] = xr & 0x00600060u; e[6] = xr & 0x01800180u; e[7] = xr & 0x06000600u;
+    e[4] = xr & 0x00030003u; e[5] = xr & 0x000C000Cu; e[6] = xr & 0x00300030u; e[7] = xr & 0x00C000C0u;
   }
 };
 template <> struct RowFmt<4> {
@@ -181,8 +180,16 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
   const float w_unit = ldexpf(1.0f, kEPV - F::pos(F::field(my_row))) / sigma_u;
 
   if (quad == 0 && kb0 + wg <= kb1) issue_block(kb0 + wg, 0);
-  bool first = true;
-  int it = 0;
+  // The tensor core adds into its fp32 accumulators without rounding to nearest, and the sums of codes
+  // times weights are all of one sign: left to grow over thousands of MMAs the loss shows in the output,
+  // which is the small difference of that sum and the zero-point sum.  So every kEpochBlocks blocks the
+  // accumulators of this thread's channel move into registers (ov) and the tensor-memory sums restart.
+  constexpr int kEpochBlocks = 16;
+  float ov[8];
+#pragma unroll
+  for (int h = 0; h < 8; ++h) ov[h] = 0.f;
+  bool first = true;  // the tensor-memory accumulators hold nothing yet
+  int it = 0, since = 0;
   for (int kb = kb0 + wg; kb <= kb1; kb += kWarpgroups, ++it) {
     const int s = it & 1;
     const int lo_i = max(t_lo - 8 * kb, 0), hi_i = min(t_hi - 8 * kb, 8);
@@ -238,6 +245,15 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
         tc_wait(tc, bar_o, tc.ph_o, 4u);
         tc.ph_o ^= 1u;
         tc05::fence_after_sync();
+        if (since == kEpochBlocks) {
+          uint32_t o[16];
+          tc05::tmem_ld16(tD_O + t_lane, o);
+          tc05::wait_ld();
+#pragma unroll
+          for (int h = 0; h < 8; ++h) ov[h] += fmaf(__uint_as_float(o[8 + h]), 0x1p-11f, __uint_as_float(o[h]));
+          first = true;
+          since = 0;
+        }
       }
       tc05::tmem_st32(tA_V + t_lane, r);
       tc05::tmem_st32(tA_V + t_lane + 32, r + 32);
@@ -295,42 +311,44 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
         m2[j] = make_float2(nx, ny);
         l2[j] = __fmul2_rn(l2[j], make_float2(f[2 * j], f[2 * j + 1]));
         zs2[j] = __fmul2_rn(zs2[j], make_float2(f[2 * j], f[2 * j + 1]));
+        ov[2 * j] *= f[2 * j];
+        ov[2 * j + 1] *= f[2 * j + 1];
         arg[j] = __fadd2_rn(sc[j], make_float2(-nx, -ny));
         if (!alive) arg[j] = make_float2(-INFINITY, -INFINITY);
       }
       if (!first) {  // the output accumulators of channel row tw (every earlier output MMA has completed)
-        uint32_t o[8];
-        tc05::tmem_ld8(tD_O + t_lane, o);
+        uint32_t o[16];
+        tc05::tmem_ld16(tD_O + t_lane, o);
         tc05::wait_ld();
 #pragma unroll
-        for (int h = 0; h < 8; ++h) o[h] = __float_as_uint(__uint_as_float(o[h]) * f[h]);
-        asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n" ::"r"(tD_O + t_lane), "r"(o[0]),
-                     "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
-                     : "memory");
+        for (int h = 0; h < 8; ++h) {
+          o[h] = __float_as_uint(__uint_as_float(o[h]) * f[h]);
+          o[8 + h] = __float_as_uint(__uint_as_float(o[8 + h]) * f[h]);
+        }
+        tc05::tmem_st16(tD_O + t_lane, o);
       }
       wg_sync(wg);  // wmax may be rewritten by the next slow path
     }
 
-    // ---- probabilities and weights ----
+    // ---- probabilities and weights: w = p * S_V goes to the output MMA as fp16 hi + lo (22 bits), in
+    //      columns h and 8 + h of the B operand; the sums take p itself ----
     {
       // a constant V group has S_V = 0 and all codes 0: any finite unit will do for it
-      const float s_e = meta.z == 0.f ? w_unit : meta.z * w_unit;   // w = p * s_e
-      const float rs = rcp_approx(s_e);
-      const bool tiny = s_e < 0x1p-10f;  // w would leave fp16's normal range: take p itself for the sums
-      uint32_t wp[4];
+      const float s_e = meta.z == 0.f ? w_unit : meta.z * w_unit;
+      uint32_t whi[4], wlo[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const float2 e = make_float2(ex2(arg[j].x), ex2(arg[j].y));
         const float2 w = __fmul2_rn(e, make_float2(s_e, s_e));
-        wp[j] = pack_half2(w.x, w.y);
-        // the probability that enters the denominator and the zero-point sum is the rounded w divided by
-        // its unit again, so numerator and denominator see the same probabilities
-        float2 pr = __fmul2_rn(__half22float2(*reinterpret_cast<const __half2 *>(&wp[j])), make_float2(rs, rs));
-        if (tiny) pr = e;
-        l2[j] = __fadd2_rn(l2[j], pr);
-        zs2[j] = __ffma2_rn(pr, make_float2(meta.w, meta.w), zs2[j]);
+        whi[j] = pack_half2(w.x, w.y);
+        const float2 back = __half22float2(*reinterpret_cast<const __half2 *>(&whi[j]));
+        const float2 rest = __fmul2_rn(__fadd2_rn(w, make_float2(-back.x, -back.y)), make_float2(2048.f, 2048.f));
+        wlo[j] = pack_half2(rest.x, rest.y);
+        l2[j] = __fadd2_rn(l2[j], e);
+        zs2[j] = __ffma2_rn(e, make_float2(meta.w, meta.w), zs2[j]);
       }
-      *reinterpret_cast<uint4 *>(wbuf + tw * 16) = make_uint4(wp[0], wp[1], wp[2], wp[3]);
+      *reinterpret_cast<uint4 *>(wbuf + tw * 16) = make_uint4(whi[0], whi[1], whi[2], whi[3]);
+      *reinterpret_cast<uint4 *>(wbuf + 2048 + tw * 16) = make_uint4(wlo[0], wlo[1], wlo[2], wlo[3]);
     }
     tc05::fence_async_smem();
     tc05::wait_st();
@@ -344,22 +362,20 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
       tc05::mma_commit(bar_o);
     }
     first = false;
+    ++since;
   }
 
   // ---- the warpgroup's partial: (m, l, o[128]) per head ----
-  float ov[8];
-#pragma unroll
-  for (int h = 0; h < 8; ++h) ov[h] = 0.f;
   if (it > 0) {
     tc_wait(tc, bar_o, tc.ph_o, 4u);
     tc.ph_o ^= 1u;
     tc05::fence_after_sync();
-    uint32_t o[8];
-    tc05::tmem_ld8(tD_O + t_lane, o);
+    uint32_t o[16];
+    tc05::tmem_ld16(tD_O + t_lane, o);
     tc05::wait_ld();
     const float f_out = ldexpf(sigma_u, 24 - kEPV);
 #pragma unroll
-    for (int h = 0; h < 8; ++h) ov[h] = __uint_as_float(o[h]) * f_out;
+    for (int h = 0; h < 8; ++h) ov[h] = (ov[h] + fmaf(__uint_as_float(o[8 + h]), 0x1p-11f, __uint_as_float(o[h]))) * f_out;
   }
   // sums over the warpgroup's 128 token rows
   float red[16];
