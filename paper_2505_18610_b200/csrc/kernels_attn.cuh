@@ -46,9 +46,9 @@ constexpr int kMaxGroup = 8;         // query heads per KV head handled by one M
 constexpr int kPartialStride = 132;  // floats per (segment, head): m, l, 2 pad, o[128]
 constexpr float kNegBig = -1.0e30f;
 constexpr float kMaxAhead = 3.0f;    // a score may exceed the reference by this much (log2 units)
-constexpr int kAttnWarps = 12;       // one CTA per SM: three warpgroups; its warps share the CTA's INT16 / 8-bit tiles dynamically
+constexpr int kAttnWarps = 16;       // one CTA per SM; these warps share the CTA's INT16 / 8- / 16-bit tiles dynamically
 constexpr int kAttnThreads = 32 * kAttnWarps;
-constexpr int kParts = kAttnWarps + 3;  // partial results a segment merges: one per warp, one per warpgroup
+constexpr int kParts = kAttnWarps + 2;  // partial results a segment merges: one per warp, two of the tensor-memory body
 
 struct AttnParams {
   LayerGeom geom;
@@ -695,11 +695,12 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
     for (int c = 0; c < (TB / 16 + 31) / 32; ++c)
       if (c * 32 + lane < TB / 16) cp_async16(dst + c * 512, src + c * 512);
   };
+  const bool worker = warp < kAttnWarps;  // the last warp of the CTA only serves the tensor-memory path
   int pending[S];  // tiles claimed and in flight, oldest first (>= n_steps: none)
   if constexpr (F::SLOTS > 0) {
 #pragma unroll
     for (int i = 0; i < S - 1; ++i) {
-      pending[i] = n_steps > 0 ? claim(1) : 0;
+      pending[i] = (n_steps > 0 && worker) ? claim(1) : n_steps;
       if (pending[i] < n_steps) issue(pending[i], i);
       cp_async_commit();
     }
@@ -719,7 +720,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
 
   // ---- INT16 tiles (sink + window ring) ----
-  if (a_hi > a_lo) {
+  if (a_hi > a_lo && worker) {
     run_int16_tiles(p, slice_base, a_lo, a_hi, st, s_frag, s_ctr, e_g, sumq, sigma16, lane);
     if constexpr (BITS != 16) {
       // accumulator units change with the width: INT16 units -> body units (exact powers of two)
@@ -737,7 +738,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
 
   // ---- body tiles ----
   const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
-  if (n_steps > 0) {
+  if (n_steps > 0 && worker) {
     QFrag qa;
     qa.mine = (BITS != 16 ? s_frag + 256 : s_frag) + lane;
     const float mu = ldexpf(1.0f, 24 - F::EQ + e_g);
@@ -777,7 +778,8 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   __syncthreads();  // every warp is done with its stages
   float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(ring);
   float *s_m = s_stat + 16, *s_l = s_stat + 16 + kParts * kMaxGroup;
-  store_warp_partial(st, [&](int J) { return ldexpf(sigma_u, 24 - F::EP - F::pos(J % F::N)); }, s_o, s_m, s_l, warp, lane);
+  if (worker)
+    store_warp_partial(st, [&](int J) { return ldexpf(sigma_u, 24 - F::EP - F::pos(J % F::N)); }, s_o, s_m, s_l, warp, lane);
   __syncthreads();
   publish_segment(p, slice, kAttnWarps, s_o, s_m, s_l, s_ctr);
 }
@@ -787,15 +789,15 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
 namespace pmkvq {
 
 // Dynamic shared memory of a CTA that may run the tensor-memory path.
-constexpr int kSmemStages = kWarpgroups * kStagesPerWg * kStageBytes;   // also the cp.async ring / outputs of the 8- and 16-bit path
+constexpr int kSmemStages = kStages * kStageBytes;
 constexpr int kSmemQOperand = kSmemStages;
 constexpr int kSmemWBuf = kSmemQOperand + kQOperandBytes;
-constexpr int kSmemParts = kSmemWBuf + kWarpgroups * kWBufBytes;
+constexpr int kSmemParts = kSmemWBuf + 2 * kWBufBytes;
 constexpr int kSmemTcTotal = kSmemParts + kParts * kMaxGroup * kHeadDim * 4;
 
 // One segment with a 4- or 2-bit body.  The INT16 tiles run as above, on the warps' own accumulators, and
-// every warp parks its partial in shared memory; the body runs on the tensor-memory path, one partial per
-// warpgroup.
+// every warp parks its partial in shared memory; the body then runs through the tensor-memory pipeline
+// and leaves one more partial.
 template <int BITS>
 __device__ __forceinline__ void run_segment_tc(const AttnParams &p, int slice, long long u_lo, long long u_hi,
                                                float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint4 *s_frag,
@@ -820,7 +822,7 @@ __device__ __forceinline__ void run_segment_tc(const AttnParams &p, int slice, l
   float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(tc.part_o);
   float *s_m = s_stat + 16, *s_l = s_stat + 16 + kParts * kMaxGroup;
 
-  {
+  if (warp < kAttnWarps) {
     WarpState st;
     st.m = kNegBig; st.l = make_float2(0.f, 0.f); st.zs = make_float2(0.f, 0.f);
 #pragma unroll
@@ -829,12 +831,12 @@ __device__ __forceinline__ void run_segment_tc(const AttnParams &p, int slice, l
     store_warp_partial(st, [&](int J) { return ldexpf(sigma16, 24 - F16::EP - F16::pos(J % F16::N)); }, s_o, s_m, s_l, warp, lane);
   }
   if (t_hi > t_lo) {
-    tc_body<BITS>(p, tc, slice_base + p.geom.body_off, t_lo, t_hi, s_stat, sigma16, s_m, s_l, kAttnWarps + (warp >> 2));
-  } else {
-    const int slot = kAttnWarps + (warp >> 2), tw = tid & 127;
+    tc_body<BITS>(p, tc, slice_base + p.geom.body_off, t_lo, t_hi, s_stat, sigma16, s_m, s_l, kAttnWarps);
+  } else if (tid < 2 * kHeadDim) {
+    const int slot = kAttnWarps + (tid >> 7), c = tid & 127;
 #pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h) s_o[slot][h][tw] = 0.f;
-    if (tw < kMaxGroup) { s_m[slot * 8 + tw] = kNegBig; s_l[slot * 8 + tw] = 0.f; }
+    for (int h = 0; h < kMaxGroup; ++h) s_o[slot][h][c] = 0.f;
+    if (c < kMaxGroup) { s_m[slot * 8 + c] = kNegBig; s_l[slot * 8 + c] = 0.f; }
   }
   __syncthreads();
   publish_segment(p, slice, kParts, s_o, s_m, s_l, s_ctr);
@@ -852,8 +854,7 @@ constexpr int attn_smem_bytes() {
   }
 }
 
-// CTA set-up of the tensor-memory path: barriers, tensor memory, the zero half of the weight operands.
-// Ends with a CTA-wide barrier.
+// CTA set-up of the tensor-memory path: barriers and tensor memory.  Ends with a CTA-wide barrier.
 __device__ __forceinline__ void tc_setup(TcShared *sh, TcCtx &tc, uint8_t *ring, unsigned *error_word) {
   const int tid = threadIdx.x, warp = tid >> 5;
   tc.sh = sh;
@@ -862,20 +863,23 @@ __device__ __forceinline__ void tc_setup(TcShared *sh, TcCtx &tc, uint8_t *ring,
   tc.wbuf = ring + kSmemWBuf;
   tc.part_o = reinterpret_cast<float *>(ring + kSmemParts);
   tc.error_word = error_word;
-  tc.ph_full = 0; tc.ph_s = 0; tc.ph_o = 0;
+  tc.gi = 0; tc.gc = 0;
   if (tid == 0) {
-    for (int w = 0; w < kWarpgroups; ++w) {
-      for (int s = 0; s < kStagesPerWg; ++s) tc05::mbar_init(tc05::smem_u32(&sh->bar_full[w][s]), 1);
-      tc05::mbar_init(tc05::smem_u32(&sh->bar_s[w]), 1);
-      tc05::mbar_init(tc05::smem_u32(&sh->bar_o[w]), 1);
+    for (int s = 0; s < kStages; ++s) {
+      tc05::mbar_init(tc05::smem_u32(&sh->full[s]), 1);
+      tc05::mbar_init(tc05::smem_u32(&sh->stage_free[s]), 16);
+    }
+    for (int b = 0; b < 2; ++b) {
+      tc05::mbar_init(tc05::smem_u32(&sh->ds_free[b]), 4);
+      tc05::mbar_init(tc05::smem_u32(&sh->bar_s[b]), 1);
+      tc05::mbar_init(tc05::smem_u32(&sh->bar_o[b]), 1);
+      sh->k_tickets[b] = sh->p_tickets[b] = 0u;
+      sh->pv_fresh[b] = 1;
     }
     sh->abort = 0;
     tc05::mbar_init_fence();
   }
   if (warp == 0) tc05::tmem_alloc(tc05::smem_u32(&sh->tmem_base), kTmemCols);
-  for (int i = tid; i < kWarpgroups * kWBufBytes / 16; i += kAttnThreads)
-    reinterpret_cast<uint4 *>(tc.wbuf)[i] = make_uint4(0u, 0u, 0u, 0u);
-  tc05::fence_async_smem();
   tc05::fence_before_sync();
   __syncthreads();
   tc05::fence_after_sync();
@@ -1010,6 +1014,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_fused_kernel(cons
   tc_teardown(tc);
 }
 
-constexpr int attn_fused_smem_bytes() { return kSmemTcTotal; }
+constexpr int attn_fused_smem_bytes() { return kSmemTcTotal > attn_smem_bytes<8>() ? kSmemTcTotal : attn_smem_bytes<8>(); }
 
 }  // namespace pmkvq

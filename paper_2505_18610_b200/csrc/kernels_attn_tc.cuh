@@ -1,96 +1,128 @@
 // Decode attention over the 4- and 2-bit body of a slice on the fifth-generation tensor cores.
 //
 // Included by kernels_attn.cuh (which holds the work decomposition, the INT16 tile path and the split-K
-// combine).  A body block is 128 consecutive tokens = the eight tiles at one index of a slice's eight
-// streams.  The CTA's three warpgroups each take every third block of the segment; per block a warpgroup
+// combine).  The body tiles [t_lo, t_hi) of a segment are taken stream by stream (tile t lives in stream
+// t mod 8, and softmax attention does not care about the order of the tokens): in every stream the
+// segment's tiles are one contiguous run of bytes, which is cut into chunks of CHUNK_TILES tiles (about
+// 20 KB: one cp.async.bulk copy each; copies of that size reach the HBM read rate from one issuing lane,
+// 1-10 KB copies do not) and every chunk into MMA blocks of up to 8 tiles = 128 tokens.  The blocks flow
+// through specialised warps that meet only on mbarriers and tickets (no CTA-wide barrier inside the
+// loop), each running ahead of the next as far as its buffers allow:
 //
-//   1. waits for the block's tiles (eight cp.async.bulk copies that complete on an mbarrier, issued one
-//      block ahead by one thread);
-//   2. K: thread t unpacks the 128 codes of token t into fp16 bit patterns (a code field left in place
-//      below bit 11 of an fp16 is exactly code * 2^(pos-24); one AND per pair of codes) and stores them as
-//      row t of the A operand in tensor memory (tcgen05.st);
-//   3. one thread issues S[token, head] = A_K . Q''^T: 8 tcgen05.mma (128 x 16 x 16, fp16 in, fp32
-//      accumulators in tensor memory), B = the query fragments in shared memory (rows 0-7 the fp16 "hi"
-//      part of up to 8 heads, rows 8-15 the "lo" remainder), then tcgen05.commit onto an mbarrier;
-//   4. V: thread c unpacks channel c's codes of the 128 tokens into row c of the second A operand while
-//      the score MMAs run;
-//   5. thread t reads its token's 16 score sums (tcgen05.ld), applies scale and zero-point
-//      (q.k = S_K (q.c) + Z_K sum(q)), takes p = 2^(s - m) against the warpgroup's reference m and writes
-//      w = p * S_V (fp16 hi + lo per head) as row t of the MN-major B operand of the output MMA;
-//   6. one thread issues O^T[channel, head] += A_V . w: one tcgen05.mma per live tile of the block.
+//   copies         one lane of the K warpgroup's first warp issues one bulk copy per chunk into a ring of
+//                  kStages stages in shared memory, kStages - 1 chunks ahead of the chunk it works on,
+//                  completing on the stage's mbarrier;
+//   K warpgroup    thread t unpacks the 128 codes of token t into fp16 bit patterns (a code field left in
+//                  place below bit 11 of an fp16 is exactly code * 2^(pos-24); one AND per pair of codes)
+//                  and stores them as row t of the score MMA's A operand in tensor memory (tcgen05.st).
+//                  The last of its four warps to finish a block issues S[token, head] = A_K . Q''^T: 8
+//                  tcgen05.mma (128 x 16 x 16, fp16 in, fp32 accumulators in tensor memory), B = the query
+//                  fragments in shared memory (rows 0-7 the fp16 "hi" part of up to 8 heads, rows 8-15 the
+//                  "lo" remainder), and tcgen05.commit onto the buffer's mbarrier;
+//   V warpgroup    thread c does the same for channel c's codes of the block's tokens: row c of the output
+//                  MMA's A operand;
+//   S warpgroups   two, taking alternate blocks.  Thread t reads its token's 16 score sums (tcgen05.ld),
+//                  applies scale and zero-point (q.k = S_K (q.c) + Z_K sum(q)), takes p = 2^(s - m)
+//                  against its warpgroup's reference m and writes w = p * S_V (fp16 hi + lo per head) as
+//                  row t of the MN-major B operand of the output MMA; it keeps the sums of p and p * Z_V.
+//                  The last of the eight warps (four V, four S) to finish a block issues
+//                  O^T[channel, head] += A_V . w, one tcgen05.mma per live tile, into the warpgroup's own
+//                  accumulators.
 //
-// The reference m only moves when some score of a block exceeds it by more than kMaxAhead (found with one
-// barrier-wide OR per block); then the warpgroup takes the block's maxima, rescales its accumulators in
-// tensor memory and its running sums, and goes on.  Each warpgroup ends a segment with one partial
-// (m, l, o[128]) per head, merged with the INT16 tiles' per-warp partials like any other split.
+// A_K, A_V, the score accumulators, the weight buffer and the output accumulators exist twice (block n
+// uses buffer n mod 2, which is also the S warpgroup that owns it).  A reference m only moves when some
+// score of a block exceeds it by more than kTcMaxAhead (one OR over the warpgroup per block); the
+// warpgroup then takes the block's maxima plus some headroom, waits for its output MMAs, rescales its
+// accumulators in tensor memory and its running sums, and goes on.  A segment ends with one partial
+// (m, l, o[128]) per head and S warpgroup, merged with the INT16 tiles' per-warp partials like any split.
 //
 // Every mbarrier wait has an iteration limit; a wait that runs out sets a CTA-wide abort flag and an
-// error word in global memory, after which the CTA skips its remaining waits, runs through its barriers,
+// error word in global memory, after which the CTA skips its remaining waits, runs through its loops,
 // frees its tensor memory and returns (the results of that launch are then meaningless and the host
 // reports PMKVQ_ERR_DEVICE_WAIT).
 #pragma once
 
 namespace pmkvq {
 
-constexpr int kWarpgroups = 3;
-constexpr int kTmemCols = 512;
-constexpr int kTmemColsPerWg = 160;        // A_K 64 | A_V 64 | D_S 16 | D_O 16
-constexpr int kStageTiles = kBlockTiles;   // one block per stage
-constexpr int kStagesPerWg = 2;
+constexpr int kTmemCols = 512;             // A_K 2 x 64 | A_V 2 x 64 | D_S 2 x 16 | D_O 2 x 16
+constexpr int kTmemAK = 0, kTmemAV = 128, kTmemDS = 256, kTmemDO = 288;
+constexpr int kStages = 6;                 // chunks in flight in shared memory
+constexpr int kStageBytes = 16 * tile_bytes(2);   // 20 480: 16 tiles at 2 bit, 8 tiles at 4 bit (18 432)
+static_assert(kStageBytes >= 8 * tile_bytes(4), "a stage holds a chunk of either width");
 constexpr int kWBufBytes = 4096;           // [hi | lo][128 tokens][8 heads] fp16: columns h and 8 + h of the weights
 constexpr int kQOperandBytes = 4096;       // [n-group 2][k-chunk 16][8 rows][8 channels] fp16
-constexpr int kEPV = 12;                   // w = p * S_V / sigma_u * 2^(kEPV - pos) stays below 2^16
+constexpr int kEPV = 7;                    // w = p * S_V / sigma_u * 2^(kEPV - pos) stays below 2^16 for p <= 2^kTcMaxAhead
+constexpr float kTcMaxAhead = 8.0f;        // a score may exceed the reference by this much (log2 units)
+constexpr float kTcHeadroom = 4.0f;        // a new reference is set this far above the maxima seen
+constexpr int kWarpK = 0, kWarpV = 4, kWarpS = 8;  // first warp of each role (S: two warpgroups, warps 8-11 and 12-15)
 
 // Shared-memory bookkeeping of the tensor-core path (static).
 struct TcShared {
-  unsigned long long bar_full[kWarpgroups][kStagesPerWg];
-  unsigned long long bar_s[kWarpgroups];
-  unsigned long long bar_o[kWarpgroups];
+  unsigned long long full[kStages];        // the stage's copy has landed
+  unsigned long long stage_free[kStages];  // K, V and both S warpgroups are done with the stage (16 warp arrivals)
+  unsigned long long ds_free[2];           // the S warpgroup has read the buffer's scores (4 warp arrivals)
+  unsigned long long bar_s[2], bar_o[2];   // score / output MMAs of the buffer's block are complete
   uint32_t tmem_base;
   int abort;
-  float wmax[kWarpgroups][4][kMaxGroup];   // per warp block maxima (slow path)
-  float sums[kWarpgroups][4][2 * kMaxGroup];
+  unsigned k_tickets[2], p_tickets[2];     // warps that have finished the buffer's block (K: 4; V and S: 8)
+  int pv_fresh[2];                         // the block's first output MMA overwrites the accumulators
+  float wmax[2][4][kMaxGroup];             // per-warp block maxima (when a reference moves)
+  float sums[2][4][2 * kMaxGroup];
 };
 
-// Per-thread view: tensor-memory base, barrier parities (one bit each), error word.
+// Per-thread view: tensor-memory base, the CTA's running block and chunk counts (barrier parities follow).
 struct TcCtx {
   TcShared *sh;
-  uint8_t *stages;    // [kWarpgroups][kStagesPerWg][8 tiles of the widest row width]
+  uint8_t *stages;    // [kStages][kStageBytes]
   uint8_t *q_operand; // kQOperandBytes
-  uint8_t *wbuf;      // [kWarpgroups] kWBufBytes
+  uint8_t *wbuf;      // [2] kWBufBytes
   float *part_o;      // [kParts][8][128]
   unsigned *error_word;
   uint32_t tmem_base;
-  uint32_t ph_full;   // bit s: parity of the next wait on bar_full[wg][s]
-  uint32_t ph_s, ph_o;
+  uint32_t gi, gc;    // body blocks / chunks this CTA has pushed through the pipeline so far (all segments)
 };
 
-constexpr int kStageBytes = kStageTiles * tile_bytes(4);
-
-__device__ __forceinline__ void wg_sync(int wg) { asm volatile("bar.sync %0, 128;\n" ::"r"(wg + 1) : "memory"); }
-// barrier over the warpgroup that also ORs a predicate
-__device__ __forceinline__ bool wg_any(int wg, bool pred) {
+// barriers over one S warpgroup (128 threads); `any` also ORs a predicate
+__device__ __forceinline__ bool swg_any(int sw, bool pred) {
   uint32_t r;
   asm volatile(
       "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, %2, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
       : "=r"(r)
-      : "r"((uint32_t)pred), "r"(wg + 1 + kWarpgroups)
+      : "r"((uint32_t)pred), "r"(1 + 2 * sw)
       : "memory");
   return r != 0;
 }
+__device__ __forceinline__ void swg_sync(int sw) { asm volatile("bar.sync %0, 128;\n" ::"r"(2 + 2 * sw) : "memory"); }
 
 // A wait that gives up: marks the CTA as aborted and leaves a trace for the host.
-__device__ __forceinline__ void tc_wait(TcCtx &tc, uint32_t bar, uint32_t parity, unsigned code) {
+__device__ __forceinline__ void tc_wait(TcCtx &tc, const unsigned long long *bar, uint32_t parity, unsigned code) {
   if (*reinterpret_cast<volatile int *>(&tc.sh->abort)) return;
-  if (!tc05::mbar_wait(bar, parity)) {
+  if (!tc05::mbar_wait(tc05::smem_u32(bar), parity & 1u)) {
     tc.sh->abort = 1;
     atomicOr(tc.error_word, code);
   }
 }
+// one arrival per warp, after all its lanes are done
+__device__ __forceinline__ void warp_arrive(const unsigned long long *bar, int lane) {
+  __syncwarp();
+  if (lane == 0) tc05::mbar_arrive(tc05::smem_u32(bar));
+}
+// One ticket per warp (release / acquire at CTA scope); true in every lane of the warp that draws the
+// last of `n`, which also puts the counter back to zero for the buffer's next block.
+__device__ __forceinline__ bool last_ticket(unsigned *counter, unsigned n, int lane) {
+  __syncwarp();
+  unsigned old = 0;
+  if (lane == 0) {
+    asm volatile("atom.acq_rel.cta.shared.add.u32 %0, [%1], 1;\n" : "=r"(old) : "r"(tc05::smem_u32(counter)) : "memory");
+    if (old == n - 1) *reinterpret_cast<volatile unsigned *>(counter) = 0u;
+  }
+  old = __shfl_sync(0xffffffffu, old, 0);
+  return old == n - 1;
+}
 
 template <int BITS> struct RowFmt;
 template <> struct RowFmt<2> {
-  static constexpr int SIGMA_LOG2 = 15;
+  static constexpr int SIGMA_LOG2 = 15, CHUNK_TILES = 16;
   __host__ __device__ static constexpr int pos(int f) { return 2 * (f & 3); }                // f = field 0..7
   __host__ __device__ static constexpr int field(int idx) { return (idx & 15) >> 1; }        // of channel / token index
   // one word (16 codes) -> 8 tensor-memory columns (column f = fields f of the two halves)
@@ -101,7 +133,7 @@ template <> struct RowFmt<2> {
   }
 };
 template <> struct RowFmt<4> {
-  static constexpr int SIGMA_LOG2 = 13;
+  static constexpr int SIGMA_LOG2 = 13, CHUNK_TILES = 8;
   __host__ __device__ static constexpr int pos(int f) { return (f & 1) ? 4 : 0; }            // f = field 0..3
   __host__ __device__ static constexpr int field(int idx) { return (idx & 7) >> 1; }
   // one word (8 codes) -> 4 columns
@@ -129,283 +161,378 @@ __device__ __forceinline__ void fill_q_operand(uint8_t *dst, const float (*s_q)[
   }
 }
 
-// One warpgroup's walk over its blocks of the segment's body tiles [t_lo, t_hi).  Leaves the warpgroup's
-// partial in slot `slot` of (s_m, s_l, part_o).
+// Walks the blocks of the segment's body tiles [t_lo, t_hi) in the order every role uses: streams 0..7,
+// in each stream the run of tiles j with t_lo <= s + 8 j < t_hi in chunks of CHUNK tiles, in each chunk
+// blocks of up to 8 tiles.  on_chunk(chunk index, stream, first stream-tile j, tiles) comes before the
+// chunk's blocks; on_block(block index, chunk index, stream, first stream-tile j of the block, tile offset
+// inside the chunk, live tiles, last block of its chunk).
+template <int CHUNK, class OnChunk, class OnBlock>
+__device__ __forceinline__ void tc_walk(int t_lo, int t_hi, OnChunk on_chunk, OnBlock on_block) {
+  int blk = 0, chunk = 0;
+  for (int s = 0; s < kStreams; ++s) {
+    const int j_lo = t_lo > s ? (t_lo - s + 7) >> 3 : 0, j_hi = t_hi > s ? (t_hi - s + 7) >> 3 : 0;
+    for (int c0 = j_lo; c0 < j_hi; c0 += CHUNK, ++chunk) {
+      const int tiles = min(CHUNK, j_hi - c0);
+      on_chunk(chunk, s, c0, tiles);
+      for (int sb = 0; sb < tiles; sb += 8, ++blk) on_block(blk, chunk, s, c0 + sb, sb, min(8, tiles - sb), sb + 8 >= tiles);
+    }
+  }
+}
+
+// The body tiles [t_lo, t_hi) of a segment, by all warps of the CTA in their roles.  Leaves the two S
+// warpgroups' partials in slots slot0, slot0 + 1 of (s_m, s_l, part_o).  Buffer / stage parities follow the
+// CTA-wide counts tc.gi / tc.gc: block number n uses buffer n mod 2, chunk number m stage m mod kStages, and
+// every completion of a barrier is either waited for or provably over before the barrier can complete again.
 template <int BITS>
 __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const uint8_t *body, int t_lo, int t_hi,
-                                        const float *s_stat, float sigma16, float *s_m, float *s_l, int slot) {
+                                        const float *s_stat, float sigma16, float *s_m, float *s_l, int slot0) {
   using F = RowFmt<BITS>;
   constexpr int TB = tile_bytes(BITS);
+  constexpr int CHUNK = F::CHUNK_TILES;
   constexpr int ROW_BYTES = 16 * BITS;      // a token's K codes
   constexpr int CH_BYTES = 2 * BITS;        // a channel's V codes of one tile
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int wg = warp >> 2, quad = warp & 3;
-  const int tw = threadIdx.x & 127;         // token row of a block (scores) and channel (output)
+  const int quad = warp & 3;
+  const int tw = threadIdx.x & 127;         // token row of a block (K, scores) and channel (V, output)
   const int my_tile = tw >> 4, my_row = tw & 15;
   TcShared *sh = tc.sh;
   const uint32_t t_lane = (uint32_t)(quad * 32) << 16;
-  const uint32_t tA_K = tc.tmem_base + wg * kTmemColsPerWg, tA_V = tA_K + 64, tD_S = tA_K + 128, tD_O = tA_K + 144;
-  uint8_t *stage_base = tc.stages + (size_t)wg * kStagesPerWg * kStageBytes;
-  uint8_t *wbuf = tc.wbuf + wg * kWBufBytes;
-  const uint32_t bar_full0 = tc05::smem_u32(&sh->bar_full[wg][0]);
-  const uint32_t bar_s = tc05::smem_u32(&sh->bar_s[wg]), bar_o = tc05::smem_u32(&sh->bar_o[wg]);
-  const uint32_t q_addr = tc05::smem_u32(tc.q_operand), w_addr = tc05::smem_u32(wbuf);
+  const uint32_t tb = tc.tmem_base;
+  const uint32_t g0 = tc.gi, c0g = tc.gc;
+  {  // every thread advances the CTA-wide counts by this segment's blocks and chunks
+    int nb = 0, nc = 0;
+    for (int s = 0; s < kStreams; ++s) {
+      const int j_lo = t_lo > s ? (t_lo - s + 7) >> 3 : 0, j_hi = t_hi > s ? (t_hi - s + 7) >> 3 : 0;
+      const int r = j_hi - j_lo;
+      nc += (r + CHUNK - 1) / CHUNK;
+      nb += (r / CHUNK) * (CHUNK / 8) + ((r % CHUNK) + 7) / 8;
+    }
+    tc.gi += (uint32_t)nb;
+    tc.gc += (uint32_t)nc;
+  }
   constexpr uint32_t idesc_qk = tc05::idesc_f16(128, 16, 0), idesc_pv = tc05::idesc_f16(128, 16, 1);
-
-  const int kb0 = t_lo >> 3, kb1 = (t_hi - 1) >> 3;
-  // issue the copies of block kb into stage s (warp 0 of the warpgroup; lane i copies tile i)
-  auto issue_block = [&](int kb, int s) {
-    const int lo_i = max(t_lo - 8 * kb, 0), hi_i = min(t_hi - 8 * kb, 8);
-    const uint32_t bar = bar_full0 + 8 * s;
-    if (lane == 0) tc05::mbar_arrive_expect_tx(bar, (uint32_t)((hi_i - lo_i) * TB));
+  // the output MMAs of a block: one per live tile, into the accumulators of the block's S warpgroup
+  auto issue_pv = [&](uint32_t b, int nv) {
+    tc05::fence_after_sync();
+    const bool fresh = *reinterpret_cast<volatile int *>(&sh->pv_fresh[b]) != 0;
+    if (tc05::elect_one()) {
+      const uint32_t w_addr = tc05::smem_u32(tc.wbuf) + kWBufBytes * b;
+      for (int j = 0; j < nv; ++j)
+        tc05::mma_f16_ts(tb + kTmemDO + 16 * b, tb + kTmemAV + 64 * b + 8 * j, tc05::smem_desc(w_addr + 256 * j, 128, 2048), idesc_pv,
+                         (fresh && j == 0) ? 0u : 1u);
+      tc05::mma_commit(tc05::smem_u32(&sh->bar_o[b]));
+    }
     __syncwarp();
-    if (lane >= lo_i && lane < hi_i)
-      tc05::bulk_g2s(tc05::smem_u32(stage_base + (size_t)s * kStageBytes + lane * TB),
-                     body + (size_t)lane * p.geom.stream_stride + (size_t)kb * TB, TB, bar);
   };
 
-  // per-head constants
-  float2 mu2[4], sumq2[4], m2[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    mu2[j] = make_float2(ldexpf(1.0f, 24 - 14 + (int)s_stat[2 * j]), ldexpf(1.0f, 24 - 14 + (int)s_stat[2 * j + 1]));
-    sumq2[j] = make_float2(s_stat[8 + 2 * j], s_stat[8 + 2 * j + 1]);
-    m2[j] = make_float2(kNegBig, kNegBig);
-  }
-  float2 l2[4], zs2[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) l2[j] = zs2[j] = make_float2(0.f, 0.f);
-  const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
-  // the weight of this thread's token row in the output MMA carries the row's code position
-  const float w_unit = ldexpf(1.0f, kEPV - F::pos(F::field(my_row))) / sigma_u;
-
-  if (quad == 0 && kb0 + wg <= kb1) issue_block(kb0 + wg, 0);
-  // The tensor core adds into its fp32 accumulators without rounding to nearest, and the sums of codes
-  // times weights are all of one sign: left to grow over thousands of MMAs the loss shows in the output,
-  // which is the small difference of that sum and the zero-point sum.  So every kEpochBlocks blocks the
-  // accumulators of this thread's channel move into registers (ov) and the tensor-memory sums restart.
-  constexpr int kEpochBlocks = 16;
-  float ov[8];
-#pragma unroll
-  for (int h = 0; h < 8; ++h) ov[h] = 0.f;
-  bool first = true;  // the tensor-memory accumulators hold nothing yet
-  int it = 0, since = 0;
-  for (int kb = kb0 + wg; kb <= kb1; kb += kWarpgroups, ++it) {
-    const int s = it & 1;
-    const int lo_i = max(t_lo - 8 * kb, 0), hi_i = min(t_hi - 8 * kb, 8);
-    const uint8_t *blk = stage_base + (size_t)s * kStageBytes;
-    tc_wait(tc, bar_full0 + 8 * s, (tc.ph_full >> s) & 1u, 1u);
-    tc.ph_full ^= 1u << s;
-
-    // ---- K: token row -> tensor memory ----
-    {
-      const uint8_t *kp = blk + my_tile * TB + my_row * ROW_BYTES;
-      constexpr int HALF_CHUNKS = ROW_BYTES / 32;  // 16-byte chunks per half row
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t r[32];
-#pragma unroll
-        for (int c = 0; c < HALF_CHUNKS; ++c) {
-          const uint4 v = *reinterpret_cast<const uint4 *>(kp + (half * HALF_CHUNKS + c) * 16);
-          const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) F::extract(w4[e], r + (4 * c + e) * (32 / (4 * HALF_CHUNKS)));
-        }
-        tc05::tmem_st32(tA_K + t_lane + 32 * half, r);
-      }
-    }
-    tc05::wait_st();
-    tc05::fence_before_sync();
-    wg_sync(wg);
-    if (tw == 0) {
-      tc05::fence_after_sync();
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        tc05::mma_f16_ts(tD_S, tA_K + 8 * ks, tc05::smem_desc(q_addr + 256 * ks, 128, 2048), idesc_qk, ks > 0 ? 1u : 0u);
-      tc05::mma_commit(bar_s);
-    }
-    // the other stage was last read in the previous block, which every thread has left: refill it
-    if (quad == 0 && kb + kWarpgroups <= kb1) issue_block(kb + kWarpgroups, s ^ 1);
-
-    // ---- V: channel row -> tensor memory (after the previous block's output MMAs have read it) ----
-    {
-      uint32_t r[64];
-      const uint8_t *vp = blk + v_part_offset(BITS) + tw * CH_BYTES;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if constexpr (BITS == 2) {
-          F::extract(*reinterpret_cast<const uint32_t *>(vp + i * TB), r + 8 * i);
-        } else {
-          const uint2 v = *reinterpret_cast<const uint2 *>(vp + i * TB);
-          F::extract(v.x, r + 8 * i);
-          F::extract(v.y, r + 8 * i + 4);
+  if (false) {
+  } else if (warp < kWarpV) {
+    // ---- K: token row -> tensor memory; the last warp of a block issues the score MMAs ----
+    const uint32_t q_addr = tc05::smem_u32(tc.q_operand);
+    // Warp 0 also feeds the ring: one bulk copy per chunk, kStages - 1 chunks ahead of the chunk it works on.
+    int cp_s = 0, cp_j = 0, cp_hi = 0, cp_n = 0;  // next chunk to copy: stream, first stream-tile, end of the stream's run, chunk index
+    auto copy_next = [&]() {
+      while (cp_s < kStreams && cp_j >= cp_hi) {  // next stream with tiles left
+        ++cp_s;
+        if (cp_s < kStreams) {
+          cp_j = t_lo > cp_s ? (t_lo - cp_s + 7) >> 3 : 0;
+          cp_hi = t_hi > cp_s ? (t_hi - cp_s + 7) >> 3 : 0;
         }
       }
-      if (it > 0) {
-        tc_wait(tc, bar_o, tc.ph_o, 4u);
-        tc.ph_o ^= 1u;
-        tc05::fence_after_sync();
-        if (since == kEpochBlocks) {
-          uint32_t o[16];
-          tc05::tmem_ld16(tD_O + t_lane, o);
-          tc05::wait_ld();
-#pragma unroll
-          for (int h = 0; h < 8; ++h) ov[h] += fmaf(__uint_as_float(o[8 + h]), 0x1p-11f, __uint_as_float(o[h]));
-          first = true;
-          since = 0;
-        }
+      if (cp_s >= kStreams) return;
+      const int tiles = min(CHUNK, cp_hi - cp_j);
+      const uint32_t m = c0g + cp_n, st = m % kStages;
+      if (cp_n >= kStages) tc_wait(tc, &sh->stage_free[st], m / kStages - 1, 8u);
+      if (lane == 0) {
+        const uint32_t bar = tc05::smem_u32(&sh->full[st]);
+        tc05::mbar_arrive_expect_tx(bar, (uint32_t)(tiles * TB));
+        tc05::bulk_g2s(tc05::smem_u32(tc.stages + (size_t)st * kStageBytes), body + (size_t)cp_s * p.geom.stream_stride + (size_t)cp_j * TB,
+                       (uint32_t)(tiles * TB), bar);
       }
-      tc05::tmem_st32(tA_V + t_lane, r);
-      tc05::tmem_st32(tA_V + t_lane + 32, r + 32);
+      __syncwarp();
+      cp_j += tiles;
+      ++cp_n;
+    };
+    if (warp == 0) {
+      cp_j = (t_lo + 7) >> 3;
+      cp_hi = (t_hi + 7) >> 3;
+      for (int c = 0; c < kStages - 1; ++c) copy_next();
     }
-
-    // ---- scores of this thread's token ----
-    tc_wait(tc, bar_s, tc.ph_s, 2u);
-    tc.ph_s ^= 1u;
-    tc05::fence_after_sync();
-    uint32_t sraw[16];
-    tc05::tmem_ld16(tD_S + t_lane, sraw);
-    tc05::wait_ld();
-    const bool alive = my_tile >= lo_i && my_tile < hi_i && ((8 * kb + my_tile) * 16 + my_row) < p.n_body;
-    float4 meta = *reinterpret_cast<const float4 *>(blk + my_tile * TB + meta_offset(BITS) + my_row * 16);  // S_K Z_K S_V Z_V
-    if (!alive) meta = make_float4(0.f, 0.f, 0.f, 0.f);  // a dead row holds arbitrary bytes
-    float2 dot[4], a2[4], arg[4];
+    tc_walk<CHUNK>(t_lo, t_hi,
+        [&](int chunk, int, int, int) {
+          if (warp == 0) copy_next();
+          tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u);
+        },
+        [&](int i, int chunk, int, int, int sb, int, bool last_of_chunk) {
+          const uint32_t n = g0 + i, b = n & 1u, st = (c0g + chunk) % kStages;
+          const uint8_t *kp = tc.stages + (size_t)st * kStageBytes + (sb + my_tile) * TB + my_row * ROW_BYTES;
+          constexpr int HALF_CHUNKS = ROW_BYTES / 32;  // 16-byte chunks per half row
+          uint4 raw[2 * HALF_CHUNKS];
+#pragma unroll
+          for (int c = 0; c < 2 * HALF_CHUNKS; ++c) raw[c] = *reinterpret_cast<const uint4 *>(kp + c * 16);
+          if (i >= 2) {  // the score MMAs of the block that used this buffer have read it
+            tc_wait(tc, &sh->bar_s[b], (n >> 1) - 1, 2u);
+            tc05::fence_after_sync();
+          }
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t r[32];
+#pragma unroll
+            for (int c = 0; c < HALF_CHUNKS; ++c) {
+              const uint4 v = raw[half * HALF_CHUNKS + c];
+              const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) F::extract(w4[e], r + (4 * c + e) * (32 / (4 * HALF_CHUNKS)));
+            }
+            tc05::tmem_st32(tb + kTmemAK + 64 * b + t_lane + 32 * half, r);
+          }
+          tc05::wait_st();
+          tc05::fence_before_sync();
+          if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
+          if (last_ticket(&sh->k_tickets[b], 4, lane)) {
+            if (i >= 2) tc_wait(tc, &sh->ds_free[b], (n >> 1) - 1, 16u);  // the scores of the buffer's last block have been read
+            tc05::fence_after_sync();
+            if (tc05::elect_one()) {
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks)
+                tc05::mma_f16_ts(tb + kTmemDS + 16 * b, tb + kTmemAK + 64 * b + 8 * ks, tc05::smem_desc(q_addr + 256 * ks, 128, 2048),
+                                 idesc_qk, ks > 0 ? 1u : 0u);
+              tc05::mma_commit(tc05::smem_u32(&sh->bar_s[b]));
+            }
+            __syncwarp();
+          }
+        });
+  } else if (warp < kWarpS) {
+    // ---- V: channel row -> tensor memory ----
+    tc_walk<CHUNK>(t_lo, t_hi,
+        [&](int chunk, int, int, int) { tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u); },
+        [&](int i, int chunk, int, int, int sb, int nv, bool last_of_chunk) {
+          const uint32_t n = g0 + i, b = n & 1u, st = (c0g + chunk) % kStages;
+          const uint8_t *vp = tc.stages + (size_t)st * kStageBytes + sb * TB + v_part_offset(BITS) + tw * CH_BYTES;
+          if (i >= 2) {  // the output MMAs of the block that used this buffer have read it
+            tc_wait(tc, &sh->bar_o[b], (n >> 1) - 1, 4u);
+            tc05::fence_after_sync();
+          }
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t r[32];
+#pragma unroll
+            for (int t4 = 0; t4 < 4; ++t4) {
+              const int t8 = 4 * half + t4;
+              if constexpr (BITS == 2) {
+                F::extract(*reinterpret_cast<const uint32_t *>(vp + t8 * TB), r + 8 * t4);
+              } else {
+                const uint2 v = *reinterpret_cast<const uint2 *>(vp + t8 * TB);
+                F::extract(v.x, r + 8 * t4);
+                F::extract(v.y, r + 8 * t4 + 4);
+              }
+            }
+            tc05::tmem_st32(tb + kTmemAV + 64 * b + t_lane + 32 * half, r);
+          }
+          tc05::wait_st();
+          tc05::fence_before_sync();
+          if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
+          if (last_ticket(&sh->p_tickets[b], 8, lane)) issue_pv(b, nv);
+        });
+  } else {
+    // ---- S: scores -> probabilities -> weights; running sums; this warpgroup's partial ----
+    const uint32_t sw = (uint32_t)(warp - kWarpS) >> 2;   // S warpgroup 0 / 1: owns the blocks with n mod 2 == sw
+    float2 mu2[4], sumq2[4], m2[4], l2[4], zs2[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      dot[j] = __fadd2_rn(make_float2(__uint_as_float(sraw[2 * j]), __uint_as_float(sraw[2 * j + 1])),
-                          make_float2(__uint_as_float(sraw[8 + 2 * j]), __uint_as_float(sraw[8 + 2 * j + 1])));
-      a2[j] = __fmul2_rn(mu2[j], make_float2(meta.x, meta.x));
-      const float2 b = __ffma2_rn(make_float2(meta.y, meta.y), sumq2[j], make_float2(-m2[j].x, -m2[j].y));
-      arg[j] = __ffma2_rn(a2[j], dot[j], b);
-      if (!alive) arg[j] = make_float2(-INFINITY, -INFINITY);
+      mu2[j] = make_float2(ldexpf(1.0f, 24 - 14 + (int)s_stat[2 * j]), ldexpf(1.0f, 24 - 14 + (int)s_stat[2 * j + 1]));
+      sumq2[j] = make_float2(s_stat[8 + 2 * j], s_stat[8 + 2 * j + 1]);
+      m2[j] = make_float2(kNegBig, kNegBig);
+      l2[j] = zs2[j] = make_float2(0.f, 0.f);
     }
-    float amax = fmaxf(fmaxf(fmaxf(arg[0].x, arg[0].y), fmaxf(arg[1].x, arg[1].y)),
-                       fmaxf(fmaxf(arg[2].x, arg[2].y), fmaxf(arg[3].x, arg[3].y)));
-    if (wg_any(wg, amax > kMaxAhead)) {
-      // ---- the reference moves: block maxima of the true scores, new reference, rescale ----
-      float2 sc[4];
+    const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
+    // the weight of this thread's token row in the output MMA carries the row's code position
+    const float w_unit = ldexpf(1.0f, kEPV - F::pos(F::field(my_row))) / sigma_u;
+    // The tensor core adds into its fp32 accumulators without rounding to nearest, and the sums of codes
+    // times weights are all of one sign: left to grow over thousands of MMAs the loss shows in the output,
+    // which is the small difference of that sum and the zero-point sum.  So every kEpochBlocks blocks the
+    // accumulators of this thread's channel move into registers (ov) and the tensor-memory sums restart.
+    constexpr int kEpochBlocks = 16;
+    float ov[8];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        sc[j] = __ffma2_rn(a2[j], dot[j], __fmul2_rn(make_float2(meta.y, meta.y), sumq2[j]));
-        if (!alive) sc[j] = make_float2(kNegBig, kNegBig);
-        float mx = sc[j].x, my = sc[j].y;
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-          my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, o));
-        }
-        if (lane == 0) { sh->wmax[wg][quad][2 * j] = mx; sh->wmax[wg][quad][2 * j + 1] = my; }
+    for (int h = 0; h < 8; ++h) ov[h] = 0.f;
+    bool fresh = true;       // the tensor-memory accumulators hold nothing yet
+    int since = 0;
+    int mine_last = -1;      // last block (segment-local index) this warpgroup has handed to the output MMA
+    int o_seen = -1;         // last such block whose output MMAs are known complete
+    const uint32_t tDO = tb + kTmemDO + 16 * sw + t_lane, tDS = tb + kTmemDS + 16 * sw + t_lane;
+    auto wait_o = [&](int blk) {  // output MMAs of this warpgroup's block blk (and its earlier ones) are complete
+      if (blk >= 0 && o_seen < blk) {
+        tc_wait(tc, &sh->bar_o[sw], (g0 + blk) >> 1, 4u);
+        tc05::fence_after_sync();
+        o_seen = blk;
       }
-      wg_sync(wg);
-      float f[8];
+    };
+    tc_walk<CHUNK>(t_lo, t_hi,
+        [&](int chunk, int, int, int) { tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u); },
+        [&](int i, int chunk, int s, int j0, int sb, int nv, bool last_of_chunk) {
+          const uint32_t n = g0 + i, b = n & 1u, st = (c0g + chunk) % kStages;
+          if (b != sw) {  // the other warpgroup's block; a chunk is released by both
+            if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
+            return;
+          }
+          const uint8_t *blk = tc.stages + (size_t)st * kStageBytes + sb * TB;
+          // token row (my_tile, my_row) of the block is token 16 (s + 8 (j0 + my_tile)) + my_row of the body
+          const bool alive = my_tile < nv && ((s + 8 * (j0 + my_tile)) * 16 + my_row) < p.n_body;
+          float4 meta = *reinterpret_cast<const float4 *>(blk + my_tile * TB + meta_offset(BITS) + my_row * 16);  // S_K Z_K S_V Z_V
+          if (!alive) meta = make_float4(0.f, 0.f, 0.f, 0.f);  // a dead row holds arbitrary bytes
+          if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
+          tc_wait(tc, &sh->bar_s[b], n >> 1, 2u);
+          tc05::fence_after_sync();
+          uint32_t sraw[16];
+          tc05::tmem_ld16(tDS, sraw);
+          tc05::wait_ld();
+          tc05::fence_before_sync();
+          warp_arrive(&sh->ds_free[b], lane);
+          float2 dot[4], a2[4], arg[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float nx = m2[j].x, ny = m2[j].y;
+          for (int j = 0; j < 4; ++j) {
+            dot[j] = __fadd2_rn(make_float2(__uint_as_float(sraw[2 * j]), __uint_as_float(sraw[2 * j + 1])),
+                                make_float2(__uint_as_float(sraw[8 + 2 * j]), __uint_as_float(sraw[8 + 2 * j + 1])));
+            a2[j] = __fmul2_rn(mu2[j], make_float2(meta.x, meta.x));
+            const float2 bb = __ffma2_rn(make_float2(meta.y, meta.y), sumq2[j], make_float2(-m2[j].x, -m2[j].y));
+            arg[j] = __ffma2_rn(a2[j], dot[j], bb);
+            if (!alive) arg[j] = make_float2(-INFINITY, -INFINITY);
+          }
+          const float amax = fmaxf(fmaxf(fmaxf(arg[0].x, arg[0].y), fmaxf(arg[1].x, arg[1].y)),
+                                   fmaxf(fmaxf(arg[2].x, arg[2].y), fmaxf(arg[3].x, arg[3].y)));
+          if (swg_any(sw, amax > kTcMaxAhead)) {
+            // ---- the reference moves: block maxima of the true scores, new reference, rescale ----
+            float2 sc[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          nx = fmaxf(nx, sh->wmax[wg][q][2 * j]);
-          ny = fmaxf(ny, sh->wmax[wg][q][2 * j + 1]);
-        }
-        f[2 * j] = ex2(m2[j].x - nx);
-        f[2 * j + 1] = ex2(m2[j].y - ny);
-        m2[j] = make_float2(nx, ny);
-        l2[j] = __fmul2_rn(l2[j], make_float2(f[2 * j], f[2 * j + 1]));
-        zs2[j] = __fmul2_rn(zs2[j], make_float2(f[2 * j], f[2 * j + 1]));
-        ov[2 * j] *= f[2 * j];
-        ov[2 * j + 1] *= f[2 * j + 1];
-        arg[j] = __fadd2_rn(sc[j], make_float2(-nx, -ny));
-        if (!alive) arg[j] = make_float2(-INFINITY, -INFINITY);
-      }
-      if (!first) {  // the output accumulators of channel row tw (every earlier output MMA has completed)
-        uint32_t o[16];
-        tc05::tmem_ld16(tD_O + t_lane, o);
-        tc05::wait_ld();
+            for (int j = 0; j < 4; ++j) {
+              sc[j] = __ffma2_rn(a2[j], dot[j], __fmul2_rn(make_float2(meta.y, meta.y), sumq2[j]));
+              if (!alive) sc[j] = make_float2(kNegBig, kNegBig);
+              float mx = sc[j].x, my = sc[j].y;
 #pragma unroll
-        for (int h = 0; h < 8; ++h) {
-          o[h] = __float_as_uint(__uint_as_float(o[h]) * f[h]);
-          o[8 + h] = __float_as_uint(__uint_as_float(o[8 + h]) * f[h]);
-        }
-        tc05::tmem_st16(tD_O + t_lane, o);
-      }
-      wg_sync(wg);  // wmax may be rewritten by the next slow path
-    }
+              for (int o = 16; o; o >>= 1) {
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, o));
+              }
+              if (lane == 0) { sh->wmax[sw][quad][2 * j] = mx; sh->wmax[sw][quad][2 * j + 1] = my; }
+            }
+            swg_sync(sw);
+            float f[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              float bx = kNegBig, by = kNegBig;
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                bx = fmaxf(bx, sh->wmax[sw][q][2 * j]);
+                by = fmaxf(by, sh->wmax[sw][q][2 * j + 1]);
+              }
+              const float nx = fmaxf(m2[j].x, bx + kTcHeadroom), ny = fmaxf(m2[j].y, by + kTcHeadroom);
+              f[2 * j] = ex2(m2[j].x - nx);
+              f[2 * j + 1] = ex2(m2[j].y - ny);
+              m2[j] = make_float2(nx, ny);
+              l2[j] = __fmul2_rn(l2[j], make_float2(f[2 * j], f[2 * j + 1]));
+              zs2[j] = __fmul2_rn(zs2[j], make_float2(f[2 * j], f[2 * j + 1]));
+              ov[2 * j] *= f[2 * j];
+              ov[2 * j + 1] *= f[2 * j + 1];
+              arg[j] = __fadd2_rn(sc[j], make_float2(-nx, -ny));
+              if (!alive) arg[j] = make_float2(-INFINITY, -INFINITY);
+            }
+            if (!fresh) {  // the output accumulators of channel row tw, once this warpgroup's output MMAs are complete
+              wait_o(mine_last);
+              uint32_t o[16];
+              tc05::tmem_ld16(tDO, o);
+              tc05::wait_ld();
+#pragma unroll
+              for (int h = 0; h < 8; ++h) {
+                o[h] = __float_as_uint(__uint_as_float(o[h]) * f[h]);
+                o[8 + h] = __float_as_uint(__uint_as_float(o[8 + h]) * f[h]);
+              }
+              tc05::tmem_st16(tDO, o);
+              tc05::wait_st();
+            }
+            swg_sync(sw);  // wmax may be rewritten by the next move
+          }
+          if (since == kEpochBlocks) {  // move the accumulators into registers; the next output MMA starts afresh
+            wait_o(mine_last);
+            uint32_t o[16];
+            tc05::tmem_ld16(tDO, o);
+            tc05::wait_ld();
+#pragma unroll
+            for (int h = 0; h < 8; ++h) ov[h] += fmaf(__uint_as_float(o[8 + h]), 0x1p-11f, __uint_as_float(o[h]));
+            fresh = true;
+            since = 0;
+          }
 
-    // ---- probabilities and weights: w = p * S_V goes to the output MMA as fp16 hi + lo (22 bits), in
-    //      columns h and 8 + h of the B operand; the sums take p itself ----
-    {
-      // a constant V group has S_V = 0 and all codes 0: any finite unit will do for it
-      const float s_e = meta.z == 0.f ? w_unit : meta.z * w_unit;
-      uint32_t whi[4], wlo[4];
+          // ---- probabilities and weights: w = p * S_V goes to the output MMA as fp16 hi + lo (22 bits), in
+          //      columns h and 8 + h of the B operand; the sums take p itself ----
+          // a constant V group has S_V = 0 and all codes 0: any finite unit will do for it
+          const float s_e = meta.z == 0.f ? w_unit : meta.z * w_unit;
+          uint32_t whi[4], wlo[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 e = make_float2(ex2(arg[j].x), ex2(arg[j].y));
-        const float2 w = __fmul2_rn(e, make_float2(s_e, s_e));
-        whi[j] = pack_half2(w.x, w.y);
-        const float2 back = __half22float2(*reinterpret_cast<const __half2 *>(&whi[j]));
-        const float2 rest = __fmul2_rn(__fadd2_rn(w, make_float2(-back.x, -back.y)), make_float2(2048.f, 2048.f));
-        wlo[j] = pack_half2(rest.x, rest.y);
-        l2[j] = __fadd2_rn(l2[j], e);
-        zs2[j] = __ffma2_rn(e, make_float2(meta.w, meta.w), zs2[j]);
-      }
-      *reinterpret_cast<uint4 *>(wbuf + tw * 16) = make_uint4(whi[0], whi[1], whi[2], whi[3]);
-      *reinterpret_cast<uint4 *>(wbuf + 2048 + tw * 16) = make_uint4(wlo[0], wlo[1], wlo[2], wlo[3]);
-    }
-    tc05::fence_async_smem();
-    tc05::wait_st();
-    tc05::fence_before_sync();
-    wg_sync(wg);
-    if (tw == 0) {
-      tc05::fence_after_sync();
-      for (int j = lo_i; j < hi_i; ++j)
-        tc05::mma_f16_ts(tD_O, tA_V + 8 * j, tc05::smem_desc(w_addr + 256 * j, 128, 2048), idesc_pv,
-                         (first && j == lo_i) ? 0u : 1u);
-      tc05::mma_commit(bar_o);
-    }
-    first = false;
-    ++since;
-  }
+          for (int j = 0; j < 4; ++j) {
+            const float2 e = make_float2(ex2(arg[j].x), ex2(arg[j].y));
+            const float2 w = __fmul2_rn(e, make_float2(s_e, s_e));
+            whi[j] = pack_half2(w.x, w.y);
+            const float2 back = __half22float2(*reinterpret_cast<const __half2 *>(&whi[j]));
+            const float2 rest = __fmul2_rn(__fadd2_rn(w, make_float2(-back.x, -back.y)), make_float2(2048.f, 2048.f));
+            wlo[j] = pack_half2(rest.x, rest.y);
+            l2[j] = __fadd2_rn(l2[j], e);
+            zs2[j] = __ffma2_rn(e, make_float2(meta.w, meta.w), zs2[j]);
+          }
+          wait_o(mine_last);  // the output MMAs that read this weight buffer are complete
+          uint8_t *wbuf = tc.wbuf + kWBufBytes * b;
+          *reinterpret_cast<uint4 *>(wbuf + tw * 16) = make_uint4(whi[0], whi[1], whi[2], whi[3]);
+          *reinterpret_cast<uint4 *>(wbuf + 2048 + tw * 16) = make_uint4(wlo[0], wlo[1], wlo[2], wlo[3]);
+          if (tw == 0) sh->pv_fresh[b] = fresh ? 1 : 0;
+          tc05::fence_async_smem();
+          tc05::fence_before_sync();
+          if (last_ticket(&sh->p_tickets[b], 8, lane)) issue_pv(b, nv);
+          mine_last = i;
+          fresh = false;
+          ++since;
+        });
 
-  // ---- the warpgroup's partial: (m, l, o[128]) per head ----
-  if (it > 0) {
-    tc_wait(tc, bar_o, tc.ph_o, 4u);
-    tc.ph_o ^= 1u;
-    tc05::fence_after_sync();
-    uint32_t o[16];
-    tc05::tmem_ld16(tD_O + t_lane, o);
-    tc05::wait_ld();
+    // ---- this warpgroup's partial: (m, l, o[128]) per head ----
+    if (mine_last >= 0) {
+      wait_o(mine_last);
+      uint32_t o[16];
+      tc05::tmem_ld16(tDO, o);
+      tc05::wait_ld();
+#pragma unroll
+      for (int h = 0; h < 8; ++h) ov[h] += fmaf(__uint_as_float(o[8 + h]), 0x1p-11f, __uint_as_float(o[h]));
+    }
     const float f_out = ldexpf(sigma_u, 24 - kEPV);
+    // sums over the 128 token rows
+    float red[16];
 #pragma unroll
-    for (int h = 0; h < 8; ++h) ov[h] = (ov[h] + fmaf(__uint_as_float(o[8 + h]), 0x1p-11f, __uint_as_float(o[h]))) * f_out;
-  }
-  // sums over the warpgroup's 128 token rows
-  float red[16];
+    for (int j = 0; j < 4; ++j) {
+      red[2 * j] = l2[j].x; red[2 * j + 1] = l2[j].y;
+      red[8 + 2 * j] = zs2[j].x; red[8 + 2 * j + 1] = zs2[j].y;
+    }
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    red[2 * j] = l2[j].x; red[2 * j + 1] = l2[j].y;
-    red[8 + 2 * j] = zs2[j].x; red[8 + 2 * j + 1] = zs2[j].y;
-  }
+    for (int k = 0; k < 16; ++k) {
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+      for (int o = 16; o; o >>= 1) red[k] += __shfl_xor_sync(0xffffffffu, red[k], o);
+    }
+    if (lane == 0) {
 #pragma unroll
-    for (int o = 16; o; o >>= 1) red[i] += __shfl_xor_sync(0xffffffffu, red[i], o);
-  }
-  if (lane == 0) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) sh->sums[wg][quad][i] = red[i];
-  }
-  tc05::fence_before_sync();
-  wg_sync(wg);
-  float (*po)[kHeadDim] = reinterpret_cast<float (*)[kHeadDim]>(tc.part_o + (size_t)slot * kMaxGroup * kHeadDim);
-#pragma unroll
-  for (int h = 0; h < 8; ++h) {
-    const float zs = sh->sums[wg][0][8 + h] + sh->sums[wg][1][8 + h] + sh->sums[wg][2][8 + h] + sh->sums[wg][3][8 + h];
-    po[h][tw] = ov[h] + zs;
-  }
-  if (tw == 0) {
+      for (int k = 0; k < 16; ++k) sh->sums[sw][quad][k] = red[k];
+    }
+    tc05::fence_before_sync();
+    swg_sync(sw);
+    const int slot = slot0 + (int)sw;
+    float (*po)[kHeadDim] = reinterpret_cast<float (*)[kHeadDim]>(tc.part_o + (size_t)slot * kMaxGroup * kHeadDim);
 #pragma unroll
     for (int h = 0; h < 8; ++h) {
-      s_m[slot * 8 + h] = (h & 1) ? m2[h >> 1].y : m2[h >> 1].x;
-      s_l[slot * 8 + h] = sh->sums[wg][0][h] + sh->sums[wg][1][h] + sh->sums[wg][2][h] + sh->sums[wg][3][h];
+      const float zs = sh->sums[sw][0][8 + h] + sh->sums[sw][1][8 + h] + sh->sums[sw][2][8 + h] + sh->sums[sw][3][8 + h];
+      po[h][tw] = fmaf(ov[h], f_out, zs);
+    }
+    if (tw == 0) {
+#pragma unroll
+      for (int h = 0; h < 8; ++h) {
+        s_m[slot * 8 + h] = (h & 1) ? m2[h >> 1].y : m2[h >> 1].x;
+        s_l[slot * 8 + h] = sh->sums[sw][0][h] + sh->sums[sw][1][h] + sh->sums[sw][2][h] + sh->sums[sw][3][h];
+      }
     }
   }
 }
