@@ -70,6 +70,10 @@ typedef struct {
   int32_t shift_variant;  /* how a halving 2b -> b is done (Sec. 4.4.1): 0 Equivalent Right Shift, Eq. 3 (the
                              method); 1 Direct Right Shift (X >> b, S_b = (2^b+1) S_2b, Z kept); 2 Modified
                              Right Shift (X >> b, S_b = 2^b S_2b, Z_b = Z_2b + (S_b - S_2b)/2) */
+  int32_t attention_path; /* which contraction the 4- and 2-bit body is laid out for (chosen once, when the cache is
+                             created, because it fixes the order of the codes inside a tile): 0 warp-level MMAs
+                             (mma.sync, register operands; the faster one as measured), 1 tensor memory
+                             (tcgen05.mma with the code operands unpacked into tensor memory) */
 } pmkvq_config;
 
 /* Bytes of device arena a cache with this configuration needs (d_arena / arena_bytes are

@@ -37,6 +37,7 @@ class _Config(ctypes.Structure):
         ("n_sink", ctypes.c_int32), ("window", ctypes.c_int32), ("evict_chunk", ctypes.c_int32),
         ("count_metadata", ctypes.c_int32), ("auto_reduce", ctypes.c_int32), ("sm_scale", ctypes.c_float),
         ("d_arena", ctypes.c_void_p), ("arena_bytes", ctypes.c_size_t), ("shift_variant", ctypes.c_int32),
+        ("attention_path", ctypes.c_int32),
     ]
 
 
@@ -172,7 +173,7 @@ class Cache:
                  fbit: Sequence[int], budget_bytes: Optional[Sequence[int]] = None,
                  lam: Optional[np.ndarray] = None, n_sink: int = 1, window: int = 128, evict_chunk: int = 1,
                  count_metadata: bool = True, auto_reduce: bool = True, sm_scale: float = 0.0,
-                 device: str = "cuda:0", shift_variant: int = 0):
+                 device: str = "cuda:0", shift_variant: int = 0, attention_path: int = 0):
         self._h = None
         self.layers, self.q_heads, self.kv_heads, self.batch = layers, q_heads, kv_heads, batch
         self._fbit = (ctypes.c_uint8 * layers)(*[int(b) for b in fbit])
@@ -189,6 +190,7 @@ class Cache:
         cfg.n_sink, cfg.window, cfg.evict_chunk = n_sink, window, evict_chunk
         cfg.count_metadata, cfg.auto_reduce, cfg.sm_scale = int(count_metadata), int(auto_reduce), float(sm_scale)
         cfg.shift_variant = int(shift_variant)
+        cfg.attention_path = int(attention_path)
         need = lib().pmkvq_arena_bytes_required(ctypes.byref(cfg))
         if need == 0:
             raise PmkvqError(INVALID_ARG, "pmkvq_arena_bytes_required")

@@ -142,6 +142,25 @@ __device__ __forceinline__ uint32_t high_bytes(uint32_t x) { return __byte_perm(
 // is also how far apart the warps of a CTA can finish, so the ring is kept shallow: 16 warps per SM
 // already keep about 70 KB in flight).
 template <int BITS> struct Fmt;
+template <> struct Fmt<2> {
+  static constexpr int N = 8, EQ = 14, EP = 12, SIGMA_LOG2 = 15, NT = 2, SLOTS = 2;
+  __host__ __device__ static constexpr int pos(int j) { return j < 5 ? 2 * j : 2 * j - 5; }
+  __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[8]) {
+    const uint32_t xr = x >> 5;
+    e[0] = x & 0x00030003u; e[1] = x & 0x000C000Cu; e[2] = x & 0x00300030u; e[3] = x & 0x00C000C0u;
+    e[4] = x & 0x03000300u;
+    e[5] = xr & 0x00600060u; e[6] = xr & 0x01800180u; e[7] = xr & 0x06000600u;
+  }
+};
+template <> struct Fmt<4> {
+  static constexpr int N = 4, EQ = 14, EP = 12, SIGMA_LOG2 = 13, NT = 2, SLOTS = 2;
+  __host__ __device__ static constexpr int pos(int j) { return (j & 1) ? 4 : 0; }
+  __device__ static __forceinline__ void extract(uint32_t x, uint32_t (&e)[4]) {
+    const uint32_t xr = x >> 8;
+    e[0] = x & 0x000F000Fu; e[1] = x & 0x00F000F0u;
+    e[2] = xr & 0x000F000Fu; e[3] = xr & 0x00F000F0u;
+  }
+};
 template <> struct Fmt<8> {
   static constexpr int N = 2, EQ = 14, EP = 12, SIGMA_LOG2 = 9, NT = 1, SLOTS = 2;
   __host__ __device__ static constexpr int pos(int) { return 0; }
@@ -656,17 +675,16 @@ __device__ __forceinline__ void segment_ranges(const AttnParams &p, long long u_
   }
 }
 
-// One segment with a 16- or 8-bit body: the part [u_lo, u_hi) (units relative to the slice) of one slice
+// One segment on the warp-level MMA path: the part [u_lo, u_hi) (units relative to the slice) of one slice
 // that this CTA owns.  Builds the slice's query, runs the INT16 tiles and then the body tiles (width
 // BITS) of the range, merges the warps and publishes one partial per head.  The warps of the CTA draw
-// work from two shared counters (INT16 tiles, then body tiles), so they all finish together whatever share
-// of the issue slots each of them gets.  `ring` is the CTA's dynamic shared memory: the per-warp cp.async
-// stages while tiles stream, then the warps' outputs.
+// work from two shared counters (INT16 tiles, then body steps of NT tiles), so they all finish together
+// whatever share of the issue slots each of them gets.  `ring` is the CTA's dynamic shared memory: the
+// per-warp cp.async stages while tiles stream, then the warps' outputs.
 template <int BITS>
 __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long long u_lo, long long u_hi,
                                             float (*s_q)[kHeadDim], float *s_stat, int *s_ctr, uint4 *s_frag,
                                             uint8_t *ring) {
-  static_assert(BITS == 16 || BITS == 8, "narrower bodies take the tensor-memory path");
   using F = Fmt<BITS>;
   using F16 = Fmt<16>;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2;
@@ -679,28 +697,35 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   segment_ranges(p, u_lo, u_hi, a_lo, a_hi, t_lo, t_hi);
   const uint8_t *slice_base = p.geom.base + (size_t)slice * p.geom.slice_stride;
 
-  // ---- body stream set-up: claim the first tiles and start their copies before anything else ----
+  // ---- body stream set-up: claim the first steps and start their copies before anything else ----
   constexpr int TB = tile_bytes(BITS);
-  constexpr int S = F::SLOTS > 0 ? F::SLOTS : 1;
-  const int n_steps = t_hi - t_lo;
+  constexpr int NT = F::NT, S = F::SLOTS > 0 ? F::SLOTS : 1, SB = NT * TB;
+  const int n_steps = (t_hi - t_lo + NT - 1) / NT;
   const uint8_t *body = slice_base + p.geom.body_off;
   const size_t stream_stride = p.geom.stream_stride;
-  uint8_t *my_ring = ring + (size_t)warp * S * TB;
+  uint8_t *my_ring = ring + (size_t)warp * S * SB;
   const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
   auto claim = [&](int which) { return claim_next(s_ctr + which, lane); };
+  // step j = tiles t_lo + NT j .. + NT - 1 (consecutive tiles sit in consecutive streams); 16-byte chunk
+  // c of the step belongs to tile c / (TB / 16)
   auto issue = [&](int j, int slot) {
-    const uint8_t *src = body + body_tile_offset(t_lo + j, BITS, stream_stride) + lane * 16;
-    const uint32_t dst = ring_addr + slot * TB + lane * 16;
+    const int t0 = t_lo + NT * j;
+    constexpr int CPT = TB / 16;  // 16-byte chunks per tile: lane l copies chunks l, l + 32, ...
 #pragma unroll
-    for (int c = 0; c < (TB / 16 + 31) / 32; ++c)
-      if (c * 32 + lane < TB / 16) cp_async16(dst + c * 512, src + c * 512);
+    for (int k = 0; k < NT; ++k) {
+      if (t0 + k < t_hi) {
+        const uint8_t *src = body + body_tile_offset(t0 + k, BITS, stream_stride) + lane * 16;
+        const uint32_t dst = ring_addr + slot * SB + k * TB + lane * 16;
+        cp_async_run<CPT / 32>(dst, src);
+        if (CPT % 32 != 0 && lane < CPT % 32) cp_async16_at<(CPT / 32) * 512>(dst, src);
+      }
+    }
   };
-  const bool worker = warp < kAttnWarps;  // the last warp of the CTA only serves the tensor-memory path
-  int pending[S];  // tiles claimed and in flight, oldest first (>= n_steps: none)
+  int pending[S];  // steps claimed and in flight, oldest first (>= n_steps: none)
   if constexpr (F::SLOTS > 0) {
 #pragma unroll
     for (int i = 0; i < S - 1; ++i) {
-      pending[i] = (n_steps > 0 && worker) ? claim(1) : n_steps;
+      pending[i] = n_steps > 0 ? claim(1) : 0;
       if (pending[i] < n_steps) issue(pending[i], i);
       cp_async_commit();
     }
@@ -720,7 +745,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   for (int mt = 0; mt < 8; ++mt) st.acc[mt][0] = st.acc[mt][1] = st.acc[mt][2] = st.acc[mt][3] = 0.f;
 
   // ---- INT16 tiles (sink + window ring) ----
-  if (a_hi > a_lo && worker) {
+  if (a_hi > a_lo) {
     run_int16_tiles(p, slice_base, a_lo, a_hi, st, s_frag, s_ctr, e_g, sumq, sigma16, lane);
     if constexpr (BITS != 16) {
       // accumulator units change with the width: INT16 units -> body units (exact powers of two)
@@ -738,7 +763,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
 
   // ---- body tiles ----
   const float sigma_u = sigma16 * ldexpf(1.0f, F::SIGMA_LOG2);
-  if (n_steps > 0 && worker) {
+  if (n_steps > 0) {
     QFrag qa;
     qa.mine = (BITS != 16 ? s_frag + 256 : s_frag) + lane;
     const float mu = ldexpf(1.0f, 24 - F::EQ + e_g);
@@ -759,10 +784,20 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
         cp_async_commit();
         cp_async_wait<S - 1>();
         __syncwarp();
-        const uint8_t *tile = my_ring + slot * TB;
-        const int t = t_lo + pending[0];
-        if (t == tail_tile) process_tiles<BITS, 1, true>(tile, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
-        else process_tiles<BITS, 1, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+        const uint8_t *tile = my_ring + slot * SB;
+        const int t = t_lo + NT * pending[0];
+        if (NT == 2 && t + 1 < t_hi && t + 1 != tail_tile) {
+          process_tiles<BITS, NT, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+        } else {
+#pragma unroll
+          for (int k = 0; k < NT; ++k) {
+            if (t + k >= t_hi) break;
+            if (t + k == tail_tile)
+              process_tiles<BITS, 1, true>(tile + k * TB, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
+            else
+              process_tiles<BITS, 1, false>(tile + k * TB, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
+          }
+        }
         __syncwarp();
 #pragma unroll
         for (int i = 0; i + 2 < S; ++i) pending[i] = pending[i + 1];
@@ -778,8 +813,7 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   __syncthreads();  // every warp is done with its stages
   float(*s_o)[kMaxGroup][kHeadDim] = reinterpret_cast<float(*)[kMaxGroup][kHeadDim]>(ring);
   float *s_m = s_stat + 16, *s_l = s_stat + 16 + kParts * kMaxGroup;
-  if (worker)
-    store_warp_partial(st, [&](int J) { return ldexpf(sigma_u, 24 - F::EP - F::pos(J % F::N)); }, s_o, s_m, s_l, warp, lane);
+  store_warp_partial(st, [&](int J) { return ldexpf(sigma_u, 24 - F::EP - F::pos(J % F::N)); }, s_o, s_m, s_l, warp, lane);
   __syncthreads();
   publish_segment(p, slice, kAttnWarps, s_o, s_m, s_l, s_ctr);
 }
@@ -842,16 +876,19 @@ __device__ __forceinline__ void run_segment_tc(const AttnParams &p, int slice, l
   publish_segment(p, slice, kParts, s_o, s_m, s_l, s_ctr);
 }
 
+// Dynamic shared memory of the warp-level MMA path at body width BITS: per-warp stages while streaming;
+// at least the warps' outputs they are reused for.
 template <int BITS>
+constexpr int attn_ring_bytes() {
+  constexpr int out_bytes = kAttnWarps * kMaxGroup * kHeadDim * 4;
+  constexpr int ring = kAttnWarps * Fmt<BITS>::SLOTS * Fmt<BITS>::NT * tile_bytes(BITS);
+  return ring > out_bytes ? ring : out_bytes;
+}
+// ... of the one-block kernel on either path
+template <int BITS, bool ROWS>
 constexpr int attn_smem_bytes() {
-  if constexpr (BITS <= 4) {
-    return kSmemTcTotal;
-  } else {
-    // per-warp stages while streaming; at least the warps' outputs they are reused for
-    constexpr int out_bytes = kAttnWarps * kMaxGroup * kHeadDim * 4;
-    constexpr int ring = kAttnWarps * Fmt<BITS>::SLOTS * tile_bytes(BITS);
-    return ring > out_bytes ? ring : out_bytes;
-  }
+  if constexpr (BITS <= 4 && ROWS) return kSmemTcTotal;
+  else return attn_ring_bytes<BITS>();
 }
 
 // CTA set-up of the tensor-memory path: barriers and tensor memory.  Ends with a CTA-wide barrier.
@@ -891,7 +928,7 @@ __device__ __forceinline__ void tc_teardown(TcCtx &tc) {
   if ((threadIdx.x >> 5) == 0) tc05::tmem_dealloc(tc.tmem_base, kTmemCols);
 }
 
-template <int BODY_BITS>
+template <int BODY_BITS, bool ROWS>
 __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(const AttnParams p, unsigned *error_word) {
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
   __shared__ float s_stat[16 + 2 * kParts * kMaxGroup];  // head stats, per-partial (m, l)
@@ -900,7 +937,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
   __shared__ TcShared s_tc;
   extern __shared__ __align__(128) uint8_t ring[];
   TcCtx tc;
-  if constexpr (BODY_BITS <= 4) tc_setup(&s_tc, tc, ring, error_word);
+  constexpr bool tensor_path = BODY_BITS <= 4 && ROWS;
+  if constexpr (tensor_path) tc_setup(&s_tc, tc, ring, error_word);
   const long long u_begin = (long long)blockIdx.x * p.units_per_cta;
   const long long u_end = min(u_begin + p.units_per_cta, p.units_total);
   for (long long u = u_begin; u < u_end;) {
@@ -908,12 +946,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_splitk_kernel(con
     const long long base = (long long)slice * p.units_slice;
     const long long hi = min(u_end - base, p.units_slice);
     if (hi > p.units_lead) {
-      if constexpr (BODY_BITS <= 4) run_segment_tc<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc);
+      if constexpr (tensor_path) run_segment_tc<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc);
       else run_segment<BODY_BITS>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
     }
     u = base + hi;
   }
-  if constexpr (BODY_BITS <= 4) tc_teardown(tc);
+  if constexpr (tensor_path) tc_teardown(tc);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -936,6 +974,7 @@ struct FusedParams {
   size_t partial_stride;
   int layers, kv_heads, group, q_heads, n_slices, batch;
   int n_sink, window, evict_chunk, sink_tiles, ring_tiles;
+  int rows;                   // 1: tensor-memory path (row tiles at 4 and 2 bit)
   float qk_scale;
   long long per_cta, total;              // fine units
   long long start[kMaxFusedLayers + 1];  // fine units before each block
@@ -974,6 +1013,7 @@ __device__ __forceinline__ void fused_layer_params(const FusedParams &fp, int l,
   p.qk_scale = fp.qk_scale;
 }
 
+template <bool ROWS>
 __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_fused_kernel(const __grid_constant__ FusedParams fp) {
   __shared__ __align__(16) float s_q[kMaxGroup][kHeadDim];
   __shared__ float s_stat[16 + 2 * kParts * kMaxGroup];
@@ -982,7 +1022,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_fused_kernel(cons
   __shared__ TcShared s_tc;
   extern __shared__ __align__(128) uint8_t ring[];
   TcCtx tc;
-  tc_setup(&s_tc, tc, ring, fp.error_word);
+  constexpr bool tensor_path = ROWS;  // the cache was created for the tensor-memory path
+  if constexpr (tensor_path) tc_setup(&s_tc, tc, ring, fp.error_word);
   const long long f_begin = (long long)blockIdx.x * fp.per_cta;
   const long long f_end = min(f_begin + fp.per_cta, fp.total);
   int l = 0;
@@ -1003,17 +1044,31 @@ __global__ void __launch_bounds__(kAttnThreads, 1) decode_attn_fused_kernel(cons
         switch (p.cur_bits) {
           case 16: run_segment<16>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
           case 8: run_segment<8>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring); break;
-          case 4: run_segment_tc<4>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc); break;
-          default: run_segment_tc<2>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc); break;
+          case 4:
+            if constexpr (tensor_path) run_segment_tc<4>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc);
+            else run_segment<4>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
+            break;
+          default:
+            if constexpr (tensor_path) run_segment_tc<2>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, tc);
+            else run_segment<2>(p, slice, u - base, hi, s_q, s_stat, s_ctr, s_frag, ring);
+            break;
         }
       }
       u = base + hi;
     }
     f = f_hi;
   }
-  tc_teardown(tc);
+  if constexpr (tensor_path) tc_teardown(tc);
 }
 
-constexpr int attn_fused_smem_bytes() { return kSmemTcTotal > attn_smem_bytes<8>() ? kSmemTcTotal : attn_smem_bytes<8>(); }
+template <bool ROWS>
+constexpr int attn_fused_smem_bytes() {
+  int m = ROWS ? kSmemTcTotal : 0;
+  m = attn_ring_bytes<16>() > m ? attn_ring_bytes<16>() : m;
+  m = attn_ring_bytes<8>() > m ? attn_ring_bytes<8>() : m;
+  m = attn_ring_bytes<4>() > m ? attn_ring_bytes<4>() : m;
+  m = attn_ring_bytes<2>() > m ? attn_ring_bytes<2>() : m;
+  return m;
+}
 
 }  // namespace pmkvq

@@ -20,6 +20,7 @@ struct LayerGeom {
   int n_sink;           // leading INT16 tokens (stored in tiles at offset 0)
   int ring_tokens;      // ring capacity in tokens (multiple of 16)
   int shift_variant;    // ShiftVariant of this cache
+  int rows;             // 1: the 4- and 2-bit body uses row tiles (tensor-memory attention path)
 };
 
 struct TokenDest {
@@ -137,16 +138,18 @@ __device__ __forceinline__ void insert_value_row(uint8_t *v_part, int row, const
 }
 
 __device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, const uint16_t *codes16, int is_value,
-                                            int lane, int variant) {
+                                            int lane, int variant, bool rows) {
   switch (bits) {
     case 16: store_token_w<16>(part, row, codes16, is_value, lane, variant); break;
     case 8: store_token_w<8>(part, row, codes16, is_value, lane, variant); break;
     case 4:
-      if (is_value) insert_value_row<4>(part, row, codes16, lane, variant);
+      if (!rows) store_token_w<4>(part, row, codes16, is_value, lane, variant);
+      else if (is_value) insert_value_row<4>(part, row, codes16, lane, variant);
       else store_key_row<4>(part, row, codes16, lane, variant);
       break;
     default:
-      if (is_value) insert_value_row<2>(part, row, codes16, lane, variant);
+      if (!rows) store_token_w<2>(part, row, codes16, is_value, lane, variant);
+      else if (is_value) insert_value_row<2>(part, row, codes16, lane, variant);
       else store_key_row<2>(part, row, codes16, lane, variant);
       break;
   }
@@ -156,8 +159,8 @@ __device__ __forceinline__ void store_token(uint8_t *part, int bits, int row, co
 __device__ __forceinline__ void load_token16(const uint8_t *part, int row, uint16_t *codes16, int is_value, int lane) {
   for (int ch = lane; ch < kHeadDim; ch += 32) {
     int byte_off, bit_off;
-    if (is_value) v_slot(16, row, ch, byte_off, bit_off);
-    else k_slot(16, row, ch, byte_off, bit_off);
+    if (is_value) v_slot(16, false, row, ch, byte_off, bit_off);
+    else k_slot(16, false, row, ch, byte_off, bit_off);
     codes16[ch] = *reinterpret_cast<const uint16_t *>(part + byte_off);
   }
 }
@@ -231,10 +234,11 @@ __device__ __forceinline__ float quantize_token16(uint2 raw, const float *__rest
 }
 
 // Writes the metadata of one stored token (S, Z of K or of V after the chain to `bits`).
-__device__ __forceinline__ void store_meta(uint8_t *tile, int bits, int row, int is_value, float s16, float z16, int variant) {
+__device__ __forceinline__ void store_meta(uint8_t *tile, int bits, int row, int is_value, float s16, float z16, int variant,
+                                           bool rows) {
   float *meta = reinterpret_cast<float *>(tile + meta_offset(bits));
-  meta[meta_slot(bits, is_value ? 2 : 0, row) >> 2] = chain_scale(s16, bits, variant);
-  meta[meta_slot(bits, is_value ? 3 : 1, row) >> 2] = chain_zero(z16, s16, bits, variant);
+  meta[meta_slot(bits, rows, is_value ? 2 : 0, row) >> 2] = chain_scale(s16, bits, variant);
+  meta[meta_slot(bits, rows, is_value ? 3 : 1, row) >> 2] = chain_zero(z16, s16, bits, variant);
 }
 
 // One warp per (new token, slice, K|V) of the new tokens i0 .. i0 + n_cnt - 1.  Values that go straight
@@ -251,7 +255,7 @@ __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int l
   int i = i0 + (int)(ts / n_slices);  // index among the new tokens
   uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
   int t = n_old + i, last = t;
-  const bool shared_rows = is_value && t >= geom.n_sink && t < win_start && row_layout(cur_bits);
+  const bool shared_rows = is_value && t >= geom.n_sink && t < win_start && row_layout(cur_bits, geom.rows != 0);
   if (shared_rows) {
     const int j = t - geom.n_sink;
     if (i != i0 && (j & 15) != 0) return;  // an earlier token of this tile does this one
@@ -264,9 +268,10 @@ __device__ __forceinline__ void append_one(long long wid, uint16_t *codes, int l
                                          codes, lane, mn);
     __syncwarp();
     const TokenDest d = token_dest(geom, slice_base, t, win_start, cur_bits);
-    store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, codes, is_value, lane, geom.shift_variant);
+    store_token(d.tile + (is_value ? v_part_offset(d.bits) : 0), d.bits, d.row, codes, is_value, lane, geom.shift_variant,
+                geom.rows != 0);
     if (lane == 0) {
-      store_meta(d.tile, d.bits, d.row, is_value, scale, mn, geom.shift_variant);
+      store_meta(d.tile, d.bits, d.row, is_value, scale, mn, geom.shift_variant, geom.rows != 0);
       if (is_value) atomicMax(vmax_bits + slice, __float_as_uint(scale));  // scale >= 0: uint order = float order
     }
     __syncwarp();
@@ -537,8 +542,14 @@ __global__ void __launch_bounds__(128, 8) append_tiles_kernel(const uint16_t *__
   switch (bits) {
     case 16: append_tile_half<16>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
     case 8: append_tile_half<8>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
-    case 4: append_tile_half_row<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]); break;
-    default: append_tile_half_row<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]); break;
+    case 4:
+      if (geom.rows) append_tile_half_row<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]);
+      else append_tile_half<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant);
+      break;
+    default:
+      if (geom.rows) append_tile_half_row<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]);
+      else append_tile_half<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant);
+      break;
   }
 }
 
@@ -555,7 +566,7 @@ __device__ __forceinline__ void evict_one(long long wid, uint16_t *codes, int la
   const int slice = (int)(ts % n_slices);
   int t = first_token + (int)(ts / n_slices), last = t;
   uint8_t *slice_base = geom.base + (size_t)slice * geom.slice_stride;
-  if (is_value && row_layout(cur_bits)) {
+  if (is_value && row_layout(cur_bits, geom.rows != 0)) {
     const int j = t - geom.n_sink;
     if (t != first_token && (j & 15) != 0) return;
     last = min(first_token + n_evict, geom.n_sink + (j | 15) + 1) - 1;
@@ -566,14 +577,14 @@ __device__ __forceinline__ void evict_one(long long wid, uint16_t *codes, int la
     const int src_row = rp & 15;
     load_token16(src_tile + (is_value ? v_part_offset(16) : 0), src_row, codes, is_value, lane);
     const float *smeta = reinterpret_cast<const float *>(src_tile + meta_offset(16));
-    const float s16 = smeta[meta_slot(16, is_value ? 2 : 0, src_row) >> 2];
-    const float z = smeta[meta_slot(16, is_value ? 3 : 1, src_row) >> 2];
+    const float s16 = smeta[meta_slot(16, false, is_value ? 2 : 0, src_row) >> 2];
+    const float z = smeta[meta_slot(16, false, is_value ? 3 : 1, src_row) >> 2];
     __syncwarp();
     const int j = t - geom.n_sink;
     uint8_t *dst_tile = slice_base + geom.body_off + body_tile_offset(j >> 4, cur_bits, geom.stream_stride);
     store_token(dst_tile + (is_value ? v_part_offset(cur_bits) : 0), cur_bits, j & 15, codes, is_value, lane,
-                geom.shift_variant);
-    if (lane == 0) store_meta(dst_tile, cur_bits, j & 15, is_value, s16, z, geom.shift_variant);
+                geom.shift_variant, geom.rows != 0);
+    if (lane == 0) store_meta(dst_tile, cur_bits, j & 15, is_value, s16, z, geom.shift_variant, geom.rows != 0);
     __syncwarp();
   }
 }
@@ -839,7 +850,7 @@ __device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *o
     if (lane < 16) {
       const float *mi = reinterpret_cast<const float *>(in + meta_offset(8));
 #pragma unroll
-      for (int kind = 0; kind < 4; ++kind) m[kind] = mi[meta_slot(8, kind, lane) >> 2];
+      for (int kind = 0; kind < 4; ++kind) m[kind] = mi[meta_slot(8, false, kind, lane) >> 2];
       halve_meta(m[0], m[1], 4, variant);
       halve_meta(m[2], m[3], 4, variant);
     }
@@ -871,8 +882,8 @@ __global__ void __launch_bounds__(kReduceWarps * 32) reduce_stream_kernel(LayerG
     const bool active = j < cnt;
     const uint8_t *in = base + (size_t)j * tile_bytes(2 * B);
     uint8_t *out = base + (size_t)j * tile_bytes(B);
-    if constexpr (B == 8) {
-      reduce_tile<8, true>(in, out, lane, geom.shift_variant, active);
+    if (B == 8 || !geom.rows) {
+      reduce_tile<B, true>(in, out, lane, geom.shift_variant, active);
     } else if constexpr (B == 4) {
       if (shr) reduce_tile_to_row<true>(in, out, lane, geom.shift_variant, active, s_scratch[warp]);
       else reduce_tile_to_row<false>(in, out, lane, geom.shift_variant, active, s_scratch[warp]);

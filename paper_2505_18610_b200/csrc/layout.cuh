@@ -8,8 +8,10 @@
 // the budget accounting of the progressive policy (Sec. 3.1) charges, nothing more.
 //
 // The arrangement of the codes inside a tile follows the unit that consumes them in the attention kernel.
+// A cache is created for one of two attention paths: warp-level MMAs (every width uses lane-owned tiles) or
+// tensor memory (the 4- and 2-bit body uses row tiles; 16 and 8 bit stay lane-owned).
 //
-// --- 16 and 8 bit: "lane-owned" tiles, read by warp-level MMAs from registers -------------------------
+// --- "lane-owned" tiles, read by warp-level MMAs from registers ---------------------------------------
 // The 32 lanes of a warp own 16-byte chunks, chunk q of lane l at byte (q*32 + l)*16, so a warp reads a
 // tile with fully coalesced 128-bit loads and every lane gets exactly the codes its fragments need, with
 // no shuffle.  With lane = 4*g + tig:
@@ -27,7 +29,7 @@
 // Metadata: for tig = 0..3 a 64-byte record {S_K[4], Z_K[4], S_V[4], Z_V[4]} of the four tokens
 // {2tig, 2tig+1, 8+2tig, 9+2tig} a lane needs for its score / probability fragments.
 //
-// --- 4 and 2 bit: "row" tiles, read by tcgen05.mma through tensor memory ------------------------------
+// --- "row" tiles (4 and 2 bit of a tensor-memory cache), read by tcgen05.mma through tensor memory ----
 // The A operand of the MMAs lives in tensor memory, where a thread writes one lane (one matrix row):
 // a token's row of K^T-side codes for the scores, a channel's row of V codes for the output.  So
 //
@@ -66,7 +68,7 @@ PMKVQ_HD constexpr int code_part_bytes(int bits) { return 256 * bits; }
 PMKVQ_HD constexpr int tile_bytes(int bits) { return 512 * bits + 256; }
 PMKVQ_HD constexpr int v_part_offset(int bits) { return 256 * bits; }
 PMKVQ_HD constexpr int meta_offset(int bits) { return 512 * bits; }
-PMKVQ_HD constexpr bool row_layout(int bits) { return bits <= 4; }
+PMKVQ_HD constexpr bool row_layout(int bits, bool rows) { return rows && bits <= 4; }
 
 // Byte offset of body tile i inside the body of a slice.
 PMKVQ_HD size_t body_tile_offset(int i, int bits, size_t stream_stride) {
@@ -93,8 +95,8 @@ PMKVQ_HD void row_slot(int bits, int idx, int &byte_off, int &bit_off) {
 }
 
 // K code of (token row 0..15, channel 0..127): half-word byte offset inside the K part, bit offset
-PMKVQ_HD void k_slot(int bits, int row, int ch, int &byte_off, int &bit_off) {
-  if (row_layout(bits)) {
+PMKVQ_HD void k_slot(int bits, bool rows, int row, int ch, int &byte_off, int &bit_off) {
+  if (row_layout(bits, rows)) {
     row_slot(bits, ch, byte_off, bit_off);
     byte_off += row * 16 * bits;
     return;
@@ -105,8 +107,8 @@ PMKVQ_HD void k_slot(int bits, int row, int ch, int &byte_off, int &bit_off) {
 }
 
 // V code of (token row 0..15, channel 0..127)
-PMKVQ_HD void v_slot(int bits, int row, int ch, int &byte_off, int &bit_off) {
-  if (row_layout(bits)) {
+PMKVQ_HD void v_slot(int bits, bool rows, int row, int ch, int &byte_off, int &bit_off) {
+  if (row_layout(bits, rows)) {
     row_slot(bits, row, byte_off, bit_off);
     byte_off += ch * 2 * bits;
     return;
@@ -117,8 +119,8 @@ PMKVQ_HD void v_slot(int bits, int row, int ch, int &byte_off, int &bit_off) {
 }
 
 // Byte offset inside the metadata block of kind (0 S_K, 1 Z_K, 2 S_V, 3 Z_V) of token row.
-PMKVQ_HD int meta_slot(int bits, int kind, int row) {
-  if (row_layout(bits)) return row * 16 + kind * 4;
+PMKVQ_HD int meta_slot(int bits, bool rows, int kind, int row) {
+  if (row_layout(bits, rows)) return row * 16 + kind * 4;
   const int tig = (row & 7) >> 1;
   const int i = (row >> 3) * 2 + (row & 1);
   return tig * 64 + kind * 16 + i * 4;

@@ -44,7 +44,7 @@ struct Layer {
 
 struct pmkvq_cache {
   int layers, q_heads, kv_heads, batch, max_tokens, group, n_slices;
-  int n_sink, window, evict_chunk, count_metadata, auto_reduce, shift_variant;
+  int n_sink, window, evict_chunk, count_metadata, auto_reduce, shift_variant, rows;
   float sm_scale;
   uint8_t *arena;
   size_t arena_bytes;
@@ -83,6 +83,7 @@ struct pmkvq_cache {
     g.n_sink = n_sink;
     g.ring_tokens = ring_tiles * 16;
     g.shift_variant = shift_variant;
+    g.rows = rows;
     return g;
   }
 };
@@ -101,6 +102,7 @@ bool check_config(const pmkvq_config *c) {
     if (!valid_bits(c->fbit[i])) return false;
   if (c->n_sink < 0 || c->window < 0 || c->evict_chunk < 1) return false;
   if (c->shift_variant < 0 || c->shift_variant > 2) return false;
+  if (c->attention_path < 0 || c->attention_path > 1) return false;
   if ((int64_t)c->n_sink + c->window + c->evict_chunk > (1 << 24)) return false;
   if ((int64_t)c->batch * c->kv_heads > 65535) return false;
   if (c->lambda) {
@@ -119,6 +121,7 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
   k.n_sink = c->n_sink; k.window = c->window; k.evict_chunk = c->evict_chunk;
   k.count_metadata = c->count_metadata ? 1 : 0; k.auto_reduce = c->auto_reduce ? 1 : 0;
   k.shift_variant = c->shift_variant;
+  k.rows = c->attention_path == 1 ? 1 : 0;
   k.sm_scale = c->sm_scale > 0.0f ? c->sm_scale : 1.0f / std::sqrt((float)kHeadDim);
   k.sink_tiles = (k.n_sink + 15) / 16;
   k.ring_tiles = std::max(1, (k.window + k.evict_chunk - 1 + 15) / 16 + 1);
@@ -173,15 +176,32 @@ cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStr
   return cudaGetLastError();
 }
 
-template <int BITS>
+template <int BITS, bool ROWS>
 cudaError_t attention_setup_one(int &resident, int sms) {
-  cudaError_t e = cudaFuncSetAttribute(decode_attn_splitk_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       attn_smem_bytes<BITS>());
+  cudaError_t e = cudaFuncSetAttribute(decode_attn_splitk_kernel<BITS, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       attn_smem_bytes<BITS, ROWS>());
   int per_sm = 0;
   if (e == cudaSuccess)
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_splitk_kernel<BITS>, kAttnThreads,
-                                                      attn_smem_bytes<BITS>());
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_splitk_kernel<BITS, ROWS>, kAttnThreads,
+                                                      attn_smem_bytes<BITS, ROWS>());
   resident = std::min(kMaxCtas, std::max(1, per_sm) * sms);
+  return e;
+}
+
+template <bool ROWS>
+cudaError_t attention_setup_path(pmkvq_cache *k, int sms) {
+  cudaError_t e = attention_setup_one<16, ROWS>(k->resident_ctas[0], sms);
+  if (e == cudaSuccess) e = attention_setup_one<8, ROWS>(k->resident_ctas[1], sms);
+  if (e == cudaSuccess) e = attention_setup_one<4, ROWS>(k->resident_ctas[2], sms);
+  if (e == cudaSuccess) e = attention_setup_one<2, ROWS>(k->resident_ctas[3], sms);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_attn_fused_kernel<ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             attn_fused_smem_bytes<ROWS>());
+  int per_sm = 0;
+  if (e == cudaSuccess)
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_fused_kernel<ROWS>, kAttnThreads,
+                                                      attn_fused_smem_bytes<ROWS>());
+  k->resident_fused = std::min(kMaxCtas, std::max(1, per_sm) * sms);
   return e;
 }
 
@@ -190,16 +210,7 @@ cudaError_t attention_setup(pmkvq_cache *k) {
   int dev = 0, sms = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (e == cudaSuccess) e = attention_setup_one<16>(k->resident_ctas[0], sms);
-  if (e == cudaSuccess) e = attention_setup_one<8>(k->resident_ctas[1], sms);
-  if (e == cudaSuccess) e = attention_setup_one<4>(k->resident_ctas[2], sms);
-  if (e == cudaSuccess) e = attention_setup_one<2>(k->resident_ctas[3], sms);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_attn_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_fused_smem_bytes());
-  int per_sm = 0;
-  if (e == cudaSuccess)
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_attn_fused_kernel, kAttnThreads, attn_fused_smem_bytes());
-  k->resident_fused = std::min(kMaxCtas, std::max(1, per_sm) * sms);
+  if (e == cudaSuccess) e = k->rows ? attention_setup_path<true>(k, sms) : attention_setup_path<false>(k, sms);
   return e;
 }
 
@@ -451,7 +462,10 @@ static pmkvq_status attn_params(pmkvq_cache *k, int32_t layer, const void *d_Q, 
 
 template <int BITS>
 static cudaError_t attn_launch_width(const AttnParams &p, unsigned n_ctas, cudaStream_t st, unsigned *error_word) {
-  decode_attn_splitk_kernel<BITS><<<n_ctas, kAttnThreads, attn_smem_bytes<BITS>(), st>>>(p, error_word);
+  if (p.geom.rows)
+    decode_attn_splitk_kernel<BITS, true><<<n_ctas, kAttnThreads, attn_smem_bytes<BITS, true>(), st>>>(p, error_word);
+  else
+    decode_attn_splitk_kernel<BITS, false><<<n_ctas, kAttnThreads, attn_smem_bytes<BITS, false>(), st>>>(p, error_word);
   return cudaGetLastError();
 }
 
@@ -496,6 +510,7 @@ static pmkvq_status attention_all_blocks(pmkvq_cache *k, const void *d_Q, float 
   fp.n_slices = k->n_slices; fp.batch = k->batch;
   fp.n_sink = k->n_sink; fp.window = k->window; fp.evict_chunk = k->evict_chunk;
   fp.sink_tiles = k->sink_tiles; fp.ring_tiles = k->ring_tiles;
+  fp.rows = k->rows;
   fp.qk_scale = k->sm_scale * 1.4426950408889634f;
   long long total = 0;
   for (int l = 0; l < k->layers; ++l) {
@@ -521,7 +536,8 @@ static pmkvq_status attention_all_blocks(pmkvq_cache *k, const void *d_Q, float 
   fp.per_cta = std::max<long long>((total + want - 1) / want,
                                    k->user_ctas > 0 ? (long long)tile_weight(16) : 50ll * kMinUnitsPerCta);
   const unsigned n_ctas = (unsigned)((total + fp.per_cta - 1) / fp.per_cta);
-  decode_attn_fused_kernel<<<n_ctas, kAttnThreads, attn_fused_smem_bytes(), st>>>(fp);
+  if (k->rows) decode_attn_fused_kernel<true><<<n_ctas, kAttnThreads, attn_fused_smem_bytes<true>(), st>>>(fp);
+  else decode_attn_fused_kernel<false><<<n_ctas, kAttnThreads, attn_fused_smem_bytes<false>(), st>>>(fp);
   k->launches += 1;
   return cudaGetLastError() == cudaSuccess ? PMKVQ_OK : PMKVQ_ERR_CUDA;
 }
@@ -688,7 +704,7 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
     std::memset(packed, 0, sizeof(packed));
     for (int ch = 0; ch < kHeadDim; ++ch) {
       int bo, sh;
-      if (is_value) v_slot(bits, row, ch, bo, sh); else k_slot(bits, row, ch, bo, sh);
+      if (is_value) v_slot(bits, k->rows != 0, row, ch, bo, sh); else k_slot(bits, k->rows != 0, row, ch, bo, sh);
       uint16_t hw;
       std::memcpy(&hw, part + bo, 2);
       const uint32_t c = (hw >> sh) & cmask;
@@ -697,8 +713,8 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
       else packed[(ch * bits) >> 3] |= (uint8_t)(c << ((ch * bits) & 7));
     }
     float sc, ze;
-    std::memcpy(&sc, tile + meta_offset(bits) + meta_slot(bits, is_value ? 2 : 0, row), 4);
-    std::memcpy(&ze, tile + meta_offset(bits) + meta_slot(bits, is_value ? 3 : 1, row), 4);
+    std::memcpy(&sc, tile + meta_offset(bits) + meta_slot(bits, k->rows != 0, is_value ? 2 : 0, row), 4);
+    std::memcpy(&ze, tile + meta_offset(bits) + meta_slot(bits, k->rows != 0, is_value ? 3 : 1, row), 4);
     if (h_scale) h_scale[t] = sc;
     if (h_zero) h_zero[t] = ze;
     if (h_bits) h_bits[t] = (uint8_t)bits;

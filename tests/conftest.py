@@ -24,3 +24,10 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_generate_tests(metafunc):
+    """GPU tests that take `attention_path` run once per attention path of the library: 0 = warp-level
+    MMAs (lane-owned tiles at every width), 1 = tensor memory (row tiles at 4 and 2 bit)."""
+    if "attention_path" in metafunc.fixturenames:
+        metafunc.parametrize("attention_path", [0, 1], ids=["warp_mma", "tensor_memory"])

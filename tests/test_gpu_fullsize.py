@@ -3,8 +3,9 @@ configuration bench.py times
 (same batch, heads, context length, default attention grid, pmkvq_decode_step), on sampled (batch,
 kv_head) slices the oracle can compute one by one: cache state bit-exact after the run (it crosses each
 block's last progressive reduce), attention outputs within tolerance at several steps.  Two blocks per
-case (one per Fbit of the schedule) keep the device footprint at a few GB; a launch works on one block,
-so the per-launch shapes are those of the full model."""
+case (one per Fbit of the schedule) keep the device footprint at a few GB,
+so the per-block shapes are those of the full model (the step's one attention launch covers both blocks).  Every case runs on
+both attention paths of the library."""
 import numpy as np
 import pytest
 import torch
@@ -34,7 +35,7 @@ CASES = {
 
 
 @pytest.mark.parametrize("name", list(CASES))
-def test_fullsize_sampled_slices(name):
+def test_fullsize_sampled_slices(name, attention_path):
     q_heads, kvh, batch, n_end, fbit, n_out, factor = CASES[name]
     layers, steps, chunk = len(fbit), 6, 8192
     n_slices, group = batch * kvh, q_heads // kvh
@@ -45,7 +46,7 @@ def test_fullsize_sampled_slices(name):
     dev = "cuda"
     lam = np.stack([synth.make_lambda(synth.make_kv(0, l, 0, 512, 1, kvh, 0, n_out, factor)[0]).numpy()
                     for l in range(layers)])
-    cache = Cache(layers, q_heads, kvh, batch, n_end, fbit, budget_bytes=budgets, lam=lam)
+    cache = Cache(layers, q_heads, kvh, batch, n_end, fbit, budget_bytes=budgets, lam=lam, attention_path=attention_path)
     oracles = []
     for l in range(layers):
         pol = O.Policy(fbit[l], n_end, n_slices, budgets[l])

@@ -16,24 +16,24 @@ def _lam(layers, kv_heads, k_sample):
 
 @pytest.mark.parametrize("fbit", [16, 8, 4, 2])
 @pytest.mark.parametrize("n", [1, 2, 3, 17])
-def test_tiny_token_counts(fbit, n):
+def test_tiny_token_counts(fbit, n, attention_path):
     """1-17 tokens, no window: sink + body at every width, brute-force sized."""
     k, v = make_inputs(1, 0, n, 1, 1)
     m = Mirror(1, 4, 1, 1, 64, [fbit], n_sink=1, window=0,
-               budget_bytes=[2 * (264 + (n - 1) * (16 * fbit + 8))])     # exactly n tokens with the body at Fbit
+               budget_bytes=[2 * (264 + (n - 1) * (16 * fbit + 8))], attention_path=attention_path)     # exactly n tokens with the body at Fbit
     m.append(0, k, v, bulk=False)
     assert m.cache.layer_state(0)["cur_bits"] == (fbit if n > 1 else 16)
     m.check_state(0)
     m.check_attention(0, synth.make_q(1, 0, 0, 1, 4, n))
 
 
-def test_config1_progressive_16_8_4():
+def test_config1_progressive_16_8_4(attention_path):
     """The small progressive case: 1 block, batch 1, 4 Q / 1 KV head, 4096 tokens fed one by one, 4 outlier channels
     x20, default budget for Fbit = 4: the block goes 16 -> 8 -> 4.  Full parity after every reduce."""
     n = 4096
     k, v = make_inputs(0, 0, n, 1, 1, n_outlier=4, factor=20.0)
     lam = _lam(1, 1, k[:512])
-    m = Mirror(1, 4, 1, 1, n, [4], lam=lam)
+    m = Mirror(1, 4, 1, 1, n, [4], lam=lam, attention_path=attention_path)
     kd, vd = k.cuda(), v.cuda()
     seen = [16]
     for t in range(n):
@@ -52,10 +52,10 @@ def test_config1_progressive_16_8_4():
 
 
 @pytest.mark.parametrize("group", [1, 4, 5, 7, 8])
-def test_gqa_groups(group):
+def test_gqa_groups(group, attention_path):
     kvh, batch, n = 2, 2, 333
     k, v = make_inputs(2, 0, n, batch, kvh)
-    m = Mirror(1, group * kvh, kvh, batch, 400, [2], lam=_lam(1, kvh, k[:64]), window=32)
+    m = Mirror(1, group * kvh, kvh, batch, 400, [2], lam=_lam(1, kvh, k[:64]), window=32, attention_path=attention_path)
     m.append(0, k, v)
     m.check_state(0)
     m.check_attention(0, synth.make_q(2, 0, 0, batch, group * kvh, n))
@@ -63,7 +63,7 @@ def test_gqa_groups(group):
 
 @pytest.mark.parametrize("fbit,chunk,n_sink,window", [(2, 1, 1, 128), (4, 16, 1, 128), (2, 16, 0, 32), (8, 3, 4, 20),
                                                      (2, 1, 0, 0), (4, 1, 17, 5)])
-def test_multi_layer_bulk_and_stepwise(fbit, chunk, n_sink, window):
+def test_multi_layer_bulk_and_stepwise(fbit, chunk, n_sink, window, attention_path):
     """Several blocks / slices, ragged bulk appends followed by single-token decode steps."""
     layers, kvh, batch, group, n_max = 2, 2, 3, 7, 1500
     m = None
@@ -73,7 +73,7 @@ def test_multi_layer_bulk_and_stepwise(fbit, chunk, n_sink, window):
         ks.append(k); vs.append(v)
     lam = np.stack([synth.make_lambda(ks[l][:256]).numpy() for l in range(layers)])
     m = Mirror(layers, group * kvh, kvh, batch, n_max, [fbit, 16 if fbit == 16 else max(fbit, 4)], lam=lam,
-               n_sink=n_sink, window=window, evict_chunk=chunk)
+               n_sink=n_sink, window=window, evict_chunk=chunk, attention_path=attention_path)
     cuts = [0, 1, 130, 131, 700, 1237, 1400]
     for l in range(layers):
         for a, b in zip(cuts[:-1], cuts[1:]):
@@ -89,11 +89,11 @@ def test_multi_layer_bulk_and_stepwise(fbit, chunk, n_sink, window):
         m.check_state(l, slices=[1, 4])
 
 
-def test_policy_thresholds_on_gpu():
+def test_policy_thresholds_on_gpu(attention_path):
     """Code-bit accounting, no sink / window, Fbit = 2, 512 max tokens: reduces at 64, 128, 256 tokens."""
     n = 512
     k, v = make_inputs(4, 0, n, 1, 2)
-    m = Mirror(1, 8, 2, 1, n, [2], n_sink=0, window=0, count_metadata=False)
+    m = Mirror(1, 8, 2, 1, n, [2], n_sink=0, window=0, count_metadata=False, attention_path=attention_path)
     kd, vd = k.cuda(), v.cuda()
     fired, bits = [], 16
     for t in range(n):
@@ -134,11 +134,11 @@ def test_manual_reduce_and_error_codes():
         B.Cache(1, 18, 2, 1, 64, [4])          # GQA group of 9 is outside 1..8
 
 
-def test_reduce_head_batches_and_waves():
+def test_reduce_head_batches_and_waves(attention_path):
     """Bodies of 378, 733 and 1385 tiles cross 16 -> 8 -> 4 -> 2: the in-place reduce runs its CTA-wide head
     batches (256 tiles) and one, two and three parallel waves behind them."""
     kvh, n_max = 2, 40000
-    m = Mirror(1, 2 * kvh, kvh, 1, n_max, [2])
+    m = Mirror(1, 2 * kvh, kvh, 1, n_max, [2], attention_path=attention_path)
     done, widths = 0, []
     for upto in (6170, 6200, 11855, 11900, 22279, 22400):
         k, v = make_inputs(31, 0, upto - done, 1, kvh, pos0=done, chunk=upto)
@@ -175,10 +175,10 @@ def test_empty_inputs_are_refused_and_empty_bodies_reduce():
     assert torch.isfinite(out).all()
 
 
-def test_split_invariance():
+def test_split_invariance(attention_path):
     kvh, batch, n, group = 2, 2, 5000, 8
     k, v = make_inputs(6, 0, n, batch, kvh)
-    m = Mirror(1, group * kvh, kvh, batch, n, [2], lam=_lam(1, kvh, k[:256]))
+    m = Mirror(1, group * kvh, kvh, batch, n, [2], lam=_lam(1, kvh, k[:256]), attention_path=attention_path)
     m.append(0, k, v)
     q = synth.make_q(6, 0, 0, batch, group * kvh, n)
     outs = []
@@ -192,14 +192,14 @@ def test_split_invariance():
         assert np.abs(o - outs[0]).max() < 1e-3
 
 
-def test_degenerate_values():
+def test_degenerate_values(attention_path):
     """Constant V groups (S = 0), zero K, zero Q, and a huge-range token."""
     n, kvh = 200, 1
     k, v = make_inputs(7, 0, n, 1, kvh)
     v[5] = 1.5; v[150] = -2.0          # constant groups: scale 0
     k[7] = 0.0
     v[9] = v[9] * 1000.0               # one token with a huge value range
-    m = Mirror(1, 4, kvh, 1, n, [2], window=16)
+    m = Mirror(1, 4, kvh, 1, n, [2], window=16, attention_path=attention_path)
     m.append(0, k, v)
     m.check_state(0)
     q = synth.make_q(7, 0, 0, 1, 4, n)
@@ -209,7 +209,7 @@ def test_degenerate_values():
 
 
 @pytest.mark.parametrize("bulk", [True, False])
-def test_quantizer_scale_extremes(bulk):
+def test_quantizer_scale_extremes(bulk, attention_path):
     """Tokens whose scale lies outside the range of the reciprocal-based quotient (below 2^-60, above 2^60,
     exactly 0) take the plain-division path; codes, scales and zero-points stay bit-exact."""
     n, kvh = 100, 2
@@ -218,17 +218,17 @@ def test_quantizer_scale_extremes(bulk):
         k[t] = (k[t].float() * f).to(k.dtype)
         v[t] = (v[t].float() * f).to(v.dtype)
     k[50] = 0.25; v[51] = 0.0
-    m = Mirror(1, 2, kvh, 1, n, [4], window=8)
+    m = Mirror(1, 2, kvh, 1, n, [4], window=8, attention_path=attention_path)
     m.append(0, k, v, bulk=bulk)
     m.check_state(0)
 
 
-def test_decode_step_over_all_blocks():
+def test_decode_step_over_all_blocks(attention_path):
     """pmkvq_decode_step = append + attention for every block; compared with the oracle block by block,
     across a reduce (block 0 crosses its budget during the steps)."""
     layers, kvh, batch, group, n0, steps = 3, 2, 2, 7, 300, 24
     fbit = [2, 4, 8]
-    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, fbit, window=32)
+    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, fbit, window=32, attention_path=attention_path)
     for l in range(layers):
         k, v = make_inputs(8, l, n0, batch, kvh)
         m.append(l, k, v)
@@ -258,11 +258,11 @@ def test_decode_step_over_all_blocks():
 
 
 @pytest.mark.parametrize("layers", [128, 130])
-def test_decode_step_with_many_blocks(layers):
+def test_decode_step_with_many_blocks(layers, attention_path):
     """128 blocks fill the argument tables of the one-launch step exactly; 130 take the block-by-block route."""
     kvh, batch, group, n0, steps = 1, 1, 2, 40, 3
     fbit = [(2, 4, 8, 16)[l % 4] for l in range(layers)]
-    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, fbit, window=8)
+    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, fbit, window=8, attention_path=attention_path)
     for l in range(layers):
         k, v = make_inputs(21, l, n0, batch, kvh)
         m.append(l, k, v)
@@ -289,11 +289,11 @@ def test_decode_step_with_many_blocks(layers):
 
 
 @pytest.mark.parametrize("variant", [1, 2])
-def test_shift_variants_direct_and_modified(variant):
+def test_shift_variants_direct_and_modified(variant, attention_path):
     """The two ablation strategies of Sec. 4.4.1 as cache options: bulk appends, evictions through the
     chain and progressive reduces down to 2 bit, state bit-exact and attention within tolerance."""
     layers, kvh, batch, group, n = 2, 2, 2, 4, 900
-    m = Mirror(layers, group * kvh, kvh, batch, n, [2, 4], window=32, shift_variant=variant)
+    m = Mirror(layers, group * kvh, kvh, batch, n, [2, 4], window=32, shift_variant=variant, attention_path=attention_path)
     for l in range(layers):
         k, v = make_inputs(10 + variant, l, n, batch, kvh)
         m.append(l, k[:500], v[:500])
@@ -332,11 +332,11 @@ def test_decode_step_budget_full_leaves_every_block_untouched():
 
 
 @pytest.mark.parametrize("chunk,n_sink,window", [(16, 4, 20), (3, 0, 7), (1, 17, 0)])
-def test_decode_step_with_chunked_eviction(chunk, n_sink, window):
+def test_decode_step_with_chunked_eviction(chunk, n_sink, window, attention_path):
     """The all-blocks append of pmkvq_decode_step with eviction in chunks, several sink tokens and small
     windows: blocks at different token counts are not supported by the call, different widths are."""
     layers, kvh, batch, group, n0, steps = 2, 2, 2, 5, 70, 45
-    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, [2, 8], n_sink=n_sink, window=window, evict_chunk=chunk)
+    m = Mirror(layers, group * kvh, kvh, batch, n0 + steps, [2, 8], n_sink=n_sink, window=window, evict_chunk=chunk, attention_path=attention_path)
     for l in range(layers):
         k, v = make_inputs(30, l, n0, batch, kvh)
         m.append(l, k, v)
