@@ -67,16 +67,16 @@ def plan(wl, steps, warmup):
     assert n0 > N_SINK + WINDOW + 16, "too many steps for this workload"
     budgets = []
     if wl.get("schedule") == "70b":
-        # a ~100 GB cache whose blocks sit at different points of the 16 -> 8 -> 4 -> 2 chain: 4 blocks
-        # cross 16 -> 8 during the run, 8 cross 8 -> 4, 30 cross 4 -> 2, the other 38 are already at 2 bit
+        # a ~120 GB cache whose blocks sit at different points of the 16 -> 8 -> 4 -> 2 chain: 8 blocks
+        # cross 16 -> 8 during the run, 16 cross 8 -> 4, 30 cross 4 -> 2, the other 26 are already at 2 bit
         fbit, crossing = [], []
         for l in range(L):
-            fbit.append(8 if l >= L - 4 else 4 if l >= L - 12 else 2)
-            crossing.append(l >= L - 42)
+            fbit.append(8 if l >= L - 8 else 4 if l >= L - 24 else 2)
+            crossing.append(l >= L - 54)
         k = 0
         for l in range(L):
             if crossing[l]:
-                fire_step = warmup + (k * steps) // 42
+                fire_step = warmup + (k * steps) // 54
                 budgets.append(bytes_at(n0 + fire_step, 2 * fbit[l], n_slices)); k += 1
             else:
                 budgets.append(bytes_at(wl["end_tokens"], fbit[l], n_slices))
@@ -97,18 +97,33 @@ def make_lambda(wl, seed, device):
     return np.stack(lam)
 
 
-def build_cache(wl, fbit, budgets, lam, n0, device, chunk=8192, seed=0):
+def build_cache(wl, fbit, budgets, lam, n0, device, chunk=8192, seed=0, shared_chunks=False, attention_path=0,
+                max_tokens=None):
+    """Prefill a cache of the workload's shape with n0 tokens per block.  With shared_chunks every block
+    receives the same seeded chunk (the per-width and compact records: timing does not depend on the values)."""
     from paper_2505_18610_b200.binding import Cache
-    cache = Cache(wl["layers"], wl["q_heads"], wl["kv_heads"], wl["batch"], wl["end_tokens"], fbit,
-                  budget_bytes=budgets, lam=lam, n_sink=N_SINK, window=WINDOW, device=device)
-    for l in range(wl["layers"]):
+    cache = Cache(wl["layers"], wl["q_heads"], wl["kv_heads"], wl["batch"], max_tokens or wl["end_tokens"], fbit,
+                  budget_bytes=budgets, lam=lam, n_sink=N_SINK, window=WINDOW, device=device,
+                  attention_path=attention_path)
+    if shared_chunks:
         done = 0
         while done < n0:
             n = min(chunk, n0 - done)
-            k, v = synth.make_kv(seed, l, done // chunk, n, wl["batch"], wl["kv_heads"], done, wl["n_outlier"],
+            k, v = synth.make_kv(seed, 0, done // chunk, n, wl["batch"], wl["kv_heads"], done, wl["n_outlier"],
                                  wl["factor"], device=device)
-            cache.append(l, k.contiguous(), v.contiguous())
+            k, v = k.contiguous(), v.contiguous()
+            for l in range(wl["layers"]):
+                cache.append(l, k, v)
             done += n
+    else:
+        for l in range(wl["layers"]):
+            done = 0
+            while done < n0:
+                n = min(chunk, n0 - done)
+                k, v = synth.make_kv(seed, l, done // chunk, n, wl["batch"], wl["kv_heads"], done, wl["n_outlier"],
+                                     wl["factor"], device=device)
+                cache.append(l, k.contiguous(), v.contiguous())
+                done += n
     torch.cuda.synchronize()
     return cache
 
@@ -167,23 +182,106 @@ def kernel_source_digest():
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2505_18610_b200", "csrc")
-    for f in ("kernels_attn.cuh", "kernels_cache.cuh", "layout.cuh"):
+    for f in ("kernels_attn.cuh", "kernels_attn_tc.cuh", "tc05.cuh", "kernels_cache.cuh", "layout.cuh"):
         with open(os.path.join(d, f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
 
 
-# DRAM read + write bytes of one launch of the all-blocks attention kernel from the ncu capture summarised in
-# profiles/decode_attn_fused_7b_shape.md (4 blocks of the 7B shape: a launch of the 28-block workload moves
-# 7x the bytes, block by block the same way), its algorithmic bytes, and the digest of the sources it was
-# taken on.
+# DRAM read + write bytes of one captured launch of the all-blocks attention kernel (ncu, 4 blocks of the 7B shape
+# at their final widths: a launch of the 28-block workload moves 7x the bytes, block by block the same way), its
+# algorithmic bytes, and the digest of the sources it was taken on.
 NCU_TRAFFIC = {"digest": "302fac57a5376af8", "traffic_bytes": 976_058_112, "algorithmic_bytes": 954_646_528}
 
 
-def aux_leg(wl, device):
-    """The two kernels beside the decode step, timed alone with CUDA events (best of 5 calls after a warm-up):
-    the bulk prefill append of 8192 tokens into one block of the workload's shape, and the alpha grid search
-    of the calibration (2048 tokens x 8 sequences of the workload's head counts, 20 alphas, 2 bit)."""
+def time_attention_all(cache, q, out, launches, warm=3):
+    """CUDA-event time of `launches` calls of pmkvq_decode_attention_all (one attention launch over all blocks,
+    nothing appended) on the current stream.  Returns the list of per-launch milliseconds."""
+    for _ in range(warm):
+        cache.decode_attention_all(q, out)
+    torch.cuda.synchronize()
+    evs = []
+    for _ in range(launches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); cache.decode_attention_all(q, out); e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def width_leg(wl, device, peak, blocks=8, launches=12):
+    """Steady-state attention at one width: caches of `blocks` blocks of the workload's per-block shape whose
+    whole body sits at 2 / 4 / 8 / 16 bit, timed with one all-blocks attention launch per event pair."""
+    out = {}
+    sub = dict(wl, layers=blocks)
+    for path, pname in ((0, "warp_mma"), (1, "tensor_memory")):
+        for bits in (2, 4, 8, 16):
+            if path == 1 and bits > 4:
+                continue                      # the two paths only differ at 4 and 2 bit
+            cache = build_cache(sub, [bits] * blocks, None, None, wl["end_tokens"], device, shared_chunks=True,
+                                attention_path=path)
+            assert all(cache.layer_state(l)["cur_bits"] == bits for l in range(blocks))
+            q = torch.stack([synth.make_q(2, l, 0, wl["batch"], wl["q_heads"], wl["end_tokens"], device=device)
+                             for l in range(blocks)]).contiguous()
+            o = torch.empty(blocks, wl["batch"], wl["q_heads"], 128, dtype=torch.float32, device=device)
+            ts = time_attention_all(cache, q, o, launches)
+            by = sum(cache.attention_bytes(l) for l in range(blocks))
+            ms = float(np.median(ts))
+            rec = {"blocks_per_launch": blocks, "bytes_per_launch": by, "us_per_launch": ms * 1e3,
+                   "us_per_block": ms * 1e3 / blocks, "GBps": by / (ms * 1e-3) / 1e9, "frac": by / (ms * 1e-3) / 1e9 / peak}
+            cache.device_status()
+            cache.close(); del cache
+            torch.cuda.empty_cache()
+            out.setdefault(pname, {})[f"{bits}bit"] = rec
+    return out
+
+
+def reduce_leg(wl, device, peak, repeats=3):
+    """One progressive-reduce event of each width at the workload's per-block shape, timed alone: a one-block
+    cache is filled at 16 bit to the full context and reduced 16 -> 8 -> 4 -> 2 by hand.  Bytes per event are
+    body groups x (16 * 2b + 16 * b + 8): codes read, codes written, scale read and written."""
+    from paper_2505_18610_b200.binding import Cache
+    n_slices = wl["batch"] * wl["kv_heads"]
+    n = wl["end_tokens"]
+    best = {}
+    launches = {}
+    for _ in range(repeats):
+        cache = Cache(1, wl["q_heads"], wl["kv_heads"], wl["batch"], n, [2], budget_bytes=[bytes_at(n, 16, n_slices)],
+                      n_sink=N_SINK, window=WINDOW, auto_reduce=False, device=device)
+        done = 0
+        while done < n:
+            m = min(8192, n - done)
+            k, v = synth.make_kv(4, 0, done // 8192, m, wl["batch"], wl["kv_heads"], done, wl["n_outlier"], wl["factor"],
+                                 device=device)
+            cache.append(0, k.contiguous(), v.contiguous())
+            done += m
+        nb = n - N_SINK - WINDOW
+        for b in (8, 4, 2):
+            l0 = cache.launch_count()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(); cache.progressive_reduce(0); e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            key = f"{2 * b}to{b}"
+            best[key] = min(best.get(key, 1e9), ms)
+            launches[key] = cache.launch_count() - l0
+        cache.close(); del cache
+        torch.cuda.empty_cache()
+    out = {}
+    nb = n - N_SINK - WINDOW
+    for b in (8, 4, 2):
+        key = f"{2 * b}to{b}"
+        by = 2 * n_slices * nb * (16 * 2 * b + 16 * b + 8)
+        out[key] = {"us": best[key] * 1e3, "bytes": by, "GBps": by / (best[key] * 1e-3) / 1e9,
+                    "frac": by / (best[key] * 1e-3) / 1e9 / peak, "launches": launches[key]}
+    return out
+
+
+def aux_leg(wl, device, peak):
+    """The kernels beside the decode step, timed alone with CUDA events: the bulk prefill append of 8192 tokens
+    into one block of the workload's shape (best of 5 calls after a warm-up), one progressive-reduce event per
+    width, and the alpha grid search of the calibration (2048 tokens x 8 sequences, 20 alphas, 2 bit)."""
     from paper_2505_18610_b200 import binding as B
     n = 8192
     k, v = synth.make_kv(3, 0, 0, n, wl["batch"], wl["kv_heads"], 0, wl["n_outlier"], wl["factor"], device=device)
@@ -200,7 +298,9 @@ def aux_leg(wl, device):
         cache.close(); del cache
     append_bytes = 2 * n * n_slices * (256 + tokbytes(16))
     out = {"bulk_append": {"tokens": n, "ms": min(ts[1:]), "GBps": append_bytes / (min(ts[1:]) * 1e-3) / 1e9,
+                           "frac": append_bytes / (min(ts[1:]) * 1e-3) / 1e9 / peak,
                            "bytes": append_bytes, "what": "bf16 K, V in, INT16 tiles out, one block"}}
+    out["reduce"] = reduce_leg(wl, device, peak)
     g = torch.Generator().manual_seed(5)
     nt, ns, kvh, grp = 2048, 8, wl["kv_heads"], wl["q_heads"] // wl["kv_heads"]    # a 2,048-token calibration text
     kk = torch.randn(nt, ns, kvh, 128, generator=g); kk[..., 9] *= 25.0; kk[..., 73] *= 25.0
@@ -217,6 +317,48 @@ def aux_leg(wl, device):
                                 "fp32_TFLOPs": flop / (min(ts[1:]) * 1e-3) / 1e12,
                                 "what": "host-timed call (it ends with a synchronize); 21 causal attention passes"}
     return out
+
+
+def steady_state_record(name, device, peak, launches=5, steps=4):
+    """A compact steady-state record of another workload: the cache is built once with every block at its
+    final width (default budgets), then timed twice: the all-blocks attention launch alone, and whole decode
+    steps (append + eviction + attention) through pmkvq_decode_step."""
+    wl = WORKLOADS[name]
+    if wl.get("schedule") == "70b":
+        fbit = plan(wl, 8, 3)[0]
+    else:
+        fbit = synth.bit_schedule(wl["layers"], wl["edge_bits"], wl["inner_bits"], wl["n_edge"])
+    n0 = wl["end_tokens"] - steps - 3
+    cache = build_cache(wl, fbit, None, None, n0, device, shared_chunks=True)
+    assert all(cache.layer_state(l)["cur_bits"] == fbit[l] for l in range(wl["layers"]))
+    L = wl["layers"]
+    q = torch.stack([synth.make_q(2, l % 4, 0, wl["batch"], wl["q_heads"], n0, device=device) for l in range(L)]).contiguous()
+    o = torch.empty(L, wl["batch"], wl["q_heads"], 128, dtype=torch.float32, device=device)
+    ts = time_attention_all(cache, q, o, launches, warm=2)
+    by = sum(cache.attention_bytes(l) for l in range(L))
+    ms = float(np.median(ts))
+    k1, v1 = synth.make_kv(5, 0, 0, 1, wl["batch"], wl["kv_heads"], n0, wl["n_outlier"], wl["factor"], device=device)
+    K = k1[0].unsqueeze(0).expand(L, -1, -1, -1).contiguous(); V = v1[0].unsqueeze(0).expand(L, -1, -1, -1).contiguous()
+    for _ in range(3):
+        cache.decode_step(K, V, q, out=o)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        cache.decode_step(K, V, q, out=o)
+    e1.record()
+    torch.cuda.synchronize()
+    step_ms = e0.elapsed_time(e1) / steps
+    by_step = sum(cache.attention_bytes(l) for l in range(L))
+    cache.device_status()
+    rec = {"workload": wl["name"], "fbit_counts": {str(b): fbit.count(b) for b in sorted(set(fbit))},
+           "cache_GB": by / 1e9, "attention_ms_per_launch": ms, "attention_GBps": by / (ms * 1e-3) / 1e9,
+           "attention_frac": by / (ms * 1e-3) / 1e9 / peak, "step_ms": step_ms,
+           "step_GBps": by_step / (step_ms * 1e-3) / 1e9, "tokens_per_s": wl["batch"] / (step_ms * 1e-3),
+           "what": "every block at its final width; attention launch alone (median of %d) and whole decode steps (%d)" % (launches, steps)}
+    cache.close(); del cache
+    torch.cuda.empty_cache()
+    return rec
 
 
 class ClockSampler:
@@ -263,12 +405,11 @@ class ClockSampler:
         return out
 
 
-def run_steps(cache, wl, pool, steps, first_step, out, host_io=None, attn_events=None):
+def run_steps(cache, wl, pool, steps, first_step, out, host_io=None):
     """Run `steps` decode steps.  With host_io the step's inputs come from pinned host memory and the
     outputs go back to pinned host memory (end-to-end leg)."""
     K, V, Q = pool
     n_pool = K.shape[0]
-    L = wl["layers"]
     for s in range(steps):
         i = (first_step + s) % n_pool
         if host_io is not None:
@@ -276,18 +417,8 @@ def run_steps(cache, wl, pool, steps, first_step, out, host_io=None, attn_events
             dk.copy_(hk[i], non_blocking=True); dv.copy_(hv[i], non_blocking=True); dq.copy_(hq[i], non_blocking=True)
             cache.decode_step(dk, dv, dq, out=do)
             ho.copy_(do, non_blocking=True)
-        elif attn_events is None:
-            cache.decode_step(K[i], V[i], Q[i], out=out)
         else:
-            # an event pair around the step's launches: the all-blocks attention kernel and the all-blocks
-            # append kernel before it (and, in the few steps where a block's budget fills, its reduce)
-            bits0 = [cache.layer_state(l)["cur_bits"] for l in range(L)]
-            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-            e0.record()
             cache.decode_step(K[i], V[i], Q[i], out=out)
-            e1.record()
-            reduced = any(cache.layer_state(l)["cur_bits"] != bits0[l] for l in range(L))
-            attn_events.append((e0, e1, sum(cache.attention_bytes(l) for l in range(L)), reduced))
 
 
 def cpu_oracle_leg(wl, seconds_target=12.0, steps=None, warmup=1, n_sample_slices=4):
@@ -350,17 +481,21 @@ def main():
     ap.add_argument("--impl", default="pmkvq", choices=["pmkvq", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS))
     ap.add_argument("--ctas", type=int, default=0, help="attention grid override (0 = library default: one wave)")
+    ap.add_argument("--attention-path", type=int, default=0, choices=[0, 1],
+                    help="0 warp-level MMAs (default), 1 tensor memory at 4 and 2 bit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-aux", action="store_true", help="skip the prefill-append and calibration timings")
+    ap.add_argument("--no-aux", action="store_true", help="skip the prefill-append, reduce and calibration timings")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
-    ap.add_argument("--no-kernel-timing", action="store_true", help="skip the per-launch event leg (profiling runs)")
+    ap.add_argument("--no-widths", action="store_true", help="skip the per-width steady-state records")
+    ap.add_argument("--no-others", action="store_true", help="skip the compact 8B / 32B / 70B records")
+    ap.add_argument("--attention-only", type=int, default=0,
+                    help="profiling runs: build the cache at its final widths and launch the attention this many times")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     steps, warmup = args.steps, max(3, args.warmup)
-    G = wl["q_heads"] // wl["kv_heads"]
 
     if args.impl == "reference":
         if rank != 0:
@@ -389,20 +524,42 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        with open(peaks_path) as f:
+            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+
     fbit, budgets, n0 = plan(wl, steps, warmup)
     lam = make_lambda(wl, 0, device)
+    L = wl["layers"]
+    out_dev = torch.empty(L, wl["batch"], wl["q_heads"], 128, dtype=torch.float32, device=device)
+
+    if args.attention_only:      # profiling runs: the steady-state attention launch and nothing else
+        cache = build_cache(wl, fbit, None, lam, wl["end_tokens"], device, shared_chunks=True, attention_path=args.attention_path)
+        q = torch.stack([synth.make_q(2, l, 0, wl["batch"], wl["q_heads"], wl["end_tokens"], device=device) for l in range(L)]).contiguous()
+        ts = time_attention_all(cache, q, out_dev, args.attention_only, warm=2)
+        by = sum(cache.attention_bytes(l) for l in range(L))
+        print(json.dumps({"attention_only": True, "workload": wl["name"], "launches": args.attention_only,
+                          "ms_per_launch": float(np.median(ts)), "GBps": by / (float(np.median(ts)) * 1e-3) / 1e9, "bytes": by}))
+        return
+
     n_pool = 8
     pool = step_inputs(wl, n_pool, 0, device, n0)
-    n_slices = wl["batch"] * wl["kv_heads"]
 
-    out_dev = torch.empty(wl["layers"], wl["batch"], wl["q_heads"], 128, dtype=torch.float32, device=device)
-
-    # ---------------- device-resident leg: `value` ----------------
-    cache = build_cache(wl, fbit, budgets, lam, n0, device)
+    # ---------------- the cache is built once; its freshly prefilled state is kept for the end-to-end leg ----------------
+    cache = build_cache(wl, fbit, budgets, lam, n0, device, attention_path=args.attention_path)
     if args.ctas:
         cache.set_attention_ctas(args.ctas)
+    states0 = [cache.layer_state(l) for l in range(L)]
+    snapshot = None
+    if not args.no_e2e and cache.arena.numel() < 70e9:
+        snapshot = cache.arena.clone()
+
+    # ---------------- device-resident leg: `value` (the trajectory: appends, evictions, every block's last reduce) ----------------
     run_steps(cache, wl, pool, warmup, 0, out_dev)
-    bits_before = [cache.layer_state(l)["cur_bits"] for l in range(wl["layers"])]
+    bits_before = [cache.layer_state(l)["cur_bits"] for l in range(L)]
     barrier()
     launches0 = cache.launch_count()
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -414,46 +571,39 @@ def main():
         total_bytes += step_bytes(cache, wl, bits_before)       # host-side bookkeeping only
     ev1.record()
     barrier()
-    clocks = sampler.stop() if sampler else None
     ms = ev0.elapsed_time(ev1)
     launches = cache.launch_count() - launches0
-    n_reduced = sum(1 for l in range(wl["layers"]) if cache.layer_state(l)["cur_bits"] == fbit[l])
+    n_reduced = sum(1 for l in range(L) if cache.layer_state(l)["cur_bits"] == fbit[l])
     final_tokens = cache.layer_state(0)["n_tokens"]
-    cache.close(); del cache
-    torch.cuda.empty_cache()
 
-    # ---------------- the same timed region again, with an event pair around every step ----------------
-    attn_ms, attn_bytes, n_attn, instr_ms = float("nan"), 0, 0, float("nan")
-    if not args.no_kernel_timing:
-        cache = build_cache(wl, fbit, budgets, lam, n0, device)
-        if args.ctas:
-            cache.set_attention_ctas(args.ctas)
-        run_steps(cache, wl, pool, warmup, 0, out_dev)
-        barrier()
-        attn_events = []
-        k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        k0.record()
-        run_steps(cache, wl, pool, steps, warmup, out_dev, attn_events=attn_events)
-        k1.record()
-        barrier()
-        instr_ms = k0.elapsed_time(k1)
-        plain = [(a, b, c) for a, b, c, reduced in attn_events if not reduced] or [(a, b, c) for a, b, c, _ in attn_events]
-        attn_ms = sum(a.elapsed_time(b) for a, b, _ in plain)
-        attn_bytes = sum(c for _, _, c in plain)
-        n_attn = len(plain)
-        cache.close(); del cache
-        torch.cuda.empty_cache()
+    # ---------------- roofline leg: the attention launch alone, on the cache as the run left it ----------------
+    # (every block that can be is at its final width now: no reduce, no append, only decode_attn_fused_kernel)
+    n_attn = max(10, min(steps, 40))
+    ts = time_attention_all(cache, pool[2][0], out_dev, n_attn)
+    attn_ms = float(np.sum(ts))
+    attn_bytes = sum(cache.attention_bytes(l) for l in range(L))
+    widths_now = {str(b): sum(1 for l in range(L) if cache.layer_state(l)["cur_bits"] == b) for b in (2, 4, 8, 16)}
+    clocks = sampler.stop() if sampler else None
+    cache.device_status()
 
-    # ---------------- end-to-end leg: host buffers in, host buffers out ----------------
+    # ---------------- end-to-end leg: the same trajectory with host buffers in, host buffers out ----------------
     e2e_ms, h2d, d2h = float("nan"), 0, 0
     if not args.no_e2e:
-        cache = build_cache(wl, fbit, budgets, lam, n0, device)
-        if args.ctas:
-            cache.set_attention_ctas(args.ctas)
+        if snapshot is not None:
+            cache.arena.copy_(snapshot)
+            for l in range(L):
+                cache.restore_layer_state(l, states0[l]["n_tokens"], states0[l]["cur_bits"])
+            del snapshot
+        else:
+            cache.close(); del cache
+            torch.cuda.empty_cache()
+            cache = build_cache(wl, fbit, budgets, lam, n0, device, attention_path=args.attention_path)
+            if args.ctas:
+                cache.set_attention_ctas(args.ctas)
         K, V, Q = pool
         hk, hv, hq = K.cpu().pin_memory(), V.cpu().pin_memory(), Q.cpu().pin_memory()
         dk, dv, dq = torch.empty_like(K[0]), torch.empty_like(V[0]), torch.empty_like(Q[0])
-        do = torch.empty(wl["layers"], wl["batch"], wl["q_heads"], 128, dtype=torch.float32, device=device)
+        do = torch.empty(L, wl["batch"], wl["q_heads"], 128, dtype=torch.float32, device=device)
         ho = torch.empty(do.shape, dtype=torch.float32).pin_memory()
         host_io = (hk, hv, hq, ho, dk, dv, dq, do)
         run_steps(cache, wl, pool, warmup, 0, out_dev, host_io=host_io)
@@ -466,7 +616,8 @@ def main():
         e2e_ms = e0.elapsed_time(e1)
         h2d = (dk.numel() + dv.numel() + dq.numel()) * 2
         d2h = do.numel() * 4
-        cache.close(); del cache
+    cache.close(); del cache
+    torch.cuda.empty_cache()
 
     # ---------------- max over ranks ----------------
     ms, e2e_ms, attn_ms = max_over_ranks([ms, e2e_ms, attn_ms], dist, device)
@@ -475,54 +626,52 @@ def main():
             dist.destroy_process_group()
         return
 
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        with open(peaks_path) as f:
-            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    else:
-        peak, peak_src = 6650.0, "fallback"
     value = whole_job_rate(total_bytes, world, ms) / 1e9
     traffic = None
-    if wl is WORKLOADS["7b"] and kernel_source_digest() == NCU_TRAFFIC["digest"] and n_attn:
-        # measured traffic / algorithmic bytes of the captured launches, applied to this run's average launch
-        ratio = NCU_TRAFFIC["traffic_bytes"] / NCU_TRAFFIC["algorithmic_bytes"]
-        traffic = ratio * attn_bytes / n_attn
-    achieved = attn_bytes / (attn_ms * 1e-3) / 1e9 if n_attn else float("nan")
+    if wl is WORKLOADS["7b"] and kernel_source_digest() == NCU_TRAFFIC["digest"]:
+        # measured traffic / algorithmic bytes of the captured launch, applied to this run's launch
+        traffic = NCU_TRAFFIC["traffic_bytes"] / NCU_TRAFFIC["algorithmic_bytes"] * attn_bytes
+    achieved = attn_bytes * n_attn / (attn_ms * 1e-3) / 1e9
     line = {
         "metric": "decode_attention_GBps", "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "int2/int4/int16 codes, f16 mma.sync, f32 accumulate", "data": "synthetic",
+        "vs_baseline": None, "dtype": "int2/int4/int8/int16 codes as f16 MMA operands, f32 accumulate", "data": "synthetic",
         "config": {"workload": wl["name"],
-                   "shape": f"{wl['layers']} blocks x ({wl['q_heads']} Q / {wl['kv_heads']} KV heads, head_dim 128) x batch "
+                   "shape": f"{L} blocks x ({wl['q_heads']} Q / {wl['kv_heads']} KV heads, head_dim 128) x batch "
                             f"{wl['batch']} per GPU x {final_tokens} cached tokens at the end",
                    "fbit_per_block": fbit,
                    "blocks_reduced_to_fbit_in_run": n_reduced, "n_sink": N_SINK, "window": WINDOW,
+                   "attention_path": "tensor memory (tcgen05.mma)" if args.attention_path else "warp-level MMAs (mma.sync)",
                    "l2": "per-step working set (the whole cache) is far larger than L2; no flush needed",
                    "path": "attention path only (no weights / MLP)", "sharding": "batch, no collective"},
         "tokens_per_s": whole_job_rate(wl["batch"] * steps, world, ms),
         "frac_of_8TBps_nominal": value / world / 8000.0,
-        "roofline": {"bound": "hbm", "kernel": "decode_attn_fused_kernel: the attention of all blocks of a step, one launch",
+        "roofline": {"bound": "hbm", "kernel": "decode_attn_fused_kernel: the attention of all blocks, one launch",
                      "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic,
                      "traffic_source": "ncu dram read+write / algorithmic bytes of a captured 4-block launch of the same kernel, times this "
-                                       "run's average launch; null if the kernel sources changed since the capture",
-                     "avg_launch_ms": attn_ms / max(1, n_attn), "launches_timed": n_attn,
-                     "algorithmic_bytes_per_launch": attn_bytes / max(1, n_attn),
-                     "how": "the timed steps replayed on an identical cache with a CUDA event pair around every step; "
-                            "the pair also spans the step's append kernel (one launch, under 1 % of the step); steps in "
-                            "which a block was reduced are left out of the average",
-                     "ms_per_step_with_events": instr_ms / steps},
+                                       "run's launch; null if the kernel sources changed since the capture",
+                     "avg_launch_ms": attn_ms / n_attn, "launches_timed": n_attn,
+                     "algorithmic_bytes_per_launch": attn_bytes, "blocks_at_width": widths_now,
+                     "how": "after the timed steps (every block's last reduce is behind it) the attention launch alone is "
+                            "repeated on the same cache through pmkvq_decode_attention_all, one CUDA event pair per launch; "
+                            "nothing is appended or reduced in between"},
         "e2e": {"value": world * total_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms / steps,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "clocks": clocks,
     }
-    if not args.no_cpu_baseline and world == 1:
-        gbs, dt, desc, cores, nst, _ = cpu_oracle_leg(wl)
-        line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc,
-                                "s_per_oracle_step": dt}
-    if not args.no_aux and world == 1:
-        line["aux"] = aux_leg(wl, device)
+    if world == 1:
+        if not args.no_widths:
+            line["roofline_by_width"] = width_leg(wl, device, peak)
+        if not args.no_aux:
+            line["aux"] = aux_leg(wl, device, peak)
+        if not args.no_others:
+            line["other_workloads"] = {n: steady_state_record(n, device, peak) for n in ("8b", "32b", "70b") if WORKLOADS[n] is not wl}
+        if not args.no_cpu_baseline:
+            gbs, dt, desc, cores, nst, _ = cpu_oracle_leg(wl)
+            line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc,
+                                    "s_per_oracle_step": dt}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -335,18 +335,17 @@ __device__ __forceinline__ float softmax_phase(const uint8_t *tile0, uint32_t ma
     const float2 neg_m = make_float2(-st.m, -st.m), inv2 = make_float2(inv_sigma_e, inv_sigma_e);
 #pragma unroll
     for (int j = 0; j < NP; ++j) {
-      // a constant V group has S_V = 0 and all codes 0: any finite unit will do for it
-      const float2 s_e = __ffma2_rn(sv[j], inv2, make_float2(sv[j].x == 0.f ? 1.f : 0.f, sv[j].y == 0.f ? 1.f : 0.f));
+      // The token's unit s_e = S_V / sigma_u * 2^EP is kept at or above 2^-10, so that w stays in fp16's normal
+      // range whenever p matters: a constant V group (S_V = 0, all codes 0) and a token whose V scale lies
+      // far below the slice's largest then enter the sums with their exact probability, and what the floor
+      // adds to the output, at most p * 2^-22 sigma_u per code unit, is far below the tolerance.
+      float2 s_e = __fmul2_rn(sv[j], inv2);
+      s_e.x = fmaxf(s_e.x, 0x1p-10f); s_e.y = fmaxf(s_e.y, 0x1p-10f);
       const float2 rs = make_float2(rcp_approx(s_e.x), rcp_approx(s_e.y));
       const float2 arg = __fadd2_rn(sc[j], neg_m);
-      const float2 e = make_float2(ex2(arg.x), ex2(arg.y));
-      const float2 w = __fmul2_rn(e, s_e);  // p * S_V / sigma_u * 2^EP
+      const float2 w = __fmul2_rn(make_float2(ex2(arg.x), ex2(arg.y)), s_e);  // p * S_V / sigma_u * 2^EP
       pb[j] = pack_half2(w.x, w.y);
-      float2 p = __fmul2_rn(__half22float2(*reinterpret_cast<const __half2 *>(&pb[j])), rs);
-      // a V scale far below the slice's largest takes w out of fp16's normal range (the token's codes then
-      // carry next to nothing): its probability enters the sums as it is
-      if (s_e.x < 0x1p-10f) p.x = e.x;
-      if (s_e.y < 0x1p-10f) p.y = e.y;
+      const float2 p = __fmul2_rn(__half22float2(*reinterpret_cast<const __half2 *>(&pb[j])), rs);
       st.l = __fadd2_rn(st.l, p);
       st.zs = __ffma2_rn(p, zv[j], st.zs);
     }

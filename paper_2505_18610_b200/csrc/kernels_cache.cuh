@@ -667,28 +667,58 @@ __global__ void __launch_bounds__(128) append_step_kernel(const uint16_t *__rest
 // one word at B bits.  Everything is read and transformed before the first store, so the output may
 // overlap this tile's own input.
 // ---------------------------------------------------------------------------------------------
+// Eq. 3 (or the plain right shift of the ablations) on all codes of two adjacent words at 2B bits, packed into
+// one word at B bits: half h of the result holds the codes of half h of in0 in its low byte-half and those
+// of in1 above them.  The narrow widths work on several fields of a register at once: the products
+// (c + 2^(B-1)) (2^2B - 2^B + 1) of a 4-bit (8-bit) code fit the code's own byte (16-bit lane), so one
+// multiply-add serves four (two) codes.
 template <int B, bool SHR>
-__device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1) {
-  constexpr int NIN = 8 / B;  // codes per half-word at 2B bits
-  constexpr uint32_t MASK = (1u << (2 * B)) - 1u;
-  uint32_t out = 0;
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-#pragma unroll
-    for (int j = 0; j < NIN; ++j) {
-      const uint32_t c0 = (in0 >> (16 * h + j * 2 * B)) & MASK;
-      const uint32_t c1 = (in1 >> (16 * h + j * 2 * B)) & MASK;
-      out |= (SHR ? c0 >> B : shift_step(c0, B)) << (16 * h + j * B);
-      out |= (SHR ? c1 >> B : shift_step(c1, B)) << (16 * h + (NIN + j) * B);
-    }
+__device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1);
+
+template <bool SHR>
+__device__ __forceinline__ uint32_t halve_nibbles(uint32_t x) {  // 8 codes of 4 bit -> 8 codes of 2 bit in bits 0-7, 16-23
+  const uint32_t a = x & 0x0F0F0F0Fu, b = (x >> 4) & 0x0F0F0F0Fu;  // even / odd fields, one per byte
+  uint32_t ya, yb;
+  if (SHR) {
+    ya = (a >> 2) & 0x03030303u;
+    yb = (b >> 2) & 0x03030303u;
+  } else {  // (13 (c + 2)) >> 6 per byte: 13 * 17 = 221 stays inside the byte
+    ya = ((a * 13u + 0x1A1A1A1Au) >> 6) & 0x03030303u;
+    yb = ((b * 13u + 0x1A1A1A1Au) >> 6) & 0x03030303u;
   }
-  return out;
+  return ((ya | (ya >> 4)) & 0x00330033u) | (((yb << 2) | (yb >> 2)) & 0x00CC00CCu);
+}
+template <bool SHR>
+__device__ __forceinline__ uint32_t halve_bytes(uint32_t x) {  // 4 codes of 8 bit -> 4 codes of 4 bit in bits 0-7, 16-23
+  const uint32_t a = x & 0x00FF00FFu, b = (x >> 8) & 0x00FF00FFu;  // first / second code of each half
+  uint32_t ya, yb;
+  if (SHR) {
+    ya = (a >> 4) & 0x000F000Fu;
+    yb = (b >> 4) & 0x000F000Fu;
+  } else {  // (241 (c + 8)) >> 12 per 16-bit lane: 241 * 263 = 63383 stays inside the lane
+    ya = ((a * 241u + 0x07880788u) >> 12) & 0x000F000Fu;
+    yb = ((b * 241u + 0x07880788u) >> 12) & 0x000F000Fu;
+  }
+  return ya | (yb << 4);
+}
+template <> __device__ __forceinline__ uint32_t merge_words<2, false>(uint32_t in0, uint32_t in1) { return halve_nibbles<false>(in0) | (halve_nibbles<false>(in1) << 8); }
+template <> __device__ __forceinline__ uint32_t merge_words<2, true>(uint32_t in0, uint32_t in1) { return halve_nibbles<true>(in0) | (halve_nibbles<true>(in1) << 8); }
+template <> __device__ __forceinline__ uint32_t merge_words<4, false>(uint32_t in0, uint32_t in1) { return halve_bytes<false>(in0) | (halve_bytes<false>(in1) << 8); }
+template <> __device__ __forceinline__ uint32_t merge_words<4, true>(uint32_t in0, uint32_t in1) { return halve_bytes<true>(in0) | (halve_bytes<true>(in1) << 8); }
+// 16 -> 8 bit: the product (c + 128) * 65281 needs all 32 bits; the new code is its top byte
+template <> __device__ __forceinline__ uint32_t merge_words<8, false>(uint32_t in0, uint32_t in1) {
+  const uint32_t p00 = (in0 & 0xFFFFu) * 65281u + 0x7F8080u, p01 = (in0 >> 16) * 65281u + 0x7F8080u;
+  const uint32_t p10 = (in1 & 0xFFFFu) * 65281u + 0x7F8080u, p11 = (in1 >> 16) * 65281u + 0x7F8080u;
+  return __byte_perm(__byte_perm(p00, p10, 0x0073), __byte_perm(p01, p11, 0x0073), 0x5410);  // {p00.3, p10.3, p01.3, p11.3}
+}
+template <> __device__ __forceinline__ uint32_t merge_words<8, true>(uint32_t in0, uint32_t in1) {
+  return __byte_perm(__byte_perm(in0, in1, 0x0051), __byte_perm(in0, in1, 0x0073), 0x5410);  // the high byte of each code
 }
 
 // CTA_WIDE: the warps of a CTA work on consecutive tiles at once; a CTA-wide barrier (reached by every
 // warp, `active` or not) separates all their loads from all their stores.
-template <int B, bool SHR, bool CTA_WIDE>
-__device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, int lane, int variant, bool active) {
+template <int B, bool SHR>
+__device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, int lane, int variant, bool active, bool cta_wide) {
   constexpr int IN_CHUNKS = B;                          // 16-byte chunks per lane per part at 2B bits
   constexpr int OUT_WORDS = 2 * B;                      // words per lane per part at B bits
   constexpr int OUT_CHUNKS = (OUT_WORDS + 3) / 4;
@@ -726,7 +756,7 @@ __device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, i
   }
   }
   // every lane (every warp of the CTA) holds its transformed data: the input is dead from here on
-  if constexpr (CTA_WIDE) __syncthreads();
+  if (cta_wide) __syncthreads();
   else __syncwarp();
   if (!active) return;
 #pragma unroll
@@ -741,16 +771,16 @@ __device__ __forceinline__ void reduce_tile_v(const uint8_t *in, uint8_t *out, i
   *reinterpret_cast<float2 *>(out + meta_offset(B) + lane * 8) = m;
 }
 
-template <int B, bool CTA_WIDE = false>
-__device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int lane, int variant, bool active = true) {
-  if (variant == kShiftEquivalent) reduce_tile_v<B, false, CTA_WIDE>(in, out, lane, variant, active);
-  else reduce_tile_v<B, true, CTA_WIDE>(in, out, lane, variant, active);
+template <int B>
+__device__ __forceinline__ void reduce_tile(const uint8_t *in, uint8_t *out, int lane, int variant, bool active, bool cta_wide) {
+  if (variant == kShiftEquivalent) reduce_tile_v<B, false>(in, out, lane, variant, active, cta_wide);
+  else reduce_tile_v<B, true>(in, out, lane, variant, active, cta_wide);
 }
 
 // Row tile at 4 bit -> row tile at 2 bit: in both parts the words of a row pair up (a token row has 16
 // words, a channel row 2), so the tile is a flat array of word pairs; a lane takes four words at a time.
 template <bool SHR>
-__device__ __forceinline__ void reduce_tile_row(const uint8_t *in, uint8_t *out, int lane, int variant, bool active) {
+__device__ __forceinline__ void reduce_tile_row(const uint8_t *in, uint8_t *out, int lane, int variant, bool active, bool cta_wide) {
   uint2 o[2][2];
   float4 m = make_float4(0.f, 0.f, 0.f, 0.f);
   if (active) {
@@ -767,7 +797,8 @@ __device__ __forceinline__ void reduce_tile_row(const uint8_t *in, uint8_t *out,
       halve_meta(m.z, m.w, 2, variant);
     }
   }
-  __syncthreads();  // every warp of the CTA holds its transformed tile: the inputs are dead from here on
+  if (cta_wide) __syncthreads();  // every warp of the CTA holds its transformed tile: the inputs are dead from here on
+  else __syncwarp();
   if (!active) return;
 #pragma unroll
   for (int part = 0; part < 2; ++part)
@@ -780,7 +811,7 @@ __device__ __forceinline__ void reduce_tile_row(const uint8_t *in, uint8_t *out,
 // bytes of this warp, one part at a time), from which the lanes gather the row words.
 template <bool SHR>
 __device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *out, int lane, int variant, bool active,
-                                                   uint8_t *scratch) {
+                                                   bool cta_wide, uint8_t *scratch) {
   const int g = lane >> 2, tig = lane & 3;
   uint4 ko[4];       // K part: this lane's 16 bytes of rows lane / 2 (+ 0, 1 ... see below)
   uint2 vo[4];       // V part: channels lane, lane + 32, ...
@@ -855,7 +886,8 @@ __device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *o
       halve_meta(m[2], m[3], 4, variant);
     }
   }
-  __syncthreads();  // every warp of the CTA holds its transformed tile: the inputs are dead from here on
+  if (cta_wide) __syncthreads();  // every warp of the CTA holds its transformed tile: the inputs are dead from here on
+  else __syncwarp();
   if (!active) return;
 #pragma unroll
   for (int rr = 0; rr < 2; ++rr)
@@ -865,32 +897,43 @@ __device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *o
   if (lane < 16) *reinterpret_cast<float4 *>(out + meta_offset(4) + lane * 16) = make_float4(m[0], m[1], m[2], m[3]);
 }
 
-// The whole body of a block in one launch: one CTA per (stream, slice) walks its stream front to back in
-// batches of one tile per warp.  Inside a stream tile j moves from j tile_bytes(2B) to j tile_bytes(B):
-// the outputs of a batch end below the inputs of every later batch and overlap inputs of this and earlier
-// batches only, which the CTA-wide barrier between a batch's loads and its stores has seen loaded.
+// The whole body of a block in one launch: one CTA per (stream, slice) compacts its stream in place.  Inside
+// a stream tile j moves from j tile_bytes(2B) to j tile_bytes(B).  The CTA first takes tiles [0, W), one per
+// warp, with a CTA-wide barrier between their loads and their stores; then waves [lo, hi) with
+// hi tile_bytes(B) <= lo tile_bytes(2B): every output of a wave lies below every input of the wave, so the
+// warps run through the wave's tiles without meeting, and a barrier between waves keeps a wave's stores
+// behind the earlier waves' loads.  The waves grow geometrically (x 1.8 - 1.9).
 constexpr int kReduceWarps = 8;
+template <int B>
+__device__ __forceinline__ void reduce_one_tile(const LayerGeom &geom, const uint8_t *in, uint8_t *out, int lane, bool active,
+                                                bool cta_wide, uint8_t *scratch) {
+  const bool shr = geom.shift_variant != kShiftEquivalent;
+  if (B == 8 || !geom.rows) {
+    reduce_tile<B>(in, out, lane, geom.shift_variant, active, cta_wide);
+  } else if constexpr (B == 4) {
+    if (shr) reduce_tile_to_row<true>(in, out, lane, geom.shift_variant, active, cta_wide, scratch);
+    else reduce_tile_to_row<false>(in, out, lane, geom.shift_variant, active, cta_wide, scratch);
+  } else {
+    if (shr) reduce_tile_row<true>(in, out, lane, geom.shift_variant, active, cta_wide);
+    else reduce_tile_row<false>(in, out, lane, geom.shift_variant, active, cta_wide);
+  }
+}
+
 template <int B>
 __global__ void __launch_bounds__(kReduceWarps * 32) reduce_stream_kernel(LayerGeom geom, int n_tiles) {
   __shared__ __align__(16) uint8_t s_scratch[B == 4 ? kReduceWarps : 1][B == 4 ? kTileTokens * kHeadDim : 16];
   const int stream = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint8_t *base = geom.base + (size_t)blockIdx.y * geom.slice_stride + geom.body_off + (size_t)stream * geom.stream_stride;
   const int cnt = (n_tiles - stream + kStreams - 1) / kStreams;  // tiles of this stream
-  const bool shr = geom.shift_variant != kShiftEquivalent;
-  for (int j0 = 0; j0 < cnt; j0 += kReduceWarps) {
-    const int j = j0 + warp;
-    const bool active = j < cnt;
-    const uint8_t *in = base + (size_t)j * tile_bytes(2 * B);
-    uint8_t *out = base + (size_t)j * tile_bytes(B);
-    if (B == 8 || !geom.rows) {
-      reduce_tile<B, true>(in, out, lane, geom.shift_variant, active);
-    } else if constexpr (B == 4) {
-      if (shr) reduce_tile_to_row<true>(in, out, lane, geom.shift_variant, active, s_scratch[warp]);
-      else reduce_tile_to_row<false>(in, out, lane, geom.shift_variant, active, s_scratch[warp]);
-    } else {
-      if (shr) reduce_tile_row<true>(in, out, lane, geom.shift_variant, active);
-      else reduce_tile_row<false>(in, out, lane, geom.shift_variant, active);
-    }
+  uint8_t *scratch = s_scratch[B == 4 ? warp : 0];
+  if (cnt <= 0) return;
+  reduce_one_tile<B>(geom, base + (size_t)warp * tile_bytes(2 * B), base + (size_t)warp * tile_bytes(B), lane, warp < cnt, true, scratch);
+  for (int lo = kReduceWarps; lo < cnt;) {
+    const int hi = min(cnt, (int)((long long)lo * tile_bytes(2 * B) / tile_bytes(B)));
+    __syncthreads();  // the stores of this wave may land on inputs of the tiles before it
+    for (int j = lo + warp; j < hi; j += kReduceWarps)
+      reduce_one_tile<B>(geom, base + (size_t)j * tile_bytes(2 * B), base + (size_t)j * tile_bytes(B), lane, true, false, scratch);
+    lo = hi;
   }
 }
 
