@@ -160,6 +160,15 @@ pmkvq_status pmkvq_device_status(pmkvq_cache *cache, uint32_t *h_wait_bits);
  * of this block (width below Fbit, over budget, beyond capacity); nothing on the device is touched. */
 pmkvq_status pmkvq_restore_layer_state(pmkvq_cache *cache, int32_t layer, int32_t n_tokens, int32_t cur_bits);
 
+/* Where a block's bytes sit inside the arena, for callers that checkpoint parts of it and for tests that watch
+ * the bytes the kernels must not touch.  h_out receives ten values: [0] the arena bytes the cache uses
+ * (= pmkvq_arena_bytes_required), [1] offset of the block's first (batch, kv_head) slice, [2] bytes between
+ * slices, and inside a slice [3] offset of the INT16 window ring (the sink tiles sit at 0), [4] offset of the
+ * body, [5] bytes between the body's eight streams (body tile i lives in stream i mod 8 at index i div 8,
+ * tile_bytes(b) = 512 b + 256 apart), [6] ring capacity in tokens; [7] offset and [8] size of the block's
+ * split-K workspace, [9] bytes of one partial slot in it. */
+pmkvq_status pmkvq_arena_layout(const pmkvq_cache *cache, int32_t layer, uint64_t *h_out);
+
 /* Split-K tuning of pmkvq_decode_attention (flash-decoding partition over the sequence): the tiles
  * of all (batch, kv_head) slices are cut into `n_ctas` equal contiguous pieces, one per CTA
  * (1..1024); 0 restores the default, one wave of resident CTAs on the GPU's SMs. */

@@ -68,6 +68,8 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.pmkvq_restore_layer_state.restype = i32
     lib.pmkvq_restore_layer_state.argtypes = [vp, i32, i32, i32]
+    lib.pmkvq_arena_layout.restype = i32
+    lib.pmkvq_arena_layout.argtypes = [vp, i32, u64p]
     lib.pmkvq_set_attention_ctas.restype = i32
     lib.pmkvq_set_attention_ctas.argtypes = [vp, i32]
     lib.pmkvq_layer_state.restype = i32
@@ -173,7 +175,8 @@ class Cache:
                  fbit: Sequence[int], budget_bytes: Optional[Sequence[int]] = None,
                  lam: Optional[np.ndarray] = None, n_sink: int = 1, window: int = 128, evict_chunk: int = 1,
                  count_metadata: bool = True, auto_reduce: bool = True, sm_scale: float = 0.0,
-                 device: str = "cuda:0", shift_variant: int = 0, attention_path: int = 0):
+                 device: str = "cuda:0", shift_variant: int = 0, attention_path: int = 0, slack_bytes: int = 0,
+                 fill_byte: Optional[int] = None):
         self._h = None
         self.layers, self.q_heads, self.kv_heads, self.batch = layers, q_heads, kv_heads, batch
         self._fbit = (ctypes.c_uint8 * layers)(*[int(b) for b in fbit])
@@ -197,8 +200,11 @@ class Cache:
         self.arena_bytes = need
         self.device = torch.device(device)
         with torch.cuda.device(self.device):
-            self.arena = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+            self.arena = torch.empty(need + 256 + int(slack_bytes), dtype=torch.uint8, device=self.device)
+            if fill_byte is not None:       # tests that watch the bytes no kernel may touch
+                self.arena.fill_(int(fill_byte))
             base = self.arena.data_ptr()
+            self.arena_offset = (base + 255) // 256 * 256 - base
             cfg.d_arena = (base + 255) // 256 * 256
             cfg.arena_bytes = need
             h = ctypes.c_void_p()
@@ -310,6 +316,15 @@ class Cache:
         st = lib().pmkvq_restore_layer_state(self._h, layer, int(n_tokens), int(cur_bits))
         if st != OK:
             raise PmkvqError(st, "pmkvq_restore_layer_state")
+
+    def arena_layout(self, layer: int):
+        out = (ctypes.c_uint64 * 10)()
+        st = lib().pmkvq_arena_layout(self._h, layer, out)
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_arena_layout")
+        keys = ("arena_bytes", "offset", "slice_stride", "ring_off", "body_off", "stream_stride", "ring_tokens",
+                "partials_off", "partials_bytes", "partial_slot_bytes")
+        return dict(zip(keys, [int(x) for x in out]))
 
     def set_attention_ctas(self, n_ctas: int):
         st = lib().pmkvq_set_attention_ctas(self._h, n_ctas)

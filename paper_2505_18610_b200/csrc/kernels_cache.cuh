@@ -903,7 +903,10 @@ __device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *o
 // hi tile_bytes(B) <= lo tile_bytes(2B): every output of a wave lies below every input of the wave, so the
 // warps run through the wave's tiles without meeting, and a barrier between waves keeps a wave's stores
 // behind the earlier waves' loads.  The waves grow geometrically (x 1.8 - 1.9).
-constexpr int kReduceWarps = 8;
+// Warps per CTA: enough tiles in flight per stream to cover the memory latency, and few enough registers
+// that every (stream, slice) CTA of the common shapes is resident at once.
+template <int B> __host__ __device__ constexpr int reduce_warps() { return B == 2 ? 16 : 8; }
+template <int B> __host__ __device__ constexpr int reduce_min_ctas() { return B == 2 ? 3 : 4; }
 template <int B>
 __device__ __forceinline__ void reduce_one_tile(const LayerGeom &geom, const uint8_t *in, uint8_t *out, int lane, bool active,
                                                 bool cta_wide, uint8_t *scratch) {
@@ -920,7 +923,8 @@ __device__ __forceinline__ void reduce_one_tile(const LayerGeom &geom, const uin
 }
 
 template <int B>
-__global__ void __launch_bounds__(kReduceWarps * 32) reduce_stream_kernel(LayerGeom geom, int n_tiles) {
+__global__ void __launch_bounds__(reduce_warps<B>() * 32, reduce_min_ctas<B>()) reduce_stream_kernel(LayerGeom geom, int n_tiles) {
+  constexpr int kReduceWarps = reduce_warps<B>();
   __shared__ __align__(16) uint8_t s_scratch[B == 4 ? kReduceWarps : 1][B == 4 ? kTileTokens * kHeadDim : 16];
   const int stream = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint8_t *base = geom.base + (size_t)blockIdx.y * geom.slice_stride + geom.body_off + (size_t)stream * geom.stream_stride;

@@ -171,7 +171,7 @@ size_t plan(pmkvq_cache &k, const pmkvq_config *c) {
 template <int B>
 cudaError_t launch_reduce(const LayerGeom &g, int n_slices, int n_tiles, cudaStream_t st, uint64_t &launches) {
   // one CTA per (stream, slice): the streams compact in place independently of one another
-  reduce_stream_kernel<B><<<dim3(kStreams, (unsigned)n_slices), kReduceWarps * 32, 0, st>>>(g, n_tiles);
+  reduce_stream_kernel<B><<<dim3(kStreams, (unsigned)n_slices), reduce_warps<B>() * 32, 0, st>>>(g, n_tiles);
   ++launches;
   return cudaGetLastError();
 }
@@ -646,6 +646,23 @@ pmkvq_status pmkvq_restore_layer_state(pmkvq_cache *k, int32_t layer, int32_t n_
     return PMKVQ_ERR_INVALID_ARG;
   l.n_tokens = n_tokens;
   l.cur_bits = cur_bits;
+  return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_arena_layout(const pmkvq_cache *k, int32_t layer, uint64_t *h_out) {
+  if (!k || !h_out || layer < 0 || layer >= k->layers) return PMKVQ_ERR_INVALID_ARG;
+  const Layer &l = k->L[layer];
+  const LayerGeom g = k->geom(l);
+  h_out[0] = k->arena_bytes;
+  h_out[1] = l.offset;
+  h_out[2] = g.slice_stride;
+  h_out[3] = g.ring_off;
+  h_out[4] = g.body_off;
+  h_out[5] = g.stream_stride;
+  h_out[6] = (uint64_t)k->ring_tiles * kTileTokens;
+  h_out[7] = k->off_partials + (uint64_t)layer * k->partial_bytes;
+  h_out[8] = k->partial_bytes;
+  h_out[9] = (uint64_t)kMaxGroup * kPartialStride * sizeof(float);
   return PMKVQ_OK;
 }
 

@@ -8,7 +8,7 @@ import torch
 from oracle import pmkvq_oracle as O
 from paper_2505_18610_b200 import synth
 
-MAX_ABS_TOL = 2e-3     # spec tolerance on attention outputs
+MAX_ABS_TOL = 2e-3     # the stated tolerance on attention outputs
 REL_L2_TOL = 1e-3
 
 
@@ -36,6 +36,7 @@ class Mirror:
             pol = O.Policy(fbit[l], max_tokens, n_slices, None if budget_bytes is None else budget_bytes[l], **okw)
             lam_s = None if self.lam is None else np.stack([self.lam[l, s % kv_heads] for s in self.slices])
             self.oracles.append(O.LayerOracle(pol, len(self.slices), lam=lam_s, shift_variant=variant))
+        self.sm_scale = kw.get("sm_scale") or None
 
     def append(self, layer, k, v, bulk=True):
         """k, v: CPU or CUDA bf16 [n, batch, kv_heads, 128]."""
@@ -73,7 +74,7 @@ class Mirror:
         torch.cuda.synchronize()
         got = out.cpu().numpy().reshape(self.batch * self.kv_heads, self.group, 128)[self.slices]
         qq = q.float().cpu().numpy().reshape(self.batch * self.kv_heads, self.group, 128)[self.slices]
-        ref = self.oracles[layer].decode_attention(qq)
+        ref = self.oracles[layer].decode_attention(qq, sm_scale=self.sm_scale)
         assert np.all(np.isfinite(got)), "non-finite attention output"
         err = float(np.abs(got.astype(np.float64) - ref).max())
         rel = float(np.linalg.norm(got.astype(np.float64) - ref) / max(np.linalg.norm(ref), 1e-30))

@@ -22,6 +22,26 @@ def test_hand_case():
     assert B.allocate_bits([2, 4], sens, mem, 20) == ([2, 2], 14.0)
     with pytest.raises(B.PmkvqError):
         B.allocate_bits([2, 4], sens, mem, 19)
+    # the same hand-computed answers pin the exhaustive oracle the other tests compare against
+    assert O.allocate_bits_brute_force(sens, mem, 30) == ([0, 1], 7.0)
+    assert O.allocate_bits_brute_force(sens, mem, 40) == ([1, 1], 3.0)
+    assert O.allocate_bits_brute_force(sens, mem, 20) == ([0, 0], 14.0)
+    assert O.allocate_bits_brute_force(sens, mem, 19) == (None, np.inf)
+
+
+def test_sensitivity_of_hand_made_tokens():
+    """The oracle's sensitivity (L1 error of the per-token quantizer) on tokens whose codes can be written down:
+    a token with values {0, 1, 2, 3} (times any scale) is exact at 2 bit, one with {0, 1.5, 3} loses 0.5 on
+    its middle value at 2 bit (code 1 or 2, S = 1) and nothing at 4 bit (S = 0.2, code 7.5 -> tie, error 0.1)."""
+    exact = np.tile(np.array([0.0, 1.0, 2.0, 3.0], np.float32), 32)[None, :] * 0.25
+    assert O.quantization_sensitivity(exact, exact, 2) == 0.0
+    tok = np.zeros((1, 128), np.float32); tok[0, 1] = 1.5; tok[0, 2] = 3.0
+    assert abs(O.quantization_sensitivity(tok, np.zeros_like(tok), 2) - 0.5) < 1e-6
+    # 4 bit: S = 3 / 15 = 0.2, 1.5 / 0.2 = 7.5 rounds to 8 (half to even) -> 1.6: error 0.1
+    assert abs(O.quantization_sensitivity(tok, np.zeros_like(tok), 4) - 0.1) < 1e-6
+    # errors add over K and V and over tokens
+    both = O.quantization_sensitivity(np.concatenate([tok, tok]), tok, 2)
+    assert abs(both - 1.5) < 1e-6
 
 
 @pytest.mark.parametrize("seed", range(6))

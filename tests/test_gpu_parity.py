@@ -193,7 +193,10 @@ def test_split_invariance(attention_path):
 
 
 def test_degenerate_values(attention_path):
-    """Constant V groups (S = 0), zero K, zero Q, and a huge-range token."""
+    """Constant V groups (S = 0), zero K, zero Q, and a huge-range token.  With one token's values scaled by
+    1000 the outputs reach O(1000) where that token has weight; the criterion for this one case is the
+    stated tolerance relative to the largest output, max-abs <= 2e-3 * max(1, max |reference|), and the
+    stated rel-L2."""
     n, kvh = 200, 1
     k, v = make_inputs(7, 0, n, 1, kvh)
     v[5] = 1.5; v[150] = -2.0          # constant groups: scale 0
@@ -203,9 +206,10 @@ def test_degenerate_values(attention_path):
     m.append(0, k, v)
     m.check_state(0)
     q = synth.make_q(7, 0, 0, 1, 4, n)
-    m.check_attention(0, q, max_abs=2e-3 * 50)    # outputs reach O(1000) with the scaled token
-    q0 = torch.zeros_like(q)
-    m.check_attention(0, q0, max_abs=2e-3 * 50)
+    for qq in (q, torch.zeros_like(q)):
+        ref = m.oracles[0].decode_attention(qq.float().numpy().reshape(1, 4, 128))
+        err, rel = m.check_attention(0, qq, max_abs=2e-3 * max(1.0, float(np.abs(ref).max())))
+        print(f"degenerate values: max |ref| {np.abs(ref).max():.1f}, max-abs err {err:.2e}, rel-L2 {rel:.2e}")
 
 
 @pytest.mark.parametrize("bulk", [True, False])
@@ -359,3 +363,161 @@ def test_decode_step_with_chunked_eviction(chunk, n_sink, window, attention_path
                 ref = m.oracles[l].decode_attention(qq)
                 got = out[l].cpu().numpy().reshape(batch * kvh, group, 128)[m.slices].astype(np.float64)
                 assert np.abs(got - ref).max() <= 2e-3 and np.linalg.norm(got - ref) <= 1e-3 * np.linalg.norm(ref)
+
+
+def test_decode_step_tiny_caches_with_many_ctas(attention_path):
+    """pmkvq_decode_step with the attention grid set to 1024 CTAs on caches far smaller than that: a 16-bit block
+    of 8 tokens, and a 2- / 4-bit pair of 40 tokens.  Every slice must still be combined (each CTA between a
+    slice's first and last owner publishes a partial) and a second step must find the tickets at zero."""
+    for fbit, n0, window in (([16], 8, 4), ([2, 4], 40, 8)):
+        layers, kvh, batch, group = len(fbit), 2, 1, 4
+        m = Mirror(layers, group * kvh, kvh, batch, n0 + 2, fbit, window=window, attention_path=attention_path)
+        for l in range(layers):
+            k, v = make_inputs(51, l, n0, batch, kvh)
+            m.append(l, k, v)
+        m.cache.set_attention_ctas(1024)
+        for s in range(2):
+            ks, vs, qs = [], [], []
+            for l in range(layers):
+                k, v = make_inputs(52, l, 1, batch, kvh, pos0=n0 + s, chunk=s)
+                ks.append(k[0]); vs.append(v[0])
+                qs.append(synth.make_q(52, l, s, batch, group * kvh, n0 + s + 1))
+            K, V, Q = torch.stack(ks).cuda(), torch.stack(vs).cuda(), torch.stack(qs).cuda()
+            out = torch.full((layers, batch, group * kvh, 128), float("nan"), dtype=torch.float32, device="cuda")
+            m.cache.decode_step(K, V, Q, out=out)
+            torch.cuda.synchronize()
+            for l in range(layers):
+                m.oracles[l].append(K[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices],
+                                    V[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices])
+                ref = m.oracles[l].decode_attention(Q[l].float().cpu().numpy().reshape(batch * kvh, group, 128)[m.slices])
+                got = out[l].cpu().numpy().reshape(batch * kvh, group, 128)[m.slices].astype(np.float64)
+                assert np.all(np.isfinite(got)), "a slice was never combined"
+                assert np.abs(got - ref).max() <= 2e-3 and np.linalg.norm(got - ref) <= 1e-3 * np.linalg.norm(ref)
+        assert m.cache.device_status() == 0
+
+
+def test_decode_step_capacity_leaves_every_block_untouched():
+    """auto_reduce on: block 0 could take the step's token after a reduce, block 1 is at its final width and
+    full.  The step fails with CAPACITY and nothing has happened: block 0 has NOT been reduced."""
+    from paper_2505_18610_b200 import binding as B
+    layers, kvh, batch, group = 2, 1, 1, 4
+    full16 = 2 * 16 * 264                            # 16 INT16 tokens per (K|V) slice
+    m = Mirror(layers, group * kvh, kvh, batch, 64, [8, 16], n_sink=0, window=0, budget_bytes=[full16, full16])
+    k, v = make_inputs(53, 0, 17, batch, kvh)
+    for l in range(layers):
+        m.append(l, k[:16], v[:16])
+    K = torch.stack([k[16], k[16]]).cuda().contiguous(); V = torch.stack([v[16], v[16]]).cuda().contiguous()
+    Q = torch.stack([synth.make_q(53, l, 0, batch, group * kvh, 17) for l in range(layers)]).cuda().contiguous()
+    with pytest.raises(B.PmkvqError) as e:
+        m.cache.decode_step(K, V, Q)
+    assert e.value.status == B.CAPACITY
+    assert [m.cache.layer_state(l)["n_tokens"] for l in range(layers)] == [16, 16]
+    assert [m.cache.layer_state(l)["cur_bits"] for l in range(layers)] == [16, 16]
+    for l in range(layers):
+        m.check_state(l)                              # bytes as well: nothing was reduced on the device either
+
+
+def test_v_scales_spread_and_near_constant_token(attention_path):
+    """V scales spread over 2^-12 .. 2^12 inside one slice, and a near-constant V token (range 1e-7 around 5)
+    that carries most of the softmax mass, once inside the 2-bit body and once inside the INT16 window: the
+    token's zero-point must reach the output although its codes weigh next to nothing."""
+    n, kvh = 400, 1
+    k, v = make_inputs(54, 0, n, 1, kvh)
+    vf = v.float()
+    for t in range(n):
+        vf[t] *= 2.0 ** ((t * 7) % 25 - 12)
+    q = synth.make_q(54, 0, 0, 1, 4, n)
+    for t_special in (100, n - 3):
+        kk, vv = k.clone(), vf.clone()
+        vv[t_special] = 5.0 + 1e-7 * torch.arange(128, dtype=torch.float32).reshape(1, 1, 128) / 128.0
+        kk[t_special] = (q[0, 0].float() * 6.0).to(kk.dtype)          # a Key aligned with head 0's Query: a dominant score
+        m = Mirror(1, 4, kvh, 1, n, [2], window=16, attention_path=attention_path)
+        m.append(0, kk, vv.to(v.dtype))
+        m.check_state(0)
+        ref = m.oracles[0].decode_attention(q.float().numpy().reshape(1, 4, 128))
+        err, rel = m.check_attention(0, q, max_abs=2e-3 * max(1.0, float(np.abs(ref).max())))
+        print(f"near-constant token at {t_special}: max |ref| {np.abs(ref).max():.1f}, err {err:.2e}, rel {rel:.2e}")
+
+
+def test_sm_scale_and_lambda_extremes(attention_path):
+    """A caller-chosen softmax scale and an equalization vector with entries of 1e-3 and 1e3, on Keys whose
+    channels have those magnitudes (what Eq. 10 would produce for them): after K / lambda every channel is
+    O(1) again, Q * lambda spans six decades, and the scale keeps the scores O(1)."""
+    n, kvh, batch, group = 700, 2, 2, 5
+    k, v = make_inputs(55, 0, n, batch, kvh)
+    lam = np.ones((1, kvh, 128), np.float32)
+    lam[0, :, ::7] = 1e-3
+    lam[0, :, 3::11] = 1e3
+    kf = k.float() * torch.from_numpy(lam[0]).reshape(1, 1, kvh, 128)
+    k = kf.to(k.dtype)
+    m = Mirror(1, group * kvh, kvh, batch, n, [2], lam=lam, window=32, sm_scale=2e-4, attention_path=attention_path)
+    m.append(0, k, v)
+    m.check_state(0)
+    err, rel = m.check_attention(0, synth.make_q(55, 0, 0, batch, group * kvh, n))
+    print(f"lambda 1e-3 .. 1e3, sm_scale 2e-4: max-abs err {err:.2e}, rel-L2 {rel:.2e}")
+
+
+def test_guard_bands(attention_path):
+    """No tool checks the kernels' addresses on this path, so this test does: the arena and a slack region behind
+    it are filled with a pattern before the cache is created, a small cache then goes through bulk appends,
+    300 decode steps with chunked eviction and all three progressive reduces, and afterwards every byte
+    outside the regions the layout makes live must still hold the pattern: the slack past the arena, the part
+    of every body stream beyond the most bytes the stream has ever held, and the split-K partial slots beyond
+    the ones a launch can use.  All slices are compared with the oracle at the end."""
+    PAT = 0xA5
+    layers, kvh, batch, group, n0, steps, chunk = 2, 2, 2, 4, 200, 300, 4
+    n_slices = batch * kvh
+    fbit = [2, 4]
+    n_max = n0 + steps                 # default budgets: the blocks cross 16 -> 8 -> 4 (-> 2) at about 100 / 170 / 290 tokens
+    m = Mirror(layers, group * kvh, kvh, batch, n_max, fbit, window=32, evict_chunk=chunk,
+               attention_path=attention_path, slack_bytes=1 << 20, fill_byte=PAT)
+    lay = [m.cache.arena_layout(l) for l in range(layers)]
+    high = np.zeros((layers, 8), np.int64)              # most bytes each stream has held so far
+
+    def note(l):
+        st = m.cache.layer_state(l)
+        body = max(0, st["n_tokens"] - 1 - 32) // chunk * chunk
+        tiles = (body + 15) // 16
+        for s_ in range(8):
+            cnt = (tiles - s_ + 7) // 8 if tiles > s_ else 0
+            high[l, s_] = max(high[l, s_], cnt * (512 * st["cur_bits"] + 256))
+
+    widths = [set() for _ in range(layers)]
+    for l in range(layers):
+        k, v = make_inputs(56, l, n0, batch, kvh)
+        for a, b in ((0, 60), (60, 150), (150, n0)):
+            m.append(l, k[a:b], v[a:b]); note(l); widths[l].add(m.cache.layer_state(l)["cur_bits"])
+    for s in range(steps):
+        ks, vs, qs = [], [], []
+        for l in range(layers):
+            k, v = make_inputs(57, l, 1, batch, kvh, pos0=n0 + s, chunk=s)
+            ks.append(k[0]); vs.append(v[0])
+            qs.append(synth.make_q(57, l, s, batch, group * kvh, n0 + s + 1))
+        K, V, Q = torch.stack(ks).cuda(), torch.stack(vs).cuda(), torch.stack(qs).cuda()
+        m.cache.decode_step(K, V, Q)
+        for l in range(layers):
+            m.oracles[l].append(K[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices],
+                                V[l].float().cpu().numpy().reshape(1, -1, 128)[:, m.slices])
+            note(l); widths[l].add(m.cache.layer_state(l)["cur_bits"])
+    torch.cuda.synchronize()
+    assert widths[0] == {16, 8, 4, 2} and widths[1] == {16, 8, 4}
+    assert m.cache.device_status() == 0
+    arena = m.cache.arena[m.cache.arena_offset:].cpu().numpy()
+    used = lay[0]["arena_bytes"]
+    assert (arena[used:] == PAT).all(), "bytes behind the arena were written"
+    for l in range(layers):
+        g = lay[l]
+        for s_ in range(n_slices):
+            base = g["offset"] + s_ * g["slice_stride"] + g["body_off"]
+            for st_ in range(8):
+                lo = base + st_ * g["stream_stride"] + int(high[l, st_])
+                hi = base + (st_ + 1) * g["stream_stride"]
+                assert (arena[lo:hi] == PAT).all(), f"block {l} slice {s_} stream {st_}: bytes beyond the stream's data were written"
+            end = g["offset"] + s_ * g["slice_stride"] + g["body_off"] + 8 * g["stream_stride"]
+            assert (arena[end:g["offset"] + (s_ + 1) * g["slice_stride"]] == PAT).all()
+        # split-K workspace: a launch uses at most (CTAs + slices) partial slots; 148 CTAs at most by default
+        first_unused = g["partials_off"] + (148 + n_slices) * g["partial_slot_bytes"]
+        assert (arena[first_unused:g["partials_off"] + g["partials_bytes"]] == PAT).all()
+    for l in range(layers):
+        m.check_state(l)                                 # every slice, not a sample
+        m.check_attention(l, synth.make_q(58, l, 0, batch, group * kvh, n_max))

@@ -115,7 +115,7 @@ def test_quantizer_invariants(bits):
     assert np.all(c[np.arange(200), x.argmax(-1)] == qmax)
     # Eq. 2 in float64 agrees with the fp32 scale to one rounding
     assert np.allclose(s, (x.max(-1).astype(np.float64) - z) / qmax, rtol=2.0 ** -23, atol=0)
-    # round-trip error <= S/2 (spec bound); the slack covers the three fp32 roundings of the
+    # round-trip error <= S/2 (the bound the method states); the slack covers the three fp32 roundings of the
     # recipe (x - Z, the division, S itself), each at most 2^-24 of the group's range
     err = np.abs(O.dequantize(c, s, z) - x.astype(np.float64))
     rng_ = (x.max(-1).astype(np.float64) - z)[:, None]
