@@ -715,6 +715,79 @@ template <> __device__ __forceinline__ uint32_t merge_words<8, true>(uint32_t in
   return __byte_perm(__byte_perm(in0, in1, 0x0051), __byte_perm(in0, in1, 0x0073), 0x5410);  // the high byte of each code
 }
 
+// One lane-owned tile at 2B bits in a lane's registers: B 16-byte chunks per part, and the lane's 8 bytes of metadata.
+template <int B>
+struct TileRegs {
+  uint4 v[2][B];
+  float2 m;
+};
+template <int B>
+__device__ __forceinline__ void load_tile_regs(const uint8_t *in, int lane, TileRegs<B> &t) {
+#pragma unroll
+  for (int part = 0; part < 2; ++part)
+#pragma unroll
+    for (int q = 0; q < B; ++q) t.v[part][q] = *reinterpret_cast<const uint4 *>(in + part * code_part_bytes(2 * B) + (q * 32 + lane) * 16);
+  t.m = *reinterpret_cast<const float2 *>(in + meta_offset(2 * B) + lane * 8);
+}
+// Eq. 3 on the loaded tile and its stores at B bits.
+template <int B, bool SHR>
+__device__ __forceinline__ void finish_tile_regs(const TileRegs<B> &t, uint8_t *out, int lane, int variant) {
+  constexpr int OUT_WORDS = 2 * B;                      // words per lane per part at B bits
+  constexpr int OUT_CHUNKS = (OUT_WORDS + 3) / 4;
+#pragma unroll
+  for (int part = 0; part < 2; ++part) {
+    uint32_t w[B * 4], o[OUT_CHUNKS * 4];
+#pragma unroll
+    for (int q = 0; q < B; ++q) {
+      w[4 * q + 0] = t.v[part][q].x; w[4 * q + 1] = t.v[part][q].y; w[4 * q + 2] = t.v[part][q].z; w[4 * q + 3] = t.v[part][q].w;
+    }
+    // out lane-word r*B + w'  <-  in lane-words r*2B + 2w', r*2B + 2w' + 1
+#pragma unroll
+    for (int lw = 0; lw < OUT_WORDS; ++lw) {
+      const int r = lw / B, wp = lw % B;
+      o[lw] = merge_words<B, SHR>(w[r * 2 * B + 2 * wp], w[r * 2 * B + 2 * wp + 1]);
+    }
+    uint8_t *dst = out + part * code_part_bytes(B);
+    if constexpr (OUT_WORDS >= 4) {
+#pragma unroll
+      for (int q = 0; q < OUT_CHUNKS; ++q)
+        *reinterpret_cast<uint4 *>(dst + (q * 32 + lane) * 16) = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+    } else {
+      *reinterpret_cast<uint4 *>(dst + lane * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+  float2 m = t.m;
+  const int kind = ((2 * lane) & 15) >> 2;  // 0 S_K, 1 Z_K, 2 S_V, 3 Z_V
+  // a zero-point lane finds the scales of its two tokens two lanes below (16 bytes earlier)
+  const float s_x = __shfl_up_sync(0xffffffffu, m.x, 2), s_y = __shfl_up_sync(0xffffffffu, m.y, 2);
+  if ((kind & 1) == 0) {
+    float unused = 0.f;
+    halve_meta(m.x, unused, B, variant);
+    halve_meta(m.y, unused, B, variant);
+  } else if (variant == kShiftModified) {
+    float sx = s_x, sy = s_y;
+    halve_meta(sx, m.x, B, variant);
+    halve_meta(sy, m.y, B, variant);
+  }
+  *reinterpret_cast<float2 *>(out + meta_offset(B) + lane * 8) = m;
+}
+// The tiles lo + warp, lo + warp + n_warps, ... below hi of a wave, by one warp: the loads of a warp's next tile
+// are in flight while it works on the current one (every output of a wave lies below every input of the wave).
+template <int B, bool SHR>
+__device__ __forceinline__ void reduce_wave_tiles(uint8_t *base, int lo, int hi, int warp, int n_warps, int lane, int variant) {
+  int j = lo + warp;
+  if (j >= hi) return;
+  TileRegs<B> cur;
+  load_tile_regs<B>(base + (size_t)j * tile_bytes(2 * B), lane, cur);
+  for (; j < hi; j += n_warps) {
+    TileRegs<B> nxt;
+    const bool more = j + n_warps < hi;
+    if (more) load_tile_regs<B>(base + (size_t)(j + n_warps) * tile_bytes(2 * B), lane, nxt);
+    finish_tile_regs<B, SHR>(cur, base + (size_t)j * tile_bytes(B), lane, variant);
+    if (more) cur = nxt;
+  }
+}
+
 // CTA_WIDE: the warps of a CTA work on consecutive tiles at once; a CTA-wide barrier (reached by every
 // warp, `active` or not) separates all their loads from all their stores.
 template <int B, bool SHR>
@@ -905,8 +978,8 @@ __device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *o
 // behind the earlier waves' loads.  The waves grow geometrically (x 1.8 - 1.9).
 // Warps per CTA: enough tiles in flight per stream to cover the memory latency, and few enough registers
 // that every (stream, slice) CTA of the common shapes is resident at once.
-template <int B> __host__ __device__ constexpr int reduce_warps() { return B == 2 ? 16 : 8; }
-template <int B> __host__ __device__ constexpr int reduce_min_ctas() { return B == 2 ? 3 : 4; }
+template <int B> __host__ __device__ constexpr int reduce_warps() { return 8; }
+template <int B> __host__ __device__ constexpr int reduce_min_ctas() { return 4; }
 template <int B>
 __device__ __forceinline__ void reduce_one_tile(const LayerGeom &geom, const uint8_t *in, uint8_t *out, int lane, bool active,
                                                 bool cta_wide, uint8_t *scratch) {
@@ -935,8 +1008,13 @@ __global__ void __launch_bounds__(reduce_warps<B>() * 32, reduce_min_ctas<B>()) 
   for (int lo = kReduceWarps; lo < cnt;) {
     const int hi = min(cnt, (int)((long long)lo * tile_bytes(2 * B) / tile_bytes(B)));
     __syncthreads();  // the stores of this wave may land on inputs of the tiles before it
-    for (int j = lo + warp; j < hi; j += kReduceWarps)
-      reduce_one_tile<B>(geom, base + (size_t)j * tile_bytes(2 * B), base + (size_t)j * tile_bytes(B), lane, true, false, scratch);
+    if (B == 2 && !geom.rows) {  // few registers per tile at this width: a warp keeps its next tile's loads in flight
+      if (geom.shift_variant == kShiftEquivalent) reduce_wave_tiles<B, false>(base, lo, hi, warp, kReduceWarps, lane, geom.shift_variant);
+      else reduce_wave_tiles<B, true>(base, lo, hi, warp, kReduceWarps, lane, geom.shift_variant);
+    } else {
+      for (int j = lo + warp; j < hi; j += kReduceWarps)
+        reduce_one_tile<B>(geom, base + (size_t)j * tile_bytes(2 * B), base + (size_t)j * tile_bytes(B), lane, true, false, scratch);
+    }
     lo = hi;
   }
 }
