@@ -209,10 +209,11 @@ def time_attention_all(cache, q, out, launches, warm=3):
     return [a.elapsed_time(b) for a, b in evs]
 
 
-def width_leg(wl, device, peak, blocks=8, launches=12):
-    """Steady-state attention at one width: caches of `blocks` blocks of the workload's per-block shape whose
-    whole body sits at 2 / 4 / 8 / 16 bit, timed with one all-blocks attention launch per event pair."""
+def width_leg(wl, device, peak, blocks=None, launches=12):
+    """Steady-state attention at one width: caches of the workload's shape (all its blocks) whose whole body
+    sits at 2 / 4 / 8 / 16 bit, timed with one all-blocks attention launch per event pair."""
     out = {}
+    blocks = blocks or wl["layers"]
     sub = dict(wl, layers=blocks)
     for path, pname in ((0, "warp_mma"), (1, "tensor_memory")):
         for bits in (2, 4, 8, 16):

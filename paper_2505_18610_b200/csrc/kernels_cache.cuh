@@ -350,20 +350,36 @@ __device__ __forceinline__ void store_words(uint8_t *part, int r, int lane, cons
   }
 }
 
+constexpr int kStageRowBytes = 272;  // a staged bf16 row of 128 channels plus 16 bytes: the owner-mapped reads below hit 32 different banks
 template <int BITS>
 __device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ src, size_t row_stride,
                                                  const float *__restrict__ il, uint8_t *dst_tile, int is_value,
-                                                 unsigned *vmax_slot, int lane, int variant) {
+                                                 unsigned *vmax_slot, int lane, int variant, uint8_t *stage) {
   const int g = lane >> 2, tig = lane & 3;
   uint32_t words[BITS];
+  // the tile's 16 rows of 256 bytes come in with eight coalesced 16-byte loads per lane, all in flight at once
+  {
+    uint4 v[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const int id = lane + 32 * c;
+      v[c] = *reinterpret_cast<const uint4 *>(src + (size_t)(id >> 4) * row_stride + (id & 15) * 8);
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const int id = lane + 32 * c;
+      *reinterpret_cast<uint4 *>(stage + (id >> 4) * kStageRowBytes + (id & 15) * 16) = v[c];
+    }
+    __syncwarp();
+  }
   if (!is_value) {
 #pragma unroll 1
     for (int r = 0; r < 2; ++r) {  // token g + 8 r
       float x[32];                 // [2 W + h]
-      const uint16_t *row = src + (size_t)(g + 8 * r) * row_stride + 2 * tig;
+      const uint8_t *row = stage + (g + 8 * r) * kStageRowBytes + 4 * tig;
 #pragma unroll
       for (int W = 0; W < 16; ++W) {
-        const uint32_t raw = *reinterpret_cast<const uint32_t *>(row + 8 * W);
+        const uint32_t raw = *reinterpret_cast<const uint32_t *>(row + 16 * W);
         const float2 l2 = __ldg(reinterpret_cast<const float2 *>(il + 8 * W + 2 * tig));  // Lambda^-1, L1-resident
         x[2 * W] = __fmul_rn(__uint_as_float(raw << 16), l2.x);
         x[2 * W + 1] = __fmul_rn(__uint_as_float(raw & 0xFFFF0000u), l2.y);
@@ -391,11 +407,12 @@ __device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ sr
 #pragma unroll 1
     for (int r = 0; r < 2; ++r) {  // tokens 2 tig + 8 r + h, h = 0, 1
       float x[2][16];              // [h][J]
-      const uint16_t *row = src + (size_t)(2 * tig + 8 * r) * row_stride + g;
+      const uint8_t *row = stage + (2 * tig + 8 * r) * kStageRowBytes + 2 * g;
 #pragma unroll
       for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int J = 0; J < 16; ++J) x[h][J] = __uint_as_float((uint32_t)row[h * row_stride + 8 * J] << 16);
+        for (int J = 0; J < 16; ++J)
+          x[h][J] = __uint_as_float((uint32_t)*reinterpret_cast<const uint16_t *>(row + h * kStageRowBytes + 16 * J) << 16);
       float S[2], Z[2];
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
@@ -527,7 +544,7 @@ __global__ void __launch_bounds__(128, 8) append_tiles_kernel(const uint16_t *__
                                                            const float *__restrict__ inv_lambda, unsigned *vmax_bits,
                                                            LayerGeom geom, int n_slices, int kv_heads, int n_old,
                                                            int tile_lo, int n_tiles, int bits) {
-  __shared__ __align__(16) uint8_t s_scratch[4][kTileTokens * kHeadDim];
+  __shared__ __align__(16) uint8_t s_scratch[4][kTileTokens * kStageRowBytes];  // the warp's staged input rows, or its code bytes (row tiles)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wid = (long long)blockIdx.x * 4 + warp;
   if (wid >= (long long)n_tiles * n_slices * 2) return;
@@ -540,15 +557,15 @@ __global__ void __launch_bounds__(128, 8) append_tiles_kernel(const uint16_t *__
   const float *il = inv_lambda + (size_t)(slice % kv_heads) * kHeadDim;
   uint8_t *dst_tile = geom.base + (size_t)slice * geom.slice_stride + geom.body_off + body_tile_offset(tile, bits, geom.stream_stride);
   switch (bits) {
-    case 16: append_tile_half<16>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
-    case 8: append_tile_half<8>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant); break;
+    case 16: append_tile_half<16>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]); break;
+    case 8: append_tile_half<8>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]); break;
     case 4:
       if (geom.rows) append_tile_half_row<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]);
-      else append_tile_half<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant);
+      else append_tile_half<4>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]);
       break;
     default:
       if (geom.rows) append_tile_half_row<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]);
-      else append_tile_half<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant);
+      else append_tile_half<2>(src, row_stride, il, dst_tile, is_value, vmax_bits + slice, lane, geom.shift_variant, s_scratch[warp]);
       break;
   }
 }
