@@ -489,6 +489,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-widths", action="store_true", help="skip the per-width steady-state records")
     ap.add_argument("--no-others", action="store_true", help="skip the compact 8B / 32B / 70B records")
+    ap.add_argument("--only", default="", choices=["", "reduce", "append"],
+                    help="profiling runs: only the progressive-reduce events or only the bulk append of the aux leg")
     ap.add_argument("--attention-only", type=int, default=0,
                     help="profiling runs: build the cache at its final widths and launch the attention this many times")
     args = ap.parse_args()
@@ -537,6 +539,18 @@ def main():
     L = wl["layers"]
     out_dev = torch.empty(L, wl["batch"], wl["q_heads"], 128, dtype=torch.float32, device=device)
 
+    if args.only == "reduce":
+        print(json.dumps({"only": "reduce", "workload": wl["name"], "reduce": reduce_leg(wl, device, peak, repeats=1)}))
+        return
+    if args.only == "append":
+        from paper_2505_18610_b200 import binding as B
+        k, v = synth.make_kv(3, 0, 0, 8192, wl["batch"], wl["kv_heads"], 0, wl["n_outlier"], wl["factor"], device=device)
+        k, v = k.contiguous(), v.contiguous()
+        for _ in range(3):
+            c = B.Cache(1, wl["q_heads"], wl["kv_heads"], wl["batch"], 32768, [16], n_sink=N_SINK, window=WINDOW, device=device)
+            c.append(0, k, v); torch.cuda.synchronize(); c.close()
+        print(json.dumps({"only": "append", "workload": wl["name"], "tokens": 8192}))
+        return
     if args.attention_only:      # profiling runs: the steady-state attention launch and nothing else
         cache = build_cache(wl, fbit, None, lam, wl["end_tokens"], device, shared_chunks=True, attention_path=args.attention_path)
         q = torch.stack([synth.make_q(2, l, 0, wl["batch"], wl["q_heads"], wl["end_tokens"], device=device) for l in range(L)]).contiguous()

@@ -154,6 +154,12 @@ pmkvq_status pmkvq_decode_attention_all(pmkvq_cache *cache, const void *d_Q_bf16
  * NULL) receives the word.  The word is never cleared: create a new cache after a failure. */
 pmkvq_status pmkvq_device_status(pmkvq_cache *cache, uint32_t *h_wait_bits);
 
+/* Self-test of the bounded waits: launches one thread that waits on a barrier nothing will ever complete, with a
+ * limit of 1024 polls.  The wait must give up, set *h_gave_up to 1 and let the kernel end normally; the CUDA
+ * context stays usable (the attention kernels use the same wait with a limit of 2^20 polls and report through
+ * pmkvq_device_status).  Synchronises `stream`. */
+pmkvq_status pmkvq_selftest_bounded_wait(pmkvq_cache *cache, void *stream, uint32_t *h_gave_up);
+
 /* Checkpoint / restore of a block's host-side state.  The device-side state of a cache is the arena; a
  * caller that saved a copy of the arena together with pmkvq_layer_state()'s (n_tokens, cur_bits) of every
  * block puts the bytes back and then calls this for every block.  INVALID_ARG if the pair cannot be a state

@@ -66,6 +66,8 @@ def load_library() -> ctypes.CDLL:
     lib.pmkvq_decode_attention_all.argtypes = [vp, vp, vp, vp]
     lib.pmkvq_device_status.restype = i32
     lib.pmkvq_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.pmkvq_selftest_bounded_wait.restype = i32
+    lib.pmkvq_selftest_bounded_wait.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.pmkvq_restore_layer_state.restype = i32
     lib.pmkvq_restore_layer_state.argtypes = [vp, i32, i32, i32]
     lib.pmkvq_arena_layout.restype = i32
@@ -311,6 +313,14 @@ class Cache:
         if check and st != OK:
             raise PmkvqError(st, f"pmkvq_device_status (bits {word.value:#x})")
         return int(word.value)
+
+    def selftest_bounded_wait(self, stream=None) -> int:
+        """1 if the deliberately unsatisfiable wait gave up as designed."""
+        got = ctypes.c_uint32()
+        st = lib().pmkvq_selftest_bounded_wait(self._h, _stream_ptr(stream), ctypes.byref(got))
+        if st != OK:
+            raise PmkvqError(st, "pmkvq_selftest_bounded_wait")
+        return int(got.value)
 
     def restore_layer_state(self, layer: int, n_tokens: int, cur_bits: int):
         st = lib().pmkvq_restore_layer_state(self._h, layer, int(n_tokens), int(cur_bits))

@@ -102,6 +102,16 @@ __device__ __forceinline__ void tc_wait(TcCtx &tc, const unsigned long long *bar
     atomicOr(tc.error_word, code);
   }
 }
+// A wait that nothing will ever satisfy, with a short limit: shows that a bounded wait gives up, reports it
+// and lets the kernel end normally (the context stays usable).  One thread.
+__global__ void bounded_wait_selftest_kernel(unsigned *word, unsigned limit) {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t b = tc05::smem_u32(&bar);
+  tc05::mbar_init(b, 1);
+  tc05::mbar_init_fence();
+  if (!tc05::mbar_wait(b, 0u, limit)) atomicOr(word, 1u);
+}
+
 // one arrival per warp, after all its lanes are done
 __device__ __forceinline__ void warp_arrive(const unsigned long long *bar, int lane) {
   __syncwarp();

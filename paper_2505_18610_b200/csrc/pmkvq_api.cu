@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <limits>
+#include <memory>
 #include <new>
 #include <vector>
 
@@ -264,20 +265,22 @@ extern "C" {
 
 size_t pmkvq_arena_bytes_required(const pmkvq_config *cfg) {
   if (!check_config(cfg)) return 0;
-  pmkvq_cache tmp{};
-  return plan(tmp, cfg);
+  try {
+    pmkvq_cache tmp{};
+    return plan(tmp, cfg);
+  } catch (...) {
+    return 0;
+  }
 }
 
-pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
+static pmkvq_status cache_create_impl(const pmkvq_config *cfg, pmkvq_cache **out) {
   if (!out || !check_config(cfg) || !cfg->d_arena) return PMKVQ_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(cfg->d_arena) % kAlign) return PMKVQ_ERR_INVALID_ARG;
-  pmkvq_cache *k = new (std::nothrow) pmkvq_cache{};
+  std::unique_ptr<pmkvq_cache> owner(new (std::nothrow) pmkvq_cache{});  // released to the caller on success only
+  pmkvq_cache *k = owner.get();
   if (!k) return PMKVQ_ERR_STATE;
   const size_t need = plan(*k, cfg);
-  if (cfg->arena_bytes < need) {
-    delete k;
-    return PMKVQ_ERR_ARENA_TOO_SMALL;
-  }
+  if (cfg->arena_bytes < need) return PMKVQ_ERR_ARENA_TOO_SMALL;
   k->arena = static_cast<uint8_t *>(cfg->d_arena);
   k->arena_bytes = cfg->arena_bytes;
   const size_t n_lam = (size_t)k->layers * k->kv_heads * kHeadDim;
@@ -300,12 +303,17 @@ pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
     e = cudaMemcpy(k->arena + k->off_geoms, geoms.data(), geoms.size() * sizeof(LayerGeom), cudaMemcpyHostToDevice);
   }
   if (e == cudaSuccess) e = attention_setup(k);
-  if (e != cudaSuccess) {
-    delete k;
-    return PMKVQ_ERR_CUDA;
-  }
-  *out = k;
+  if (e != cudaSuccess) return PMKVQ_ERR_CUDA;
+  *out = owner.release();
   return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_cache_create(const pmkvq_config *cfg, pmkvq_cache **out) {
+  try {
+    return cache_create_impl(cfg, out);
+  } catch (...) {
+    return PMKVQ_ERR_STATE;
+  }
 }
 
 void pmkvq_cache_destroy(pmkvq_cache *cache) { delete cache; }
@@ -636,6 +644,21 @@ pmkvq_status pmkvq_device_status(pmkvq_cache *k, uint32_t *h_wait_bits) {
   return word ? PMKVQ_ERR_DEVICE_WAIT : PMKVQ_OK;
 }
 
+pmkvq_status pmkvq_selftest_bounded_wait(pmkvq_cache *k, void *stream, uint32_t *h_gave_up) {
+  if (!k || !h_gave_up) return PMKVQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned *word = reinterpret_cast<unsigned *>(k->arena + k->off_error) + 1;  // beside the error word, never read by it
+  if (cudaMemsetAsync(word, 0, sizeof(unsigned), st) != cudaSuccess) return PMKVQ_ERR_CUDA;
+  bounded_wait_selftest_kernel<<<1, 1, 0, st>>>(word, 1u << 10);
+  ++k->launches;
+  unsigned got = 0;
+  if (cudaGetLastError() != cudaSuccess || cudaMemcpyAsync(&got, word, sizeof(got), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return PMKVQ_ERR_CUDA;
+  *h_gave_up = got;
+  return PMKVQ_OK;
+}
+
 pmkvq_status pmkvq_restore_layer_state(pmkvq_cache *k, int32_t layer, int32_t n_tokens, int32_t cur_bits) {
   if (!k || layer < 0 || layer >= k->layers || n_tokens < 0 || n_tokens > k->max_tokens || !valid_bits(cur_bits))
     return PMKVQ_ERR_INVALID_ARG;
@@ -688,8 +711,8 @@ uint64_t pmkvq_attention_bytes(const pmkvq_cache *k, int32_t layer) {
   return kv + qo + (uint64_t)k->kv_heads * kHeadDim * 4;
 }
 
-pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx, int32_t kv_head, int32_t is_value,
-                                uint16_t *h_codes, float *h_scale, float *h_zero, uint8_t *h_bits, uint8_t *h_packed) {
+static pmkvq_status export_slice_impl(pmkvq_cache *k, int32_t layer, int32_t batch_idx, int32_t kv_head, int32_t is_value,
+                                      uint16_t *h_codes, float *h_scale, float *h_zero, uint8_t *h_bits, uint8_t *h_packed) {
   if (!k || layer < 0 || layer >= k->layers || batch_idx < 0 || batch_idx >= k->batch || kv_head < 0 ||
       kv_head >= k->kv_heads)
     return PMKVQ_ERR_INVALID_ARG;
@@ -739,6 +762,15 @@ pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx
     packed_off += 16 * bits;
   }
   return PMKVQ_OK;
+}
+
+pmkvq_status pmkvq_export_slice(pmkvq_cache *k, int32_t layer, int32_t batch_idx, int32_t kv_head, int32_t is_value,
+                                uint16_t *h_codes, float *h_scale, float *h_zero, uint8_t *h_bits, uint8_t *h_packed) {
+  try {
+    return export_slice_impl(k, layer, batch_idx, kv_head, is_value, h_codes, h_scale, h_zero, h_bits, h_packed);
+  } catch (...) {
+    return PMKVQ_ERR_STATE;
+  }
 }
 
 pmkvq_status pmkvq_set_attention_ctas(pmkvq_cache *k, int32_t n_ctas) {
@@ -853,8 +885,8 @@ pmkvq_status pmkvq_alpha_grid_search(const void *d_K, const void *d_Q, const voi
   return PMKVQ_OK;
 }
 
-pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_t *h_widths, const double *h_sens,
-                                 const uint64_t *h_mem, uint64_t budget, uint8_t *h_fbit_out, double *h_cost_out) {
+static pmkvq_status allocate_bits_impl(int32_t layers, int32_t n_choices, const uint8_t *h_widths, const double *h_sens,
+                                       const uint64_t *h_mem, uint64_t budget, uint8_t *h_fbit_out, double *h_cost_out) {
   if (layers <= 0 || n_choices <= 0 || n_choices > 8 || !h_widths || !h_sens || !h_mem || !h_fbit_out)
     return PMKVQ_ERR_INVALID_ARG;
   for (int i = 0; i < layers * n_choices; ++i)
@@ -881,7 +913,7 @@ pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_
     max_extra += m;
   }
   const uint64_t cap = std::min((budget - floor_sum) / g, max_extra);
-  if ((cap + 1) * (uint64_t)layers > (1ull << 26)) return PMKVQ_ERR_INVALID_ARG;
+  if (cap >= (1ull << 26) / (uint64_t)layers) return PMKVQ_ERR_INVALID_ARG;  // table of (cap + 1) * layers cells
   const size_t W = (size_t)cap + 1;
   const double inf = std::numeric_limits<double>::infinity();
   // best[i][w]: minimal sensitivity of blocks 0..i-1 using exactly w units; pick[i][w]: choice of block i-1
@@ -913,6 +945,16 @@ pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_
     w -= (size_t)(extra[(size_t)i * n_choices + c] / g);
   }
   return PMKVQ_OK;
+}
+
+// host allocations (std::vector) must not throw across the C boundary
+pmkvq_status pmkvq_allocate_bits(int32_t layers, int32_t n_choices, const uint8_t *h_widths, const double *h_sens,
+                                 const uint64_t *h_mem, uint64_t budget, uint8_t *h_fbit_out, double *h_cost_out) {
+  try {
+    return allocate_bits_impl(layers, n_choices, h_widths, h_sens, h_mem, budget, h_fbit_out, h_cost_out);
+  } catch (...) {
+    return PMKVQ_ERR_STATE;
+  }
 }
 
 const char *pmkvq_status_string(pmkvq_status s) {

@@ -521,3 +521,29 @@ def test_guard_bands(attention_path):
     for l in range(layers):
         m.check_state(l)                                 # every slice, not a sample
         m.check_attention(l, synth.make_q(58, l, 0, batch, group * kvh, n_max))
+
+
+def test_bounded_wait_gives_up_and_the_context_lives():
+    """A barrier wait that nothing can satisfy runs out after its poll limit, the kernel reports it and ends;
+    afterwards the same cache still computes attention, and its error word (the attention kernels' own waits)
+    is clean.  Also: a checkpoint of the arena plus pmkvq_restore_layer_state brings a cache back."""
+    from paper_2505_18610_b200 import binding as B
+    kvh, batch, group, n = 2, 1, 4, 600
+    k, v = make_inputs(61, 0, n, batch, kvh)
+    m = Mirror(1, group * kvh, kvh, batch, n + 8, [2], window=16, attention_path=1)
+    m.append(0, k, v)
+    assert m.cache.selftest_bounded_wait() == 1
+    q = synth.make_q(61, 0, 0, batch, group * kvh, n)
+    m.check_attention(0, q)
+    assert m.cache.device_status() == 0
+    # checkpoint, move on, restore
+    snap, st0 = m.cache.arena.clone(), m.cache.layer_state(0)
+    before = m.cache.decode_attention(0, q.cuda()).clone()
+    k2, v2 = make_inputs(62, 0, 8, batch, kvh, pos0=n)
+    m.cache.append(0, k2.cuda().contiguous(), v2.cuda().contiguous())
+    m.cache.arena.copy_(snap)
+    m.cache.restore_layer_state(0, st0["n_tokens"], st0["cur_bits"])
+    assert m.cache.layer_state(0) == st0
+    assert torch.equal(m.cache.decode_attention(0, q.cuda()), before)
+    with pytest.raises(B.PmkvqError):
+        m.cache.restore_layer_state(0, 5, 1)        # not a width
