@@ -699,24 +699,32 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
   // ---- body stream set-up: claim the first steps and start their copies before anything else ----
   constexpr int TB = tile_bytes(BITS);
   constexpr int NT = F::NT, S = F::SLOTS > 0 ? F::SLOTS : 1, SB = NT * TB;
-  const int n_steps = (t_hi - t_lo + NT - 1) / NT;
   const uint8_t *body = slice_base + p.geom.body_off;
   const size_t stream_stride = p.geom.stream_stride;
+  // A step is NT tiles.  With NT = 2 these are the tiles 16 G + s and 16 G + 8 + s: neighbours in stream s, one
+  // contiguous run of 2 TB bytes (attention does not care about the order of the tokens).  The first and
+  // the last group of 16 tiles of a segment may reach beyond [t_lo, t_hi): such tiles are left out.
+  const int g_lo = t_lo >> 4;
+  const int n_steps = t_hi <= t_lo ? 0 : (NT == 2 ? 8 * (((t_hi - 1) >> 4) - g_lo + 1) : t_hi - t_lo);
+  auto step_tile = [&](int j, int k) { return NT == 2 ? 16 * (g_lo + (j >> 3)) + (j & 7) + 8 * k : t_lo + j; };
+  auto live = [&](int t) { return t >= t_lo && t < t_hi; };
   uint8_t *my_ring = ring + (size_t)warp * S * SB;
   const uint32_t ring_addr = (uint32_t)__cvta_generic_to_shared(my_ring);
   auto claim = [&](int which) { return claim_next(s_ctr + which, lane); };
-  // step j = tiles t_lo + NT j .. + NT - 1 (consecutive tiles sit in consecutive streams); 16-byte chunk
-  // c of the step belongs to tile c / (TB / 16)
   auto issue = [&](int j, int slot) {
-    const int t0 = t_lo + NT * j;
     constexpr int CPT = TB / 16;  // 16-byte chunks per tile: lane l copies chunks l, l + 32, ...
+    const int ta = step_tile(j, 0);
+    const uint8_t *src = body + body_tile_offset(ta, BITS, stream_stride) + lane * 16;
+    const uint32_t dst = ring_addr + slot * SB + lane * 16;
+    if (NT == 2 && (NT * CPT) % 32 == 0 && live(ta) && live(ta + 8)) {  // the whole step, every lane the same number of chunks
+      cp_async_run<NT * CPT / 32>(dst, src);
+    } else {
 #pragma unroll
-    for (int k = 0; k < NT; ++k) {
-      if (t0 + k < t_hi) {
-        const uint8_t *src = body + body_tile_offset(t0 + k, BITS, stream_stride) + lane * 16;
-        const uint32_t dst = ring_addr + slot * SB + k * TB + lane * 16;
-        cp_async_run<CPT / 32>(dst, src);
-        if (CPT % 32 != 0 && lane < CPT % 32) cp_async16_at<(CPT / 32) * 512>(dst, src);
+      for (int k = 0; k < NT; ++k) {
+        if (live(step_tile(j, k))) {
+          cp_async_run<CPT / 32>(dst + k * TB, src + k * TB);
+          if (CPT % 32 != 0 && lane < CPT % 32) cp_async16_at<(CPT / 32) * 512>(dst + k * TB, src + k * TB);
+        }
       }
     }
   };
@@ -784,14 +792,15 @@ __device__ __forceinline__ void run_segment(const AttnParams &p, int slice, long
         cp_async_wait<S - 1>();
         __syncwarp();
         const uint8_t *tile = my_ring + slot * SB;
-        const int t = t_lo + NT * pending[0];
-        if (NT == 2 && t + 1 < t_hi && t + 1 != tail_tile) {
+        const int t = step_tile(pending[0], 0);
+        if (NT == 2 && live(t) && live(t + 8) && t != tail_tile && t + 8 != tail_tile) {
           process_tiles<BITS, NT, false>(tile, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
         } else {
 #pragma unroll
           for (int k = 0; k < NT; ++k) {
-            if (t + k >= t_hi) break;
-            if (t + k == tail_tile)
+            const int tk = step_tile(pending[0], k);
+            if (!live(tk)) continue;
+            if (tk == tail_tile)
               process_tiles<BITS, 1, true>(tile + k * TB, tail_mask, st, qa, mu, sumq, inv_sigma_e, lane);
             else
               process_tiles<BITS, 1, false>(tile + k * TB, 0xFFFFu, st, qa, mu, sumq, inv_sigma_e, lane);
