@@ -237,6 +237,19 @@ def width_leg(wl, device, peak, blocks=None, launches=12):
     return out
 
 
+def busy_wait_warm(device, ms=30.0):
+    """Keep the GPU busy for about `ms` with plain copies (1 GiB each, larger than L2) and return with the queue
+    still holding the last of them, so that what is timed next starts on a GPU at its working clocks."""
+    global _WARM
+    if _WARM is None or _WARM[0].device != torch.device(device):
+        _WARM = (torch.empty(1 << 28, dtype=torch.float32, device=device), torch.empty(1 << 28, dtype=torch.float32, device=device))
+    for _ in range(max(1, int(ms / 0.35))):
+        _WARM[1].copy_(_WARM[0])
+
+
+_WARM = None
+
+
 def reduce_leg(wl, device, peak, repeats=3):
     """One progressive-reduce event of each width at the workload's per-block shape, timed alone: a one-block
     cache is filled at 16 bit to the full context and reduced 16 -> 8 -> 4 -> 2 by hand.  Bytes per event are
@@ -260,7 +273,7 @@ def reduce_leg(wl, device, peak, repeats=3):
         for b in (8, 4, 2):
             l0 = cache.launch_count()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
+            busy_wait_warm(device)           # an event fires between decode steps, on a GPU that is busy
             e0.record(); cache.progressive_reduce(0); e1.record()
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1)
@@ -292,7 +305,7 @@ def aux_leg(wl, device, peak):
     for _ in range(6):
         cache = B.Cache(1, wl["q_heads"], wl["kv_heads"], wl["batch"], 32768, [16], n_sink=N_SINK, window=WINDOW, device=device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
+        busy_wait_warm(device)
         e0.record(); cache.append(0, k, v); e1.record()
         torch.cuda.synchronize()
         ts.append(e0.elapsed_time(e1))
@@ -376,6 +389,12 @@ class ClockSampler:
                                       stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
+
+    def wait_first(self, timeout=5.0):
+        """Block until the sampler has written its first line (nvidia-smi takes a moment to start)."""
+        t0 = time.time()
+        while self.p is not None and time.time() - t0 < timeout and os.path.getsize(self.f.name) == 0:
+            time.sleep(0.01)
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -573,11 +592,15 @@ def main():
         snapshot = cache.arena.clone()
 
     # ---------------- device-resident leg: `value` (the trajectory: appends, evictions, every block's last reduce) ----------------
+    # the clock sampler runs from the warm-up steps to the end of the end-to-end leg (the GPU is under this
+    # workload's load the whole time); the timed region starts once it has delivered its first sample
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     run_steps(cache, wl, pool, warmup, 0, out_dev)
     bits_before = [cache.layer_state(l)["cur_bits"] for l in range(L)]
+    if sampler:
+        sampler.wait_first()
     barrier()
     launches0 = cache.launch_count()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     total_bytes = 0
     ev0.record()
@@ -598,7 +621,6 @@ def main():
     attn_ms = float(np.sum(ts))
     attn_bytes = sum(cache.attention_bytes(l) for l in range(L))
     widths_now = {str(b): sum(1 for l in range(L) if cache.layer_state(l)["cur_bits"] == b) for b in (2, 4, 8, 16)}
-    clocks = sampler.stop() if sampler else None
     cache.device_status()
 
     # ---------------- end-to-end leg: the same trajectory with host buffers in, host buffers out ----------------
@@ -631,6 +653,7 @@ def main():
         e2e_ms = e0.elapsed_time(e1)
         h2d = (dk.numel() + dv.numel() + dq.numel()) * 2
         d2h = do.numel() * 4
+    clocks = sampler.stop() if sampler else None
     cache.close(); del cache
     torch.cuda.empty_cache()
 

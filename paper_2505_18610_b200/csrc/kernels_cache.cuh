@@ -305,10 +305,28 @@ template <int BITS, int N>
 __device__ __forceinline__ float quantize_owned(float (&x)[N], float mn, float mx, int variant) {
   const float scale = __fdiv_rn(__fsub_rn(mx, mn), 65535.0f);
   if (scale >= 0x1p-60f && scale <= 0x1p60f) {  // one scale per token: the branch is uniform in the warp
+    // two values per instruction (packed fp32 pairs, each component rounded to nearest like the scalar form):
+    // x - mn as x + (-mn), the residual d - q s as q (-s) + d
+    static_assert(N % 2 == 0, "values are taken in pairs");
     const float y = __frcp_rn(scale);
+    const float2 y2 = make_float2(y, y), ns2 = make_float2(-scale, -scale), nmn2 = make_float2(-mn, -mn);
 #pragma unroll
-    for (int i = 0; i < N; ++i)
-      x[i] = __uint_as_float(shift_chain((uint32_t)code_of_quotient(quotient_rn(__fsub_rn(x[i], mn), scale, y)), BITS, variant));
+    for (int i = 0; i < N; i += 2) {
+      const float2 d = __fadd2_rn(make_float2(x[i], x[i + 1]), nmn2);
+      float2 q = __fmul2_rn(d, y2);
+      float2 r = __ffma2_rn(q, ns2, d);
+      q = __ffma2_rn(r, y2, q);
+      r = __ffma2_rn(q, ns2, d);
+      q = __ffma2_rn(r, y2, q);
+      const float2 c = __fadd2_rn(q, make_float2(8388608.0f, 8388608.0f));  // code_of_quotient, both at once
+      if constexpr (BITS == 16) {  // the code is the low half of the sum's bit pattern; the packing keeps only that
+        x[i] = c.x;
+        x[i + 1] = c.y;
+      } else {
+        x[i] = __uint_as_float(shift_chain((uint32_t)(__float_as_int(c.x) - 0x4B000000), BITS, variant));
+        x[i + 1] = __uint_as_float(shift_chain((uint32_t)(__float_as_int(c.y) - 0x4B000000), BITS, variant));
+      }
+    }
   } else {  // constant tokens (0 / 0 converts to code 0) and scales far outside any real tensor's range
 #pragma unroll
     for (int i = 0; i < N; ++i) {
@@ -325,6 +343,11 @@ __device__ __forceinline__ float quantize_owned(float (&x)[N], float mn, float m
 template <int BITS>
 __device__ __forceinline__ void pack_words(const float *lo, const float *hi, int step, uint32_t *words) {
   constexpr int n = 16 / BITS;
+  if constexpr (BITS == 16) {  // one code per half; only the low 16 bits of a pattern are the code
+#pragma unroll
+    for (int w = 0; w < 16; ++w) words[w] = __byte_perm(__float_as_uint(lo[w * step]), __float_as_uint(hi[w * step]), 0x5410);
+    return;
+  }
 #pragma unroll
   for (int w = 0; w < BITS; ++w) {
     uint32_t a = 0, b = 0;
@@ -381,8 +404,9 @@ __device__ __forceinline__ void append_tile_half(const uint16_t *__restrict__ sr
       for (int W = 0; W < 16; ++W) {
         const uint32_t raw = *reinterpret_cast<const uint32_t *>(row + 16 * W);
         const float2 l2 = __ldg(reinterpret_cast<const float2 *>(il + 8 * W + 2 * tig));  // Lambda^-1, L1-resident
-        x[2 * W] = __fmul_rn(__uint_as_float(raw << 16), l2.x);
-        x[2 * W + 1] = __fmul_rn(__uint_as_float(raw & 0xFFFF0000u), l2.y);
+        const float2 xl = __fmul2_rn(make_float2(__uint_as_float(raw << 16), __uint_as_float(raw & 0xFFFF0000u)), l2);
+        x[2 * W] = xl.x;
+        x[2 * W + 1] = xl.y;
       }
       float mn = x[0], mx = x[0];
 #pragma unroll
@@ -718,7 +742,24 @@ __device__ __forceinline__ uint32_t halve_bytes(uint32_t x) {  // 4 codes of 8 b
   }
   return ya | (yb << 4);
 }
-template <> __device__ __forceinline__ uint32_t merge_words<2, false>(uint32_t in0, uint32_t in1) { return halve_nibbles<false>(in0) | (halve_nibbles<false>(in1) << 8); }
+// 4 -> 2 bit without spreading the codes out: Eq. 3 at b = 2, (13 (c + 2)) >> 6, is [c >= 3] + [c >= 8] + [c >= 13]
+// for the sixteen 4-bit codes.  The result's high bit is the code's bit 3; its low bit is the carry of
+// (c & 7) + 5 - 2 [c >= 8] into bit 3 ((c & 7) >= 3 below 8, (c & 7) >= 5 from 8 on), a sum that stays inside 3..12,
+// so all eight fields of a word are served by one add with no carry between them.
+__device__ __forceinline__ uint32_t halve_nibbles_in_place(uint32_t x) {  // -> 2-bit results at the bottom of every nibble
+  const uint32_t h2 = (x >> 2) & 0x22222222u;
+  const uint32_t s = (x & 0x77777777u) + 0x55555555u - h2;
+  return ((s >> 3) & 0x11111111u) | h2;
+}
+// The four results of each half (fields at the bottom of the nibbles) gathered into 8 adjacent bits, at bits 6-13
+// (half 0) and 22-29 (half 1): y * 5 puts an even nibble's result right below its odd neighbour's (bits 2-5 of
+// every byte), * 17 puts byte 0's four bits right below byte 1's.  The fields never overlap, so the products are
+// ORs of shifted copies, done on the multiply-add pipe, which this kernel leaves idle otherwise.
+__device__ __forceinline__ uint32_t gather_nibble_results(uint32_t y) { return ((y * 5u) & 0x3C3C3C3Cu) * 17u; }
+template <> __device__ __forceinline__ uint32_t merge_words<2, false>(uint32_t in0, uint32_t in1) {
+  return __byte_perm(gather_nibble_results(halve_nibbles_in_place(in0)) >> 6, gather_nibble_results(halve_nibbles_in_place(in1)) >> 6,
+                     0x6240);
+}
 template <> __device__ __forceinline__ uint32_t merge_words<2, true>(uint32_t in0, uint32_t in1) { return halve_nibbles<true>(in0) | (halve_nibbles<true>(in1) << 8); }
 template <> __device__ __forceinline__ uint32_t merge_words<4, false>(uint32_t in0, uint32_t in1) { return halve_bytes<false>(in0) | (halve_bytes<false>(in1) << 8); }
 template <> __device__ __forceinline__ uint32_t merge_words<4, true>(uint32_t in0, uint32_t in1) { return halve_bytes<true>(in0) | (halve_bytes<true>(in1) << 8); }
@@ -794,14 +835,19 @@ template <int B, bool SHR>
 __device__ __forceinline__ void reduce_wave_tiles(uint8_t *base, int lo, int hi, int warp, int n_warps, int lane, int variant) {
   int j = lo + warp;
   if (j >= hi) return;
-  TileRegs<B> cur;
-  load_tile_regs<B>(base + (size_t)j * tile_bytes(2 * B), lane, cur);
-  for (; j < hi; j += n_warps) {
-    TileRegs<B> nxt;
-    const bool more = j + n_warps < hi;
-    if (more) load_tile_regs<B>(base + (size_t)(j + n_warps) * tile_bytes(2 * B), lane, nxt);
-    finish_tile_regs<B, SHR>(cur, base + (size_t)j * tile_bytes(B), lane, variant);
-    if (more) cur = nxt;
+  TileRegs<B> a, b;  // two tiles take turns, so no tile is ever copied from one set of registers to another
+  load_tile_regs<B>(base + (size_t)j * tile_bytes(2 * B), lane, a);
+  while (true) {
+    const bool more_b = j + n_warps < hi;
+    if (more_b) load_tile_regs<B>(base + (size_t)(j + n_warps) * tile_bytes(2 * B), lane, b);
+    finish_tile_regs<B, SHR>(a, base + (size_t)j * tile_bytes(B), lane, variant);
+    if (!more_b) break;
+    j += n_warps;
+    const bool more_a = j + n_warps < hi;
+    if (more_a) load_tile_regs<B>(base + (size_t)(j + n_warps) * tile_bytes(2 * B), lane, a);
+    finish_tile_regs<B, SHR>(b, base + (size_t)j * tile_bytes(B), lane, variant);
+    if (!more_a) break;
+    j += n_warps;
   }
 }
 
@@ -994,8 +1040,12 @@ __device__ __forceinline__ void reduce_tile_to_row(const uint8_t *in, uint8_t *o
 // warps run through the wave's tiles without meeting, and a barrier between waves keeps a wave's stores
 // behind the earlier waves' loads.  The waves grow geometrically (x 1.8 - 1.9).
 // Warps per CTA: enough tiles in flight per stream to cover the memory latency, and few enough registers
-// that every (stream, slice) CTA of the common shapes is resident at once.
-template <int B> __host__ __device__ constexpr int reduce_warps() { return 8; }
+// that every (stream, slice) CTA of the common shapes is resident at once.  4 -> 2 bit keeps two tiles per warp
+// in registers (80 registers at 6 warps); measured at 64 slices x 32K tokens, 6 warps 84 us,
+// 5 warps 85, 8 warps (64 registers, spilling) 90, 4 warps 89; a cp.async ring of 2-4 tiles per warp in shared
+// memory instead of the registers changed nothing (88 us at 8 warps): the three widths all sit on
+// 14 us + bytes / 6.4 TB/s, the 14 us being the launch, the short first waves and the uneven end.
+template <int B> __host__ __device__ constexpr int reduce_warps() { return B == 2 ? 6 : 8; }
 template <int B> __host__ __device__ constexpr int reduce_min_ctas() { return 4; }
 template <int B>
 __device__ __forceinline__ void reduce_one_tile(const LayerGeom &geom, const uint8_t *in, uint8_t *out, int lane, bool active,
