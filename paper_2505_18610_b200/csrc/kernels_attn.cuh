@@ -912,13 +912,15 @@ __device__ __forceinline__ void tc_setup(TcShared *sh, TcCtx &tc, uint8_t *ring,
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       tc05::mbar_init(tc05::smem_u32(&sh->full[s]), 1);
-      tc05::mbar_init(tc05::smem_u32(&sh->stage_free[s]), 16);
+      tc05::mbar_init(tc05::smem_u32(&sh->stage_free[s]), 12);
     }
     for (int b = 0; b < 2; ++b) {
+      tc05::mbar_init(tc05::smem_u32(&sh->ak_full[b]), 4);
+      tc05::mbar_init(tc05::smem_u32(&sh->av_full[b]), 4);
+      tc05::mbar_init(tc05::smem_u32(&sh->w_full[b]), 4);
       tc05::mbar_init(tc05::smem_u32(&sh->ds_free[b]), 4);
       tc05::mbar_init(tc05::smem_u32(&sh->bar_s[b]), 1);
       tc05::mbar_init(tc05::smem_u32(&sh->bar_o[b]), 1);
-      sh->k_tickets[b] = sh->p_tickets[b] = 0u;
       sh->pv_fresh[b] = 1;
     }
     sh->abort = 0;
@@ -933,6 +935,13 @@ __device__ __forceinline__ void tc_setup(TcShared *sh, TcCtx &tc, uint8_t *ring,
 __device__ __forceinline__ void tc_teardown(TcCtx &tc) {
   tc05::fence_before_sync();
   __syncthreads();
+  if (*reinterpret_cast<volatile int *>(&tc.sh->abort)) {
+    // a wait gave up: copies into this CTA's shared memory may still be in flight; give them about a
+    // millisecond (a bounded delay) to land before the CTA goes away
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) {}
+    __syncthreads();
+  }
   if ((threadIdx.x >> 5) == 0) tc05::tmem_dealloc(tc.tmem_base, kTmemCols);
 }
 

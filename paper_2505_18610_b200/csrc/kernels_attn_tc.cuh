@@ -54,17 +54,20 @@ constexpr int kQOperandBytes = 4096;       // [n-group 2][k-chunk 16][8 rows][8 
 constexpr int kEPV = 7;                    // w = p * S_V / sigma_u * 2^(kEPV - pos) stays below 2^16 for p <= 2^kTcMaxAhead
 constexpr float kTcMaxAhead = 8.0f;        // a score may exceed the reference by this much (log2 units)
 constexpr float kTcHeadroom = 4.0f;        // a new reference is set this far above the maxima seen
-constexpr int kWarpK = 0, kWarpV = 4, kWarpS = 8;  // first warp of each role (S: two warpgroups, warps 8-11 and 12-15)
+// first warp of each role: one warpgroup unpacks K and V, two take the scores, three single warps serve them
+constexpr int kWarpKV = 0, kWarpS = 4, kWarpCopy = 12, kWarpMmaS = 13, kWarpMmaO = 14;
 
 // Shared-memory bookkeeping of the tensor-core path (static).
 struct TcShared {
   unsigned long long full[kStages];        // the stage's copy has landed
-  unsigned long long stage_free[kStages];  // K, V and both S warpgroups are done with the stage (16 warp arrivals)
+  unsigned long long stage_free[kStages];  // the unpacking warpgroup and both S warpgroups are done with the stage (12 warp arrivals)
+  unsigned long long ak_full[2];           // the block's K operand is in tensor memory (4 warp arrivals)
+  unsigned long long av_full[2];           // the block's V operand is in tensor memory (4 warp arrivals)
+  unsigned long long w_full[2];            // the block's weights are in shared memory (4 warp arrivals)
   unsigned long long ds_free[2];           // the S warpgroup has read the buffer's scores (4 warp arrivals)
   unsigned long long bar_s[2], bar_o[2];   // score / output MMAs of the buffer's block are complete
   uint32_t tmem_base;
   int abort;
-  unsigned k_tickets[2], p_tickets[2];     // warps that have finished the buffer's block (K: 4; V and S: 8)
   int pv_fresh[2];                         // the block's first output MMA overwrites the accumulators
   float wmax[2][4][kMaxGroup];             // per-warp block maxima (when a reference moves)
   float sums[2][4][2 * kMaxGroup];
@@ -117,19 +120,6 @@ __device__ __forceinline__ void warp_arrive(const unsigned long long *bar, int l
   __syncwarp();
   if (lane == 0) tc05::mbar_arrive(tc05::smem_u32(bar));
 }
-// One ticket per warp (release / acquire at CTA scope); true in every lane of the warp that draws the
-// last of `n`, which also puts the counter back to zero for the buffer's next block.
-__device__ __forceinline__ bool last_ticket(unsigned *counter, unsigned n, int lane) {
-  __syncwarp();
-  unsigned old = 0;
-  if (lane == 0) {
-    asm volatile("atom.acq_rel.cta.shared.add.u32 %0, [%1], 1;\n" : "=r"(old) : "r"(tc05::smem_u32(counter)) : "memory");
-    if (old == n - 1) *reinterpret_cast<volatile unsigned *>(counter) = 0u;
-  }
-  old = __shfl_sync(0xffffffffu, old, 0);
-  return old == n - 1;
-}
-
 template <int BITS> struct RowFmt;
 template <> struct RowFmt<2> {
   static constexpr int SIGMA_LOG2 = 15, CHUNK_TILES = 16;
@@ -221,58 +211,96 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
     tc.gc += (uint32_t)nc;
   }
   constexpr uint32_t idesc_qk = tc05::idesc_f16(128, 16, 0), idesc_pv = tc05::idesc_f16(128, 16, 1);
-  // the output MMAs of a block: one per live tile, into the accumulators of the block's S warpgroup
-  auto issue_pv = [&](uint32_t b, int nv) {
-    tc05::fence_after_sync();
-    const bool fresh = *reinterpret_cast<volatile int *>(&sh->pv_fresh[b]) != 0;
-    if (tc05::elect_one()) {
-      const uint32_t w_addr = tc05::smem_u32(tc.wbuf) + kWBufBytes * b;
-      for (int j = 0; j < nv; ++j)
-        tc05::mma_f16_ts(tb + kTmemDO + 16 * b, tb + kTmemAV + 64 * b + 8 * j, tc05::smem_desc(w_addr + 256 * j, 128, 2048), idesc_pv,
-                         (fresh && j == 0) ? 0u : 1u);
-      tc05::mma_commit(tc05::smem_u32(&sh->bar_o[b]));
-    }
-    __syncwarp();
-  };
 
-  if (false) {
-  } else if (warp < kWarpV) {
-    // ---- K: token row -> tensor memory; the last warp of a block issues the score MMAs ----
-    const uint32_t q_addr = tc05::smem_u32(tc.q_operand);
-    // Warp 0 also feeds the ring: one bulk copy per chunk, kStages - 1 chunks ahead of the chunk it works on.
-    int cp_s = 0, cp_j = 0, cp_hi = 0, cp_n = 0;  // next chunk to copy: stream, first stream-tile, end of the stream's run, chunk index
-    auto copy_next = [&]() {
-      while (cp_s < kStreams && cp_j >= cp_hi) {  // next stream with tiles left
-        ++cp_s;
-        if (cp_s < kStreams) {
-          cp_j = t_lo > cp_s ? (t_lo - cp_s + 7) >> 3 : 0;
-          cp_hi = t_hi > cp_s ? (t_hi - cp_s + 7) >> 3 : 0;
+  if (warp == kWarpCopy) {
+    // ---- copies: one bulk copy per chunk into the ring, as far ahead as the ring has free stages ----
+    int n_chunk = 0;
+    for (int s = 0; s < kStreams; ++s) {
+      const int j_lo = t_lo > s ? (t_lo - s + 7) >> 3 : 0, j_hi = t_hi > s ? (t_hi - s + 7) >> 3 : 0;
+      for (int j = j_lo; j < j_hi; j += CHUNK, ++n_chunk) {
+        const int tiles = min(CHUNK, j_hi - j);
+        const uint32_t m = c0g + n_chunk, st = m % kStages;
+        if (n_chunk >= kStages) tc_wait(tc, &sh->stage_free[st], m / kStages - 1, 8u);  // the stage's last chunk has been used up
+        if (lane == 0) {
+          const uint32_t bar = tc05::smem_u32(&sh->full[st]);
+          tc05::mbar_arrive_expect_tx(bar, (uint32_t)(tiles * TB));
+          tc05::bulk_g2s(tc05::smem_u32(tc.stages + (size_t)st * kStageBytes), body + (size_t)s * p.geom.stream_stride + (size_t)j * TB,
+                         (uint32_t)(tiles * TB), bar);
         }
+        __syncwarp();
       }
-      if (cp_s >= kStreams) return;
-      const int tiles = min(CHUNK, cp_hi - cp_j);
-      const uint32_t m = c0g + cp_n, st = m % kStages;
-      if (cp_n >= kStages) tc_wait(tc, &sh->stage_free[st], m / kStages - 1, 8u);
-      if (lane == 0) {
-        const uint32_t bar = tc05::smem_u32(&sh->full[st]);
-        tc05::mbar_arrive_expect_tx(bar, (uint32_t)(tiles * TB));
-        tc05::bulk_g2s(tc05::smem_u32(tc.stages + (size_t)st * kStageBytes), body + (size_t)cp_s * p.geom.stream_stride + (size_t)cp_j * TB,
-                       (uint32_t)(tiles * TB), bar);
-      }
-      __syncwarp();
-      cp_j += tiles;
-      ++cp_n;
-    };
-    if (warp == 0) {
-      cp_j = (t_lo + 7) >> 3;
-      cp_hi = (t_hi + 7) >> 3;
-      for (int c = 0; c < kStages - 1; ++c) copy_next();
     }
+  } else if (warp == kWarpMmaS) {
+    // ---- score MMAs: S[token, head] = A_K . Q''^T once the block's K operand is in tensor memory ----
+    const uint32_t q_addr = tc05::smem_u32(tc.q_operand);
+    tc_walk<CHUNK>(t_lo, t_hi, [&](int, int, int, int) {},
+        [&](int i, int, int, int, int, int, bool) {
+          const uint32_t n = g0 + i, b = n & 1u;
+          tc_wait(tc, &sh->ak_full[b], n >> 1, 32u);
+          if (i >= 2) tc_wait(tc, &sh->ds_free[b], (n >> 1) - 1, 16u);  // the scores of the buffer's last block have been read
+          __syncwarp();
+          tc05::fence_after_sync();
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            tc05::mma_f16_ts_elect(tb + kTmemDS + 16 * b, tb + kTmemAK + 64 * b + 8 * ks, tc05::smem_desc(q_addr + 256 * ks, 128, 2048),
+                                   idesc_qk, ks > 0 ? 1u : 0u);
+          tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_s[b]));
+        });
+  } else if (warp == kWarpMmaO) {
+    // ---- output MMAs: O^T[channel, head] += A_V . w, one per live tile, into the accumulators of the block's S warpgroup ----
+    const uint32_t w_base = tc05::smem_u32(tc.wbuf);
+    tc_walk<CHUNK>(t_lo, t_hi, [&](int, int, int, int) {},
+        [&](int i, int, int, int, int, int nv, bool) {
+          const uint32_t n = g0 + i, b = n & 1u;
+          tc_wait(tc, &sh->av_full[b], n >> 1, 64u);
+          tc_wait(tc, &sh->w_full[b], n >> 1, 128u);
+          __syncwarp();
+          tc05::fence_after_sync();
+          const uint32_t fresh = *reinterpret_cast<volatile int *>(&sh->pv_fresh[b]) != 0 ? 1u : 0u;
+          const uint32_t w_addr = w_base + kWBufBytes * b;
+          for (int j = 0; j < nv; ++j)
+            tc05::mma_f16_ts_elect(tb + kTmemDO + 16 * b, tb + kTmemAV + 64 * b + 8 * j, tc05::smem_desc(w_addr + 256 * j, 128, 2048), idesc_pv,
+                                   (fresh && j == 0) ? 0u : 1u);
+          tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_o[b]));
+        });
+  } else if (warp < kWarpS) {
+    // ---- K and V: thread tw writes token row tw of A_K and channel row tw of A_V.  The Keys run two blocks
+    //      ahead of the Values: a block's scores are wanted as early as possible, its Values only when its
+    //      softmax ends, and the Value buffer of block n is free only once the output MMAs of block n - 2
+    //      are complete. ----
+    struct Pending { int i, chunk, sb; bool last_of_chunk; };
+    Pending pend[2];
+    int n_pend = 0;
+    auto do_v = [&](const Pending &d) {
+      const uint32_t n = g0 + d.i, b = n & 1u, st = (c0g + d.chunk) % kStages;
+      const uint8_t *vp = tc.stages + (size_t)st * kStageBytes + d.sb * TB + v_part_offset(BITS) + tw * CH_BYTES;
+      if (d.i >= 2) {  // the output MMAs of the block that used this buffer have read it
+        tc_wait(tc, &sh->bar_o[b], (n >> 1) - 1, 4u);
+        tc05::fence_after_sync();
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t r[32];
+#pragma unroll
+        for (int t4 = 0; t4 < 4; ++t4) {
+          const int t8 = 4 * half + t4;
+          if constexpr (BITS == 2) {
+            F::extract(*reinterpret_cast<const uint32_t *>(vp + t8 * TB), r + 8 * t4);
+          } else {
+            const uint2 v = *reinterpret_cast<const uint2 *>(vp + t8 * TB);
+            F::extract(v.x, r + 8 * t4);
+            F::extract(v.y, r + 8 * t4 + 4);
+          }
+        }
+        tc05::tmem_st32(tb + kTmemAV + 64 * b + t_lane + 32 * half, r);
+      }
+      tc05::wait_st();
+      tc05::fence_before_sync();
+      warp_arrive(&sh->av_full[b], lane);
+      if (d.last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
+    };
     tc_walk<CHUNK>(t_lo, t_hi,
-        [&](int chunk, int, int, int) {
-          if (warp == 0) copy_next();
-          tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u);
-        },
+        [&](int chunk, int, int, int) { tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u); },
         [&](int i, int chunk, int, int, int sb, int, bool last_of_chunk) {
           const uint32_t n = g0 + i, b = n & 1u, st = (c0g + chunk) % kStages;
           const uint8_t *kp = tc.stages + (size_t)st * kStageBytes + (sb + my_tile) * TB + my_row * ROW_BYTES;
@@ -298,53 +326,16 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
           }
           tc05::wait_st();
           tc05::fence_before_sync();
-          if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
-          if (last_ticket(&sh->k_tickets[b], 4, lane)) {
-            if (i >= 2) tc_wait(tc, &sh->ds_free[b], (n >> 1) - 1, 16u);  // the scores of the buffer's last block have been read
-            tc05::fence_after_sync();
-            if (tc05::elect_one()) {
-#pragma unroll
-              for (int ks = 0; ks < 8; ++ks)
-                tc05::mma_f16_ts(tb + kTmemDS + 16 * b, tb + kTmemAK + 64 * b + 8 * ks, tc05::smem_desc(q_addr + 256 * ks, 128, 2048),
-                                 idesc_qk, ks > 0 ? 1u : 0u);
-              tc05::mma_commit(tc05::smem_u32(&sh->bar_s[b]));
-            }
-            __syncwarp();
+          warp_arrive(&sh->ak_full[b], lane);
+          if (n_pend == 2) {
+            do_v(pend[0]);
+            pend[0] = pend[1];
+            n_pend = 1;
           }
+          pend[n_pend++] = Pending{i, chunk, sb, last_of_chunk};
         });
-  } else if (warp < kWarpS) {
-    // ---- V: channel row -> tensor memory ----
-    tc_walk<CHUNK>(t_lo, t_hi,
-        [&](int chunk, int, int, int) { tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u); },
-        [&](int i, int chunk, int, int, int sb, int nv, bool last_of_chunk) {
-          const uint32_t n = g0 + i, b = n & 1u, st = (c0g + chunk) % kStages;
-          const uint8_t *vp = tc.stages + (size_t)st * kStageBytes + sb * TB + v_part_offset(BITS) + tw * CH_BYTES;
-          if (i >= 2) {  // the output MMAs of the block that used this buffer have read it
-            tc_wait(tc, &sh->bar_o[b], (n >> 1) - 1, 4u);
-            tc05::fence_after_sync();
-          }
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            uint32_t r[32];
-#pragma unroll
-            for (int t4 = 0; t4 < 4; ++t4) {
-              const int t8 = 4 * half + t4;
-              if constexpr (BITS == 2) {
-                F::extract(*reinterpret_cast<const uint32_t *>(vp + t8 * TB), r + 8 * t4);
-              } else {
-                const uint2 v = *reinterpret_cast<const uint2 *>(vp + t8 * TB);
-                F::extract(v.x, r + 8 * t4);
-                F::extract(v.y, r + 8 * t4 + 4);
-              }
-            }
-            tc05::tmem_st32(tb + kTmemAV + 64 * b + t_lane + 32 * half, r);
-          }
-          tc05::wait_st();
-          tc05::fence_before_sync();
-          if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
-          if (last_ticket(&sh->p_tickets[b], 8, lane)) issue_pv(b, nv);
-        });
-  } else {
+    for (int k = 0; k < n_pend; ++k) do_v(pend[k]);
+  } else if (warp < kWarpCopy) {
     // ---- S: scores -> probabilities -> weights; running sums; this warpgroup's partial ----
     const uint32_t sw = (uint32_t)(warp - kWarpS) >> 2;   // S warpgroup 0 / 1: owns the blocks with n mod 2 == sw
     float2 mu2[4], sumq2[4], m2[4], l2[4], zs2[4];
@@ -496,7 +487,7 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
           if (tw == 0) sh->pv_fresh[b] = fresh ? 1 : 0;
           tc05::fence_async_smem();
           tc05::fence_before_sync();
-          if (last_ticket(&sh->p_tickets[b], 8, lane)) issue_pv(b, nv);
+          warp_arrive(&sh->w_full[b], lane);
           mine_last = i;
           fresh = false;
           ++since;

@@ -346,17 +346,17 @@ __device__ __forceinline__ void pack_words(const float *lo, const float *hi, int
   if constexpr (BITS == 16) {  // one code per half; only the low 16 bits of a pattern are the code
 #pragma unroll
     for (int w = 0; w < 16; ++w) words[w] = __byte_perm(__float_as_uint(lo[w * step]), __float_as_uint(hi[w * step]), 0x5410);
-    return;
-  }
+  } else {
 #pragma unroll
-  for (int w = 0; w < BITS; ++w) {
-    uint32_t a = 0, b = 0;
+    for (int w = 0; w < BITS; ++w) {
+      uint32_t a = 0, b = 0;
 #pragma unroll
-    for (int j = 0; j < n; ++j) {
-      a |= __float_as_uint(lo[(w * n + j) * step]) << (j * BITS);
-      b |= __float_as_uint(hi[(w * n + j) * step]) << (j * BITS);
+      for (int j = 0; j < n; ++j) {
+        a |= __float_as_uint(lo[(w * n + j) * step]) << (j * BITS);
+        b |= __float_as_uint(hi[(w * n + j) * step]) << (j * BITS);
+      }
+      words[w] = a | (b << 16);
     }
-    words[w] = a | (b << 16);
   }
 }
 
