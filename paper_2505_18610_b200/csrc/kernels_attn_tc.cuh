@@ -99,8 +99,11 @@ __device__ __forceinline__ void swg_sync(int sw) { asm volatile("bar.sync %0, 12
 
 // A wait that gives up: marks the CTA as aborted and leaves a trace for the host.
 __device__ __forceinline__ void tc_wait(TcCtx &tc, const unsigned long long *bar, uint32_t parity, unsigned code) {
+  const uint32_t addr = tc05::smem_u32(bar);
+  if (tc05::mbar_test_wait(addr, parity & 1u)) return;  // the common case costs one barrier operation
   if (*reinterpret_cast<volatile int *>(&tc.sh->abort)) return;
-  if (!tc05::mbar_wait(tc05::smem_u32(bar), parity & 1u)) {
+  const bool ok = tc05::mbar_wait(addr, parity & 1u);
+  if (!ok) {
     tc.sh->abort = 1;
     atomicOr(tc.error_word, code);
   }

@@ -40,12 +40,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Waits for the phase with the given parity to complete; gives up after kWaitLimit polls (each poll
-// itself blocks for a hardware-defined time slice), far beyond anything a healthy launch needs.
-constexpr uint32_t kWaitLimit = 1u << 20;
+// A blocking poll with a time hint: the thread sleeps in hardware until the phase completes or about `ns`
+// nanoseconds have passed, instead of coming back after the (short) default time and spinning through the
+// issue slots that the working warps of the same scheduler need.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {  // never blocks
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Waits for the phase with the given parity to complete; gives up after kWaitLimit polls of up to kWaitHintNs
+// each (about a second in all), far beyond anything a healthy launch needs.
+constexpr uint32_t kWaitLimit = 1u << 16;
+constexpr uint32_t kWaitHintNs = 16384;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = kWaitLimit) {
+  if (mbar_test_wait(bar, parity)) return true;
   for (uint32_t i = 0; i < limit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_hint(bar, parity, kWaitHintNs)) return true;
   return false;
 }
 
