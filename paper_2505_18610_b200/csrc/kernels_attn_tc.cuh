@@ -125,7 +125,7 @@ __device__ __forceinline__ void warp_arrive(const unsigned long long *bar, int l
 }
 template <int BITS> struct RowFmt;
 template <> struct RowFmt<2> {
-  static constexpr int SIGMA_LOG2 = 15, CHUNK_TILES = 16;
+  static constexpr int SIGMA_LOG2 = 15, CHUNK_TILES = 8;
   __host__ __device__ static constexpr int pos(int f) { return 2 * (f & 3); }                // f = field 0..7
   __host__ __device__ static constexpr int field(int idx) { return (idx & 15) >> 1; }        // of channel / token index
   // one word (16 codes) -> 8 tensor-memory columns (column f = fields f of the two halves)
