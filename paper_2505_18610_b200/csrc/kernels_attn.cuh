@@ -48,7 +48,7 @@ constexpr float kNegBig = -1.0e30f;
 constexpr float kMaxAhead = 3.0f;    // a score may exceed the reference by this much (log2 units)
 constexpr int kAttnWarps = 16;       // one CTA per SM; these warps share the CTA's INT16 / 8- / 16-bit tiles dynamically
 constexpr int kAttnThreads = 32 * kAttnWarps;
-constexpr int kParts = kAttnWarps + 2;  // partial results a segment merges: one per warp, two of the tensor-memory body
+constexpr int kParts = kAttnWarps + 3;  // partial results a segment merges: one per warp, three of the tensor-memory body
 
 struct AttnParams {
   LayerGeom geom;
@@ -834,7 +834,7 @@ namespace pmkvq {
 constexpr int kSmemStages = kStages * kStageBytes;
 constexpr int kSmemQOperand = kSmemStages;
 constexpr int kSmemWBuf = kSmemQOperand + kQOperandBytes;
-constexpr int kSmemParts = kSmemWBuf + 2 * kWBufBytes;
+constexpr int kSmemParts = kSmemWBuf + kTcGroups * kWBufBytes;
 constexpr int kSmemTcTotal = kSmemParts + kParts * kMaxGroup * kHeadDim * 4;
 
 // One segment with a 4- or 2-bit body.  The INT16 tiles run as above, on the warps' own accumulators, and
@@ -874,7 +874,7 @@ __device__ __forceinline__ void run_segment_tc(const AttnParams &p, int slice, l
   }
   if (t_hi > t_lo) {
     tc_body<BITS>(p, tc, slice_base + p.geom.body_off, t_lo, t_hi, s_stat, sigma16, s_m, s_l, kAttnWarps);
-  } else if (tid < 2 * kHeadDim) {
+  } else if (tid < kTcGroups * kHeadDim) {
     const int slot = kAttnWarps + (tid >> 7), c = tid & 127;
 #pragma unroll
     for (int h = 0; h < kMaxGroup; ++h) s_o[slot][h][c] = 0.f;
@@ -912,13 +912,12 @@ __device__ __forceinline__ void tc_setup(TcShared *sh, TcCtx &tc, uint8_t *ring,
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       tc05::mbar_init(tc05::smem_u32(&sh->full[s]), 1);
-      tc05::mbar_init(tc05::smem_u32(&sh->stage_free[s]), 12);
+      tc05::mbar_init(tc05::smem_u32(&sh->stage_free[s]), 4);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kTcGroups; ++b) {
       tc05::mbar_init(tc05::smem_u32(&sh->ak_full[b]), 4);
       tc05::mbar_init(tc05::smem_u32(&sh->av_full[b]), 4);
       tc05::mbar_init(tc05::smem_u32(&sh->w_full[b]), 4);
-      tc05::mbar_init(tc05::smem_u32(&sh->ds_free[b]), 4);
       tc05::mbar_init(tc05::smem_u32(&sh->bar_s[b]), 1);
       tc05::mbar_init(tc05::smem_u32(&sh->bar_o[b]), 1);
       sh->pv_fresh[b] = 1;

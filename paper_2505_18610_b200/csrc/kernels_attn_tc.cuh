@@ -44,33 +44,32 @@
 
 namespace pmkvq {
 
-constexpr int kTmemCols = 512;             // A_K 2 x 64 | A_V 2 x 64 | D_S 2 x 16 | D_O 2 x 16
-constexpr int kTmemAK = 0, kTmemAV = 128, kTmemDS = 256, kTmemDO = 288;
+constexpr int kTcGroups = 3;               // warpgroups that each take every third block through K, V and softmax
+constexpr int kTmemCols = 512;             // A_K 3 x 64 | A_V 3 x 64 | D_S 3 x 16 | D_O 3 x 16
+constexpr int kTmemAK = 0, kTmemAV = 192, kTmemDS = 384, kTmemDO = 432;
 constexpr int kStages = 6;                 // chunks in flight in shared memory
-constexpr int kStageBytes = 16 * tile_bytes(2);   // 20 480: 16 tiles at 2 bit, 8 tiles at 4 bit (18 432)
-static_assert(kStageBytes >= 8 * tile_bytes(4), "a stage holds a chunk of either width");
+constexpr int kStageBytes = 8 * tile_bytes(4);    // 18 432: a chunk is 8 tiles = one MMA block at either width
 constexpr int kWBufBytes = 4096;           // [hi | lo][128 tokens][8 heads] fp16: columns h and 8 + h of the weights
 constexpr int kQOperandBytes = 4096;       // [n-group 2][k-chunk 16][8 rows][8 channels] fp16
 constexpr int kEPV = 7;                    // w = p * S_V / sigma_u * 2^(kEPV - pos) stays below 2^16 for p <= 2^kTcMaxAhead
 constexpr float kTcMaxAhead = 8.0f;        // a score may exceed the reference by this much (log2 units)
 constexpr float kTcHeadroom = 4.0f;        // a new reference is set this far above the maxima seen
-// first warp of each role: one warpgroup unpacks K and V, two take the scores, three single warps serve them
-constexpr int kWarpKV = 0, kWarpS = 4, kWarpCopy = 12, kWarpMmaS = 13, kWarpMmaO = 14;
+// warps 0-11 are the three block warpgroups; three single warps serve them
+constexpr int kWarpCopy = 12, kWarpMmaS = 13, kWarpMmaO = 14;
 
 // Shared-memory bookkeeping of the tensor-core path (static).
 struct TcShared {
-  unsigned long long full[kStages];        // the stage's copy has landed
-  unsigned long long stage_free[kStages];  // the unpacking warpgroup and both S warpgroups are done with the stage (12 warp arrivals)
-  unsigned long long ak_full[2];           // the block's K operand is in tensor memory (4 warp arrivals)
-  unsigned long long av_full[2];           // the block's V operand is in tensor memory (4 warp arrivals)
-  unsigned long long w_full[2];            // the block's weights are in shared memory (4 warp arrivals)
-  unsigned long long ds_free[2];           // the S warpgroup has read the buffer's scores (4 warp arrivals)
-  unsigned long long bar_s[2], bar_o[2];   // score / output MMAs of the buffer's block are complete
+  unsigned long long full[kStages];           // the stage's copy has landed
+  unsigned long long stage_free[kStages];     // the block's warpgroup is done with the stage (4 warp arrivals)
+  unsigned long long ak_full[kTcGroups];      // the block's K operand is in tensor memory (4 warp arrivals)
+  unsigned long long av_full[kTcGroups];      // the block's V operand is in tensor memory (4 warp arrivals)
+  unsigned long long w_full[kTcGroups];       // the block's weights are in shared memory (4 warp arrivals)
+  unsigned long long bar_s[kTcGroups], bar_o[kTcGroups];  // score / output MMAs of the warpgroup's block are complete
   uint32_t tmem_base;
   int abort;
-  int pv_fresh[2];                         // the block's first output MMA overwrites the accumulators
-  float wmax[2][4][kMaxGroup];             // per-warp block maxima (when a reference moves)
-  float sums[2][4][2 * kMaxGroup];
+  int pv_fresh[kTcGroups];                    // the block's first output MMA overwrites the accumulators
+  float wmax[kTcGroups][4][kMaxGroup];        // per-warp block maxima (when a reference moves)
+  float sums[kTcGroups][4][2 * kMaxGroup];
 };
 
 // Per-thread view: tensor-memory base, the CTA's running block and chunk counts (barrier parities follow).
@@ -215,6 +214,7 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
   }
   constexpr uint32_t idesc_qk = tc05::idesc_f16(128, 16, 0), idesc_pv = tc05::idesc_f16(128, 16, 1);
 
+  static_assert(CHUNK == 8, "a chunk is one MMA block: the stage belongs to the block's warpgroup alone");
   if (warp == kWarpCopy) {
     // ---- copies: one bulk copy per chunk into the ring, as far ahead as the ring has free stages ----
     int n_chunk = 0;
@@ -234,113 +234,43 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
       }
     }
   } else if (warp == kWarpMmaS) {
-    // ---- score MMAs: S[token, head] = A_K . Q''^T once the block's K operand is in tensor memory ----
+    // ---- score MMAs: S[token, head] = A_K . Q''^T once the block's K operand is in tensor memory.  The K
+    //      operand and the score accumulators belong to the block's warpgroup, which has finished with both
+    //      (its previous block's scores read, its softmax done) before it writes the next K operand. ----
     const uint32_t q_addr = tc05::smem_u32(tc.q_operand);
     tc_walk<CHUNK>(t_lo, t_hi, [&](int, int, int, int) {},
         [&](int i, int, int, int, int, int, bool) {
-          const uint32_t n = g0 + i, b = n & 1u;
-          tc_wait(tc, &sh->ak_full[b], n >> 1, 32u);
-          if (i >= 2) tc_wait(tc, &sh->ds_free[b], (n >> 1) - 1, 16u);  // the scores of the buffer's last block have been read
+          const uint32_t n = g0 + i, wg = n % kTcGroups, use = n / kTcGroups;
+          tc_wait(tc, &sh->ak_full[wg], use, 32u);
           __syncwarp();
           tc05::fence_after_sync();
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            tc05::mma_f16_ts_elect(tb + kTmemDS + 16 * b, tb + kTmemAK + 64 * b + 8 * ks, tc05::smem_desc(q_addr + 256 * ks, 128, 2048),
+            tc05::mma_f16_ts_elect(tb + kTmemDS + 16 * wg, tb + kTmemAK + 64 * wg + 8 * ks, tc05::smem_desc(q_addr + 256 * ks, 128, 2048),
                                    idesc_qk, ks > 0 ? 1u : 0u);
-          tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_s[b]));
+          tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_s[wg]));
         });
   } else if (warp == kWarpMmaO) {
-    // ---- output MMAs: O^T[channel, head] += A_V . w, one per live tile, into the accumulators of the block's S warpgroup ----
+    // ---- output MMAs: O^T[channel, head] += A_V . w, one per live tile, into the accumulators of the block's warpgroup ----
     const uint32_t w_base = tc05::smem_u32(tc.wbuf);
     tc_walk<CHUNK>(t_lo, t_hi, [&](int, int, int, int) {},
         [&](int i, int, int, int, int, int nv, bool) {
-          const uint32_t n = g0 + i, b = n & 1u;
-          tc_wait(tc, &sh->av_full[b], n >> 1, 64u);
-          tc_wait(tc, &sh->w_full[b], n >> 1, 128u);
+          const uint32_t n = g0 + i, wg = n % kTcGroups, use = n / kTcGroups;
+          tc_wait(tc, &sh->av_full[wg], use, 64u);
+          tc_wait(tc, &sh->w_full[wg], use, 128u);
           __syncwarp();
           tc05::fence_after_sync();
-          const uint32_t fresh = *reinterpret_cast<volatile int *>(&sh->pv_fresh[b]) != 0 ? 1u : 0u;
-          const uint32_t w_addr = w_base + kWBufBytes * b;
+          const uint32_t fresh = *reinterpret_cast<volatile int *>(&sh->pv_fresh[wg]) != 0 ? 1u : 0u;
+          const uint32_t w_addr = w_base + kWBufBytes * wg;
           for (int j = 0; j < nv; ++j)
-            tc05::mma_f16_ts_elect(tb + kTmemDO + 16 * b, tb + kTmemAV + 64 * b + 8 * j, tc05::smem_desc(w_addr + 256 * j, 128, 2048), idesc_pv,
+            tc05::mma_f16_ts_elect(tb + kTmemDO + 16 * wg, tb + kTmemAV + 64 * wg + 8 * j, tc05::smem_desc(w_addr + 256 * j, 128, 2048), idesc_pv,
                                    (fresh && j == 0) ? 0u : 1u);
-          tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_o[b]));
+          tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_o[wg]));
         });
-  } else if (warp < kWarpS) {
-    // ---- K and V: thread tw writes token row tw of A_K and channel row tw of A_V.  The Keys run two blocks
-    //      ahead of the Values: a block's scores are wanted as early as possible, its Values only when its
-    //      softmax ends, and the Value buffer of block n is free only once the output MMAs of block n - 2
-    //      are complete. ----
-    struct Pending { int i, chunk, sb; bool last_of_chunk; };
-    Pending pend[2];
-    int n_pend = 0;
-    auto do_v = [&](const Pending &d) {
-      const uint32_t n = g0 + d.i, b = n & 1u, st = (c0g + d.chunk) % kStages;
-      const uint8_t *vp = tc.stages + (size_t)st * kStageBytes + d.sb * TB + v_part_offset(BITS) + tw * CH_BYTES;
-      if (d.i >= 2) {  // the output MMAs of the block that used this buffer have read it
-        tc_wait(tc, &sh->bar_o[b], (n >> 1) - 1, 4u);
-        tc05::fence_after_sync();
-      }
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t r[32];
-#pragma unroll
-        for (int t4 = 0; t4 < 4; ++t4) {
-          const int t8 = 4 * half + t4;
-          if constexpr (BITS == 2) {
-            F::extract(*reinterpret_cast<const uint32_t *>(vp + t8 * TB), r + 8 * t4);
-          } else {
-            const uint2 v = *reinterpret_cast<const uint2 *>(vp + t8 * TB);
-            F::extract(v.x, r + 8 * t4);
-            F::extract(v.y, r + 8 * t4 + 4);
-          }
-        }
-        tc05::tmem_st32(tb + kTmemAV + 64 * b + t_lane + 32 * half, r);
-      }
-      tc05::wait_st();
-      tc05::fence_before_sync();
-      warp_arrive(&sh->av_full[b], lane);
-      if (d.last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
-    };
-    tc_walk<CHUNK>(t_lo, t_hi,
-        [&](int chunk, int, int, int) { tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u); },
-        [&](int i, int chunk, int, int, int sb, int, bool last_of_chunk) {
-          const uint32_t n = g0 + i, b = n & 1u, st = (c0g + chunk) % kStages;
-          const uint8_t *kp = tc.stages + (size_t)st * kStageBytes + (sb + my_tile) * TB + my_row * ROW_BYTES;
-          constexpr int HALF_CHUNKS = ROW_BYTES / 32;  // 16-byte chunks per half row
-          uint4 raw[2 * HALF_CHUNKS];
-#pragma unroll
-          for (int c = 0; c < 2 * HALF_CHUNKS; ++c) raw[c] = *reinterpret_cast<const uint4 *>(kp + c * 16);
-          if (i >= 2) {  // the score MMAs of the block that used this buffer have read it
-            tc_wait(tc, &sh->bar_s[b], (n >> 1) - 1, 2u);
-            tc05::fence_after_sync();
-          }
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            uint32_t r[32];
-#pragma unroll
-            for (int c = 0; c < HALF_CHUNKS; ++c) {
-              const uint4 v = raw[half * HALF_CHUNKS + c];
-              const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) F::extract(w4[e], r + (4 * c + e) * (32 / (4 * HALF_CHUNKS)));
-            }
-            tc05::tmem_st32(tb + kTmemAK + 64 * b + t_lane + 32 * half, r);
-          }
-          tc05::wait_st();
-          tc05::fence_before_sync();
-          warp_arrive(&sh->ak_full[b], lane);
-          if (n_pend == 2) {
-            do_v(pend[0]);
-            pend[0] = pend[1];
-            n_pend = 1;
-          }
-          pend[n_pend++] = Pending{i, chunk, sb, last_of_chunk};
-        });
-    for (int k = 0; k < n_pend; ++k) do_v(pend[k]);
   } else if (warp < kWarpCopy) {
-    // ---- S: scores -> probabilities -> weights; running sums; this warpgroup's partial ----
-    const uint32_t sw = (uint32_t)(warp - kWarpS) >> 2;   // S warpgroup 0 / 1: owns the blocks with n mod 2 == sw
+    // ---- a block warpgroup: every third block, through all its steps.  Thread tw writes token row tw of A_K
+    //      (the score MMAs start), then channel row tw of A_V, then turns the block's scores into weights. ----
+    const uint32_t sw = (uint32_t)warp >> 2;   // this warpgroup: owns the blocks with n mod 3 == sw
     float2 mu2[4], sumq2[4], m2[4], l2[4], zs2[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -367,32 +297,74 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
     const uint32_t tDO = tb + kTmemDO + 16 * sw + t_lane, tDS = tb + kTmemDS + 16 * sw + t_lane;
     auto wait_o = [&](int blk) {  // output MMAs of this warpgroup's block blk (and its earlier ones) are complete
       if (blk >= 0 && o_seen < blk) {
-        tc_wait(tc, &sh->bar_o[sw], (g0 + blk) >> 1, 4u);
+        tc_wait(tc, &sh->bar_o[sw], (g0 + blk) / kTcGroups, 4u);
         tc05::fence_after_sync();
         o_seen = blk;
       }
     };
-    tc_walk<CHUNK>(t_lo, t_hi,
-        [&](int chunk, int, int, int) { tc_wait(tc, &sh->full[(c0g + chunk) % kStages], (c0g + chunk) / kStages, 1u); },
-        [&](int i, int chunk, int s, int j0, int sb, int nv, bool last_of_chunk) {
-          const uint32_t n = g0 + i, b = n & 1u, st = (c0g + chunk) % kStages;
-          if (b != sw) {  // the other warpgroup's block; a chunk is released by both
-            if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
-            return;
+    tc_walk<CHUNK>(t_lo, t_hi, [&](int, int, int, int) {},
+        [&](int i, int chunk, int s, int j0, int sb, int nv, bool) {
+          const uint32_t n = g0 + i;
+          if (n % kTcGroups != sw) return;
+          const uint32_t b = sw, use = n / kTcGroups, st = (c0g + chunk) % kStages;
+          tc_wait(tc, &sh->full[st], (c0g + chunk) / kStages, 1u);
+          {  // ---- K: this thread's token row ----
+            const uint8_t *kp = tc.stages + (size_t)st * kStageBytes + (sb + my_tile) * TB + my_row * ROW_BYTES;
+            constexpr int HALF_CHUNKS = ROW_BYTES / 32;  // 16-byte chunks per half row
+            uint4 raw[2 * HALF_CHUNKS];
+#pragma unroll
+            for (int c = 0; c < 2 * HALF_CHUNKS; ++c) raw[c] = *reinterpret_cast<const uint4 *>(kp + c * 16);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              uint32_t r[32];
+#pragma unroll
+              for (int c = 0; c < HALF_CHUNKS; ++c) {
+                const uint4 v = raw[half * HALF_CHUNKS + c];
+                const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) F::extract(w4[e], r + (4 * c + e) * (32 / (4 * HALF_CHUNKS)));
+              }
+              tc05::tmem_st32(tb + kTmemAK + 64 * b + t_lane + 32 * half, r);
+            }
+            tc05::wait_st();
+            tc05::fence_before_sync();
+            warp_arrive(&sh->ak_full[b], lane);
+          }
+          wait_o(mine_last);  // the output MMAs of this warpgroup's last block have read its V operand and weights
+          {  // ---- V: this thread's channel row ----
+            const uint8_t *vp = tc.stages + (size_t)st * kStageBytes + sb * TB + v_part_offset(BITS) + tw * CH_BYTES;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              uint32_t r[32];
+#pragma unroll
+              for (int t4 = 0; t4 < 4; ++t4) {
+                const int t8 = 4 * half + t4;
+                if constexpr (BITS == 2) {
+                  F::extract(*reinterpret_cast<const uint32_t *>(vp + t8 * TB), r + 8 * t4);
+                } else {
+                  const uint2 v = *reinterpret_cast<const uint2 *>(vp + t8 * TB);
+                  F::extract(v.x, r + 8 * t4);
+                  F::extract(v.y, r + 8 * t4 + 4);
+                }
+              }
+              tc05::tmem_st32(tb + kTmemAV + 64 * b + t_lane + 32 * half, r);
+            }
+            tc05::wait_st();
+            tc05::fence_before_sync();
+            warp_arrive(&sh->av_full[b], lane);
           }
           const uint8_t *blk = tc.stages + (size_t)st * kStageBytes + sb * TB;
           // token row (my_tile, my_row) of the block is token 16 (s + 8 (j0 + my_tile)) + my_row of the body
           const bool alive = my_tile < nv && ((s + 8 * (j0 + my_tile)) * 16 + my_row) < p.n_body;
           float4 meta = *reinterpret_cast<const float4 *>(blk + my_tile * TB + meta_offset(BITS) + my_row * 16);  // S_K Z_K S_V Z_V
           if (!alive) meta = make_float4(0.f, 0.f, 0.f, 0.f);  // a dead row holds arbitrary bytes
-          if (last_of_chunk) warp_arrive(&sh->stage_free[st], lane);
-          tc_wait(tc, &sh->bar_s[b], n >> 1, 2u);
+          warp_arrive(&sh->stage_free[st], lane);  // K, V and metadata of the block are in registers / tensor memory
+          tc_wait(tc, &sh->bar_s[b], use, 2u);
           tc05::fence_after_sync();
           uint32_t sraw[16];
           tc05::tmem_ld16(tDS, sraw);
           tc05::wait_ld();
           tc05::fence_before_sync();
-          warp_arrive(&sh->ds_free[b], lane);
           float2 dot[4], a2[4], arg[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -495,7 +467,6 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
           fresh = false;
           ++since;
         });
-
     // ---- this warpgroup's partial: (m, l, o[128]) per head ----
     if (mine_last >= 0) {
       wait_o(mine_last);
