@@ -237,34 +237,38 @@ __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const ui
     // ---- score MMAs: S[token, head] = A_K . Q''^T once the block's K operand is in tensor memory.  The K
     //      operand and the score accumulators belong to the block's warpgroup, which has finished with both
     //      (its previous block's scores read, its softmax done) before it writes the next K operand. ----
-    const uint32_t q_addr = tc05::smem_u32(tc.q_operand);
+    const uint64_t q_desc = tc05::smem_desc(tc05::smem_u32(tc.q_operand), 128, 2048);  // + 16 per k-step (256 bytes)
     tc_walk<CHUNK>(t_lo, t_hi, [&](int, int, int, int) {},
         [&](int i, int, int, int, int, int, bool) {
           const uint32_t n = g0 + i, wg = n % kTcGroups, use = n / kTcGroups;
           tc_wait(tc, &sh->ak_full[wg], use, 32u);
           __syncwarp();
           tc05::fence_after_sync();
+          const uint32_t d_s = tb + kTmemDS + 16 * wg, a_k = tb + kTmemAK + 64 * wg;
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            tc05::mma_f16_ts_elect(tb + kTmemDS + 16 * wg, tb + kTmemAK + 64 * wg + 8 * ks, tc05::smem_desc(q_addr + 256 * ks, 128, 2048),
-                                   idesc_qk, ks > 0 ? 1u : 0u);
+          for (int ks = 0; ks < 8; ++ks) tc05::mma_f16_ts_elect(d_s, a_k + 8 * ks, q_desc + 16 * ks, idesc_qk, ks > 0 ? 1u : 0u);
           tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_s[wg]));
         });
-  } else if (warp == kWarpMmaO) {
-    // ---- output MMAs: O^T[channel, head] += A_V . w, one per live tile, into the accumulators of the block's warpgroup ----
+  } else if (warp >= kWarpMmaO) {
+    // ---- output MMAs: O^T[channel, head] += A_V . w, one per live tile, into the accumulators of the block's
+    //      warpgroup.  Two warps take alternate blocks: the blocks of different warpgroups do not depend on one
+    //      another, and one warp issuing in block order holds every block behind the slowest softmax. ----
     const uint32_t w_base = tc05::smem_u32(tc.wbuf);
+    const uint32_t mine = (uint32_t)(warp - kWarpMmaO);
     tc_walk<CHUNK>(t_lo, t_hi, [&](int, int, int, int) {},
         [&](int i, int, int, int, int, int nv, bool) {
           const uint32_t n = g0 + i, wg = n % kTcGroups, use = n / kTcGroups;
+          if ((n & 1u) != mine) return;
           tc_wait(tc, &sh->av_full[wg], use, 64u);
           tc_wait(tc, &sh->w_full[wg], use, 128u);
           __syncwarp();
           tc05::fence_after_sync();
           const uint32_t fresh = *reinterpret_cast<volatile int *>(&sh->pv_fresh[wg]) != 0 ? 1u : 0u;
-          const uint32_t w_addr = w_base + kWBufBytes * wg;
-          for (int j = 0; j < nv; ++j)
-            tc05::mma_f16_ts_elect(tb + kTmemDO + 16 * wg, tb + kTmemAV + 64 * wg + 8 * j, tc05::smem_desc(w_addr + 256 * j, 128, 2048), idesc_pv,
-                                   (fresh && j == 0) ? 0u : 1u);
+          const uint64_t w_desc = tc05::smem_desc(w_base + kWBufBytes * wg, 128, 2048);  // + 16 per tile (256 bytes) in the address field
+          const uint32_t d_o = tb + kTmemDO + 16 * wg, a_v = tb + kTmemAV + 64 * wg;
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (j < nv) tc05::mma_f16_ts_elect(d_o, a_v + 8 * j, w_desc + 16 * j, idesc_pv, (fresh && j == 0) ? 0u : 1u);
           tc05::mma_commit_elect(tc05::smem_u32(&sh->bar_o[wg]));
         });
   } else if (warp < kWarpCopy) {
