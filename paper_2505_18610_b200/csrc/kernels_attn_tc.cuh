@@ -3,43 +3,42 @@
 // Included by kernels_attn.cuh (which holds the work decomposition, the INT16 tile path and the split-K
 // combine).  The body tiles [t_lo, t_hi) of a segment are taken stream by stream (tile t lives in stream
 // t mod 8, and softmax attention does not care about the order of the tokens): in every stream the
-// segment's tiles are one contiguous run of bytes, which is cut into chunks of CHUNK_TILES tiles (about
-// 20 KB: one cp.async.bulk copy each; copies of that size reach the HBM read rate from one issuing lane,
-// 1-10 KB copies do not) and every chunk into MMA blocks of up to 8 tiles = 128 tokens.  The blocks flow
-// through specialised warps that meet only on mbarriers and tickets (no CTA-wide barrier inside the
-// loop), each running ahead of the next as far as its buffers allow:
+// segment's tiles are one contiguous run of bytes, which is cut into MMA blocks of up to 8 tiles = 128
+// tokens, one cp.async.bulk copy each (10 KB at 2 bit, 18 KB at 4 bit) into a ring of kStages stages in
+// shared memory.  Block n belongs to warpgroup n mod 3.  Warps meet only on mbarriers (no CTA-wide barrier
+// inside the loop):
 //
-//   copies         one lane of the K warpgroup's first warp issues one bulk copy per chunk into a ring of
-//                  kStages stages in shared memory, kStages - 1 chunks ahead of the chunk it works on,
-//                  completing on the stage's mbarrier;
-//   K warpgroup    thread t unpacks the 128 codes of token t into fp16 bit patterns (a code field left in
-//                  place below bit 11 of an fp16 is exactly code * 2^(pos-24); one AND per pair of codes)
-//                  and stores them as row t of the score MMA's A operand in tensor memory (tcgen05.st).
-//                  The last of its four warps to finish a block issues S[token, head] = A_K . Q''^T: 8
-//                  tcgen05.mma (128 x 16 x 16, fp16 in, fp32 accumulators in tensor memory), B = the query
-//                  fragments in shared memory (rows 0-7 the fp16 "hi" part of up to 8 heads, rows 8-15 the
-//                  "lo" remainder), and tcgen05.commit onto the buffer's mbarrier;
-//   V warpgroup    thread c does the same for channel c's codes of the block's tokens: row c of the output
-//                  MMA's A operand;
-//   S warpgroups   two, taking alternate blocks.  Thread t reads its token's 16 score sums (tcgen05.ld),
-//                  applies scale and zero-point (q.k = S_K (q.c) + Z_K sum(q)), takes p = 2^(s - m)
-//                  against its warpgroup's reference m and writes w = p * S_V (fp16 hi + lo per head) as
-//                  row t of the MN-major B operand of the output MMA; it keeps the sums of p and p * Z_V.
-//                  The last of the eight warps (four V, four S) to finish a block issues
-//                  O^T[channel, head] += A_V . w, one tcgen05.mma per live tile, into the warpgroup's own
-//                  accumulators.
+//   warps 0-11     three block warpgroups of 128 threads.  For its block, thread t
+//                  - unpacks the 128 codes of token t into fp16 bit patterns (a code field left in place
+//                    below bit 11 of an fp16 is exactly code * 2^(pos-24); one AND per pair of codes) and
+//                    stores them as row t of the score MMA's A operand in tensor memory (tcgen05.st);
+//                  - does the same for channel t's codes of the block's tokens: row t of the output MMA's
+//                    A operand (while the score MMAs run);
+//                  - reads its token's 16 score sums (tcgen05.ld), applies scale and zero-point
+//                    (q.k = S_K (q.c) + Z_K sum(q)), takes p = 2^(s - m) against its warpgroup's
+//                    reference m and writes w = p * S_V (fp16 hi + lo per head) as row t of the MN-major
+//                    B operand of the output MMA; it keeps the sums of p and p * Z_V.
+//   warp 12        the copies, as far ahead as the ring has free stages;
+//   warp 13        the score MMAs S[token, head] = A_K . Q''^T of every block, in block order: 8 tcgen05.mma
+//                  (128 x 16 x 16, fp16 in, fp32 accumulators in tensor memory), B = the query fragments in
+//                  shared memory (rows 0-7 the fp16 "hi" part of up to 8 heads, rows 8-15 the "lo"
+//                  remainder), and tcgen05.commit onto the warpgroup's mbarrier;
+//   warps 14, 15   the output MMAs O^T[channel, head] += A_V . w of alternate blocks, one tcgen05.mma per
+//                  live tile, into the block's warpgroup's own accumulators.
 //
-// A_K, A_V, the score accumulators, the weight buffer and the output accumulators exist twice (block n
-// uses buffer n mod 2, which is also the S warpgroup that owns it).  A reference m only moves when some
-// score of a block exceeds it by more than kTcMaxAhead (one OR over the warpgroup per block); the
-// warpgroup then takes the block's maxima plus some headroom, waits for its output MMAs, rescales its
-// accumulators in tensor memory and its running sums, and goes on.  A segment ends with one partial
-// (m, l, o[128]) per head and S warpgroup, merged with the INT16 tiles' per-warp partials like any split.
+// A_K, A_V, the score accumulators, the weight buffer and the output accumulators exist three times, one
+// set per warpgroup (480 of the 512 columns of tensor memory).  A reference m only moves when some score
+// of a block exceeds it by more than kTcMaxAhead (one OR over the warpgroup per block); the warpgroup
+// then takes the block's maxima plus some headroom, rescales its accumulators in tensor memory and its
+// running sums, and goes on.  A segment ends with one partial (m, l, o[128]) per head and warpgroup,
+// merged with the INT16 tiles' per-warp partials like any split.
 //
-// Every mbarrier wait has an iteration limit; a wait that runs out sets a CTA-wide abort flag and an
-// error word in global memory, after which the CTA skips its remaining waits, runs through its loops,
-// frees its tensor memory and returns (the results of that launch are then meaningless and the host
-// reports PMKVQ_ERR_DEVICE_WAIT).
+// Every mbarrier wait first tests its barrier without blocking, then polls with a time hint (the waiting
+// warp sleeps in hardware instead of spinning through the issue slots of the working warps) under an
+// iteration limit; a wait that runs out sets a CTA-wide abort flag and an error word in global memory,
+// after which the CTA skips its remaining waits, runs through its loops, gives copies still in flight a
+// bounded time to land, frees its tensor memory and returns (the results of that launch are then
+// meaningless and the host reports PMKVQ_ERR_DEVICE_WAIT).
 #pragma once
 
 namespace pmkvq {
@@ -84,7 +83,7 @@ struct TcCtx {
   uint32_t gi, gc;    // body blocks / chunks this CTA has pushed through the pipeline so far (all segments)
 };
 
-// barriers over one S warpgroup (128 threads); `any` also ORs a predicate
+// barriers over one block warpgroup (128 threads); `any` also ORs a predicate
 __device__ __forceinline__ bool swg_any(int sw, bool pred) {
   uint32_t r;
   asm volatile(
@@ -183,7 +182,7 @@ __device__ __forceinline__ void tc_walk(int t_lo, int t_hi, OnChunk on_chunk, On
 
 // The body tiles [t_lo, t_hi) of a segment, by all warps of the CTA in their roles.  Leaves the two S
 // warpgroups' partials in slots slot0, slot0 + 1 of (s_m, s_l, part_o).  Buffer / stage parities follow the
-// CTA-wide counts tc.gi / tc.gc: block number n uses buffer n mod 2, chunk number m stage m mod kStages, and
+// CTA-wide counts tc.gi / tc.gc: block number n uses the buffers of warpgroup n mod 3, chunk number m stage m mod kStages, and
 // every completion of a barrier is either waited for or provably over before the barrier can complete again.
 template <int BITS>
 __device__ __forceinline__ void tc_body(const AttnParams &p, TcCtx &tc, const uint8_t *body, int t_lo, int t_hi,
