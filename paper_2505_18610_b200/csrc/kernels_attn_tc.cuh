@@ -180,8 +180,8 @@ __device__ __forceinline__ void tc_walk(int t_lo, int t_hi, OnChunk on_chunk, On
   }
 }
 
-// The body tiles [t_lo, t_hi) of a segment, by all warps of the CTA in their roles.  Leaves the two S
-// warpgroups' partials in slots slot0, slot0 + 1 of (s_m, s_l, part_o).  Buffer / stage parities follow the
+// The body tiles [t_lo, t_hi) of a segment, by all warps of the CTA in their roles.  Leaves the three block
+// warpgroups' partials in slots slot0 .. slot0 + 2 of (s_m, s_l, part_o).  Buffer / stage parities follow the
 // CTA-wide counts tc.gi / tc.gc: block number n uses the buffers of warpgroup n mod 3, chunk number m stage m mod kStages, and
 // every completion of a barrier is either waited for or provably over before the barrier can complete again.
 template <int BITS>
