@@ -221,15 +221,17 @@ pmkvq_status pmkvq_calibrate_lambda(const void *d_K_pre_bf16, int32_t n_tokens, 
  * way; loss[alpha] = mean squared difference between the causal self-attention output (softmax of
  * Q K^T / sqrt(128), query head h reads KV head h / group, token t attends to tokens 0..t) of the
  * unquantized rotated tensors and of the quantized ones, over tokens, sequences, heads and channels.
- * Arithmetic: fp32 throughout (quantizer decisions as in pmkvq_append), sums of squared errors in fp64.
+ * Arithmetic: rotation, equalization and quantizer decisions in fp32 (as in pmkvq_append); the attention
+ * contractions run on the tensor cores with every operand carried as the sum of two fp16 numbers (22
+ * significant bits) and fp32 accumulation; softmax in fp32; sums of squared errors in fp64.
  * 2 + 2 (n_alphas + 1) launches: abs-max, rotation table, then per pass one launch that writes the pass's
- * Keys (and once the Values) as fp32 into the workspace and one attention launch.
+ * Keys (and once the Values) into the workspace and one attention launch.
  *   d_K_pre_bf16, d_V_bf16  DEVICE bf16 [n_tokens][n_seq][kv_heads][128]; Keys before RoPE, token t at position t
  *   d_Q_pre_bf16            DEVICE bf16 [n_tokens][n_seq][kv_heads * group][128], before RoPE
  *   bits                    2, 4, 8 or 16: the width whose loss is minimised (the block's Fbit)
  *   h_alphas                HOST [n_alphas], 1 <= n_alphas <= 64 (the section's grid: j / 20, j = 0..19)
  *   d_workspace             DEVICE, 256-byte aligned, pmkvq_alpha_grid_workspace_bytes(...) bytes of the same sizes
- *                           (fp32 copies of each pass's Keys and Values and of the unquantized output)
+ *                           (each pass's Keys and Values at 4 bytes per element, the unquantized output in fp32)
  *   h_losses                HOST [n_alphas], written
  *   h_best                  HOST, may be NULL: index of the smallest loss (the first one on ties)
  * The call synchronises `stream` before it returns (its results are host values).  The paper states

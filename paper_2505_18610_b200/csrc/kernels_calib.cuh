@@ -81,16 +81,43 @@ __global__ void rope_table_kernel(float2 *table, int n_tokens, double pos_scale,
   table[i] = make_float2((float)c, (float)s);
 }
 
-constexpr int kQPT = 4;                     // queries per thread
-constexpr int kGridQueries = 16 * kQPT;     // queries of one CTA: 16 groups of kQPT queries, 8 threads per group
-constexpr int kGridKeys = 32;     // keys per shared-memory tile
+constexpr int kGridQueries = 64;            // queries of one CTA: four warps of 16
+constexpr int kGridKeys = 32;               // keys per shared-memory tile
 constexpr int kMaxAlphas = 64;
 __device__ __forceinline__ float ex2_fast(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-constexpr int kGridSmemBytes = 2 * 2 * kGridKeys * kHeadDim * 4;  // two stages of a K tile and a V tile
+// A tile in shared memory: four planes (K hi, K lo, V hi, V lo) of kGridKeys rows of 128 fp16; a row takes 272
+// bytes so that the eight 16-byte rows of an 8 x 8 ldmatrix tile fall into different banks.
+constexpr int kGridRowBytes = 2 * kHeadDim + 16;
+constexpr int kGridPlaneBytes = kGridKeys * kGridRowBytes;
+constexpr int kGridStageBytes = 4 * kGridPlaneBytes;
+constexpr int kGridSmemBytes = 2 * kGridStageBytes;  // two stages
+
+// x = hi + lo with both parts fp16: 22 significant bits (an absolute 2^-25 below 1/8), which three tensor-core
+// products hi*hi + hi*lo + lo*hi carry into the fp32 accumulator.
+__device__ __forceinline__ void split_half(float x, __half &hi, __half &lo) {
+  hi = __float2half_rn(x);
+  lo = __float2half_rn(x - __half2float(hi));
+}
+__device__ __forceinline__ void split_half2(float x, float y, uint32_t &hi, uint32_t &lo) {
+  __half hx, lx, hy, ly;
+  split_half(x, hx, lx);
+  split_half(y, hy, ly);
+  const __half2 h = __halves2half2(hx, hy), l = __halves2half2(lx, ly);
+  hi = *reinterpret_cast<const uint32_t *>(&h);
+  lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
 
 // One token's 4 channels per lane (channels 4 lane .. 4 lane + 3): rotate by the token's angles.  The
 // partner channel (+-64) sits in lane ^ 16.
@@ -137,7 +164,19 @@ __device__ __forceinline__ void load_bf16x4(const uint16_t *src, float (&x)[4]) 
   x[3] = __uint_as_float(raw.y & 0xFFFF0000u);
 }
 
-// One pass's Keys and Values as the attention kernel reads them: fp32 [n_tokens][n_seq][kv_heads][128].
+// Four values of vector `vec` (channels 4 lane ..) as fp16 hi and lo parts: the hi plane [n_vectors][128] fp16
+// is followed by the lo plane, together the 4 bytes per element of the fp32 buffer they replace.
+__device__ __forceinline__ void store_split4(float *out, long long n_vectors, long long vec, int lane, const float (&x)[4]) {
+  uint2 hi, lo;
+  split_half2(x[0], x[1], hi.x, lo.x);
+  split_half2(x[2], x[3], hi.y, lo.y);
+  __half *planes = reinterpret_cast<__half *>(out);
+  *reinterpret_cast<uint2 *>(planes + vec * kHeadDim + 4 * lane) = hi;
+  *reinterpret_cast<uint2 *>(planes + (n_vectors + vec) * kHeadDim + 4 * lane) = lo;
+}
+
+// One pass's Keys and Values as the attention kernel reads them: [n_tokens][n_seq][kv_heads][128] as fp16 hi and
+// lo planes (see store_split4).
 // One warp per (token, sequence, KV head) vector, lane l on channels 4 l .. 4 l + 3.
 //   alpha_index < 0  (the unquantized operator): k_out = rotated Keys, v_out = Values
 //   alpha_index >= 0: k_out = dequantized Q_bits(rotated Keys * Lambda^-1), lambda = max(amax, floor)^alpha;
@@ -164,55 +203,57 @@ __global__ void __launch_bounds__(128) alpha_grid_prep_kernel(const uint16_t *__
     xk[3] = __fmul_rn(xk[3], __fdiv_rn(1.0f, powf(fmaxf(am.w, floor_value), alpha)));
     quantize_dequantize_token(xk, bits);
   }
-  *reinterpret_cast<float4 *>(k_out + vec * kHeadDim + 4 * lane) = make_float4(xk[0], xk[1], xk[2], xk[3]);
+  store_split4(k_out, n_vectors, vec, lane, xk);
   if (v_out) {
     float xv[4];
     load_bf16x4(V + vec * kHeadDim + 4 * lane, xv);
     if (alpha_index >= 0) quantize_dequantize_token(xv, bits);
-    *reinterpret_cast<float4 *>(v_out + vec * kHeadDim + 4 * lane) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+    store_split4(v_out, n_vectors, vec, lane, xv);
   }
 }
 
-// One pass of causal self-attention in fp32.  Grid: (query blocks, query heads, sequences).
+// One pass of causal self-attention on the tensor cores at fp32-like precision.  Grid: (query blocks, query
+// heads, sequences); a CTA takes 64 queries, a warp 16 of them against all their keys.
 // Q: bf16 [n_tokens][n_seq][kv_heads * group][128] before RoPE (rotated here, and scaled by lambda(alpha)
-// when alpha_index >= 0, Eq. 9); k_in, v_in: this pass's tensors from alpha_grid_prep_kernel.
-// alpha_index < 0: the outputs go to o_ref [n_tokens][n_seq][q_heads][128]; otherwise the squared
+// when alpha_index >= 0, Eq. 9); k_in, v_in: this pass's tensors from alpha_grid_prep_kernel (fp16 hi and lo
+// planes).  alpha_index < 0: the outputs go to o_ref [n_tokens][n_seq][q_heads][128]; otherwise the squared
 // differences to o_ref are added to loss_sums[alpha_index] (fp64).
-// Thread (group, part) works on the group's kQPT consecutive queries and on channels 32 c + 4 part + e
-// (c < 4, e < 4): a rotation pair (i, i + 64) stays in one thread, the 8 parts read one 128-byte run of a
-// key row, every value read from shared memory feeds kQPT multiply-adds (one per query), and two keys are
-// taken per turn so that their score chains, shuffles and exponentials overlap.  Key / Value tiles of 32
-// tokens arrive through a two-stage cp.async ring.
-__global__ void __launch_bounds__(128) alpha_grid_attn_kernel(const uint16_t *__restrict__ Q, const float *__restrict__ k_in,
-                                                              const float *__restrict__ v_in, const float *__restrict__ amax,
-                                                              const float2 *__restrict__ table,
-                                                              const float *__restrict__ alphas, int alpha_index, int n_tokens,
-                                                              int n_seq, int kv_heads, int group, float floor_value,
-                                                              float *__restrict__ o_ref, double *loss_sums) {
-  extern __shared__ __align__(16) float s_dyn[];  // [stage][K | V][32 keys][128]
+// Every operand of the two contractions is a sum of two fp16 numbers (queries and probabilities split in
+// registers, keys and values by the prep kernel), and a product takes three mma.sync.m16n8k16 (hi hi, hi lo,
+// lo hi; the lo lo term is below 2^-22 of the product): the loss is a small difference of two attention
+// outputs, so plain fp16 or bf16 operands would drown it.  Key / Value tiles of 32 tokens arrive through a
+// two-stage cp.async ring; ldmatrix (transposed for the Values) builds the B fragments.
+__global__ void __launch_bounds__(128, 2) alpha_grid_attn_kernel(const uint16_t *__restrict__ Q, const float *__restrict__ k_in,
+                                                                 const float *__restrict__ v_in, const float *__restrict__ amax,
+                                                                 const float2 *__restrict__ table,
+                                                                 const float *__restrict__ alphas, int alpha_index, int n_tokens,
+                                                                 int n_seq, int kv_heads, int group, float floor_value,
+                                                                 float *__restrict__ o_ref, double *loss_sums) {
+  extern __shared__ __align__(16) uint8_t s_tiles[];  // [stage][K hi | K lo | V hi | V lo][32 keys][272 bytes]
   __shared__ float s_lam[kHeadDim];
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, tig = lane & 3;
   const int qb = (int)gridDim.x - 1 - (int)blockIdx.x;  // long rows first
   const int q_head = blockIdx.y, seq = blockIdx.z, kv_head = q_head / group, q_heads = kv_heads * group;
-  const int ql0 = (tid >> 3) * kQPT, part = tid & 7;  // first of the thread's queries inside the CTA
-  const int q0 = qb * kGridQueries + ql0;
+  const int q0 = qb * kGridQueries + 16 * warp;                   // first of the warp's queries
   const int q_last = min(n_tokens, (qb + 1) * kGridQueries) - 1;  // last live query of the CTA
-  const size_t kv_row = (size_t)n_seq * kv_heads * kHeadDim;
-  const float *k_base = k_in + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
-  const float *v_base = v_in + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
+  const size_t kv_row = (size_t)n_seq * kv_heads * kHeadDim;      // halfs from one token to the next
+  const size_t plane = (size_t)n_tokens * kv_row;                 // halfs from the hi plane to the lo plane
+  const __half *kv_base[4];
+  kv_base[0] = reinterpret_cast<const __half *>(k_in) + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
+  kv_base[1] = kv_base[0] + plane;
+  kv_base[2] = reinterpret_cast<const __half *>(v_in) + ((size_t)seq * kv_heads + kv_head) * kHeadDim;
+  kv_base[3] = kv_base[2] + plane;
   const float scale_log2 = 1.4426950408889634f * rsqrtf((float)kHeadDim);
-  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(s_dyn);
-  constexpr int kStageFloats = 2 * kGridKeys * kHeadDim;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(s_tiles);
 
-  // tile j -> stage j & 1: thread i copies 16-byte pieces i, i + 128, ... of the 32 x 512-byte rows
+  // tile j -> stage j & 1: thread i copies 16-byte pieces i, i + 128, ... of the 4 x 32 rows of 256 bytes
   auto issue = [&](int j) {
-    const uint32_t dst = ring + (uint32_t)((j & 1) * kStageFloats * 4);
+    const uint32_t dst = ring + (uint32_t)((j & 1) * kGridStageBytes);
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const int piece = tid + 128 * c, row = piece >> 5, col = (piece & 31) * 4;
+    for (int c = 0; c < 16; ++c) {
+      const int piece = tid + 128 * c, pl = piece >> 9, row = (piece >> 4) & 31, col = piece & 15;
       const int t = min(j * kGridKeys + row, n_tokens - 1);  // rows behind the last token are masked below
-      cp_async16(dst + (uint32_t)((row * kHeadDim + col) * 4), k_base + (size_t)t * kv_row + col);
-      cp_async16(dst + (uint32_t)(((kGridKeys + row) * kHeadDim + col) * 4), v_base + (size_t)t * kv_row + col);
+      cp_async16(dst + (uint32_t)(pl * kGridPlaneBytes + row * kGridRowBytes + col * 16), kv_base[pl] + (size_t)t * kv_row + col * 8);
     }
   };
   const int n_tiles = q_last / kGridKeys + 1;
@@ -221,35 +262,43 @@ __global__ void __launch_bounds__(128) alpha_grid_attn_kernel(const uint16_t *__
 
   s_lam[tid] = alpha_index >= 0 ? powf(fmaxf(amax[(size_t)kv_head * kHeadDim + tid], floor_value), alphas[alpha_index]) : 1.0f;
   __syncthreads();
-  // the thread's rotated, equalized, pre-scaled query channels: qe[n][4 c + e]
-  float qe[kQPT][16], acc[kQPT][16], m[kQPT], l[kQPT];
+
+  // ---- the warp's queries as A fragments: rotated, equalized, pre-scaled, split; qh / ql[k-step][register] ----
+  // register 0: row g, channels 16 ks + 2 tig, + 1; 1: row g + 8; 2: row g, channels + 8; 3: row g + 8, channels + 8
+  uint32_t qh[8][4], ql[8][4];
 #pragma unroll
-  for (int n = 0; n < kQPT; ++n) {
-    m[n] = -INFINITY;
-    l[n] = 0.f;
+  for (int rr = 0; rr < 2; ++rr) {
+    const int qi = min(q0 + g + 8 * rr, n_tokens - 1);  // a dead row repeats the last query; its output is dropped
+    const uint16_t *src = Q + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim;
+    const float2 *tab = table + (size_t)qi * 64;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) { qe[n][i] = 0.f; acc[n][i] = 0.f; }
-    const int qi = q0 + n;
-    if (qi < n_tokens) {
-      const uint16_t *src = Q + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim;
-      const float2 *tab = table + (size_t)qi * 64;
+    for (int ks = 0; ks < 4; ++ks)
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        float x1[4], x2[4];
-        load_bf16x4(src + 32 * c + 4 * part, x1);
-        load_bf16x4(src + 64 + 32 * c + 4 * part, x2);
+      for (int c8 = 0; c8 < 2; ++c8) {
+        const int ch = 16 * ks + 8 * c8 + 2 * tig;  // channels ch, ch + 1 and their rotation partners + 64
+        const uint32_t r1 = *reinterpret_cast<const uint32_t *>(src + ch), r2 = *reinterpret_cast<const uint32_t *>(src + ch + 64);
+        float y1[2], y2[2];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int ch = 32 * c + 4 * part + e;
-          const float2 cs = tab[ch];
-          const float y1 = __fsub_rn(__fmul_rn(x1[e], cs.x), __fmul_rn(x2[e], cs.y));
-          const float y2 = __fadd_rn(__fmul_rn(x1[e], cs.y), __fmul_rn(x2[e], cs.x));
-          qe[n][4 * c + e] = y1 * s_lam[ch] * scale_log2;
-          qe[n][4 * (c + 2) + e] = y2 * s_lam[ch + 64] * scale_log2;
+        for (int e = 0; e < 2; ++e) {
+          const float x1 = __uint_as_float(e ? (r1 & 0xFFFF0000u) : (r1 << 16));
+          const float x2 = __uint_as_float(e ? (r2 & 0xFFFF0000u) : (r2 << 16));
+          const float2 cs = tab[ch + e];
+          y1[e] = __fsub_rn(__fmul_rn(x1, cs.x), __fmul_rn(x2, cs.y)) * s_lam[ch + e] * scale_log2;
+          y2[e] = __fadd_rn(__fmul_rn(x1, cs.y), __fmul_rn(x2, cs.x)) * s_lam[ch + e + 64] * scale_log2;
         }
+        split_half2(y1[0], y1[1], qh[ks][2 * c8 + rr], ql[ks][2 * c8 + rr]);
+        split_half2(y2[0], y2[1], qh[ks + 4][2 * c8 + rr], ql[ks + 4][2 * c8 + rr]);
       }
-    }
   }
+
+  float acc[16][4];          // O[16 queries][128]: n-block nb holds channels 8 nb + 2 tig, + 1 of rows g (0, 1) and g + 8 (2, 3)
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};  // rows g, g + 8 (l: this thread's columns only)
+#pragma unroll
+  for (int nb = 0; nb < 16; ++nb) acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
+  // ldmatrix row addresses of this lane inside a plane: lane = 8 mat + row
+  const int lm_row = lane & 7, lm_mat = lane >> 3;
+  const uint32_t k_lane_off = (uint32_t)((((lm_mat >> 1) * 8 + lm_row) * kGridRowBytes) + (lm_mat & 1) * 16);  // keys of two n-blocks, channels k0 / k0 + 8
+  const uint32_t v_lane_off = (uint32_t)((((lm_mat & 1) * 8 + lm_row) * kGridRowBytes) + (lm_mat >> 1) * 16);  // keys k0 / k0 + 8, channels of two n-blocks
 
   for (int j = 0; j < n_tiles; ++j) {
     __syncthreads();  // everyone is done with the stage that tile j + 1 will overwrite
@@ -257,64 +306,80 @@ __global__ void __launch_bounds__(128) alpha_grid_attn_kernel(const uint16_t *__
     cp_async_commit();
     cp_async_wait<1>();  // tile j has landed (this thread's pieces)
     __syncthreads();     // ... and everyone else's
-    const float(*s_k)[kHeadDim] = reinterpret_cast<const float(*)[kHeadDim]>(s_dyn + (j & 1) * kStageFloats);
-    const float(*s_v)[kHeadDim] = s_k + kGridKeys;
     const int k0 = j * kGridKeys;
-    const int k_hi = min(kGridKeys, q_last - k0 + 1);
-    for (int kk = 0; kk < k_hi; kk += 2) {  // two keys per turn: their dependent chains overlap
-      // (a second key beyond k_hi lies behind every query of the CTA and is masked below; its row exists)
-      float s[2][kQPT];
+    if (k0 > q0 + 15) continue;  // every key of the tile lies behind every query of this warp (the barriers above still run)
+    const uint32_t st = ring + (uint32_t)((j & 1) * kGridStageBytes);
+    // ---- S[16 queries][32 keys] = Q K^T ----
+    float sc[4][4];
 #pragma unroll
-      for (int n = 0; n < kQPT; ++n) s[0][n] = s[1][n] = 0.f;
+    for (int nb = 0; nb < 4; ++nb) sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const float4 ka = *reinterpret_cast<const float4 *>(&s_k[kk][32 * c + 4 * part]);
-        const float4 kb = *reinterpret_cast<const float4 *>(&s_k[kk + 1][32 * c + 4 * part]);
+    for (int ks = 0; ks < 8; ++ks) {
 #pragma unroll
-        for (int n = 0; n < kQPT; ++n) {
-          s[0][n] = fmaf(qe[n][4 * c], ka.x, s[0][n]); s[1][n] = fmaf(qe[n][4 * c], kb.x, s[1][n]);
-          s[0][n] = fmaf(qe[n][4 * c + 1], ka.y, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 1], kb.y, s[1][n]);
-          s[0][n] = fmaf(qe[n][4 * c + 2], ka.z, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 2], kb.z, s[1][n]);
-          s[0][n] = fmaf(qe[n][4 * c + 3], ka.w, s[0][n]); s[1][n] = fmaf(qe[n][4 * c + 3], kb.w, s[1][n]);
-        }
+      for (int np = 0; np < 2; ++np) {  // n-blocks 2 np, 2 np + 1
+        uint32_t bh[4], bl[4];
+        const uint32_t a = st + k_lane_off + (uint32_t)(np * 16 * kGridRowBytes + ks * 32);
+        ldsm_x4(a, bh);
+        ldsm_x4(a + kGridPlaneBytes, bl);
+        mma_f16(sc[2 * np], qh[ks], bh[0], bh[1]);
+        mma_f16(sc[2 * np], qh[ks], bl[0], bl[1]);
+        mma_f16(sc[2 * np], ql[ks], bh[0], bh[1]);
+        mma_f16(sc[2 * np + 1], qh[ks], bh[2], bh[3]);
+        mma_f16(sc[2 * np + 1], qh[ks], bl[2], bl[3]);
+        mma_f16(sc[2 * np + 1], ql[ks], bh[2], bh[3]);
       }
+    }
+    // ---- causal mask, running maximum, probabilities ----
+    const bool diagonal = k0 + kGridKeys - 1 > q0;  // some key of the tile may lie behind some query of the warp
 #pragma unroll
-      for (int o = 1; o <= 4; o <<= 1)
+    for (int rr = 0; rr < 2; ++rr) {
+      const int qi = q0 + g + 8 * rr;
+      float mx = -INFINITY;
 #pragma unroll
-        for (int n = 0; n < kQPT; ++n) {
-          s[0][n] += __shfl_xor_sync(0xffffffffu, s[0][n], o);
-          s[1][n] += __shfl_xor_sync(0xffffffffu, s[1][n], o);
+      for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          if (diagonal && k0 + 8 * nb + 2 * tig + e > qi) sc[nb][2 * rr + e] = -INFINITY;
+          mx = fmaxf(mx, sc[nb][2 * rr + e]);
         }
-      float p[2][kQPT];
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      // key 0 is live for every query and sits in the first tile, so m is finite from the first tile on
+      const float m_new = fmaxf(m[rr], mx);
+      const float corr = ex2_fast(m[rr] - m_new);  // 0 on the first tile
+      m[rr] = m_new;
+      l[rr] *= corr;
 #pragma unroll
-      for (int n = 0; n < kQPT; ++n) {
-        // causal mask (the eight threads of a group agree); key 0 is live for every query, so m is finite
-        // from the first turn on
-        const float sa = (k0 + kk <= q0 + n) ? s[0][n] : -INFINITY;
-        const float sb = (k0 + kk + 1 <= q0 + n) ? s[1][n] : -INFINITY;
-        const float mx = fmaxf(sa, sb);
-        if (mx > m[n]) {
-          const float corr = ex2_fast(m[n] - mx);  // 0 on the first key
-          l[n] *= corr;
+      for (int nb = 0; nb < 16; ++nb) { acc[nb][2 * rr] *= corr; acc[nb][2 * rr + 1] *= corr; }
 #pragma unroll
-          for (int i = 0; i < 16; ++i) acc[n][i] *= corr;
-          m[n] = mx;
+      for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float pe = ex2_fast(sc[nb][2 * rr + e] - m_new);
+          sc[nb][2 * rr + e] = pe;
+          l[rr] += pe;
         }
-        p[0][n] = ex2_fast(sa - m[n]);
-        p[1][n] = ex2_fast(sb - m[n]);
-        l[n] += p[0][n] + p[1][n];
-      }
+    }
+    // ---- O += P V: the probability fragments of two key n-blocks are the A fragment of one k-step ----
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const float4 va = *reinterpret_cast<const float4 *>(&s_v[kk][32 * c + 4 * part]);
-        const float4 vb = *reinterpret_cast<const float4 *>(&s_v[kk + 1][32 * c + 4 * part]);
+    for (int ks = 0; ks < 2; ++ks) {
+      uint32_t ph[4], pl[4];
+      split_half2(sc[2 * ks][0], sc[2 * ks][1], ph[0], pl[0]);
+      split_half2(sc[2 * ks][2], sc[2 * ks][3], ph[1], pl[1]);
+      split_half2(sc[2 * ks + 1][0], sc[2 * ks + 1][1], ph[2], pl[2]);
+      split_half2(sc[2 * ks + 1][2], sc[2 * ks + 1][3], ph[3], pl[3]);
 #pragma unroll
-        for (int n = 0; n < kQPT; ++n) {
-          acc[n][4 * c] = fmaf(p[1][n], vb.x, fmaf(p[0][n], va.x, acc[n][4 * c]));
-          acc[n][4 * c + 1] = fmaf(p[1][n], vb.y, fmaf(p[0][n], va.y, acc[n][4 * c + 1]));
-          acc[n][4 * c + 2] = fmaf(p[1][n], vb.z, fmaf(p[0][n], va.z, acc[n][4 * c + 2]));
-          acc[n][4 * c + 3] = fmaf(p[1][n], vb.w, fmaf(p[0][n], va.w, acc[n][4 * c + 3]));
-        }
+      for (int np = 0; np < 8; ++np) {  // channel n-blocks 2 np, 2 np + 1
+        uint32_t bh[4], bl[4];
+        const uint32_t a = st + 2 * kGridPlaneBytes + v_lane_off + (uint32_t)(ks * 16 * kGridRowBytes + np * 32);
+        ldsm_x4_trans(a, bh);
+        ldsm_x4_trans(a + kGridPlaneBytes, bl);
+        mma_f16(acc[2 * np], ph, bh[0], bh[1]);
+        mma_f16(acc[2 * np], ph, bl[0], bl[1]);
+        mma_f16(acc[2 * np], pl, bh[0], bh[1]);
+        mma_f16(acc[2 * np + 1], ph, bh[2], bh[3]);
+        mma_f16(acc[2 * np + 1], ph, bl[2], bl[3]);
+        mma_f16(acc[2 * np + 1], pl, bh[2], bh[3]);
       }
     }
   }
@@ -323,20 +388,23 @@ __global__ void __launch_bounds__(128) alpha_grid_attn_kernel(const uint16_t *__
   // ---- the pass's output: keep it (the unquantized pass) or compare with the kept one ----
   float err = 0.f;
 #pragma unroll
-  for (int n = 0; n < kQPT; ++n) {
-    if (q0 + n < n_tokens) {
-      const float inv_l = __fdiv_rn(1.0f, l[n]);
-      float *kept = o_ref + (((size_t)(q0 + n) * n_seq + seq) * q_heads + q_head) * kHeadDim + 4 * part;
+  for (int rr = 0; rr < 2; ++rr) {
+    float ls = l[rr];
+    ls += __shfl_xor_sync(0xffffffffu, ls, 1);
+    ls += __shfl_xor_sync(0xffffffffu, ls, 2);
+    const int qi = q0 + g + 8 * rr;
+    if (qi < n_tokens) {
+      const float inv_l = __fdiv_rn(1.0f, ls);
+      float *kept = o_ref + (((size_t)qi * n_seq + seq) * q_heads + q_head) * kHeadDim + 2 * tig;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        float4 o = make_float4(acc[n][4 * c] * inv_l, acc[n][4 * c + 1] * inv_l, acc[n][4 * c + 2] * inv_l,
-                               acc[n][4 * c + 3] * inv_l);
+      for (int nb = 0; nb < 16; ++nb) {
+        float2 o = make_float2(acc[nb][2 * rr] * inv_l, acc[nb][2 * rr + 1] * inv_l);
         if (alpha_index < 0) {
-          *reinterpret_cast<float4 *>(kept + 32 * c) = o;
+          *reinterpret_cast<float2 *>(kept + 8 * nb) = o;
         } else {
-          const float4 r = *reinterpret_cast<const float4 *>(kept + 32 * c);
-          o.x -= r.x; o.y -= r.y; o.z -= r.z; o.w -= r.w;
-          err = fmaf(o.x, o.x, err); err = fmaf(o.y, o.y, err); err = fmaf(o.z, o.z, err); err = fmaf(o.w, o.w, err);
+          const float2 r = *reinterpret_cast<const float2 *>(kept + 8 * nb);
+          o.x -= r.x; o.y -= r.y;
+          err = fmaf(o.x, o.x, err); err = fmaf(o.y, o.y, err);
         }
       }
     }

@@ -190,7 +190,8 @@ def test_device_alpha_grid_matches_oracle(n_tokens, n_seq, kv_heads, group, bits
     want = O.attention_reconstruction_losses(k, q, v, group, bits, alphas, pos_scale=scale)
     dev = [torch.tensor(t).to(torch.bfloat16).cuda().contiguous() for t in (k, q, v)]
     best, got = B.alpha_grid_search(dev[0], dev[1], dev[2], bits, alphas=alphas, pos_scale=scale)
-    # fp32 attention on both operators: the loss is a squared difference of two fp32 outputs, so its
+    # fp32-like attention on both operators (operands of 22 significant bits, fp32 sums): the loss is a squared
+    # difference of two such outputs, so its
     # relative error grows as the quantization error shrinks (2e-2 covers 8 bit)
     assert np.allclose(got, want, rtol=2e-2 if bits == 8 else 2e-3, atol=0)
     order = np.sort(want)
