@@ -510,8 +510,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-widths", action="store_true", help="skip the per-width steady-state records")
     ap.add_argument("--no-others", action="store_true", help="skip the compact 8B / 32B / 70B records")
-    ap.add_argument("--only", default="", choices=["", "reduce", "append"],
-                    help="profiling runs: only the progressive-reduce events or only the bulk append of the aux leg")
+    ap.add_argument("--only", default="", choices=["", "reduce", "append", "agrid"],
+                    help="profiling runs: only the progressive-reduce events, only the bulk append, or only a (small) alpha "
+                         "grid search of the aux leg")
     ap.add_argument("--attention-only", type=int, default=0,
                     help="profiling runs: build the cache at its final widths and launch the attention this many times")
     args = ap.parse_args()
@@ -571,6 +572,17 @@ def main():
             c = B.Cache(1, wl["q_heads"], wl["kv_heads"], wl["batch"], 32768, [16], n_sink=N_SINK, window=WINDOW, device=device)
             c.append(0, k, v); torch.cuda.synchronize(); c.close()
         print(json.dumps({"only": "append", "workload": wl["name"], "tokens": 8192}))
+        return
+    if args.only == "agrid":     # 3 alphas on 2048 tokens x 2 sequences: 4 attention passes, small enough to capture
+        from paper_2505_18610_b200 import binding as B
+        g = torch.Generator().manual_seed(5)
+        nt, ns, kvh, grp = 2048, 2, wl["kv_heads"], wl["q_heads"] // wl["kv_heads"]
+        kk = torch.randn(nt, ns, kvh, 128, generator=g); kk[..., 9] *= 25.0; kk[..., 73] *= 25.0
+        qq = torch.randn(nt, ns, kvh * grp, 128, generator=g)
+        vv = torch.randn(nt, ns, kvh, 128, generator=g)
+        kk, qq, vv = (t.to(torch.bfloat16).to(device).contiguous() for t in (kk, qq, vv))
+        best, losses = B.alpha_grid_search(kk, qq, vv, 2, alphas=np.array([0.0, 0.5, 0.8], dtype=np.float32), pos_scale=4.0)
+        print(json.dumps({"only": "agrid", "tokens": nt, "sequences": ns, "best_alpha": best, "losses": [float(x) for x in losses]}))
         return
     if args.attention_only:      # profiling runs: the steady-state attention launch and nothing else
         cache = build_cache(wl, fbit, None, lam, wl["end_tokens"], device, shared_chunks=True, attention_path=args.attention_path)
