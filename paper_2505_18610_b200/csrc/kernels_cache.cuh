@@ -710,23 +710,15 @@ __global__ void __launch_bounds__(128) append_step_kernel(const uint16_t *__rest
 // ---------------------------------------------------------------------------------------------
 // Eq. 3 (or the plain right shift of the ablations) on all codes of two adjacent words at 2B bits, packed into
 // one word at B bits: half h of the result holds the codes of half h of in0 in its low byte-half and those
-// of in1 above them.  The narrow widths work on several fields of a register at once: the products
-// (c + 2^(B-1)) (2^2B - 2^B + 1) of a 4-bit (8-bit) code fit the code's own byte (16-bit lane), so one
-// multiply-add serves four (two) codes.
+// of in1 above them.  The narrow widths work on several fields of a register at once: the product
+// (c + 8) 241 of an 8-bit code fits the code's own 16-bit lane, so one multiply-add serves two codes; the eight
+// 4-bit codes of a word are served by one add in place (halve_nibbles_in_place).
 template <int B, bool SHR>
 __device__ __forceinline__ uint32_t merge_words(uint32_t in0, uint32_t in1);
 
-template <bool SHR>
-__device__ __forceinline__ uint32_t halve_nibbles(uint32_t x) {  // 8 codes of 4 bit -> 8 codes of 2 bit in bits 0-7, 16-23
-  const uint32_t a = x & 0x0F0F0F0Fu, b = (x >> 4) & 0x0F0F0F0Fu;  // even / odd fields, one per byte
-  uint32_t ya, yb;
-  if (SHR) {
-    ya = (a >> 2) & 0x03030303u;
-    yb = (b >> 2) & 0x03030303u;
-  } else {  // (13 (c + 2)) >> 6 per byte: 13 * 17 = 221 stays inside the byte
-    ya = ((a * 13u + 0x1A1A1A1Au) >> 6) & 0x03030303u;
-    yb = ((b * 13u + 0x1A1A1A1Au) >> 6) & 0x03030303u;
-  }
+// the plain right shift of the ablations: 8 codes of 4 bit -> 8 codes of 2 bit in bits 0-7, 16-23
+__device__ __forceinline__ uint32_t shift_nibbles(uint32_t x) {
+  const uint32_t ya = (x >> 2) & 0x03030303u, yb = (x >> 6) & 0x03030303u;  // even / odd fields, one per byte
   return ((ya | (ya >> 4)) & 0x00330033u) | (((yb << 2) | (yb >> 2)) & 0x00CC00CCu);
 }
 template <bool SHR>
@@ -760,7 +752,7 @@ template <> __device__ __forceinline__ uint32_t merge_words<2, false>(uint32_t i
   return __byte_perm(gather_nibble_results(halve_nibbles_in_place(in0)) >> 6, gather_nibble_results(halve_nibbles_in_place(in1)) >> 6,
                      0x6240);
 }
-template <> __device__ __forceinline__ uint32_t merge_words<2, true>(uint32_t in0, uint32_t in1) { return halve_nibbles<true>(in0) | (halve_nibbles<true>(in1) << 8); }
+template <> __device__ __forceinline__ uint32_t merge_words<2, true>(uint32_t in0, uint32_t in1) { return shift_nibbles(in0) | (shift_nibbles(in1) << 8); }
 template <> __device__ __forceinline__ uint32_t merge_words<4, false>(uint32_t in0, uint32_t in1) { return halve_bytes<false>(in0) | (halve_bytes<false>(in1) << 8); }
 template <> __device__ __forceinline__ uint32_t merge_words<4, true>(uint32_t in0, uint32_t in1) { return halve_bytes<true>(in0) | (halve_bytes<true>(in1) << 8); }
 // 16 -> 8 bit: the product (c + 128) * 65281 needs all 32 bits; the new code is its top byte
