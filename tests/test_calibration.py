@@ -182,7 +182,8 @@ def test_device_calibration_matches_oracle(n_tokens, n_seq, kv_heads, scale):
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("n_tokens,n_seq,kv_heads,group,bits,scale",
-                         [(1, 1, 1, 1, 2, 1.0), (45, 2, 2, 3, 2, 1.0), (130, 1, 2, 7, 4, 4.0), (97, 2, 1, 2, 8, 2.0)])
+                         [(1, 1, 1, 1, 2, 1.0), (45, 2, 2, 3, 2, 1.0), (130, 1, 2, 7, 4, 4.0), (97, 2, 1, 2, 8, 2.0),
+                          (300, 2, 2, 4, 4, 1.0), (257, 1, 1, 8, 2, 2.0)])   # several query blocks and key tiles, ragged ends
 def test_device_alpha_grid_matches_oracle(n_tokens, n_seq, kv_heads, group, bits, scale):
     from paper_2505_18610_b200 import binding as B
     k, q, v = _calib_tensors(n_tokens, n_seq, kv_heads, group, seed=100 + n_tokens, outlier=(9, 25.0))
